@@ -1,0 +1,312 @@
+"""CPU oracle for the per-layer chunked-prefill step with retaining-head eviction.
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain fp64 restatement of the
+method that the CUDA library is checked against.  It shares no code with the
+CUDA path and must never be imported by the product package; only the tests,
+the smoke check and the benchmark's CPU-baseline leg may use it.
+
+What each function follows:
+
+* ``project_qkv``          – the per-layer projection [Q, K, V] = H · [W^Q, W^K, W^V]
+                             (Section 3.1, "Transformer Architecture").
+* ``rope``                 – rotary embedding at re-assigned contiguous positions
+                             (Section 3.4: the cache is kept pre-RoPE and positions are
+                             re-assigned from the beginning at every step).
+* ``attention_rows``       – Eq. 1: chunk queries over retained cache + causal chunk,
+                             GQA map ceil(j/g), scale 1/sqrt(d_m).
+* ``retaining_scores``     – S~ = sigma([Q, K, V] W1) W2 (Section 3.3).
+* ``select_keep``          – Algorithm 1: last n_s scores set to +inf, top-b, gather
+                             (stated without infinities: protected ∪ top-(b − n_prot) of the rest).
+* ``OracleLayer.prefill_chunk`` – one iteration of Algorithm 1's loop body for one layer.
+* ``quantize_int4`` / ``dequantize_int4`` – the 4-bit cache variant (Appendix H combines
+                             a 4-bit KV cache with the method; the number format is the
+                             workload's: symmetric, one fp16 scale per head vector).
+
+Readings taken where the paper is silent are listed in the design notes of the
+repository; the ones that matter here: W1 has (h + 2 h_kv)·d rows (all heads
+concatenated, order Q heads, K heads, V heads); the activation is SiLU by
+default; the retaining head sees the pre-RoPE projections by default; kept
+units stay in temporal order; ties prefer the more recent unit; NaN scores rank
+as −inf; the protected units are the last min(n_s, n) entries of cache ‖ chunk.
+
+Two modes.  ``mirror=False``: no rounding anywhere (used for the pins).
+``mirror=True``: values are rounded to bfloat16 exactly where the CUDA path
+stores them (Q, K, V after projection; Q, K after RoPE; dequantised int4
+values); everything else stays fp64.
+"""
+
+from __future__ import annotations
+
+import numpy as np
+
+NO_EVICT = 1
+LAST_CHUNK = 2
+
+
+class CapacityError(RuntimeError):
+    pass
+
+
+# --------------------------------------------------------------------------- rounding
+
+def _round_sig(x, sig_bits: int, min_frexp_exp: int):
+    """Round fp64 to a binary format with `sig_bits` significant bits (ties to even)."""
+    x = np.asarray(x, dtype=np.float64)
+    _, e = np.frexp(x)
+    e = np.maximum(e, min_frexp_exp)
+    q = np.ldexp(1.0, e - sig_bits)
+    with np.errstate(invalid="ignore"):
+        r = np.rint(x / q) * q
+    return np.where(np.isfinite(x), r, x)
+
+
+def round_bf16(x):
+    """Nearest bfloat16 (8 significant bits), returned as fp64."""
+    return _round_sig(x, 8, -125)
+
+
+def round_fp16(x):
+    """Nearest IEEE half (11 significant bits, subnormals below 2^-14), as fp64."""
+    return _round_sig(x, 11, -13)
+
+
+# --------------------------------------------------------------------------- steps
+
+def project_qkv(X, w_qkv, h: int, h_kv: int, d: int):
+    """[Q ‖ K ‖ V] = X · W_qkv; columns: h query heads, h_kv key heads, h_kv value heads."""
+    qkv = np.asarray(X, np.float64) @ np.asarray(w_qkv, np.float64)
+    return qkv
+
+
+def split_qkv(qkv, h: int, h_kv: int, d: int):
+    n = qkv.shape[0]
+    Q = qkv[:, : h * d].reshape(n, h, d)
+    K = qkv[:, h * d: (h + h_kv) * d].reshape(n, h_kv, d)
+    V = qkv[:, (h + h_kv) * d:].reshape(n, h_kv, d)
+    return Q, K, V
+
+
+def rope(x, pos, theta: float):
+    """Rotate-half rotary embedding: pairs (i, i + d/2), angle pos · theta^(−2i/d).
+
+    x: [..., d]; pos broadcastable to x.shape[:-1].
+    """
+    x = np.asarray(x, np.float64)
+    d = x.shape[-1]
+    half = d // 2
+    inv_freq = np.float64(theta) ** (-2.0 * np.arange(half, dtype=np.float64) / d)
+    ang = np.asarray(pos, np.float64)[..., None] * inv_freq
+    c, s = np.cos(ang), np.sin(ang)
+    x1, x2 = x[..., :half], x[..., half:]
+    return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
+
+
+def attention_rows(Qr, Kr_cache, V_cache, Kr_chunk, V_chunk, group: int, rows=None):
+    """Eq. 1 for the chunk's query rows.
+
+    Qr [n, h, d] (roped); Kr_cache/V_cache [h_kv, len, d]; Kr_chunk/V_chunk [n, h_kv, d].
+    Query t attends to every cache unit and to chunk units u <= t.
+    Returns out [n, h*d]; rows not listed in `rows` are NaN.
+    """
+    n, h, d = Qr.shape
+    ln = Kr_cache.shape[1]
+    rows = np.arange(n) if rows is None else np.asarray(rows, dtype=np.int64)
+    out = np.full((n, h * d), np.nan)
+    scale = 1.0 / np.sqrt(np.float64(d))
+    u = np.arange(n)
+    for j in range(h):
+        m = j // group                      # 0-based form of ceil(j/g)
+        Kall = np.concatenate([Kr_cache[m], Kr_chunk[:, m, :]], axis=0)
+        Vall = np.concatenate([V_cache[m], V_chunk[:, m, :]], axis=0)
+        logits = (Qr[rows, j, :] @ Kall.T) * scale
+        masked = u[None, :] > rows[:, None]              # chunk unit after the query
+        logits[:, ln:][masked] = -np.inf
+        logits -= logits.max(axis=1, keepdims=True)
+        p = np.exp(logits)
+        p /= p.sum(axis=1, keepdims=True)
+        out[rows, j * d:(j + 1) * d] = p @ Vall
+    return out
+
+
+def activation(x, act: int):
+    if act == 0:      # SiLU
+        return x / (1.0 + np.exp(-x))
+    if act == 1:      # GELU, tanh form
+        return 0.5 * x * (1.0 + np.tanh(np.sqrt(2.0 / np.pi) * (x + 0.044715 * x ** 3)))
+    if act == 2:
+        return np.maximum(x, 0.0)
+    raise ValueError(act)
+
+
+def retaining_scores(z, w1, w2, act: int = 0):
+    """S~ = sigma(z W1) W2, one score per KV head per token; z = [Q ‖ K ‖ V] of the token."""
+    hidden = activation(np.asarray(z, np.float64) @ np.asarray(w1, np.float64), act)
+    return hidden @ np.asarray(w2, np.float64)
+
+
+def select_keep(scores, budget: int, n_prot: int):
+    """Slots kept by one head: the last n_prot, plus the best (budget − n_prot) of the rest.
+
+    Order among the rest: higher score first; equal scores: more recent slot first;
+    NaN ranks as −inf.  Returns ascending slot indices (temporal order).
+    """
+    s = np.array(scores, dtype=np.float64)
+    n = s.shape[0]
+    if n <= budget:
+        return np.arange(n, dtype=np.int64)
+    n_prot = min(n_prot, n, budget)
+    rest = n - n_prot
+    sr = np.where(np.isnan(s[:rest]), -np.inf, s[:rest])
+    idx = np.arange(rest, dtype=np.int64)
+    order = np.lexsort((-idx, -sr))          # primary: score desc; secondary: slot desc
+    chosen = order[: budget - n_prot]
+    keep = np.concatenate([chosen, np.arange(rest, n, dtype=np.int64)])
+    return np.sort(keep)
+
+
+def quantize_int4(x):
+    """Symmetric 4-bit codes for one group per leading index: x [..., d] -> (codes int8, scale).
+
+    scale = fp16(absmax / 7) (1 if the vector is all zero); code = clamp(rne(x / scale), −8, 7).
+    The division that decides the code is taken in float32, the precision the
+    CUDA kernel decides it in.
+    """
+    xf = np.asarray(x, dtype=np.float32)
+    amax = np.max(np.abs(xf), axis=-1, keepdims=True)
+    scale = (amax / np.float32(7.0)).astype(np.float16)
+    scale = np.where(scale == 0, np.float16(1.0), scale)
+    q = np.rint(xf / scale.astype(np.float32))
+    codes = np.clip(q, -8, 7).astype(np.int8)
+    return codes, scale[..., 0].astype(np.float64)
+
+
+def dequantize_int4(codes, scale):
+    return codes.astype(np.float64) * np.asarray(scale, np.float64)[..., None]
+
+
+# --------------------------------------------------------------------------- layer
+
+class OracleLayer:
+    """State and step of one decoder layer's attention block under Algorithm 1."""
+
+    def __init__(self, shape, w_qkv, w1, w2, budget: int, chunk: int, n_stab: int,
+                 reserve: int = 0, mirror: bool = False):
+        if n_stab > budget or budget < 1 or chunk < 1 or n_stab < 0:
+            raise ValueError("need 0 <= n_stab <= budget, budget >= 1, chunk >= 1")
+        if shape.n_q_heads % shape.n_kv_heads:
+            raise ValueError("n_q_heads must be a multiple of n_kv_heads")
+        self.s = shape
+        self.h, self.hk, self.d = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+        self.g = self.h // self.hk
+        self.w_qkv = np.asarray(w_qkv, np.float64)
+        self.w1 = np.asarray(w1, np.float64)
+        self.w2 = np.asarray(w2, np.float64)
+        self.budget, self.chunk, self.n_stab = budget, chunk, n_stab
+        self.cap = budget + chunk + reserve
+        self.mirror = mirror
+        self.int4 = shape.kv_dtype == 1
+        self.reset()
+
+    # ---- state
+    def reset(self):
+        hk, d = self.hk, self.d
+        self.K = np.zeros((hk, 0, d))          # pre-RoPE keys (dequantised if int4)
+        self.V = np.zeros((hk, 0, d))
+        self.S = np.zeros((hk, 0))
+        self.T = np.zeros((hk, 0), dtype=np.int64)   # absolute token index of each unit
+        if self.int4:
+            self.Kc = np.zeros((hk, 0, d), np.int8); self.Ks = np.zeros((hk, 0))
+            self.Vc = np.zeros((hk, 0, d), np.int8); self.Vs = np.zeros((hk, 0))
+        self.seen = 0
+        self.last_scores = None
+        self.last_keep = None
+
+    @property
+    def len(self) -> int:
+        return self.K.shape[1]
+
+    def export_state(self):
+        st = dict(K=self.K.copy(), V=self.V.copy(), S=self.S.copy(), T=self.T.copy(),
+                  seen=self.seen)
+        if self.int4:
+            st.update(Kc=self.Kc.copy(), Ks=self.Ks.copy(), Vc=self.Vc.copy(), Vs=self.Vs.copy())
+        return st
+
+    def import_state(self, st):
+        self.K, self.V = st["K"].copy(), st["V"].copy()
+        self.S, self.T = st["S"].copy(), st["T"].copy()
+        self.seen = int(st["seen"])
+        if self.int4:
+            self.Kc, self.Ks = st["Kc"].copy(), st["Ks"].copy()
+            self.Vc, self.Vs = st["Vc"].copy(), st["Vs"].copy()
+
+    def _r(self, x):
+        return round_bf16(x) if self.mirror else x
+
+    # ---- one chunk
+    def prefill_chunk(self, X, flags: int = 0, rows=None):
+        """One loop iteration of Algorithm 1 for this layer.  Returns attn_out [n_tok, h·d]."""
+        X = np.asarray(X, np.float64)
+        n_tok = X.shape[0]
+        h, hk, d, g = self.h, self.hk, self.d, self.g
+        ln = self.len
+        if n_tok < 1 or n_tok > self.chunk:
+            raise ValueError("n_tok must be in [1, chunk]")
+        if ln + n_tok > self.cap:
+            raise CapacityError("cache capacity exceeded")
+
+        # (a) projections; the staging buffer is a storage point
+        qkv = self._r(project_qkv(X, self.w_qkv, h, hk, d))
+        Q, K, V = split_qkv(qkv, h, hk, d)
+
+        # positions: cache slot i -> i, chunk token t -> len + t
+        pos_chunk = (ln + np.arange(n_tok))[:, None]
+        Qr = self._r(rope(Q, pos_chunk, self.s.rope_theta))
+        Kr_chunk = self._r(rope(K, pos_chunk, self.s.rope_theta))
+        Kr_cache = self._r(rope(self.K, np.arange(ln)[None, :], self.s.rope_theta))
+        V_cache = self._r(self.V) if self.int4 else self.V
+
+        # (b) Eq. 1
+        out = attention_rows(Qr, Kr_cache, V_cache, Kr_chunk, V, g, rows)
+
+        # (c) retaining head on the token's concatenated [Q ‖ K ‖ V]
+        if self.s.rh_input == 0:
+            z = qkv
+        else:
+            z = np.concatenate([Qr.reshape(n_tok, -1), Kr_chunk.reshape(n_tok, -1),
+                                V.reshape(n_tok, -1)], axis=1)
+        s_chunk = retaining_scores(z, self.w1, self.w2, self.s.act)     # [n_tok, h_kv]
+        self.last_scores = s_chunk
+
+        # (d) concat, protect, top-b, gather
+        Kn = np.transpose(K, (1, 0, 2))
+        Vn = np.transpose(V, (1, 0, 2))
+        if self.int4:
+            kc, ks = quantize_int4(Kn)
+            vc, vs = quantize_int4(Vn)
+            self.Kc = np.concatenate([self.Kc, kc], axis=1); self.Ks = np.concatenate([self.Ks, ks], axis=1)
+            self.Vc = np.concatenate([self.Vc, vc], axis=1); self.Vs = np.concatenate([self.Vs, vs], axis=1)
+            Kn, Vn = dequantize_int4(kc, ks), dequantize_int4(vc, vs)
+        self.K = np.concatenate([self.K, Kn], axis=1)
+        self.V = np.concatenate([self.V, Vn], axis=1)
+        self.S = np.concatenate([self.S, s_chunk.T], axis=1)
+        tid = np.broadcast_to(self.seen + np.arange(n_tok, dtype=np.int64), (hk, n_tok))
+        self.T = np.concatenate([self.T, tid], axis=1)
+        n = ln + n_tok
+        self.seen += n_tok
+
+        self.last_keep = None
+        if not (flags & NO_EVICT) and n > self.budget:
+            n_prot = 0 if (flags & LAST_CHUNK) else min(self.n_stab, n)
+            keep = np.stack([select_keep(self.S[m], self.budget, n_prot) for m in range(hk)])
+            self.last_keep = keep
+            take = lambda a: np.stack([a[m][keep[m]] for m in range(hk)])
+            self.K, self.V, self.S, self.T = take(self.K), take(self.V), take(self.S), take(self.T)
+            if self.int4:
+                self.Kc, self.Ks = take(self.Kc), take(self.Ks)
+                self.Vc, self.Vs = take(self.Vc), take(self.Vs)
+        return out
+
+    def decode_step(self, x):
+        """The B = 1 case of Eq. 1: append without eviction."""
+        return self.prefill_chunk(np.asarray(x, np.float64).reshape(1, -1), NO_EVICT)

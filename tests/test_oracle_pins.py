@@ -1,0 +1,413 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+None of these tests needs a GPU and none touches the CUDA path.
+"""
+
+import itertools
+import math
+import os
+import types
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import locret_oracle as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def shape(**kw):
+    base = dict(d_model=16, n_q_heads=4, n_kv_heads=2, head_dim=8, d_retain=12,
+                rope_theta=10000.0, act=0, rh_input=0, kv_dtype=0)
+    base.update(kw)
+    return types.SimpleNamespace(**base)
+
+
+def rand_layer(sh, budget, chunk, n_stab, seed=0, **kw):
+    g = np.random.default_rng(seed)
+    d_in = (sh.n_q_heads + 2 * sh.n_kv_heads) * sh.head_dim
+    wqkv = g.standard_normal((sh.d_model, d_in)) / math.sqrt(sh.d_model)
+    w1 = g.standard_normal((d_in, sh.d_retain)) / math.sqrt(d_in)
+    w2 = g.standard_normal((sh.d_retain, sh.n_kv_heads)) / math.sqrt(sh.d_retain)
+    return O.OracleLayer(sh, wqkv, w1, w2, budget, chunk, n_stab, **kw), (wqkv, w1, w2)
+
+
+def run_chunks(layer, X, B, flags=0):
+    outs = []
+    for s in range(0, X.shape[0], B):
+        outs.append(layer.prefill_chunk(X[s:s + B], flags))
+    return np.concatenate(outs, axis=0)
+
+
+# ------------------------------------------------------------------ rounding
+
+def test_round_bf16_matches_library_conversion():
+    g = np.random.default_rng(1)
+    x = np.concatenate([g.standard_normal(20000) * 10.0 ** g.integers(-6, 6, 20000),
+                        [0.0, -0.0, 1.0, 1.00390625, 1.01171875, 3.0e38, 1e-30]])
+    # inputs restricted to float32 so the library conversion is a single rounding
+    x32 = x.astype(np.float32)
+    want = torch.from_numpy(x32).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(O.round_bf16(x32.astype(np.float64)), want)
+    # ties go to even: 1 + 2^-8 is halfway between 1 and 1 + 2^-7
+    assert O.round_bf16(1.0 + 2.0 ** -8) == 1.0
+    assert O.round_bf16(1.0 + 3 * 2.0 ** -8) == 1.0 + 2.0 ** -6
+
+
+def test_round_fp16_matches_library_conversion():
+    g = np.random.default_rng(2)
+    x = (g.standard_normal(20000) * 10.0 ** g.integers(-7, 4, 20000)).astype(np.float32)
+    want = x.astype(np.float16).astype(np.float64)
+    assert np.array_equal(O.round_fp16(x.astype(np.float64)), want)
+
+
+# ------------------------------------------------------------------ RoPE
+
+def test_rope_is_complex_rotation_of_half_split_pairs():
+    g = np.random.default_rng(3)
+    d, theta = 16, 500000.0
+    x = g.standard_normal((5, 3, d))
+    pos = np.array([0, 1, 7, 100, 5000])[:, None]
+    got = O.rope(x, pos, theta)
+    # independent statement: z_i = x_i + i x_{i+d/2}; z_i <- z_i * exp(i pos theta^(-2i/d))
+    z = x[..., : d // 2] + 1j * x[..., d // 2:]
+    w = np.exp(1j * pos[..., None] * theta ** (-2.0 * np.arange(d // 2) / d))
+    zr = z * w
+    want = np.concatenate([zr.real, zr.imag], axis=-1)
+    assert np.allclose(got, want, rtol=0, atol=1e-12)
+    assert np.array_equal(got[0], x[0])                     # position 0 is the identity
+    assert np.allclose(np.linalg.norm(got, axis=-1), np.linalg.norm(x, axis=-1))
+
+
+def test_rope_inner_product_depends_on_relative_position_only():
+    g = np.random.default_rng(4)
+    q, k = g.standard_normal(32), g.standard_normal(32)
+    a = O.rope(q, 17, 1e4) @ O.rope(k, 5, 1e4)
+    b = O.rope(q, 1017, 1e4) @ O.rope(k, 1005, 1e4)
+    assert abs(a - b) < 1e-9
+
+
+# ------------------------------------------------------------------ Pin 1: budget >= context
+
+def brute_force_causal_attention(X, wqkv, sh):
+    """One-shot causal GQA attention with RoPE at true positions, in explicit loops."""
+    h, hk, d = sh.n_q_heads, sh.n_kv_heads, sh.head_dim
+    g = h // hk
+    n = X.shape[0]
+    out = np.zeros((n, h * d))
+    half = d // 2
+    freq = [sh.rope_theta ** (-2.0 * i / d) for i in range(half)]
+
+    def rot(v, p):
+        r = np.zeros(d)
+        for i in range(half):
+            c, s = math.cos(p * freq[i]), math.sin(p * freq[i])
+            r[i] = v[i] * c - v[i + half] * s
+            r[i + half] = v[i + half] * c + v[i] * s
+        return r
+
+    proj = X @ wqkv
+    for j in range(h):
+        m = j // g
+        q = [rot(proj[t, j * d:(j + 1) * d], t) for t in range(n)]
+        k = [rot(proj[t, (h + m) * d:(h + m + 1) * d], t) for t in range(n)]
+        v = [proj[t, (h + hk + m) * d:(h + hk + m + 1) * d] for t in range(n)]
+        for t in range(n):
+            lg = np.array([q[t] @ k[u] / math.sqrt(d) for u in range(t + 1)])
+            p = np.exp(lg - lg.max())
+            p /= p.sum()
+            out[t, j * d:(j + 1) * d] = sum(p[u] * v[u] for u in range(t + 1))
+    return out
+
+
+@pytest.mark.parametrize("B", [1, 5, 16, 37])
+@pytest.mark.parametrize("heads", [(4, 2), (4, 4), (6, 1)])
+def test_chunked_equals_full_attention_when_budget_covers_context(B, heads):
+    sh = shape(n_q_heads=heads[0], n_kv_heads=heads[1])
+    ctx = 37
+    layer, (wqkv, _, _) = rand_layer(sh, budget=ctx, chunk=max(B, 1), n_stab=3, seed=5)
+    X = np.random.default_rng(6).standard_normal((ctx, sh.d_model))
+    got = run_chunks(layer, X, B)
+    want = brute_force_causal_attention(X, wqkv, sh)
+    assert np.allclose(got, want, rtol=0, atol=1e-11)
+    assert layer.len == ctx and np.array_equal(layer.T[0], np.arange(ctx))
+
+
+def test_full_attention_matches_library_sdpa():
+    sh = shape(n_q_heads=4, n_kv_heads=2, head_dim=16, d_model=24)
+    ctx = 50
+    layer, (wqkv, _, _) = rand_layer(sh, budget=64, chunk=7, n_stab=0, seed=7)
+    X = np.random.default_rng(8).standard_normal((ctx, sh.d_model))
+    got = run_chunks(layer, X, 7)
+    h, hk, d = 4, 2, 16
+    proj = torch.from_numpy(X @ wqkv)
+    pos = np.arange(ctx)[:, None]
+    Q = torch.from_numpy(O.rope(proj[:, : h * d].reshape(ctx, h, d).numpy(), pos, sh.rope_theta))
+    K = torch.from_numpy(O.rope(proj[:, h * d:(h + hk) * d].reshape(ctx, hk, d).numpy(), pos, sh.rope_theta))
+    V = proj[:, (h + hk) * d:].reshape(ctx, hk, d)
+    K = K.repeat_interleave(h // hk, dim=1)
+    V = V.repeat_interleave(h // hk, dim=1)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        Q.permute(1, 0, 2)[None], K.permute(1, 0, 2)[None], V.permute(1, 0, 2)[None], is_causal=True)
+    ref = ref[0].permute(1, 0, 2).reshape(ctx, h * d).numpy()
+    assert np.allclose(got, ref, rtol=0, atol=1e-11)
+
+
+def test_decode_step_is_chunk_of_one():
+    sh = shape()
+    ctx = 20
+    layer, (wqkv, _, _) = rand_layer(sh, budget=8, chunk=6, n_stab=2, reserve=40, seed=9)
+    X = np.random.default_rng(10).standard_normal((ctx, sh.d_model))
+    outs = [layer.decode_step(X[t]) for t in range(ctx)]
+    want = brute_force_causal_attention(X, wqkv, sh)
+    assert np.allclose(np.concatenate(outs), want, atol=1e-11)
+    assert layer.len == ctx          # decode never evicts
+
+
+# ------------------------------------------------------------------ attention with an evicted cache
+
+def test_attention_over_evicted_cache_uses_reassigned_positions():
+    """After eviction the kept units sit at positions 0..len-1 and the chunk follows."""
+    sh = shape(n_q_heads=2, n_kv_heads=1)
+    layer, (wqkv, w1, w2) = rand_layer(sh, budget=6, chunk=5, n_stab=2, seed=11)
+    X = np.random.default_rng(12).standard_normal((15, sh.d_model))
+    layer.prefill_chunk(X[:5]); layer.prefill_chunk(X[5:10])
+    kept = layer.T[0].copy()
+    assert len(kept) == 6
+    out = layer.prefill_chunk(X[10:15])
+    # explicit: gather kept tokens + the chunk, positions 0..10, causal inside the chunk
+    h, d = 2, 8
+    proj = X @ wqkv
+    toks = list(kept) + list(range(10, 15))
+    pos = np.arange(len(toks))
+    Kr = O.rope(proj[toks, h * d:(h + 1) * d], pos, sh.rope_theta)
+    Vv = proj[toks, (h + 1) * d:]
+    for j in range(h):
+        for t in range(5):
+            q = O.rope(proj[10 + t, j * d:(j + 1) * d], 6 + t, sh.rope_theta)
+            lg = Kr[: 6 + t + 1] @ q / math.sqrt(d)
+            p = np.exp(lg - lg.max()); p /= p.sum()
+            assert np.allclose(out[t, j * d:(j + 1) * d], p @ Vv[: 6 + t + 1], atol=1e-12)
+
+
+# ------------------------------------------------------------------ retaining head (Pin 4)
+
+@pytest.mark.parametrize("act", [0, 1, 2])
+def test_retaining_head_matches_library_mlp(act):
+    g = np.random.default_rng(13)
+    z, w1, w2 = g.standard_normal((9, 20)), g.standard_normal((20, 7)), g.standard_normal((7, 3))
+    tz, t1, t2 = map(torch.from_numpy, (z, w1, w2))
+    F = torch.nn.functional
+    fn = {0: F.silu, 1: lambda v: F.gelu(v, approximate="tanh"), 2: F.relu}[act]
+    want = (fn(tz @ t1) @ t2).numpy()
+    assert np.allclose(O.retaining_scores(z, w1, w2, act), want, atol=1e-12)
+
+
+def test_retaining_head_hand_case():
+    # W1 picks input columns 0 and 2; W2 maps hidden 0 -> head 0 (x2) and hidden 1 -> head 1 (x-1)
+    z = np.array([[1.0, 5.0, -2.0]])
+    w1 = np.array([[1.0, 0.0], [0.0, 0.0], [0.0, 1.0]])
+    w2 = np.array([[2.0, 0.0], [0.0, -1.0]])
+    silu = lambda v: v / (1 + math.exp(-v))
+    got = O.retaining_scores(z, w1, w2, 0)
+    assert np.allclose(got, [[2 * silu(1.0), -silu(-2.0)]], atol=1e-15)
+
+
+def test_retaining_head_sees_all_heads_in_q_k_v_order():
+    sh = shape()
+    layer, (wqkv, w1, w2) = rand_layer(sh, budget=50, chunk=10, n_stab=0, seed=14)
+    X = np.random.default_rng(15).standard_normal((10, sh.d_model))
+    layer.prefill_chunk(X)
+    z = X @ wqkv                       # all Q heads, then K heads, then V heads
+    t = torch.from_numpy
+    want = (torch.nn.functional.silu(t(z) @ t(w1)) @ t(w2)).numpy()
+    assert np.allclose(layer.last_scores, want, atol=1e-12)
+    assert np.allclose(layer.S, want.T, atol=1e-12)
+    # a per-head-sized W1 (the other reading of the printed dimension) does not even fit
+    with pytest.raises(ValueError):
+        O.retaining_scores(z, w1[: 3 * sh.head_dim], w2)
+
+
+# ------------------------------------------------------------------ selection
+
+def literal_algorithm1_selection(scores, b, n_s, last_chunk):
+    """Algorithm 1 as printed: overwrite the last n_s scores with +inf, then top-b."""
+    s = np.array(scores, dtype=np.float64)
+    n = len(s)
+    if not last_chunk and n_s > 0:
+        s[max(0, n - n_s):] = np.inf
+    order = sorted(range(n), key=lambda i: (-s[i], -i))
+    return sorted(order[:b])
+
+
+def test_select_keep_equals_literal_algorithm1_bruteforce():
+    g = np.random.default_rng(16)
+    for n, b, n_s in itertools.product([1, 2, 5, 9, 14], [1, 3, 5, 8], [0, 1, 3, 5]):
+        if n_s > b:
+            continue
+        for trial in range(4):
+            s = g.standard_normal(n)
+            if trial == 1:
+                s = np.round(s)                       # many ties
+            want = literal_algorithm1_selection(s, b, n_s, False)
+            got = O.select_keep(s, b, n_s)
+            assert list(got) == want, (n, b, n_s, s)
+            assert list(O.select_keep(s, b, 0)) == literal_algorithm1_selection(s, b, n_s, True)
+
+
+def test_select_keep_ties_prefer_recent_and_nan_ranks_last():
+    assert list(O.select_keep([1.0, 1.0, 1.0, 1.0], 2, 0)) == [2, 3]
+    assert list(O.select_keep([np.nan, 0.0, -5.0, np.nan], 2, 0)) == [1, 2]
+    assert list(O.select_keep([np.nan, np.nan, -np.inf], 2, 0)) == [1, 2]
+
+
+# ------------------------------------------------------------------ Pin 2 / Pin 3
+
+@pytest.mark.parametrize("n_stab", [0, 3, 11, 40])
+@pytest.mark.parametrize("B", [4, 16, 25])
+def test_size_and_stabilizer_invariants_and_cache_problem_condition(n_stab, B):
+    sh = shape()
+    b = 40
+    layer, _ = rand_layer(sh, budget=b, chunk=B, n_stab=n_stab, seed=17)
+    X = np.random.default_rng(18).standard_normal((203, sh.d_model))
+    prev = [set() for _ in range(sh.n_kv_heads)]
+    for s in range(0, 203, B):
+        n_tok = min(B, 203 - s)
+        layer.prefill_chunk(X[s:s + B])
+        seen = s + n_tok
+        for m in range(sh.n_kv_heads):
+            T = layer.T[m]
+            assert len(T) == min(b, seen)                                  # size
+            assert np.all(np.diff(T) > 0)                                  # temporal order
+            ns = min(n_stab, seen)
+            assert set(range(seen - ns, seen)) <= set(T)                   # stabilizers kept
+            assert set(T) - prev[m] <= set(range(s, seen))                 # cache-problem cond. 2
+            prev[m] = set(T)
+
+
+@pytest.mark.parametrize("n_stab", [0, 7, 30])
+def test_final_retained_set_has_closed_form(n_stab):
+    """Scores depend on the token alone, so after any chunking the cache is
+    Last_{n_s} ∪ Top_{b − n_s}(all earlier tokens)."""
+    sh = shape()
+    b, ctx = 30, 157
+    X = np.random.default_rng(19).standard_normal((ctx, sh.d_model))
+    finals = []
+    for B in [1, 5, 30, 64]:
+        layer, (wqkv, w1, w2) = rand_layer(sh, budget=b, chunk=B, n_stab=n_stab, seed=20)
+        run_chunks(layer, X, B)
+        t = torch.from_numpy
+        s_all = (torch.nn.functional.silu(t(X @ wqkv) @ t(w1)) @ t(w2)).numpy()   # [ctx, hk]
+        for m in range(sh.n_kv_heads):
+            rest = ctx - n_stab
+            order = sorted(range(rest), key=lambda i: (-s_all[i, m], -i))
+            want = sorted(order[: b - n_stab] + list(range(rest, ctx)))
+            assert list(layer.T[m]) == want
+            assert np.allclose(layer.S[m], s_all[want, m], atol=1e-12)
+        finals.append(layer.T.copy())
+    for f in finals[1:]:
+        assert np.array_equal(f, finals[0])           # chunk-size invariance
+
+
+def test_last_chunk_flag_drops_protection_and_no_evict_appends():
+    sh = shape(n_kv_heads=1, n_q_heads=2)
+    layer, _ = rand_layer(sh, budget=5, chunk=8, n_stab=5, reserve=8, seed=21)
+    X = np.random.default_rng(22).standard_normal((24, sh.d_model))
+    layer.prefill_chunk(X[:8])
+    assert list(layer.T[0]) == [3, 4, 5, 6, 7]                 # all five slots are stabilizers
+    layer.prefill_chunk(X[8:16], O.LAST_CHUNK)
+    s = layer.S[0]
+    assert len(s) == 5
+    layer.prefill_chunk(X[16:24], O.NO_EVICT)
+    assert layer.len == 13 and list(layer.T[0][5:]) == list(range(16, 24))
+    with pytest.raises(O.CapacityError):
+        layer.prefill_chunk(X[:8], O.NO_EVICT)
+        layer.prefill_chunk(X[:8], O.NO_EVICT)
+
+
+# ------------------------------------------------------------------ Pin 5: arithmetic the paper prints
+
+def read_golden():
+    rows = {}
+    with open(os.path.join(GOLDEN, "paper_arithmetic.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            name, val, tol, _ = [p.strip() for p in line.split("|")]
+            rows[name] = (float(val), float(tol))
+    return rows
+
+
+def test_paper_printed_arithmetic_fixes_shapes():
+    gold = read_golden()
+
+    def near(name, x):
+        v, tol = gold[name]
+        assert abs(x - v) <= tol * v + 1e-12, (name, x, v)
+
+    # retaining-head size under the all-heads reading of W1: (h + 2 h_kv) d x d_R, d_R x h_kv
+    def rh_params(h, hk, d, dR, layers):
+        z = np.zeros((1, (h + 2 * hk) * d))
+        w1, w2 = np.zeros(((h + 2 * hk) * d, dR)), np.zeros((dR, hk))
+        assert O.retaining_scores(z, w1, w2).shape == (1, hk)
+        return layers * (w1.size + w2.size)
+
+    near("llama_retaining_param_share", rh_params(32, 8, 128, 1024, 32) / 8.03e9)
+    near("phi3_retaining_param_share", rh_params(32, 32, 96, 1024, 32) / 3.82e9)
+    # a cache unit is one token of one KV head of one layer, K and V, 16-bit
+    unit_bytes = 2 * 96 * 2
+    near("phi3_full_kv_128k_gb", 131072 * 32 * 32 * unit_bytes / 2 ** 30)
+    near("phi3_2bit_kv_128k_gb", 131072 * 32 * 32 * unit_bytes / 8 / 2 ** 30)
+    # the budget counts units per head: compression = context / budget
+    near("compression_10m", 10 * 2 ** 20 / 6000)
+    near("compression_phi3", 131072 / 6000)
+    near("compression_llama", 131072 / 16384)
+
+
+# ------------------------------------------------------------------ Pin 6: int4 cache
+
+def test_int4_roundtrip_properties():
+    g = np.random.default_rng(23)
+    x = O.round_bf16(g.standard_normal((4, 50, 128)) * 3)
+    codes, scale = O.quantize_int4(x)
+    assert codes.min() >= -8 and codes.max() <= 7
+    assert np.array_equal(scale, O.round_fp16(scale))                 # scales are fp16 values
+    deq = O.dequantize_int4(codes, scale)
+    assert np.all(np.abs(deq - x) <= scale[..., None] * 0.5 * (1 + 1e-6) + 1e-12)
+    # exact multiples of the scale survive
+    sc = 0.25
+    y = np.arange(-7, 8).astype(np.float64) * sc
+    y = np.concatenate([y, np.zeros(128 - 15)])[None]
+    c2, s2 = O.quantize_int4(y)
+    assert s2[0] == sc and np.array_equal(O.dequantize_int4(c2, s2), y)
+    # all-zero vector: scale 1, codes 0
+    c3, s3 = O.quantize_int4(np.zeros((1, 128)))
+    assert s3[0] == 1.0 and not c3.any()
+
+
+def test_int4_layer_quantises_on_append_and_moves_codes_unchanged():
+    sh = shape(kv_dtype=1, head_dim=8)
+    layer, (wqkv, _, _) = rand_layer(sh, budget=10, chunk=6, n_stab=2, seed=24, mirror=True)
+    X = O.round_bf16(np.random.default_rng(25).standard_normal((18, sh.d_model)))
+    layer.prefill_chunk(X[:6]); layer.prefill_chunk(X[6:12])
+    before = layer.export_state()
+    layer.prefill_chunk(X[12:18])
+    # every cached unit is codes * scale, and kept units carry identical codes
+    assert np.array_equal(layer.K, O.dequantize_int4(layer.Kc, layer.Ks))
+    for m in range(sh.n_kv_heads):
+        for slot, tok in enumerate(layer.T[m]):
+            if tok < 12:
+                old = list(before["T"][m]).index(tok)
+                assert np.array_equal(layer.Kc[m, slot], before["Kc"][m, old])
+                assert layer.Vs[m, slot] == before["Vs"][m, old]
+
+
+def test_mirror_mode_rounds_only_storage_points():
+    sh = shape()
+    lp, (wqkv, w1, w2) = rand_layer(sh, budget=64, chunk=16, n_stab=0, seed=26)
+    lm = O.OracleLayer(sh, wqkv, w1, w2, 64, 16, 0, mirror=True)
+    X = O.round_bf16(np.random.default_rng(27).standard_normal((16, sh.d_model)))
+    a, b = lp.prefill_chunk(X), lm.prefill_chunk(X)
+    assert np.array_equal(lm.K, O.round_bf16(lm.K))            # cached K is on the bf16 grid
+    assert np.max(np.abs(a - b)) < 0.05 and not np.array_equal(a, b)
