@@ -1,0 +1,163 @@
+/*
+ * locret.h — C ABI of the B200 (sm_100a) library for the per-layer chunked-prefill
+ * step with retaining-head eviction (Locret, arXiv 2410.01805).
+ *
+ * One `locret_layer` holds the state of one decoder layer's attention block: the
+ * retained cache units (pre-RoPE K, V), their causal importance scores, their token
+ * ids, and scratch.  One `locret_prefill_chunk` call is one iteration of the loop
+ * body of Algorithm 1 for that layer:
+ *
+ *   (a) [Q ‖ K ‖ V] = hidden_in · W_qkv                                  (Section 3.1)
+ *   (b) attention of the chunk's queries over the retained cache plus the causal
+ *       chunk, positions re-assigned contiguously from 0                 (Eq. 1, Section 3.4)
+ *   (c) retaining head  S~ = sigma([Q ‖ K ‖ V] W1) W2, one score per KV head per
+ *       token, W1 of size (h + 2 h_kv) d × d_R                           (Section 3.3)
+ *   (d) concatenate cache and chunk, protect the last n_stab units, keep the
+ *       top-`budget` per KV head, gather K, V, scores in temporal order  (Algorithm 1)
+ *
+ * Conventions
+ *   - Every function returns 0 (LOCRET_OK) or a negative LOCRET_ERR_* code; nothing
+ *     throws, aborts or exits.  Arguments are validated before anything is launched.
+ *   - "device" pointers are CUDA device memory of the current device, 16-byte aligned;
+ *     "host" pointers are ordinary host memory.  The caller owns every buffer it
+ *     passes; the library owns the cache, scores, token ids, scratch and its own
+ *     repacked copy of the weights (taken at create; the caller's weights may be
+ *     freed afterwards).
+ *   - All device work of a layer is enqueued on the stream given at create, without
+ *     host synchronisation unless stated.  A handle is bound to that stream and is
+ *     not thread-safe.  Layers created on the same stream share scratch.
+ *   - There is no CPU fallback: without a CUDA device every call that needs one
+ *     returns LOCRET_ERR_CUDA.
+ */
+#ifndef LOCRET_H_
+#define LOCRET_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LOCRET_OK                  0
+#define LOCRET_ERR_INVALID        (-1)  /* bad argument or configuration                    */
+#define LOCRET_ERR_ALLOC          (-2)  /* device or host allocation failed                 */
+#define LOCRET_ERR_CAPACITY       (-3)  /* len + n_tok exceeds budget + chunk + reserve     */
+#define LOCRET_ERR_CUDA           (-4)  /* a CUDA runtime/driver call failed                */
+#define LOCRET_ERR_DEVICE_TIMEOUT (-5)  /* a bounded device-side wait gave up (sticky)      */
+
+/* flags of locret_prefill_chunk */
+#define LOCRET_NO_EVICT    1u  /* append only (Algorithm 1's n_loc tail pass and decode)     */
+#define LOCRET_LAST_CHUNK  2u  /* evict without protecting stabilizers (Algorithm 1's
+                                  "if chunk is not the last chunk" test, negated)            */
+
+/* kernel families, indices into locret_read_timing's arrays */
+enum {
+  LOCRET_K_QKV = 0,     /* (a) projection GEMM                                   */
+  LOCRET_K_ROPE,        /* position assignment + RoPE + append of the chunk       */
+  LOCRET_K_ATTN,        /* (b) attention                                          */
+  LOCRET_K_RH,          /* (c) retaining head GEMM -> activation -> GEMM          */
+  LOCRET_K_RH_REDUCE,   /* (c) sum of the retaining head's partial scores         */
+  LOCRET_K_TOPK,        /* (d) per-head selection                                 */
+  LOCRET_K_COMPACT,     /* (d) gather / compaction + re-RoPE of kept keys         */
+  LOCRET_K_COUNT
+};
+
+typedef struct locret_layer locret_layer;   /* opaque */
+
+typedef struct {
+  int32_t d_model;      /* D: width of hidden_in                                              */
+  int32_t n_q_heads;    /* h                                                                  */
+  int32_t n_kv_heads;   /* h_kv = h / g; h must be a multiple of it                           */
+  int32_t head_dim;     /* d_m in the paper: 64, 96 or 128                                    */
+  int32_t d_retain;     /* d_R, hidden size of the retaining head (Section 4.1: 1024)         */
+  int32_t act;          /* sigma: 0 SiLU, 1 GELU (tanh form), 2 ReLU (Appendix A: the
+                           backbone's own non-linearity)                                      */
+  float   rope_theta;   /* RoPE base                                                          */
+  int32_t rh_input;     /* 0: retaining head reads pre-RoPE [Q ‖ K ‖ V]; 1: post-RoPE Q, K    */
+  int32_t kv_dtype;     /* 0: bf16 cache; 1: int4 codes + one fp16 scale per head vector      */
+  int32_t reserve;      /* cache slots beyond budget + chunk, for NO_EVICT appends            */
+  const void *w_qkv;    /* device bf16 [d_model × (h + 2 h_kv) d] row-major; columns: the h
+                           query heads, then the h_kv key heads, then the h_kv value heads    */
+  const void *w1;       /* device bf16 [(h + 2 h_kv) d × d_R] row-major                       */
+  const void *w2;       /* device bf16 [d_R × h_kv] row-major                                 */
+  void *stream;         /* cudaStream_t; NULL = the legacy default stream                     */
+} locret_layer_cfg;
+
+/*
+ * Create one layer's state for chunked prefill with a fixed cache budget (Section 3.4;
+ * hyper-parameters b, B, n_s of Table 4).  Requires 1 <= chunk, 1 <= budget,
+ * 0 <= n_stab <= budget.  Allocates device memory (cache for budget + chunk + reserve
+ * units per KV head, double-buffered; scratch), repacks the weights, and synchronises
+ * the stream once.  On failure *out is NULL and nothing stays allocated.
+ */
+int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, int32_t n_stab,
+                  locret_layer **out);
+
+/*
+ * One chunked-prefill step (loop body of Algorithm 1; attention per Eq. 1; scores per
+ * Section 3.3).  hidden_in: device bf16 [n_tok × d_model], row-major, 1 <= n_tok <= chunk.
+ * attn_out: device bf16 [n_tok × h·d] (concatenated heads, before W^O).
+ * With flags = 0 the last min(n_stab, len + n_tok) units are protected and the cache is
+ * cut to `budget` units per KV head; afterwards len = min(budget, len + n_tok).
+ * Asynchronous on the layer's stream.  LOCRET_ERR_CAPACITY if a NO_EVICT append does
+ * not fit.
+ */
+int locret_prefill_chunk(locret_layer *layer, const void *hidden_in, int32_t n_tok,
+                         uint32_t flags, void *attn_out);
+
+/*
+ * Decoding: the B = 1 case of Eq. 1 (Algorithm 1's generate).  hidden_in: device bf16
+ * [d_model]; attn_out: device bf16 [h·d].  Scores the new unit and appends it without
+ * eviction (uses a `reserve` slot).
+ */
+int locret_decode_step(locret_layer *layer, const void *hidden_in, void *attn_out);
+
+/* Number of retained units per KV head (the same for every head).  No device work. */
+int locret_cache_len(const locret_layer *layer, int32_t *len);
+
+/*
+ * Copy the retained state to HOST buffers (any may be NULL to skip it): K and V as bf16
+ * [h_kv × len × d] (K pre-RoPE; for an int4 cache the dequantised values rounded to
+ * bf16), scores fp32 [h_kv × len], token_ids int64 [h_kv × len] (index of the token in
+ * the stream), *len, *tokens_seen.  Synchronises the stream.
+ */
+int locret_export_state(locret_layer *layer, void *K, void *V, float *scores,
+                        int64_t *token_ids, int32_t *len, int64_t *tokens_seen);
+
+/*
+ * Replace the retained state from HOST buffers laid out as in locret_export_state
+ * (all four required), 0 <= len <= budget + chunk + reserve.  Rebuilds the rotated-key
+ * scratch at positions 0..len-1.  For an int4 cache the given K, V are quantised on
+ * entry.  Synchronises the stream.
+ */
+int locret_import_state(locret_layer *layer, const void *K, const void *V, const float *scores,
+                        const int64_t *token_ids, int32_t len, int64_t tokens_seen);
+
+/* Synchronise the stream; return the sticky device status (0, or LOCRET_ERR_*). */
+int locret_sync_status(locret_layer *layer);
+
+/* Forget all units: len = 0, tokens_seen = 0.  Asynchronous. */
+int locret_reset(locret_layer *layer);
+
+/*
+ * Per-kernel timing.  With enable != 0 every kernel launched for this layer is
+ * bracketed by CUDA events on the layer's stream.  locret_read_timing synchronises the
+ * stream, adds up the elapsed time and the number of launches per kernel family since
+ * the last read into ms[LOCRET_K_COUNT] and launches[LOCRET_K_COUNT] (host arrays), and
+ * clears the record.
+ */
+int locret_set_timing(locret_layer *layer, int32_t enable);
+int locret_read_timing(locret_layer *layer, float *ms, int64_t *launches);
+
+/* Total number of this library's kernels launched for the layer since create. */
+int locret_launch_count(const locret_layer *layer, int64_t *count);
+
+/* Free everything the layer owns.  Synchronises the stream.  NULL is allowed. */
+void locret_destroy(locret_layer *layer);
+
+const char *locret_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOCRET_H_ */

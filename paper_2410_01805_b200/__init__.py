@@ -1,0 +1,17 @@
+"""B200-native chunked-prefill step with retaining-head eviction (Locret).
+
+The package is a thin ctypes binding over ``liblocret.so`` (hand-written CUDA for
+sm_100a).  Every step of the path runs in the library's kernels; Python only
+marshals pointers.  There is no CPU fallback: importing the binding without the
+built library raises.
+"""
+
+from .binding import (  # noqa: F401
+    K_NAMES,
+    LAST_CHUNK,
+    NO_EVICT,
+    LocretError,
+    LocretLayer,
+    lib,
+    lib_path,
+)

@@ -1,0 +1,161 @@
+"""ctypes binding with the same names as the C ABI in include/locret.h."""
+
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+lib_path = os.path.join(_HERE, "liblocret.so")
+
+NO_EVICT = 1
+LAST_CHUNK = 2
+K_NAMES = ["qkv", "rope", "attn", "rh", "rh_reduce", "topk", "compact"]
+
+
+class LocretError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {lib.locret_strerror(code).decode()} ({code})")
+
+
+class locret_layer_cfg(C.Structure):
+    _fields_ = [
+        ("d_model", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+        ("head_dim", C.c_int32), ("d_retain", C.c_int32), ("act", C.c_int32),
+        ("rope_theta", C.c_float), ("rh_input", C.c_int32), ("kv_dtype", C.c_int32),
+        ("reserve", C.c_int32),
+        ("w_qkv", C.c_void_p), ("w1", C.c_void_p), ("w2", C.c_void_p), ("stream", C.c_void_p),
+    ]
+
+
+def _load():
+    if not os.path.exists(lib_path):
+        raise ImportError(
+            f"{lib_path} is missing: build it with `python -m paper_2410_01805_b200.build` "
+            "(there is no CPU fallback)")
+    l = C.CDLL(lib_path)
+    P = C.c_void_p
+    l.locret_strerror.restype = C.c_char_p
+    l.locret_strerror.argtypes = [C.c_int]
+    l.locret_create.argtypes = [C.POINTER(locret_layer_cfg), C.c_int32, C.c_int32, C.c_int32, C.POINTER(P)]
+    l.locret_prefill_chunk.argtypes = [P, P, C.c_int32, C.c_uint32, P]
+    l.locret_decode_step.argtypes = [P, P, P]
+    l.locret_cache_len.argtypes = [P, C.POINTER(C.c_int32)]
+    l.locret_export_state.argtypes = [P, P, P, P, P, C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
+    l.locret_import_state.argtypes = [P, P, P, P, P, C.c_int32, C.c_int64]
+    l.locret_sync_status.argtypes = [P]
+    l.locret_reset.argtypes = [P]
+    l.locret_set_timing.argtypes = [P, C.c_int32]
+    l.locret_read_timing.argtypes = [P, P, P]
+    l.locret_launch_count.argtypes = [P, C.POINTER(C.c_int64)]
+    l.locret_destroy.argtypes = [P]
+    l.locret_destroy.restype = None
+    return l
+
+
+lib = _load()
+
+
+def _check(code: int, what: str):
+    if code != 0:
+        raise LocretError(code, what)
+
+
+def _bf16_bits(t: torch.Tensor) -> np.ndarray:
+    return t.contiguous().view(torch.int16).numpy()
+
+
+class LocretLayer:
+    """One decoder layer's state; methods mirror the C entry points one to one."""
+
+    def __init__(self, shape, w_qkv: torch.Tensor, w1: torch.Tensor, w2: torch.Tensor,
+                 budget: int, chunk: int, n_stab: int, reserve: int = 0, stream=None):
+        for w in (w_qkv, w1, w2):
+            if not (w.is_cuda and w.dtype == torch.bfloat16 and w.is_contiguous()):
+                raise ValueError("weights must be contiguous CUDA bfloat16 tensors")
+        self.shape = shape
+        self.h, self.h_kv, self.d = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+        self.chunk, self.budget, self.n_stab = chunk, budget, n_stab
+        self.stream = stream if stream is not None else torch.cuda.current_stream()
+        cfg = locret_layer_cfg(
+            shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.d_retain,
+            shape.act, float(shape.rope_theta), shape.rh_input, shape.kv_dtype, reserve,
+            w_qkv.data_ptr(), w1.data_ptr(), w2.data_ptr(), self.stream.cuda_stream)
+        self._h = C.c_void_p()
+        _check(lib.locret_create(C.byref(cfg), budget, chunk, n_stab, C.byref(self._h)), "locret_create")
+
+    # -- the hot path
+    def prefill_chunk(self, hidden_in: torch.Tensor, attn_out: torch.Tensor, flags: int = 0,
+                      n_tok: int | None = None):
+        n_tok = hidden_in.shape[0] if n_tok is None else n_tok
+        _check(lib.locret_prefill_chunk(self._h, hidden_in.data_ptr(), n_tok, flags,
+                                        attn_out.data_ptr()), "locret_prefill_chunk")
+
+    def decode_step(self, hidden_in: torch.Tensor, attn_out: torch.Tensor):
+        _check(lib.locret_decode_step(self._h, hidden_in.data_ptr(), attn_out.data_ptr()),
+               "locret_decode_step")
+
+    # -- state
+    @property
+    def cache_len(self) -> int:
+        n = C.c_int32()
+        _check(lib.locret_cache_len(self._h, C.byref(n)), "locret_cache_len")
+        return n.value
+
+    def export_state(self):
+        """dict(K, V [h_kv, len, d] float32 holding bf16 values; S [h_kv, len]; T int64; seen)."""
+        n = self.cache_len
+        K = torch.empty((self.h_kv, n, self.d), dtype=torch.bfloat16)
+        V = torch.empty_like(K)
+        S = np.empty((self.h_kv, n), dtype=np.float32)
+        T = np.empty((self.h_kv, n), dtype=np.int64)
+        ln, seen = C.c_int32(), C.c_int64()
+        _check(lib.locret_export_state(self._h, K.data_ptr(), V.data_ptr(), S.ctypes.data,
+                                       T.ctypes.data, C.byref(ln), C.byref(seen)), "locret_export_state")
+        return dict(K=K.float().numpy(), V=V.float().numpy(), S=S, T=T, seen=seen.value)
+
+    def import_state(self, K, V, S, T, seen: int):
+        Kb = torch.from_numpy(np.ascontiguousarray(K, dtype=np.float32)).to(torch.bfloat16).contiguous()
+        Vb = torch.from_numpy(np.ascontiguousarray(V, dtype=np.float32)).to(torch.bfloat16).contiguous()
+        Sb = np.ascontiguousarray(S, dtype=np.float32)
+        Tb = np.ascontiguousarray(T, dtype=np.int64)
+        n = Kb.shape[1]
+        _check(lib.locret_import_state(self._h, Kb.data_ptr(), Vb.data_ptr(), Sb.ctypes.data,
+                                       Tb.ctypes.data, n, int(seen)), "locret_import_state")
+
+    def sync_status(self) -> int:
+        return lib.locret_sync_status(self._h)
+
+    def reset(self):
+        _check(lib.locret_reset(self._h), "locret_reset")
+
+    # -- measurement
+    def set_timing(self, on: bool):
+        _check(lib.locret_set_timing(self._h, int(on)), "locret_set_timing")
+
+    def read_timing(self):
+        ms = np.zeros(len(K_NAMES), dtype=np.float32)
+        cnt = np.zeros(len(K_NAMES), dtype=np.int64)
+        _check(lib.locret_read_timing(self._h, ms.ctypes.data, cnt.ctypes.data), "locret_read_timing")
+        return ms, cnt
+
+    @property
+    def launch_count(self) -> int:
+        n = C.c_int64()
+        _check(lib.locret_launch_count(self._h, C.byref(n)), "locret_launch_count")
+        return n.value
+
+    def destroy(self):
+        if self._h:
+            lib.locret_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass

@@ -1,0 +1,132 @@
+// Shared device helpers and the launcher declarations of the library's kernels.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace locret {
+
+typedef __nv_bfloat16 bf16;
+
+// ---------------------------------------------------------------- small device helpers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+// 16-byte async copy global -> shared; when !pred the destination is zero-filled.
+__device__ __forceinline__ void cp_async16(void *smem, const void *gmem, bool pred) {
+  uint32_t s = smem_u32(smem);
+  int sz = pred ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(s), "l"(gmem), "r"(sz));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3,
+                                            const void *smem) {
+  uint32_t s = smem_u32(smem);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(s));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t &r0, uint32_t &r1, uint32_t &r2,
+                                                  uint32_t &r3, const void *smem) {
+  uint32_t s = smem_u32(smem);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(s));
+}
+
+// D (16x8 fp32) += A (16x16 bf16, row) * B (16x8 bf16, col)
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4],
+                                               uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};\n"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+
+__device__ __forceinline__ float apply_act(float x, int act) {
+  if (act == 0) return x / (1.0f + __expf(-x));  // SiLU
+  if (act == 1) {                                // GELU, tanh form
+    float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
+    return 0.5f * x * (1.0f + tanhf(u));
+  }
+  return fmaxf(x, 0.0f);                         // ReLU
+}
+
+// ---------------------------------------------------------------- launchers (host)
+// Every launcher enqueues on `st` and returns the cudaError_t of the launch.
+
+// C[M x N] (bf16, row-major, leading dimension ldc) = A[M x K] · Bt[N x K]^T, both K-major bf16.
+cudaError_t launch_gemm_bf16(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, int ldc,
+                             int M, int N, int K, cudaStream_t st);
+
+// Retaining head: partial[nt][M][h_kv] = sum over the N-tile nt of act(A·W1t^T)[:, n] * W2[n][:]
+// A [M x K] bf16 (K = d_in), W1t [d_R x K] bf16, W2 [d_R x h_kv] fp32.  Returns the number of
+// N-tiles through *n_tiles.
+cudaError_t launch_rh_gemm(const bf16 *A, int lda, const bf16 *W1t, const float *W2, float *partial,
+                           int M, int d_R, int K, int h_kv, int act, int *n_tiles, cudaStream_t st);
+int rh_num_tiles(int d_R);
+
+// scores[m][slot0 + t] = sum_nt partial[nt][t][m]
+cudaError_t launch_rh_reduce(const float *partial, int n_tiles, int M, int h_kv, float *scores,
+                             int score_stride, int slot0, cudaStream_t st);
+
+struct RopeAppendArgs {
+  const bf16 *staging;  // [n_tok x d_in]  pre-RoPE Q | K | V
+  bf16 *q_rot;          // [n_tok x h*d]
+  bf16 *z_post;         // [n_tok x d_in] or nullptr: post-RoPE Q | K, V (retaining-head input variant)
+  bf16 *k_pre;          // [h_kv][cap][d]
+  bf16 *k_rot;          // [h_kv][cap][d]
+  bf16 *v;              // [h_kv][cap][d]
+  int64_t *tid;         // [h_kv][cap]
+  const float2 *cs;     // [cap][d/2] (cos, sin)
+  int n_tok, h, h_kv, d, cap, len;
+  int64_t seen;
+};
+cudaError_t launch_rope_append(const RopeAppendArgs &a, cudaStream_t st);
+
+// Attention (Eq. 1): query row t of head j sees keys [0, len + t] of KV head j / g.
+cudaError_t launch_attention_mma(const bf16 *q_rot, const bf16 *k_rot, const bf16 *v, bf16 *out,
+                                 int n_tok, int h, int h_kv, int d, int cap, int len,
+                                 cudaStream_t st);
+
+// keep[m][0..budget) = ascending slots kept among n candidates (the last n_prot protected).
+cudaError_t launch_topk(const float *scores, int score_stride, int h_kv, int n, int budget,
+                        int n_prot, int32_t *keep, cudaStream_t st);
+
+struct CompactArgs {
+  const bf16 *k_src, *v_src;
+  const float *s_src;
+  const int64_t *t_src;
+  bf16 *k_dst, *v_dst, *k_rot;
+  float *s_dst;
+  int64_t *t_dst;
+  const int32_t *keep;  // [h_kv][budget]
+  const float2 *cs;
+  int h_kv, d, cap, budget;
+};
+cudaError_t launch_compact(const CompactArgs &a, cudaStream_t st);
+
+// k_rot[m][i] = RoPE(k_pre[m][i], i) for i < len (used after an import).
+cudaError_t launch_rerope(const bf16 *k_pre, bf16 *k_rot, const float2 *cs, int h_kv, int d, int cap,
+                          int len, cudaStream_t st);
+
+// dst[c][r] = src[r][c]  (weight repack at create)
+cudaError_t launch_transpose_bf16(const bf16 *src, bf16 *dst, int rows, int cols, cudaStream_t st);
+cudaError_t launch_bf16_to_f32(const bf16 *src, float *dst, int n, cudaStream_t st);
+
+}  // namespace locret

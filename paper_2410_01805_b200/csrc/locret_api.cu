@@ -1,0 +1,421 @@
+// C ABI of the library: argument checks, state, and the per-chunk launch sequence.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <map>
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "../../include/locret.h"
+#include "common.cuh"
+
+using namespace locret;
+
+namespace {
+
+// Scratch shared by every layer bound to the same stream (only one layer's step is in
+// flight on a stream at a time).
+struct ScratchPool {
+  cudaStream_t st = nullptr;
+  int refs = 0;
+  size_t staging_b = 0, qrot_b = 0, zpost_b = 0, partial_b = 0, keep_b = 0;
+  bf16 *staging = nullptr, *q_rot = nullptr, *z_post = nullptr;
+  float *partial = nullptr;
+  int32_t *keep = nullptr;
+  struct CsTable { float theta; int d, cap; float2 *ptr; };
+  std::vector<CsTable> cs;
+};
+
+std::mutex g_mu;
+std::map<cudaStream_t, ScratchPool *> g_pools;
+
+template <typename T>
+bool grow(T **p, size_t *have, size_t want, cudaStream_t st) {
+  if (want <= *have) return true;
+  T *np_ = nullptr;
+  if (cudaMalloc(&np_, want) != cudaSuccess) { cudaGetLastError(); return false; }
+  if (*p) { cudaStreamSynchronize(st); cudaFree(*p); }
+  *p = np_;
+  *have = want;
+  return true;
+}
+
+struct TimedEvent { cudaEvent_t a, b; int kind; };
+
+}  // namespace
+
+struct locret_layer {
+  locret_layer_cfg cfg;
+  int budget, chunk, n_stab, cap, d_in, h, h_kv, d, D, d_R;
+  cudaStream_t st;
+  ScratchPool *pool;
+  bf16 *wqkv_t, *w1_t;
+  float *w2f;
+  bf16 *k_pre[2], *v[2], *k_rot;
+  float *s[2];
+  int64_t *tid[2];
+  int cur;
+  const float2 *cs;
+  int *d_status;
+  int len;
+  int64_t seen;
+  int64_t launches;
+  bool timing;
+  std::vector<TimedEvent> events;
+  size_t events_used;
+};
+
+namespace {
+
+void free_layer_memory(locret_layer *L) {
+  cudaFree(L->wqkv_t); cudaFree(L->w1_t); cudaFree(L->w2f);
+  for (int i = 0; i < 2; i++) { cudaFree(L->k_pre[i]); cudaFree(L->v[i]); cudaFree(L->s[i]); cudaFree(L->tid[i]); }
+  cudaFree(L->k_rot); cudaFree(L->d_status);
+  for (auto &e : L->events) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
+  cudaGetLastError();
+}
+
+void release_pool(ScratchPool *p) {
+  std::lock_guard<std::mutex> lk(g_mu);
+  if (!p) return;
+  if (--p->refs > 0) return;
+  cudaFree(p->staging); cudaFree(p->q_rot); cudaFree(p->z_post); cudaFree(p->partial); cudaFree(p->keep);
+  for (auto &t : p->cs) cudaFree(t.ptr);
+  g_pools.erase(p->st);
+  delete p;
+  cudaGetLastError();
+}
+
+const float2 *get_cs_table(ScratchPool *p, float theta, int d, int cap, cudaStream_t st) {
+  for (auto &t : p->cs)
+    if (t.theta == theta && t.d == d && t.cap >= cap) return t.ptr;
+  const int half = d / 2;
+  std::vector<float2> host((size_t)cap * half);
+  std::vector<double> inv(half);
+  for (int i = 0; i < half; i++) inv[i] = pow((double)theta, -2.0 * i / d);
+  for (int pos = 0; pos < cap; pos++)
+    for (int i = 0; i < half; i++) {
+      double ang = (double)pos * inv[i];
+      host[(size_t)pos * half + i] = make_float2((float)cos(ang), (float)sin(ang));
+    }
+  float2 *dev = nullptr;
+  if (cudaMalloc(&dev, host.size() * sizeof(float2)) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+  if (cudaMemcpyAsync(dev, host.data(), host.size() * sizeof(float2), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) {
+    cudaFree(dev); cudaGetLastError(); return nullptr;
+  }
+  p->cs.push_back({theta, d, cap, dev});
+  return dev;
+}
+
+// Bracket one launch with events when timing is on; count it.
+struct Timed {
+  locret_layer *L; int kind; TimedEvent *ev = nullptr;
+  Timed(locret_layer *l, int k) : L(l), kind(k) {
+    L->launches++;
+    if (!L->timing) return;
+    if (L->events_used == L->events.size()) {
+      TimedEvent e; e.kind = k;
+      if (cudaEventCreate(&e.a) != cudaSuccess || cudaEventCreate(&e.b) != cudaSuccess) { cudaGetLastError(); return; }
+      L->events.push_back(e);
+    }
+    ev = &L->events[L->events_used++];
+    ev->kind = k;
+    cudaEventRecord(ev->a, L->st);
+  }
+  ~Timed() { if (ev) cudaEventRecord(ev->b, L->st); }
+};
+
+#define CK(call)                                         \
+  do {                                                   \
+    cudaError_t e__ = (call);                            \
+    if (e__ != cudaSuccess) { cudaGetLastError(); return LOCRET_ERR_CUDA; } \
+  } while (0)
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+const char *locret_strerror(int code) {
+  switch (code) {
+    case LOCRET_OK: return "ok";
+    case LOCRET_ERR_INVALID: return "invalid argument or configuration";
+    case LOCRET_ERR_ALLOC: return "allocation failed";
+    case LOCRET_ERR_CAPACITY: return "cache capacity exceeded";
+    case LOCRET_ERR_CUDA: return "CUDA call failed";
+    case LOCRET_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown error";
+}
+
+int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, int32_t n_stab,
+                  locret_layer **out) {
+  if (!out) return LOCRET_ERR_INVALID;
+  *out = nullptr;
+  if (!cfg) return LOCRET_ERR_INVALID;
+  const int h = cfg->n_q_heads, hk = cfg->n_kv_heads, d = cfg->head_dim, D = cfg->d_model,
+            dR = cfg->d_retain;
+  if (h < 1 || hk < 1 || hk > 32 || h % hk != 0) return LOCRET_ERR_INVALID;
+  if (d != 64 && d != 96 && d != 128) return LOCRET_ERR_INVALID;
+  if (D < 32 || D % 32 != 0 || dR < 8 || dR % 8 != 0) return LOCRET_ERR_INVALID;
+  if (cfg->act < 0 || cfg->act > 2 || cfg->rh_input < 0 || cfg->rh_input > 1) return LOCRET_ERR_INVALID;
+  if (cfg->kv_dtype != 0) return LOCRET_ERR_INVALID;
+  if (!(cfg->rope_theta > 1.0f) || cfg->reserve < 0) return LOCRET_ERR_INVALID;
+  if (budget < 1 || chunk < 1 || n_stab < 0 || n_stab > budget) return LOCRET_ERR_INVALID;
+  if (!cfg->w_qkv || !cfg->w1 || !cfg->w2) return LOCRET_ERR_INVALID;
+  if (!aligned16(cfg->w_qkv) || !aligned16(cfg->w1)) return LOCRET_ERR_INVALID;
+  const long long cap_ll = (long long)budget + chunk + cfg->reserve;
+  if (cap_ll > (1ll << 24)) return LOCRET_ERR_INVALID;
+
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) { cudaGetLastError(); return LOCRET_ERR_CUDA; }
+
+  locret_layer *L = new (std::nothrow) locret_layer();
+  if (!L) return LOCRET_ERR_ALLOC;
+  L->cfg = *cfg;
+  L->budget = budget; L->chunk = chunk; L->n_stab = n_stab; L->cap = (int)cap_ll;
+  L->h = h; L->h_kv = hk; L->d = d; L->D = D; L->d_R = dR;
+  L->d_in = (h + 2 * hk) * d;
+  L->st = (cudaStream_t)cfg->stream;
+  L->cur = 0; L->len = 0; L->seen = 0; L->launches = 0; L->timing = false; L->events_used = 0;
+  L->pool = nullptr;
+
+  const size_t kv_b = (size_t)hk * L->cap * d * sizeof(bf16);
+  const size_t sc_b = (size_t)hk * L->cap * sizeof(float);
+  const size_t td_b = (size_t)hk * L->cap * sizeof(int64_t);
+  bool ok = true;
+  ok = ok && cudaMalloc(&L->wqkv_t, (size_t)L->d_in * D * sizeof(bf16)) == cudaSuccess;
+  ok = ok && cudaMalloc(&L->w1_t, (size_t)dR * L->d_in * sizeof(bf16)) == cudaSuccess;
+  ok = ok && cudaMalloc(&L->w2f, (size_t)dR * hk * sizeof(float)) == cudaSuccess;
+  for (int i = 0; i < 2 && ok; i++) {
+    ok = ok && cudaMalloc(&L->k_pre[i], kv_b) == cudaSuccess;
+    ok = ok && cudaMalloc(&L->v[i], kv_b) == cudaSuccess;
+    ok = ok && cudaMalloc(&L->s[i], sc_b) == cudaSuccess;
+    ok = ok && cudaMalloc(&L->tid[i], td_b) == cudaSuccess;
+  }
+  ok = ok && cudaMalloc(&L->k_rot, kv_b) == cudaSuccess;
+  ok = ok && cudaMalloc(&L->d_status, sizeof(int)) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); free_layer_memory(L); delete L; return LOCRET_ERR_ALLOC; }
+
+  // shared scratch
+  {
+    std::lock_guard<std::mutex> lk(g_mu);
+    ScratchPool *&p = g_pools[L->st];
+    if (!p) { p = new (std::nothrow) ScratchPool(); if (p) p->st = L->st; }
+    if (p) {
+      p->refs++;
+      L->pool = p;
+      bool g = true;
+      g = g && grow(&p->staging, &p->staging_b, (size_t)chunk * L->d_in * sizeof(bf16), L->st);
+      g = g && grow(&p->q_rot, &p->qrot_b, (size_t)chunk * h * d * sizeof(bf16), L->st);
+      if (cfg->rh_input == 1)
+        g = g && grow(&p->z_post, &p->zpost_b, (size_t)chunk * L->d_in * sizeof(bf16), L->st);
+      g = g && grow(&p->partial, &p->partial_b, (size_t)rh_num_tiles(dR) * chunk * hk * sizeof(float), L->st);
+      g = g && grow(&p->keep, &p->keep_b, (size_t)hk * budget * sizeof(int32_t), L->st);
+      if (g) L->cs = get_cs_table(p, cfg->rope_theta, d, L->cap, L->st);
+      ok = g && L->cs;
+    } else {
+      ok = false;
+    }
+  }
+  if (!ok) { ScratchPool *p = L->pool; free_layer_memory(L); delete L; release_pool(p); return LOCRET_ERR_ALLOC; }
+
+  // repack the weights: K-major copies for both GEMMs, W2 in fp32
+  cudaError_t e = cudaSuccess;
+  if (e == cudaSuccess) e = launch_transpose_bf16((const bf16 *)cfg->w_qkv, L->wqkv_t, D, L->d_in, L->st);
+  if (e == cudaSuccess) e = launch_transpose_bf16((const bf16 *)cfg->w1, L->w1_t, L->d_in, dR, L->st);
+  if (e == cudaSuccess) e = launch_bf16_to_f32((const bf16 *)cfg->w2, L->w2f, dR * hk, L->st);
+  for (int i = 0; i < 2 && e == cudaSuccess; i++) {
+    e = cudaMemsetAsync(L->k_pre[i], 0, kv_b, L->st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(L->v[i], 0, kv_b, L->st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(L->s[i], 0, sc_b, L->st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(L->tid[i], 0, td_b, L->st);
+  }
+  if (e == cudaSuccess) e = cudaMemsetAsync(L->k_rot, 0, kv_b, L->st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(L->d_status, 0, sizeof(int), L->st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(L->st);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    ScratchPool *p = L->pool; free_layer_memory(L); delete L; release_pool(p);
+    return LOCRET_ERR_CUDA;
+  }
+  *out = L;
+  return LOCRET_OK;
+}
+
+int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t flags,
+                         void *attn_out) {
+  if (!L || !hidden_in || !attn_out) return LOCRET_ERR_INVALID;
+  if (n_tok < 1 || n_tok > L->chunk) return LOCRET_ERR_INVALID;
+  if (flags & ~(LOCRET_NO_EVICT | LOCRET_LAST_CHUNK)) return LOCRET_ERR_INVALID;
+  if (!aligned16(hidden_in) || !aligned16(attn_out)) return LOCRET_ERR_INVALID;
+  const int n = L->len + n_tok;
+  if (n > L->cap) return LOCRET_ERR_CAPACITY;
+  ScratchPool *P = L->pool;
+  const int c = L->cur;
+
+  {  // (a) projections
+    Timed t(L, LOCRET_K_QKV);
+    CK(launch_gemm_bf16((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, P->staging, L->d_in, n_tok,
+                        L->d_in, L->D, L->st));
+  }
+  {  // positions, RoPE, append of the chunk's units at slots [len, len + n_tok)
+    Timed t(L, LOCRET_K_ROPE);
+    RopeAppendArgs a;
+    a.staging = P->staging; a.q_rot = P->q_rot;
+    a.z_post = L->cfg.rh_input == 1 ? P->z_post : nullptr;
+    a.k_pre = L->k_pre[c]; a.k_rot = L->k_rot; a.v = L->v[c]; a.tid = L->tid[c]; a.cs = L->cs;
+    a.n_tok = n_tok; a.h = L->h; a.h_kv = L->h_kv; a.d = L->d; a.cap = L->cap; a.len = L->len;
+    a.seen = L->seen;
+    CK(launch_rope_append(a, L->st));
+  }
+  {  // (b) Eq. 1
+    Timed t(L, LOCRET_K_ATTN);
+    CK(launch_attention_mma(P->q_rot, L->k_rot, L->v[c], (bf16 *)attn_out, n_tok, L->h, L->h_kv,
+                            L->d, L->cap, L->len, L->st));
+  }
+  int n_tiles = 0;
+  {  // (c) retaining head
+    Timed t(L, LOCRET_K_RH);
+    const bf16 *z = L->cfg.rh_input == 1 ? P->z_post : P->staging;
+    CK(launch_rh_gemm(z, L->d_in, L->w1_t, L->w2f, P->partial, n_tok, L->d_R, L->d_in, L->h_kv,
+                      L->cfg.act, &n_tiles, L->st));
+  }
+  {
+    Timed t(L, LOCRET_K_RH_REDUCE);
+    CK(launch_rh_reduce(P->partial, n_tiles, n_tok, L->h_kv, L->s[c], L->cap, L->len, L->st));
+  }
+  // (d) protect, top-b, gather
+  if (!(flags & LOCRET_NO_EVICT) && n > L->budget) {
+    const int n_prot = (flags & LOCRET_LAST_CHUNK) ? 0 : (L->n_stab < n ? L->n_stab : n);
+    {
+      Timed t(L, LOCRET_K_TOPK);
+      CK(launch_topk(L->s[c], L->cap, L->h_kv, n, L->budget, n_prot, P->keep, L->st));
+    }
+    {
+      Timed t(L, LOCRET_K_COMPACT);
+      CompactArgs a;
+      a.k_src = L->k_pre[c]; a.v_src = L->v[c]; a.s_src = L->s[c]; a.t_src = L->tid[c];
+      a.k_dst = L->k_pre[c ^ 1]; a.v_dst = L->v[c ^ 1]; a.s_dst = L->s[c ^ 1]; a.t_dst = L->tid[c ^ 1];
+      a.k_rot = L->k_rot; a.keep = P->keep; a.cs = L->cs;
+      a.h_kv = L->h_kv; a.d = L->d; a.cap = L->cap; a.budget = L->budget;
+      CK(launch_compact(a, L->st));
+    }
+    L->cur = c ^ 1;
+    L->len = L->budget;
+  } else {
+    L->len = n;
+  }
+  L->seen += n_tok;
+  return LOCRET_OK;
+}
+
+int locret_decode_step(locret_layer *L, const void *hidden_in, void *attn_out) {
+  return locret_prefill_chunk(L, hidden_in, 1, LOCRET_NO_EVICT, attn_out);
+}
+
+int locret_cache_len(const locret_layer *L, int32_t *len) {
+  if (!L || !len) return LOCRET_ERR_INVALID;
+  *len = L->len;
+  return LOCRET_OK;
+}
+
+int locret_export_state(locret_layer *L, void *K, void *V, float *scores, int64_t *token_ids,
+                        int32_t *len, int64_t *tokens_seen) {
+  if (!L) return LOCRET_ERR_INVALID;
+  const int c = L->cur, n = L->len;
+  if (len) *len = n;
+  if (tokens_seen) *tokens_seen = L->seen;
+  if (n > 0) {
+    const size_t row = (size_t)n * L->d * sizeof(bf16), pitch = (size_t)L->cap * L->d * sizeof(bf16);
+    if (K) CK(cudaMemcpy2DAsync(K, row, L->k_pre[c], pitch, row, L->h_kv, cudaMemcpyDeviceToHost, L->st));
+    if (V) CK(cudaMemcpy2DAsync(V, row, L->v[c], pitch, row, L->h_kv, cudaMemcpyDeviceToHost, L->st));
+    if (scores)
+      CK(cudaMemcpy2DAsync(scores, (size_t)n * 4, L->s[c], (size_t)L->cap * 4, (size_t)n * 4, L->h_kv,
+                           cudaMemcpyDeviceToHost, L->st));
+    if (token_ids)
+      CK(cudaMemcpy2DAsync(token_ids, (size_t)n * 8, L->tid[c], (size_t)L->cap * 8, (size_t)n * 8,
+                           L->h_kv, cudaMemcpyDeviceToHost, L->st));
+  }
+  CK(cudaStreamSynchronize(L->st));
+  return LOCRET_OK;
+}
+
+int locret_import_state(locret_layer *L, const void *K, const void *V, const float *scores,
+                        const int64_t *token_ids, int32_t len, int64_t tokens_seen) {
+  if (!L || len < 0 || len > L->cap || tokens_seen < 0) return LOCRET_ERR_INVALID;
+  if (len > 0 && (!K || !V || !scores || !token_ids)) return LOCRET_ERR_INVALID;
+  const int c = L->cur;
+  if (len > 0) {
+    const size_t row = (size_t)len * L->d * sizeof(bf16), pitch = (size_t)L->cap * L->d * sizeof(bf16);
+    CK(cudaMemcpy2DAsync(L->k_pre[c], pitch, K, row, row, L->h_kv, cudaMemcpyHostToDevice, L->st));
+    CK(cudaMemcpy2DAsync(L->v[c], pitch, V, row, row, L->h_kv, cudaMemcpyHostToDevice, L->st));
+    CK(cudaMemcpy2DAsync(L->s[c], (size_t)L->cap * 4, scores, (size_t)len * 4, (size_t)len * 4, L->h_kv,
+                         cudaMemcpyHostToDevice, L->st));
+    CK(cudaMemcpy2DAsync(L->tid[c], (size_t)L->cap * 8, token_ids, (size_t)len * 8, (size_t)len * 8,
+                         L->h_kv, cudaMemcpyHostToDevice, L->st));
+    L->launches++;
+    CK(launch_rerope(L->k_pre[c], L->k_rot, L->cs, L->h_kv, L->d, L->cap, len, L->st));
+  }
+  CK(cudaStreamSynchronize(L->st));
+  L->len = len;
+  L->seen = tokens_seen;
+  return LOCRET_OK;
+}
+
+int locret_sync_status(locret_layer *L) {
+  if (!L) return LOCRET_ERR_INVALID;
+  int host = 0;
+  CK(cudaMemcpyAsync(&host, L->d_status, sizeof(int), cudaMemcpyDeviceToHost, L->st));
+  CK(cudaStreamSynchronize(L->st));
+  CK(cudaGetLastError());
+  return host;
+}
+
+int locret_reset(locret_layer *L) {
+  if (!L) return LOCRET_ERR_INVALID;
+  L->len = 0;
+  L->seen = 0;
+  return LOCRET_OK;
+}
+
+int locret_set_timing(locret_layer *L, int32_t enable) {
+  if (!L) return LOCRET_ERR_INVALID;
+  L->timing = enable != 0;
+  return LOCRET_OK;
+}
+
+int locret_read_timing(locret_layer *L, float *ms, int64_t *launches) {
+  if (!L || !ms || !launches) return LOCRET_ERR_INVALID;
+  for (int i = 0; i < LOCRET_K_COUNT; i++) { ms[i] = 0.f; launches[i] = 0; }
+  CK(cudaStreamSynchronize(L->st));
+  for (size_t i = 0; i < L->events_used; i++) {
+    float t = 0.f;
+    CK(cudaEventElapsedTime(&t, L->events[i].a, L->events[i].b));
+    ms[L->events[i].kind] += t;
+    launches[L->events[i].kind]++;
+  }
+  L->events_used = 0;
+  return LOCRET_OK;
+}
+
+int locret_launch_count(const locret_layer *L, int64_t *count) {
+  if (!L || !count) return LOCRET_ERR_INVALID;
+  *count = L->launches;
+  return LOCRET_OK;
+}
+
+void locret_destroy(locret_layer *L) {
+  if (!L) return;
+  cudaStreamSynchronize(L->st);
+  ScratchPool *p = L->pool;
+  free_layer_memory(L);
+  delete L;
+  release_pool(p);
+}
+
+}  // extern "C"

@@ -1,0 +1,137 @@
+"""Lock-step comparison of the CUDA library with the CPU oracle.
+
+Direction of data: the oracle's state is imported INTO the CUDA layer before each
+compared chunk; nothing computed by the CUDA path is ever fed to the oracle.
+"""
+
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import locret_oracle as O
+
+ATTN_TOL = 2e-2       # |delta| <= ATTN_TOL * max(1, |ref|)
+SCORE_TOL = 1e-2      # |delta| <= SCORE_TOL * max(|ref|, rms(ref over the chunk))
+BAND = 1e-2           # index sets must agree outside this band around the cut
+
+
+def bf16_dev(x: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(torch.bfloat16).cuda()
+
+
+def make_pair(shape, weights, budget, chunk, n_stab, reserve=0):
+    from paper_2410_01805_b200 import LocretLayer
+    wqkv, w1, w2 = weights
+    ora = O.OracleLayer(shape, wqkv, w1, w2, budget, chunk, n_stab, reserve=reserve, mirror=True)
+    gpu = LocretLayer(shape, bf16_dev(wqkv), bf16_dev(w1), bf16_dev(w2), budget, chunk, n_stab,
+                      reserve=reserve)
+    return ora, gpu
+
+
+def check_attention(got: np.ndarray, ref: np.ndarray, what=""):
+    ok = ~np.isnan(ref)
+    err = np.abs(got[ok] - ref[ok])
+    bound = ATTN_TOL * np.maximum(1.0, np.abs(ref[ok]))
+    worst = float(np.max(err / bound)) if err.size else 0.0
+    assert worst <= 1.0, f"{what} attention: worst err/bound {worst:.3f}, max abs {err.max():.4g}"
+    return float(err.max()) if err.size else 0.0
+
+
+def check_scores(got: np.ndarray, ref: np.ndarray, what=""):
+    rms = np.sqrt(np.mean(ref ** 2, axis=0, keepdims=True))
+    bound = SCORE_TOL * np.maximum(np.abs(ref), rms) + 1e-30
+    worst = float(np.max(np.abs(got - ref) / bound))
+    assert worst <= 1.0, f"{what} scores: worst err/bound {worst:.3f}"
+    return worst
+
+
+def check_keep_band(kept_slots, s_ref, budget, n_prot, oracle_keep, what=""):
+    """kept_slots: ascending slot indices (into cache ‖ chunk) kept by the CUDA path for one head."""
+    n = len(s_ref)
+    kept = np.zeros(n, dtype=bool)
+    kept[kept_slots] = True
+    assert kept.sum() == min(budget, n), f"{what}: kept {kept.sum()} units"
+    assert kept[n - n_prot:].all(), f"{what}: a protected unit was evicted"
+    rest = n - n_prot
+    k = budget - n_prot
+    if k == 0:
+        assert not kept[:rest].any()
+        return True
+    if k >= rest:
+        return True
+    sr = np.where(np.isnan(s_ref[:rest]), -np.inf, s_ref[:rest])
+    srt = np.sort(sr)[::-1]
+    tau_hi, tau_lo = srt[k - 1], srt[k]
+    must = sr >= tau_hi + BAND
+    never = sr <= tau_lo - BAND
+    assert kept[:rest][must].all(), f"{what}: a unit above the band was evicted"
+    assert not kept[:rest][never].any(), f"{what}: a unit below the band was kept"
+    exact = np.array_equal(np.flatnonzero(kept), np.asarray(oracle_keep))
+    if tau_hi - tau_lo > BAND:
+        assert exact, f"{what}: index set differs although the gap is {tau_hi - tau_lo:.3g}"
+    return exact
+
+
+def lockstep_chunk(ora, gpu, x: np.ndarray, flags: int = 0, rows=None, what=""):
+    """Import the oracle's state, run one chunk on both, compare everything.  Advances the oracle."""
+    shape = ora.s
+    h, hk, d = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+    n_tok = x.shape[0]
+    st = ora.export_state()
+    ln = ora.len
+    xd = bf16_dev(x)
+    out_a = torch.zeros((n_tok, h * d), dtype=torch.bfloat16, device="cuda")
+    out_b = torch.zeros_like(out_a)
+
+    # pass 1: append only, to read the chunk's K, V and scores before compaction
+    gpu.import_state(st["K"], st["V"], st["S"], st["T"], st["seen"])
+    gpu.prefill_chunk(xd, out_a, O.NO_EVICT)
+    pre = gpu.export_state()
+    assert gpu.sync_status() == 0
+    # pass 2: the step as asked
+    gpu.import_state(st["K"], st["V"], st["S"], st["T"], st["seen"])
+    gpu.prefill_chunk(xd, out_b, flags)
+    post = gpu.export_state()
+    assert gpu.sync_status() == 0
+    assert torch.equal(out_a, out_b), f"{what}: attention output not reproducible"
+
+    ref_out = ora.prefill_chunk(x, flags, rows=rows)
+    stats = {}
+    stats["attn_max_abs"] = check_attention(out_b.float().cpu().numpy().astype(np.float64), ref_out, what)
+
+    n = ln + n_tok
+    assert pre["K"].shape[1] == n and pre["seen"] == st["seen"] + n_tok
+    # imported part untouched, token ids appended
+    assert np.array_equal(pre["K"][:, :ln], st["K"].astype(np.float32))
+    assert np.array_equal(pre["T"][:, ln:], np.broadcast_to(st["seen"] + np.arange(n_tok), (hk, n_tok)))
+    # chunk K, V as stored (bf16 of fp32 accumulation vs bf16 of fp64: rare one-ulp flips allowed)
+    qkv = O.round_bf16(O.project_qkv(x, ora.w_qkv, h, hk, d))
+    _, Kc, Vc = O.split_qkv(qkv, h, hk, d)
+    for name, got, ref in (("K", pre["K"][:, ln:], np.transpose(Kc, (1, 0, 2))),
+                           ("V", pre["V"][:, ln:], np.transpose(Vc, (1, 0, 2)))):
+        diff = np.abs(got - ref)
+        assert np.all(diff <= np.abs(ref) * 2.0 ** -7 + 1e-30), f"{what}: chunk {name} off by more than one bf16 ulp"
+        assert np.mean(diff != 0) < 2e-3, f"{what}: too many rounding flips in chunk {name}"
+    stats["score_worst"] = check_scores(pre["S"][:, ln:].T.astype(np.float64), ora.last_scores, what)
+
+    evict = not (flags & O.NO_EVICT) and n > ora.budget
+    if evict:
+        n_prot = 0 if (flags & O.LAST_CHUNK) else min(ora.n_stab, n)
+        s_ref = np.concatenate([st["S"], ora.last_scores.T], axis=1)
+        exact = True
+        for m in range(hk):
+            pos = np.searchsorted(pre["T"][m], post["T"][m])
+            assert np.array_equal(pre["T"][m][pos], post["T"][m]), f"{what}: unknown token id after compaction"
+            assert np.all(np.diff(pos) > 0), f"{what}: temporal order lost"
+            exact &= check_keep_band(pos, s_ref[m], ora.budget, n_prot, ora.last_keep[m], f"{what} head {m}")
+            # compaction is a bit-exact gather of the pre-compaction arrays
+            assert np.array_equal(post["K"][m], pre["K"][m][pos])
+            assert np.array_equal(post["V"][m], pre["V"][m][pos])
+            assert np.array_equal(post["S"][m].view(np.uint32), pre["S"][m][pos].view(np.uint32))
+        stats["sets_identical"] = exact
+    else:
+        for key in ("K", "V", "T"):
+            assert np.array_equal(post[key], pre[key])
+    assert gpu.cache_len == ora.len
+    return stats
