@@ -1,0 +1,345 @@
+#!/usr/bin/env python
+"""Chunked-prefill throughput of the Locret hot path on B200.
+
+One "step" = one whole prefill of the workload's context through the whole layer stack:
+every chunk, every layer, all kernels of the per-layer step (projection, position
+assignment + RoPE + append, attention, retaining head, top-b selection, compaction).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs the same workload
+on an independent request (the path is a sequential recurrence over chunks and shards
+only by request: "replicas only", weak scaling, no data-path collective).
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads as W  # noqa: E402
+
+METRIC = "chunked-prefill tokens/sec at 128K ctx (1 B200); % tensor/HBM roofline per kernel"
+UNIT = "tokens/s"
+DEFAULT_WORKLOAD = "c3_llama_128k"
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], tf=d["bf16_tflops"], tf_sustained=d["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, tf=1590.0, tf_sustained=1400.0, source="fallback")
+
+
+# ----------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self.index = index
+        self.t = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True,
+                                     timeout=5).stdout.strip().splitlines()[0]
+                f = [x.strip() for x in out.split(",")]
+                self.samples.append(float(f[0])); self.max_mhz = float(f[1])
+                for n, v in zip(names, f[2:]):
+                    if v.lower().startswith("active"):
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            self._stop.wait(0.2)
+
+    def __enter__(self):
+        self.t.start(); return self
+
+    def __exit__(self, *a):
+        self._stop.set(); self.t.join(timeout=6)
+
+    def summary(self):
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ----------------------------------------------------------------------------- work counts
+
+def chunk_layer_flops(w: W.Workload, ln: int, n_tok: int):
+    s = w.shape
+    qkv = 2.0 * n_tok * s.d_model * s.d_in
+    attn = 4.0 * s.n_q_heads * s.head_dim * (n_tok * ln + n_tok * (n_tok + 1) / 2)
+    rh = 2.0 * n_tok * s.d_in * s.d_retain + 2.0 * n_tok * s.d_retain * s.n_kv_heads
+    return qkv, attn, rh
+
+
+def step_flops(w: W.Workload):
+    ln, tot = 0, np.zeros(3)
+    for n_tok in w.chunk_sizes():
+        tot += np.array(chunk_layer_flops(w, ln, n_tok))
+        ln = min(w.budget, ln + n_tok)
+    return tot * w.n_layers
+
+
+# ----------------------------------------------------------------------------- reference arm (oracle on CPU)
+
+def oracle_sample(w: W.Workload, n_chunks: int):
+    """Time the oracle, as it stands, on `n_chunks` steady-state chunk-layers of layer 0."""
+    from threadpoolctl import threadpool_info
+    from oracle import locret_oracle as O
+    wts = W.layer_weights(w.shape, 0)
+    ora = O.OracleLayer(w.shape, *wts, w.budget, w.chunk, w.n_stab, mirror=True)
+    # bring the cache to its steady size without paying for attention: NO-rows calls
+    start, sizes = 0, w.chunk_sizes()
+    fill = 0
+    while ora.len < min(w.budget, w.context - w.chunk) and fill < len(sizes) - 1:
+        ora.prefill_chunk(W.hidden_states(w, start, sizes[fill]), 0, rows=[0])
+        start += sizes[fill]; fill += 1
+    times, toks = [], 0
+    for i in range(n_chunks):
+        idx = min(fill + i, len(sizes) - 1)
+        x = W.hidden_states(w, start, sizes[idx])
+        t0 = time.perf_counter()
+        ora.prefill_chunk(x, 0)
+        times.append(time.perf_counter() - t0)
+        toks += sizes[idx]; start += sizes[idx]
+    cores = max([p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"] + [1])
+    sec = float(np.sum(times))
+    # one chunk-layer handles n_tok tokens of ONE layer; the whole job does n_layers of them per chunk
+    tok_s = toks / sec / w.n_layers
+    sample = (f"{n_chunks} steady-state chunk-layer(s) of layer 0 ({toks} tokens, cache {ora.len} units/head), "
+              f"{sec:.1f} s; tokens/s = tokens / time / {w.n_layers} layers")
+    return tok_s, cores, sample, sec
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    t_all = time.perf_counter()
+    vals = []
+    total = args.steps + args.warmup
+    n_per = 1
+    sample = ""
+    cores = 1
+    for i in range(total):
+        v, cores, sample, _ = oracle_sample(w, n_per)
+        if i >= args.warmup:
+            vals.append(v)
+    value = float(np.mean(vals))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": w.context / value * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "note": "CPU oracle (numpy fp64), bounded sample extrapolated linearly"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0, "wall_s": time.perf_counter() - t_all,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- our arm
+
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_2410_01805_b200 import K_NAMES, LocretLayer
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    s = w.shape
+    peaks = measured_peaks()
+
+    # ---- inputs: seeded host arrays -> pinned host memory -> HBM
+    sizes = w.chunk_sizes()
+    t0 = time.perf_counter()
+    x_host = torch.empty((w.context, s.d_model), dtype=torch.bfloat16).pin_memory()
+    pos = 0
+    for n_tok in sizes:
+        x_host[pos:pos + n_tok] = torch.from_numpy(W.hidden_states(w, pos, n_tok)).to(torch.bfloat16)
+        pos += n_tok
+    x_dev = x_host.to(dev, non_blocking=True)
+    stream = torch.cuda.current_stream()
+    layers = []
+    for l in range(w.n_layers):
+        wq, w1, w2 = (torch.from_numpy(a).to(torch.bfloat16).to(dev) for a in W.layer_weights(s, l))
+        layers.append(LocretLayer(s, wq, w1, w2, w.budget, w.chunk, w.n_stab, stream=stream))
+        del wq, w1, w2
+    gen_s = time.perf_counter() - t0
+
+    hd = s.n_q_heads * s.head_dim
+    out = torch.empty((w.chunk, hd), dtype=torch.bfloat16, device=dev)
+    out_host = torch.empty((w.chunk, hd), dtype=torch.bfloat16).pin_memory()
+    x_stage = torch.empty((w.chunk, s.d_model), dtype=torch.bfloat16, device=dev)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)  # > 126 MB L2
+
+    def prefill_resident():
+        for L in layers:
+            L.reset()
+        p = 0
+        for n_tok in sizes:
+            xc = x_dev[p:p + n_tok]
+            for L in layers:
+                L.prefill_chunk(xc, out, 0, n_tok)
+            p += n_tok
+
+    def prefill_e2e():
+        # inputs start in pinned host memory; every chunk is copied in, the last layer's
+        # attention output of every chunk is copied back
+        for L in layers:
+            L.reset()
+        p = 0
+        for n_tok in sizes:
+            x_stage[:n_tok].copy_(x_host[p:p + n_tok], non_blocking=True)
+            for L in layers:
+                L.prefill_chunk(x_stage, out, 0, n_tok)
+            out_host[:n_tok].copy_(out[:n_tok], non_blocking=True)
+            p += n_tok
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps, timing=False):
+        evs = []
+        for L in layers:
+            L.set_timing(timing)
+        for _ in range(steps):
+            flush.zero_()                       # flush L2 between timed iterations
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); fn(); b.record(stream)
+            evs.append((a, b))
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b) for a, b in evs]
+
+    for _ in range(args.warmup):
+        prefill_resident()
+    barrier()
+    launches0 = sum(L.launch_count for L in layers)
+    with ClockSampler(local) as clk:
+        ms = timed(prefill_resident, args.steps, timing=True)
+    barrier()
+    launches = sum(L.launch_count for L in layers) - launches0
+    k_ms = np.zeros(len(K_NAMES)); k_cnt = np.zeros(len(K_NAMES), dtype=np.int64)
+    for L in layers:
+        a, c = L.read_timing(); k_ms += a; k_cnt += c
+        L.set_timing(False)
+    status = max(abs(L.sync_status()) for L in layers)
+    assert status == 0, "device status word set"
+
+    prefill_e2e(); torch.cuda.synchronize()
+    ms_e2e = timed(prefill_e2e, max(1, min(args.steps, 3)))
+    barrier()
+
+    t_ms = float(np.mean(ms)); t_e2e = float(np.mean(ms_e2e))
+    if world > 1:
+        tt = torch.tensor([t_ms, t_e2e], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        t_ms, t_e2e = tt.tolist()
+    value = world * w.context / (t_ms * 1e-3)
+    e2e = world * w.context / (t_e2e * 1e-3)
+
+    # ---- roofline of the dominant kernel (attention: a dense contraction -> tensor peak)
+    fl = step_flops(w) * args.steps                       # [qkv, attn, rh] flops over the timed region
+    ia = K_NAMES.index("attn")
+    dom = int(np.argmax(k_ms))
+    attn_tf = fl[1] / (k_ms[ia] * 1e-3) / 1e12 if k_ms[ia] > 0 else 0.0
+    per_kernel = {}
+    for i, name in enumerate(K_NAMES):
+        if k_cnt[i]:
+            per_kernel[name] = {"launches": int(k_cnt[i]), "ms_total": float(k_ms[i]),
+                                "share": float(k_ms[i] / k_ms.sum())}
+    per_kernel["qkv"]["tflops"] = float(fl[0] / (k_ms[0] * 1e-3) / 1e12)
+    per_kernel["attn"]["tflops"] = float(attn_tf)
+    per_kernel["rh"]["tflops"] = float(fl[2] / (k_ms[K_NAMES.index("rh")] * 1e-3) / 1e12)
+    ic = K_NAMES.index("compact")
+    if k_cnt[ic]:
+        unit_b = 2 * s.head_dim * 2 * 2 + 2 * (4 + 8)        # K, V read + write; score, token id
+        rope_b = s.head_dim * 2                               # rotated key written for the next step
+        bytes_c = k_cnt[ic] * s.n_kv_heads * w.budget * (unit_b + rope_b)
+        per_kernel["compact"]["gbs"] = float(bytes_c / (k_ms[ic] * 1e-3) / 1e9)
+    roofline = {"kernel": "attn", "bound": "tensor", "achieved": float(attn_tf), "peak": peaks["tf_sustained"],
+                "unit": "TFLOP/s", "frac": float(attn_tf / peaks["tf_sustained"]), "traffic": None,
+                "peak_source": f"bf16 sustained, {peaks['source']}", "dominant_by_time": K_NAMES[dom]}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": t_ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "layers": w.n_layers, "context": w.context, "chunk": w.chunk,
+                   "budget": w.budget, "n_stab": w.n_stab, "heads": f"{s.n_q_heads}q/{s.n_kv_heads}kv x {s.head_dim}",
+                   "d_model": s.d_model, "d_retain": s.d_retain, "l2": "flushed between timed iterations (256 MB write)",
+                   "parallelism": "replicas only" if world > 1 else "1 GPU"},
+        "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": int(w.context * s.d_model * 2),
+                "d2h_bytes_per_step": int(w.context * hd * 2), "ms_per_step": t_e2e},
+        "gpu_launches": int(launches),
+        "clocks": clk.summary(),
+        "roofline": roofline,
+        "kernels": per_kernel,
+        "tflops_step": float(fl.sum() / args.steps / (t_ms * 1e-3) / 1e12),
+        "setup_s": gen_s,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, cores, sample, _ = oracle_sample(w, 1)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    for L in layers:
+        L.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling only)")
+    ap.add_argument("--context", type=int, default=0, help="override the context length (profiling only)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = W.get_workload(args.workload)
+    if args.layers:
+        w = w.with_(n_layers=args.layers)
+    if args.context:
+        w = w.with_(context=args.context)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        import __graft_entry__ as G
+        G.build()
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -101,12 +101,14 @@ def rope(x, pos, theta: float):
     return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
 
 
-def attention_rows(Qr, Kr_cache, V_cache, Kr_chunk, V_chunk, group: int, rows=None):
+def attention_rows(Qr, Kr_cache, V_cache, Kr_chunk, V_chunk, group: int, rows=None, abs_out=None):
     """Eq. 1 for the chunk's query rows.
 
     Qr [n, h, d] (roped); Kr_cache/V_cache [h_kv, len, d]; Kr_chunk/V_chunk [n, h_kv, d].
     Query t attends to every cache unit and to chunk units u <= t.
     Returns out [n, h*d]; rows not listed in `rows` are NaN.
+    If `abs_out` (same shape) is given it receives sum_i p_i |V_i|, the magnitude of the
+    terms the output sums, which error bounds of reduced-precision kernels scale with.
     """
     n, h, d = Qr.shape
     ln = Kr_cache.shape[1]
@@ -125,6 +127,8 @@ def attention_rows(Qr, Kr_cache, V_cache, Kr_chunk, V_chunk, group: int, rows=No
         p = np.exp(logits)
         p /= p.sum(axis=1, keepdims=True)
         out[rows, j * d:(j + 1) * d] = p @ Vall
+        if abs_out is not None:
+            abs_out[rows, j * d:(j + 1) * d] = p @ np.abs(Vall)
     return out
 
 
@@ -220,6 +224,7 @@ class OracleLayer:
         self.seen = 0
         self.last_scores = None
         self.last_keep = None
+        self.last_abs_out = None
 
     @property
     def len(self) -> int:
@@ -267,7 +272,8 @@ class OracleLayer:
         V_cache = self._r(self.V) if self.int4 else self.V
 
         # (b) Eq. 1
-        out = attention_rows(Qr, Kr_cache, V_cache, Kr_chunk, V, g, rows)
+        self.last_abs_out = np.full((n_tok, h * d), np.nan)
+        out = attention_rows(Qr, Kr_cache, V_cache, Kr_chunk, V, g, rows, self.last_abs_out)
 
         # (c) retaining head on the token's concatenated [Q ‖ K ‖ V]
         if self.s.rh_input == 0:

@@ -11,7 +11,9 @@ import torch
 
 from oracle import locret_oracle as O
 
-ATTN_TOL = 2e-2       # |delta| <= ATTN_TOL * max(1, |ref|)
+ATTN_TOL = 2e-2       # |delta| <= ATTN_TOL * max(1, |ref|) + (P_ULP + V_ULP) * sum_i p_i |v_i|
+P_ULP = 2.0 ** -8     # the probabilities enter the second contraction as bf16 operands
+V_ULP = 2.0 ** -7     # a stored V element may round to either bf16 neighbour (fp32 vs fp64 sum)
 SCORE_TOL = 1e-2      # |delta| <= SCORE_TOL * max(|ref|, rms(ref over the chunk))
 BAND = 1e-2           # index sets must agree outside this band around the cut
 
@@ -29,10 +31,17 @@ def make_pair(shape, weights, budget, chunk, n_stab, reserve=0):
     return ora, gpu
 
 
-def check_attention(got: np.ndarray, ref: np.ndarray, what=""):
+def check_attention(got: np.ndarray, ref: np.ndarray, what="", abs_ref=None):
+    """abs_ref = sum_i p_i |v_i| from the oracle: rows that attend to outlier tokens sum terms
+    far larger than their result; a bf16 probability operand carries up to 2^-9 relative error
+    per term, and a value element whose exact projection lies next to a bf16 rounding boundary
+    may be stored one ulp apart by the two sides (checked separately), which moves the output
+    by up to p_i * ulp(v_i).  Without abs_ref the bound is the plain mixed absolute/relative one."""
     ok = ~np.isnan(ref)
     err = np.abs(got[ok] - ref[ok])
     bound = ATTN_TOL * np.maximum(1.0, np.abs(ref[ok]))
+    if abs_ref is not None:
+        bound = bound + (P_ULP + V_ULP) * abs_ref[ok]
     worst = float(np.max(err / bound)) if err.size else 0.0
     assert worst <= 1.0, f"{what} attention: worst err/bound {worst:.3f}, max abs {err.max():.4g}"
     return float(err.max()) if err.size else 0.0
@@ -98,7 +107,8 @@ def lockstep_chunk(ora, gpu, x: np.ndarray, flags: int = 0, rows=None, what=""):
 
     ref_out = ora.prefill_chunk(x, flags, rows=rows)
     stats = {}
-    stats["attn_max_abs"] = check_attention(out_b.float().cpu().numpy().astype(np.float64), ref_out, what)
+    stats["attn_max_abs"] = check_attention(out_b.float().cpu().numpy().astype(np.float64), ref_out, what,
+                                            ora.last_abs_out)
 
     n = ln + n_tok
     assert pre["K"].shape[1] == n and pre["seen"] == st["seen"] + n_tok
@@ -111,7 +121,10 @@ def lockstep_chunk(ora, gpu, x: np.ndarray, flags: int = 0, rows=None, what=""):
     for name, got, ref in (("K", pre["K"][:, ln:], np.transpose(Kc, (1, 0, 2))),
                            ("V", pre["V"][:, ln:], np.transpose(Vc, (1, 0, 2)))):
         diff = np.abs(got - ref)
-        assert np.all(diff <= np.abs(ref) * 2.0 ** -7 + 1e-30), f"{what}: chunk {name} off by more than one bf16 ulp"
+        # one bf16 ulp of the value, plus the absolute error of an fp32 accumulation (matters
+        # only for results that cancel to nearly zero)
+        assert np.all(diff <= np.abs(ref) * 2.0 ** -7 + 1e-5 * np.abs(ref).max()), \
+            f"{what}: chunk {name} off by more than one bf16 ulp"
         assert np.mean(diff != 0) < 2e-3, f"{what}: too many rounding flips in chunk {name}"
     stats["score_worst"] = check_scores(pre["S"][:, ln:].T.astype(np.float64), ora.last_scores, what)
 
