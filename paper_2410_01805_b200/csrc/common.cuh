@@ -81,6 +81,16 @@ cudaError_t launch_rh_gemm(const bf16 *A, int lda, const bf16 *W1t, const float 
                            int M, int d_R, int K, int h_kv, int act, int *n_tiles, cudaStream_t st);
 int rh_num_tiles(int d_R);
 
+// The same two GEMMs on tcgen05 tensor cores (TMA-fed, TMEM accumulators); `status` is the
+// layer's device status word (set if a bounded wait gives up).
+bool gemm_tc_supported(int M, int N, int K, int lda, int ldb);
+cudaError_t launch_gemm_tc(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, int ldc, int M,
+                           int N, int K, int *status, cudaStream_t st);
+cudaError_t launch_rh_gemm_tc(const bf16 *A, int lda, const bf16 *W1t, const float *W2, float *partial,
+                              int M, int d_R, int K, int h_kv, int act, int *n_tiles, int *status,
+                              cudaStream_t st);
+int rh_tc_num_tiles(int d_R);
+
 // scores[m][slot0 + t] = sum_nt partial[nt][t][m]
 cudaError_t launch_rh_reduce(const float *partial, int n_tiles, int M, int h_kv, float *scores,
                              int score_stride, int slot0, cudaStream_t st);

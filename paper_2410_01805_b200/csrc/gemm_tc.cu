@@ -1,0 +1,305 @@
+// bf16 GEMM on tcgen05 tensor cores: C[M x N] = A[M x K] · Bt[N x K]^T, fp32 accumulation in
+// tensor memory.  One CTA computes a 128 x BN tile: warp 0 feeds shared memory with TMA
+// (128-byte swizzled K-blocks of 64), warp 1 issues tcgen05.mma, warps 2..5 read the
+// accumulator from TMEM and run the epilogue:
+//   MODE 0: bf16 store (the QKV projection);
+//   MODE 1: the retaining head's activation and its second, thin GEMM with W2, written as one
+//           partial score per (N-tile, row, KV head)                       (Section 3.3).
+#include "tc_common.cuh"
+
+namespace locret {
+
+// ------------------------------------------------------------------ tensor-map encoding (host)
+namespace {
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+    else
+      cudaGetLastError();
+  }
+  return fn;
+}
+}  // namespace
+
+bool tmap_encode_2d_bf16(CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer,
+                         uint64_t outer_stride_bytes, uint32_t box_inner, uint32_t box_outer) {
+  EncodeTiledFn fn = get_encode();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {outer_stride_bytes};
+  cuuint32_t box[2] = {box_inner, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box,
+            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool tmap_encode_3d_bf16(CUtensorMap *map, const void *base, uint64_t d0, uint64_t d1, uint64_t d2,
+                         uint64_t stride1_bytes, uint64_t stride2_bytes, uint32_t b0, uint32_t b1,
+                         uint32_t b2) {
+  EncodeTiledFn fn = get_encode();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {d0, d1, d2};
+  cuuint64_t strides[2] = {stride1_bytes, stride2_bytes};
+  cuuint32_t box[3] = {b0, b1, b2};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box,
+            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+namespace {
+
+using namespace tc;
+
+constexpr int BM = 128, BK = 64, GT_THREADS = 192;
+constexpr int MAX_HKV = 32;
+
+template <int BN>
+struct GemmCfg {
+  static constexpr int STAGES = BN == 256 ? 4 : 6;
+  static constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int W2_BYTES = BN * MAX_HKV * 4;
+  // 1024 for alignment slack, barriers + tmem pointer in a small tail
+  static constexpr int smem_bytes(int mode) {
+    return 1024 + STAGES * STAGE_BYTES + (mode == 1 ? W2_BYTES : 0) + 256;
+  }
+};
+
+template <int BN, int MODE>
+__global__ void __launch_bounds__(GT_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               bf16 *__restrict__ C, int ldc, int M, int N, int K, const float *__restrict__ W2,
+               float *__restrict__ partial, int h_kv, int act, int *status) {
+  using Cfg = GemmCfg<BN>;
+  constexpr int STAGES = Cfg::STAGES;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char *smem = reinterpret_cast<unsigned char *>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  unsigned char *tiles = smem;
+  float *sW2 = reinterpret_cast<float *>(tiles + STAGES * Cfg::STAGE_BYTES);
+  unsigned char *tail = tiles + STAGES * Cfg::STAGE_BYTES + (MODE == 1 ? Cfg::W2_BYTES : 0);
+  uint64_t *full = reinterpret_cast<uint64_t *>(tail);
+  uint64_t *empty = full + STAGES;
+  uint64_t *acc_full = empty + STAGES;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  const int KB = K / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; s++) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(acc_full, 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+    prefetch_tmap(&map_a);
+    prefetch_tmap(&map_b);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, BN);
+    tmem_relinquish();
+  }
+  if (MODE == 1) {
+    for (int v = threadIdx.x; v < BN * h_kv; v += GT_THREADS) {
+      int c = v / h_kv;
+      sW2[v] = (n0 + c < N) ? W2[(size_t)(n0 + c) * h_kv + (v - c * h_kv)] : 0.f;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int kb = 0; kb < KB; kb++) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, status)) break;
+        mbar_expect_tx(&full[s], Cfg::STAGE_BYTES);
+        unsigned char *a_dst = tiles + s * Cfg::STAGE_BYTES;
+        tma_load_2d(a_dst, &map_a, kb * BK, m0, &full[s]);
+        tma_load_2d(a_dst + Cfg::A_BYTES, &map_b, kb * BK, n0, &full[s]);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_bf16(BM, BN, 0, 0);
+      bool ok = true;
+      for (int kb = 0; kb < KB && ok; kb++) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        ok = mbar_wait(&full[s], ph, abort_flag, status);
+        if (!ok) break;
+        tc_fence_after();
+        unsigned char *a_src = tiles + s * Cfg::STAGE_BYTES;
+        const uint64_t da = desc_kmajor_sw128(a_src), db = desc_kmajor_sw128(a_src + Cfg::A_BYTES);
+#pragma unroll
+        for (int k = 0; k < BK / 16; k++)
+          mma_ss(tmem_base, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+        mma_commit(&empty[s]);  // frees the stage once these MMAs have read it
+      }
+      mma_commit(acc_full);
+    }
+  } else {
+    // epilogue warps 2..5: TMEM lane quarter = warp % 4
+    const int quarter = warp & 3;
+    const int row = m0 + quarter * 32 + lane;
+    const bool ok = mbar_wait(acc_full, 0, abort_flag, status);
+    tc_fence_after();
+    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    if (MODE == 0) {
+      if (ok) {
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c0, r);
+          tmem_wait_ld();
+          if (row < M && n0 + c0 < N) {
+            uint4 *dst = reinterpret_cast<uint4 *>(C + (size_t)row * ldc + n0 + c0);
+#pragma unroll
+            for (int v = 0; v < 4; v++) {
+              uint4 o;
+              o.x = pack_bf16(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1]));
+              o.y = pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
+              o.z = pack_bf16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]));
+              o.w = pack_bf16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]));
+              dst[v] = o;
+            }
+          }
+        }
+      }
+    } else {
+      float sc[MAX_HKV];
+#pragma unroll
+      for (int m = 0; m < MAX_HKV; m++) sc[m] = 0.f;
+      if (ok) {
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c0, r);
+          tmem_wait_ld();
+          if (h_kv <= 8) {
+#pragma unroll
+            for (int i = 0; i < 32; i++) {
+              const float a = apply_act(__uint_as_float(r[i]), act);
+              const float *w = sW2 + (c0 + i) * h_kv;
+#pragma unroll
+              for (int m = 0; m < 8; m++)
+                if (m < h_kv) sc[m] = fmaf(a, w[m], sc[m]);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; i++) {
+              const float a = apply_act(__uint_as_float(r[i]), act);
+              const float *w = sW2 + (c0 + i) * h_kv;
+#pragma unroll
+              for (int m = 0; m < MAX_HKV; m++)
+                if (m < h_kv) sc[m] = fmaf(a, w[m], sc[m]);
+            }
+          }
+        }
+        if (row < M) {
+          float *dst = partial + ((size_t)blockIdx.x * M + row) * h_kv;
+#pragma unroll
+          for (int m = 0; m < MAX_HKV; m++)
+            if (m < h_kv) dst[m] = sc[m];
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc(tmem_base, BN);
+}
+
+struct MapCache {
+  const void *base = nullptr;
+  uint64_t inner = 0, outer = 0, stride = 0;
+  uint32_t box_outer = 0;
+  CUtensorMap map;
+};
+
+// Small per-thread cache of encoded maps (weights and staging buffers repeat every call).
+const CUtensorMap *cached_map(const void *base, uint64_t inner, uint64_t outer, uint64_t stride_bytes,
+                              uint32_t box_outer) {
+  constexpr int SLOTS = 256;
+  static thread_local MapCache cache[SLOTS];
+  static thread_local int next = 0;
+  for (int i = 0; i < SLOTS; i++) {
+    MapCache &c = cache[i];
+    if (c.base == base && c.inner == inner && c.outer == outer && c.stride == stride_bytes &&
+        c.box_outer == box_outer)
+      return &c.map;
+  }
+  MapCache &c = cache[next];
+  next = (next + 1) % SLOTS;
+  if (!tmap_encode_2d_bf16(&c.map, base, inner, outer, stride_bytes, BK, box_outer)) {
+    c.base = nullptr;
+    return nullptr;
+  }
+  c.base = base; c.inner = inner; c.outer = outer; c.stride = stride_bytes; c.box_outer = box_outer;
+  return &c.map;
+}
+
+template <int BN, int MODE>
+cudaError_t launch_t(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, int ldc, int M, int N,
+                     int K, const float *W2, float *partial, int h_kv, int act, int *status,
+                     cudaStream_t st) {
+  using Cfg = GemmCfg<BN>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, MODE>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         Cfg::smem_bytes(MODE));
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const CUtensorMap *ma = cached_map(A, K, M, (uint64_t)lda * 2, BM);
+  const CUtensorMap *mb = cached_map(Bt, K, N, (uint64_t)ldb * 2, BN);
+  if (!ma || !mb) return cudaErrorInvalidValue;
+  dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM);
+  gemm_tc_kernel<BN, MODE><<<grid, GT_THREADS, Cfg::smem_bytes(MODE), st>>>(
+      *ma, *mb, C, ldc, M, N, K, W2, partial, h_kv, act, status);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool gemm_tc_supported(int M, int N, int K, int lda, int ldb) {
+  return K % BK == 0 && N % 32 == 0 && lda % 8 == 0 && ldb % 8 == 0 && M >= 1;
+}
+
+cudaError_t launch_gemm_tc(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, int ldc, int M,
+                           int N, int K, int *status, cudaStream_t st) {
+  if (N >= 256)
+    return launch_t<256, 0>(A, lda, Bt, ldb, C, ldc, M, N, K, nullptr, nullptr, 0, 0, status, st);
+  return launch_t<128, 0>(A, lda, Bt, ldb, C, ldc, M, N, K, nullptr, nullptr, 0, 0, status, st);
+}
+
+int rh_tc_num_tiles(int d_R) { return (d_R + 127) / 128; }
+
+cudaError_t launch_rh_gemm_tc(const bf16 *A, int lda, const bf16 *W1t, const float *W2, float *partial,
+                              int M, int d_R, int K, int h_kv, int act, int *n_tiles, int *status,
+                              cudaStream_t st) {
+  *n_tiles = rh_tc_num_tiles(d_R);
+  return launch_t<128, 1>(A, lda, W1t, K, nullptr, 0, M, d_R, K, W2, partial, h_kv, act, status, st);
+}
+
+}  // namespace locret

@@ -1,6 +1,7 @@
 // C ABI of the library: argument checks, state, and the per-chunk launch sequence.
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <map>
@@ -63,6 +64,7 @@ struct locret_layer {
   int64_t seen;
   int64_t launches;
   bool timing;
+  bool use_tc;  // tcgen05 kernels (default); LOCRET_LEGACY_MMA=1 keeps the mma.sync kernels for A/B runs
   std::vector<TimedEvent> events;
   size_t events_used;
 };
@@ -183,6 +185,10 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   L->st = (cudaStream_t)cfg->stream;
   L->cur = 0; L->len = 0; L->seen = 0; L->launches = 0; L->timing = false; L->events_used = 0;
   L->pool = nullptr;
+  {
+    const char *e = getenv("LOCRET_LEGACY_MMA");
+    L->use_tc = !(e && e[0] == '1');
+  }
 
   const size_t kv_b = (size_t)hk * L->cap * d * sizeof(bf16);
   const size_t sc_b = (size_t)hk * L->cap * sizeof(float);
@@ -214,7 +220,10 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
       g = g && grow(&p->q_rot, &p->qrot_b, (size_t)chunk * h * d * sizeof(bf16), L->st);
       if (cfg->rh_input == 1)
         g = g && grow(&p->z_post, &p->zpost_b, (size_t)chunk * L->d_in * sizeof(bf16), L->st);
-      g = g && grow(&p->partial, &p->partial_b, (size_t)rh_num_tiles(dR) * chunk * hk * sizeof(float), L->st);
+      {
+        int nt = rh_num_tiles(dR) > rh_tc_num_tiles(dR) ? rh_num_tiles(dR) : rh_tc_num_tiles(dR);
+        g = g && grow(&p->partial, &p->partial_b, (size_t)nt * chunk * hk * sizeof(float), L->st);
+      }
       g = g && grow(&p->keep, &p->keep_b, (size_t)hk * budget * sizeof(int32_t), L->st);
       if (g) L->cs = get_cs_table(p, cfg->rope_theta, d, L->cap, L->st);
       ok = g && L->cs;
@@ -260,8 +269,12 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
 
   {  // (a) projections
     Timed t(L, LOCRET_K_QKV);
-    CK(launch_gemm_bf16((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, P->staging, L->d_in, n_tok,
-                        L->d_in, L->D, L->st));
+    if (L->use_tc && n_tok >= 32 && gemm_tc_supported(n_tok, L->d_in, L->D, L->D, L->D))
+      CK(launch_gemm_tc((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, P->staging, L->d_in, n_tok,
+                        L->d_in, L->D, L->d_status, L->st));
+    else
+      CK(launch_gemm_bf16((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, P->staging, L->d_in, n_tok,
+                          L->d_in, L->D, L->st));
   }
   {  // positions, RoPE, append of the chunk's units at slots [len, len + n_tok)
     Timed t(L, LOCRET_K_ROPE);
@@ -282,8 +295,12 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
   {  // (c) retaining head
     Timed t(L, LOCRET_K_RH);
     const bf16 *z = L->cfg.rh_input == 1 ? P->z_post : P->staging;
-    CK(launch_rh_gemm(z, L->d_in, L->w1_t, L->w2f, P->partial, n_tok, L->d_R, L->d_in, L->h_kv,
-                      L->cfg.act, &n_tiles, L->st));
+    if (L->use_tc && n_tok >= 32 && gemm_tc_supported(n_tok, L->d_R, L->d_in, L->d_in, L->d_in))
+      CK(launch_rh_gemm_tc(z, L->d_in, L->w1_t, L->w2f, P->partial, n_tok, L->d_R, L->d_in, L->h_kv,
+                           L->cfg.act, &n_tiles, L->d_status, L->st));
+    else
+      CK(launch_rh_gemm(z, L->d_in, L->w1_t, L->w2f, P->partial, n_tok, L->d_R, L->d_in, L->h_kv,
+                        L->cfg.act, &n_tiles, L->st));
   }
   {
     Timed t(L, LOCRET_K_RH_REDUCE);

@@ -72,7 +72,9 @@ def test_c1_free_running_matches_oracle_sets():
 @pytest.mark.parametrize("heads", [(4, 2), (3, 3), (8, 1)])
 def test_ragged_chunks_lockstep(d, heads):
     from parity_util import lockstep_chunk, make_pair
-    sh = small_shape(h=heads[0], hk=heads[1], d=d, D=96, dR=72, rope_theta=500000.0)
+    # D = 96 / d_R = 72 take the general-shape kernels, D = 128 / d_R = 96 the tcgen05 GEMMs
+    D, dR = (96, 72) if heads[1] == 3 else (128, 96)
+    sh = small_shape(h=heads[0], hk=heads[1], d=d, D=D, dR=dR, rope_theta=500000.0)
     ora, gpu = make_pair(sh, weights_for(sh, d), budget=300, chunk=200, n_stab=17)
     start = 0
     for i, n_tok in enumerate([1, 127, 129, 200, 64, 200, 3]):
