@@ -1,0 +1,318 @@
+// Eq. 1 on tcgen05 tensor cores with TMEM accumulators, head_dim 128.
+//
+// One CTA owns two 128-row query tiles that share a KV head (two query heads of one GQA
+// group over the same rows, or two consecutive row blocks of one head) and streams the
+// keys/values of that head in tiles of 128 through shared memory with TMA.  Roles:
+//   warps 0-3 / 4-7  softmax of query tile 0 / 1: one thread per query row reads its row of
+//                    S = Q K^T from TMEM, keeps a running maximum and sum, writes
+//                    P = exp2(S - max) as bf16 back into TMEM over S, and rescales the
+//                    accumulator in TMEM only when the maximum has grown by more than 2^8;
+//   warp 8           TMA producer (Q once, then K and V tiles, two stages each);
+//   warp 9           issues S_t = Q_t K_j^T (both operands in shared memory) and
+//                    O_t += P_t V_j (P from TMEM, V from shared memory), alternating the two
+//                    tiles so that one tile's softmax overlaps the other tile's MMAs.
+// TMEM columns: S0/P0 [0,128), S1/P1 [128,256), O0 [256,384), O1 [384,512).
+// Query row t sees keys [0, len + t]: the retained cache unmasked, the chunk causally.
+#include "tc_common.cuh"
+
+namespace locret {
+
+namespace {
+
+using namespace tc;
+
+constexpr int AT_THREADS = 320;
+constexpr int TILE = 128;               // query rows per tile and keys per tile
+constexpr int HD = 128;                 // head_dim
+constexpr int HALF_BYTES = TILE * 128;  // one 64-column swizzled box of 128 rows: 16 KB
+constexpr int TILE_BYTES = 2 * HALF_BYTES;
+constexpr int AT_SMEM = 1024 + 6 * TILE_BYTES + 256;  // Q0,Q1,K0,K1,V0,V1 + barriers
+
+struct AttnParams {
+  bf16 *out;
+  int n_tok, h, h_kv, len, pair_heads;
+  float scale_log2;
+  int *status;
+};
+
+__global__ void __launch_bounds__(AT_THREADS, 1)
+attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+               const __grid_constant__ CUtensorMap map_v, const AttnParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char *smem = reinterpret_cast<unsigned char *>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  unsigned char *sQ = smem;                   // [2][TILE_BYTES]
+  unsigned char *sK = smem + 2 * TILE_BYTES;  // [2 stages][TILE_BYTES]
+  unsigned char *sV = smem + 4 * TILE_BYTES;  // [2 stages][TILE_BYTES]
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + 6 * TILE_BYTES);
+  uint64_t *q_full = bars;          // 1
+  uint64_t *k_full = bars + 1;      // 2
+  uint64_t *v_full = bars + 3;      // 2
+  uint64_t *k_empty = bars + 5;     // 2
+  uint64_t *v_empty = bars + 7;     // 2
+  uint64_t *s_full = bars + 9;      // 2
+  uint64_t *p_full = bars + 11;     // 2
+  uint64_t *o_full = bars + 13;     // 2
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 15);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = p.h / p.h_kv;
+  const int n = p.len + p.n_tok;
+  const int n_rb = (p.n_tok + TILE - 1) / TILE;
+
+  // which two query tiles; longest key ranges first
+  int row0[2], head[2];
+  if (p.pair_heads) {
+    const int hp = p.h / 2;
+    const int rb = n_rb - 1 - (int)blockIdx.x / hp;
+    const int hq = (int)blockIdx.x % hp;
+    row0[0] = row0[1] = rb * TILE;
+    head[0] = 2 * hq; head[1] = 2 * hq + 1;
+  } else {
+    const int n_rp = (n_rb + 1) / 2;
+    const int rp = n_rp - 1 - (int)blockIdx.x / p.h;
+    row0[0] = rp * 2 * TILE; row0[1] = row0[0] + TILE;
+    head[0] = head[1] = (int)blockIdx.x % p.h;
+  }
+  const int kvh = head[0] / g;
+  int NK = (p.len + row0[1] + TILE + TILE - 1) / TILE;
+  NK = min(NK, (n + TILE - 1) / TILE);
+
+  if (threadIdx.x == 0) {
+    mbar_init(q_full, 1);
+    for (int s = 0; s < 2; s++) {
+      mbar_init(&k_full[s], 1); mbar_init(&v_full[s], 1);
+      mbar_init(&k_empty[s], 1); mbar_init(&v_empty[s], 1);
+      mbar_init(&s_full[s], 1); mbar_init(&p_full[s], 4); mbar_init(&o_full[s], 1);
+    }
+    *abort_flag = 0;
+    fence_barrier_init();
+    prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
+  }
+  if (warp == 9) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 8) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      mbar_expect_tx(q_full, 2 * TILE_BYTES);
+      for (int t = 0; t < 2; t++)
+        for (int hh = 0; hh < 2; hh++)
+          tma_load_2d(sQ + t * TILE_BYTES + hh * HALF_BYTES, &map_q, head[t] * HD + hh * 64, row0[t],
+                      q_full);
+      for (int j = 0; j < NK; j++) {
+        const int s = j & 1;
+        const uint32_t ph = (j >> 1) & 1;
+        if (!mbar_wait(&k_empty[s], ph ^ 1, abort_flag, p.status)) break;
+        mbar_expect_tx(&k_full[s], TILE_BYTES);
+        for (int hh = 0; hh < 2; hh++)
+          tma_load_3d(sK + s * TILE_BYTES + hh * HALF_BYTES, &map_k, hh * 64, j * TILE, kvh, &k_full[s]);
+        if (!mbar_wait(&v_empty[s], ph ^ 1, abort_flag, p.status)) break;
+        mbar_expect_tx(&v_full[s], TILE_BYTES);
+        for (int hh = 0; hh < 2; hh++)
+          tma_load_3d(sV + s * TILE_BYTES + hh * HALF_BYTES, &map_v, hh * 64, j * TILE, kvh, &v_full[s]);
+      }
+    }
+  } else if (warp == 9) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = idesc_bf16(TILE, TILE, 0, 0);
+      constexpr uint32_t idesc_pv = idesc_bf16(TILE, HD, 0, 1);
+      auto issue_s = [&](int t, int ks) {
+        const unsigned char *q = sQ + t * TILE_BYTES, *k = sK + ks * TILE_BYTES;
+#pragma unroll
+        for (int kk = 0; kk < HD / 16; kk++) {
+          const int off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
+          mma_ss(tmem_base + t * TILE, desc_kmajor_sw128(q + off), desc_kmajor_sw128(k + off), idesc_qk,
+                 kk != 0);
+        }
+        mma_commit(&s_full[t]);
+      };
+      auto issue_pv = [&](int t, int vs, bool acc) {
+        const unsigned char *v = sV + vs * TILE_BYTES;
+#pragma unroll
+        for (int kk = 0; kk < TILE / 16; kk++)
+          mma_ts(tmem_base + 2 * TILE + t * HD, tmem_base + t * TILE + kk * 8,
+                 desc_mnmajor_sw128(v + kk * 16 * 128, HALF_BYTES), idesc_pv, acc || kk != 0);
+        mma_commit(&o_full[t]);
+      };
+      bool ok = mbar_wait(q_full, 0, abort_flag, p.status);
+      ok = ok && mbar_wait(&k_full[0], 0, abort_flag, p.status);
+      if (ok) {
+        tc_fence_after();
+        issue_s(0, 0);
+        issue_s(1, 0);
+        mma_commit(&k_empty[0]);
+      }
+      for (int j = 0; j < NK && ok; j++) {
+        const int sv = j & 1;
+        ok = mbar_wait(&v_full[sv], (j >> 1) & 1, abort_flag, p.status);
+        for (int t = 0; t < 2 && ok; t++) {
+          ok = mbar_wait(&p_full[t], j & 1, abort_flag, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          issue_pv(t, sv, j > 0);
+          if (j + 1 < NK) {
+            const int sk = (j + 1) & 1;
+            if (t == 0) {
+              ok = mbar_wait(&k_full[sk], ((j + 1) >> 1) & 1, abort_flag, p.status);
+              if (!ok) break;
+              tc_fence_after();
+            }
+            issue_s(t, sk);
+            if (t == 1) mma_commit(&k_empty[sk]);
+          }
+        }
+        if (ok) mma_commit(&v_empty[sv]);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ softmax, one row per thread
+    const int t = warp >> 2, quarter = warp & 3;
+    const int r = quarter * 32 + lane;
+    const int row = row0[t] + r;
+    const int limit = p.len + row;  // last visible key
+    const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+    const uint32_t s_addr = tmem_base + lane_off + t * TILE;
+    const uint32_t o_addr = tmem_base + lane_off + 2 * TILE + t * HD;
+    const float c = p.scale_log2;
+    float m_used = -INFINITY, l = 0.f;
+    bool ok = true;
+
+    for (int j = 0; j < NK && ok; j++) {
+      ok = mbar_wait(&s_full[t], j & 1, abort_flag, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t s[TILE];
+#pragma unroll
+      for (int q = 0; q < 4; q++) tmem_ld32(s_addr + q * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[q * 32]));
+      tmem_wait_ld();
+
+      const int key0 = j * TILE;
+      float tmax = -INFINITY;
+      if (key0 + TILE - 1 > p.len + row0[t]) {  // a tile that crosses the causal boundary
+#pragma unroll
+        for (int i = 0; i < TILE; i++) {
+          float x = (key0 + i <= limit) ? __uint_as_float(s[i]) : -INFINITY;
+          s[i] = __float_as_uint(x);
+          tmax = fmaxf(tmax, x);
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < TILE; i++) tmax = fmaxf(tmax, __uint_as_float(s[i]));
+      }
+      tmax *= c;
+
+      if (j == 0) {
+        m_used = tmax;
+      } else {
+        const bool need = tmax > m_used + 8.0f;
+        if (__any_sync(0xffffffffu, need)) {
+          // the accumulator must hold every product issued so far before it is rescaled
+          ok = mbar_wait(&o_full[t], (j - 1) & 1, abort_flag, p.status);
+          tc_fence_after();
+          float alpha = 1.0f;
+          if (need) { alpha = exp2f(m_used - tmax); m_used = tmax; }
+          l *= alpha;
+#pragma unroll 1
+          for (int q = 0; q < 4; q++) {
+            uint32_t o[32];
+            tmem_ld32(o_addr + q * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; i++) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+            tmem_st32(o_addr + q * 32, o);
+          }
+          tmem_wait_st();
+        }
+      }
+
+      const float neg_m = -m_used;
+#pragma unroll
+      for (int q = 0; q < 2; q++) {
+        uint32_t pk[32];
+#pragma unroll
+        for (int i = 0; i < 32; i++) {
+          float p0 = exp2f(fmaf(__uint_as_float(s[q * 64 + 2 * i]), c, neg_m));
+          float p1 = exp2f(fmaf(__uint_as_float(s[q * 64 + 2 * i + 1]), c, neg_m));
+          l += p0 + p1;
+          pk[i] = pack_bf16(p0, p1);
+        }
+        tmem_st32(s_addr + q * 32, pk);
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&p_full[t]);
+    }
+
+    if (ok && NK > 0) ok = mbar_wait(&o_full[t], (NK - 1) & 1, abort_flag, p.status);
+    tc_fence_after();
+    if (ok) {
+      const float inv = 1.0f / l;
+      bf16 *dst = p.out + (size_t)row * p.h * HD + (size_t)head[t] * HD;
+#pragma unroll 1
+      for (int q = 0; q < 4; q++) {
+        uint32_t o[32];
+        tmem_ld32(o_addr + q * 32, o);
+        tmem_wait_ld();
+        if (row < p.n_tok) {
+#pragma unroll
+          for (int v = 0; v < 4; v++) {
+            uint4 w;
+            w.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
+            w.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
+            w.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
+            w.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
+            *reinterpret_cast<uint4 *>(dst + q * 32 + v * 8) = w;
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 9) {
+    __syncwarp();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+}  // namespace
+
+bool attention_tc_supported(int n_tok, int h, int h_kv, int d) {
+  return d == HD && n_tok >= 64 && h % h_kv == 0;
+}
+
+// map_k / map_v: 3-D maps {d, cap, h_kv} with box {64, 128, 1}; map_q: 2-D {h*d, rows} box {64, 128}.
+cudaError_t launch_attention_tc(const CUtensorMap *map_q, const CUtensorMap *map_k,
+                                const CUtensorMap *map_v, bf16 *out, int n_tok, int h, int h_kv, int len,
+                                int *status, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         AT_SMEM);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  AttnParams p;
+  p.out = out; p.n_tok = n_tok; p.h = h; p.h_kv = h_kv; p.len = len;
+  p.pair_heads = ((h / h_kv) % 2 == 0) ? 1 : 0;
+  p.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
+  p.status = status;
+  const int n_rb = (n_tok + TILE - 1) / TILE;
+  const int grid = p.pair_heads ? n_rb * (h / 2) : ((n_rb + 1) / 2) * h;
+  attn_tc_kernel<<<grid, AT_THREADS, AT_SMEM, st>>>(*map_q, *map_k, *map_v, p);
+  return cudaGetLastError();
+}
+
+}  // namespace locret

@@ -11,6 +11,7 @@
 
 #include "../../include/locret.h"
 #include "common.cuh"
+#include "tc_common.cuh"
 
 using namespace locret;
 
@@ -65,6 +66,9 @@ struct locret_layer {
   int64_t launches;
   bool timing;
   bool use_tc;  // tcgen05 kernels (default); LOCRET_LEGACY_MMA=1 keeps the mma.sync kernels for A/B runs
+  bool tc_attn;  // tensor maps for the tcgen05 attention kernel are valid
+  CUtensorMap map_k, map_v[2], map_q;
+  const void *map_q_base;
   std::vector<TimedEvent> events;
   size_t events_used;
 };
@@ -233,6 +237,16 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   }
   if (!ok) { ScratchPool *p = L->pool; free_layer_memory(L); delete L; release_pool(p); return LOCRET_ERR_ALLOC; }
 
+  // tensor maps of the cache for the tcgen05 attention kernel
+  L->map_q_base = nullptr;
+  L->tc_attn = L->use_tc && d == 128 &&
+               tmap_encode_3d_bf16(&L->map_k, L->k_rot, d, L->cap, hk, (uint64_t)d * 2,
+                                   (uint64_t)L->cap * d * 2, 64, 128, 1) &&
+               tmap_encode_3d_bf16(&L->map_v[0], L->v[0], d, L->cap, hk, (uint64_t)d * 2,
+                                   (uint64_t)L->cap * d * 2, 64, 128, 1) &&
+               tmap_encode_3d_bf16(&L->map_v[1], L->v[1], d, L->cap, hk, (uint64_t)d * 2,
+                                   (uint64_t)L->cap * d * 2, 64, 128, 1);
+
   // repack the weights: K-major copies for both GEMMs, W2 in fp32
   cudaError_t e = cudaSuccess;
   if (e == cudaSuccess) e = launch_transpose_bf16((const bf16 *)cfg->w_qkv, L->wqkv_t, D, L->d_in, L->st);
@@ -288,8 +302,18 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
   }
   {  // (b) Eq. 1
     Timed t(L, LOCRET_K_ATTN);
-    CK(launch_attention_mma(P->q_rot, L->k_rot, L->v[c], (bf16 *)attn_out, n_tok, L->h, L->h_kv,
-                            L->d, L->cap, L->len, L->st));
+    bool tc_ok = L->tc_attn && attention_tc_supported(n_tok, L->h, L->h_kv, L->d);
+    if (tc_ok && L->map_q_base != P->q_rot) {
+      tc_ok = tmap_encode_2d_bf16(&L->map_q, P->q_rot, (uint64_t)L->h * L->d, (uint64_t)L->chunk,
+                                  (uint64_t)L->h * L->d * 2, 64, 128);
+      L->map_q_base = tc_ok ? P->q_rot : nullptr;
+    }
+    if (tc_ok)
+      CK(launch_attention_tc(&L->map_q, &L->map_k, &L->map_v[c], (bf16 *)attn_out, n_tok, L->h, L->h_kv,
+                             L->len, L->d_status, L->st));
+    else
+      CK(launch_attention_mma(P->q_rot, L->k_rot, L->v[c], (bf16 *)attn_out, n_tok, L->h, L->h_kv,
+                              L->d, L->cap, L->len, L->st));
   }
   int n_tiles = 0;
   {  // (c) retaining head

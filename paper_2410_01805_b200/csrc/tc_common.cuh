@@ -196,4 +196,12 @@ bool tmap_encode_3d_bf16(CUtensorMap *map, const void *base, uint64_t d0, uint64
                          uint64_t stride1_bytes, uint64_t stride2_bytes, uint32_t b0, uint32_t b1,
                          uint32_t b2);
 
+
+// Eq. 1 on tcgen05 (attn_tc.cu).  map_k / map_v: 3-D maps {d, cap, h_kv}, box {64, 128, 1};
+// map_q: 2-D map {h*d, rows}, box {64, 128}.
+bool attention_tc_supported(int n_tok, int h, int h_kv, int d);
+cudaError_t launch_attention_tc(const CUtensorMap *map_q, const CUtensorMap *map_k,
+                                const CUtensorMap *map_v, bf16 *out, int n_tok, int h, int h_kv, int len,
+                                int *status, cudaStream_t st);
+
 }  // namespace locret
