@@ -152,6 +152,36 @@ int locret_read_timing(locret_layer *layer, float *ms, int64_t *launches);
 /* Total number of this library's kernels launched for the layer since create. */
 int locret_launch_count(const locret_layer *layer, int64_t *count);
 
+/*
+ * Retaining-head scores without any allocation.  (The paper has no counterpart: this entry
+ * point exists for hosts that may not allocate device memory where they need scores, e.g. code
+ * that runs inside a pool owning the whole device, or under an allocator that is locked while
+ * a request is in flight.)
+ *
+ * Computes scores[m][t] = sum_r act( sum_c z[t][c] * w1_t[r][c] ) * w2[r][m], the same
+ * arithmetic, kernels and summation order as step (c) of locret_prefill_chunk.
+ *   z       device bf16 [n_tok x d_in], row-major: the tokens' concatenated [Q ‖ K ‖ V]
+ *   w1_t    device bf16 [d_retain x d_in], row-major: W1 TRANSPOSED (the layer API repacks W1
+ *           into this form at create; here the caller supplies it, since repacking allocates)
+ *   w2      device fp32 [d_retain x n_kv_heads], row-major
+ *   scores  device fp32 [n_kv_heads x n_tok], written entirely
+ * Requires d_in % 64 == 0, d_retain % 32 == 0, 1 <= n_kv_heads <= 32, act in {0,1,2}, z and w1_t
+ * 16-byte aligned.  The per-tile partial sums live in a fixed array inside the library image of
+ * LOCRET_STATIC_SCRATCH_FLOATS floats (4 MiB, present on every GPU that loads the library until
+ * the process exits); a call needs ceil(d_retain / 128) * n_tok * n_kv_heads of them and returns
+ * LOCRET_ERR_CAPACITY, launching nothing, if that is more.
+ * The call makes no cudaMalloc/cudaFree and uses no allocating library routine.  Its first call on
+ * a device looks up the array's device address (cudaGetSymbolAddress, with that device current);
+ * make that first call outside of any stream capture.  All calls share the one array, which
+ * keeps the previous call's contents (nothing in it needs clearing: a call writes every value it
+ * later reads); two calls whose kernels overlap on the GPU (different streams, no dependency)
+ * race on it.  Asynchronous on `stream` (cudaStream_t; NULL = legacy default stream).
+ */
+#define LOCRET_STATIC_SCRATCH_FLOATS (1 << 20)
+int locret_rh_scores_static(const void *z, int32_t n_tok, int32_t d_in, const void *w1_t,
+                            int32_t d_retain, const float *w2, int32_t n_kv_heads, int32_t act,
+                            float *scores, void *stream);
+
 /* Free everything the layer owns.  Synchronises the stream.  NULL is allowed. */
 void locret_destroy(locret_layer *layer);
 

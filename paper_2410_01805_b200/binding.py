@@ -52,6 +52,7 @@ def _load():
     l.locret_set_timing.argtypes = [P, C.c_int32]
     l.locret_read_timing.argtypes = [P, P, P]
     l.locret_launch_count.argtypes = [P, C.POINTER(C.c_int64)]
+    l.locret_rh_scores_static.argtypes = [P, C.c_int32, C.c_int32, P, C.c_int32, P, C.c_int32, C.c_int32, P, P]
     l.locret_destroy.argtypes = [P]
     l.locret_destroy.restype = None
     return l
