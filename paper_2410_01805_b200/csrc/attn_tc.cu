@@ -21,12 +21,44 @@ namespace {
 
 using namespace tc;
 
-constexpr int AT_THREADS = 320;
+constexpr int AT_THREADS = 384;  // 3 warpgroups: softmax 0, softmax 1, {TMA, MMA, 2 idle warps}
 constexpr int TILE = 128;               // query rows per tile and keys per tile
 constexpr int HD = 128;                 // head_dim
 constexpr int HALF_BYTES = TILE * 128;  // one 64-column swizzled box of 128 rows: 16 KB
 constexpr int TILE_BYTES = 2 * HALF_BYTES;
 constexpr int AT_SMEM = 1024 + 6 * TILE_BYTES + 256;  // Q0,Q1,K0,K1,V0,V1 + barriers
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float &lo, float &hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+template <int N>
+__device__ __forceinline__ void setmaxnreg_inc() {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void setmaxnreg_dec() {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
 
 struct AttnParams {
   bf16 *out;
@@ -99,7 +131,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 8) {
+  if (warp >= 8) {
+    setmaxnreg_dec<56>();
+  if (warp >= 10) {
+    // idle warps of the third warpgroup
+  } else if (warp == 8) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       mbar_expect_tx(q_full, 2 * TILE_BYTES);
@@ -173,8 +209,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         if (ok) mma_commit(&v_empty[sv]);
       }
     }
+  }
   } else {
     // ------------------------------------------------------------ softmax, one row per thread
+    setmaxnreg_inc<224>();
     const int t = warp >> 2, quarter = warp & 3;
     const int r = quarter * 32 + lane;
     const int row = row0[t] + r;
@@ -205,8 +243,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           tmax = fmaxf(tmax, x);
         }
       } else {
+        float t0 = -INFINITY, t1 = -INFINITY, t2 = -INFINITY, t3 = -INFINITY;
 #pragma unroll
-        for (int i = 0; i < TILE; i++) tmax = fmaxf(tmax, __uint_as_float(s[i]));
+        for (int i = 0; i < TILE; i += 8) {
+          t0 = fmaxf(t0, fmaxf(__uint_as_float(s[i]), __uint_as_float(s[i + 1])));
+          t1 = fmaxf(t1, fmaxf(__uint_as_float(s[i + 2]), __uint_as_float(s[i + 3])));
+          t2 = fmaxf(t2, fmaxf(__uint_as_float(s[i + 4]), __uint_as_float(s[i + 5])));
+          t3 = fmaxf(t3, fmaxf(__uint_as_float(s[i + 6]), __uint_as_float(s[i + 7])));
+        }
+        tmax = fmaxf(fmaxf(t0, t1), fmaxf(t2, t3));
       }
       tmax *= c;
 
@@ -234,18 +279,31 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
 
-      const float neg_m = -m_used;
+      const uint64_t c2 = pack_f32x2(c, c), nm2 = pack_f32x2(-m_used, -m_used);
+      uint64_t la = pack_f32x2(0.f, 0.f), lb = la;
 #pragma unroll
       for (int q = 0; q < 2; q++) {
         uint32_t pk[32];
 #pragma unroll
-        for (int i = 0; i < 32; i++) {
-          float p0 = exp2f(fmaf(__uint_as_float(s[q * 64 + 2 * i]), c, neg_m));
-          float p1 = exp2f(fmaf(__uint_as_float(s[q * 64 + 2 * i + 1]), c, neg_m));
-          l += p0 + p1;
+        for (int i = 0; i < 32; i += 2) {
+          float x0, x1, x2, x3;
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[q * 64 + 2 * i]),
+                                            __uint_as_float(s[q * 64 + 2 * i + 1])), c2, nm2), x0, x1);
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[q * 64 + 2 * i + 2]),
+                                            __uint_as_float(s[q * 64 + 2 * i + 3])), c2, nm2), x2, x3);
+          const float p0 = ex2_approx(x0), p1 = ex2_approx(x1), p2 = ex2_approx(x2), p3 = ex2_approx(x3);
+          la = add_f32x2(la, pack_f32x2(p0, p1));
+          lb = add_f32x2(lb, pack_f32x2(p2, p3));
           pk[i] = pack_bf16(p0, p1);
+          pk[i + 1] = pack_bf16(p2, p3);
         }
         tmem_st32(s_addr + q * 32, pk);
+      }
+      {
+        float a0, a1, b0, b1;
+        unpack_f32x2(la, a0, a1);
+        unpack_f32x2(lb, b0, b1);
+        l += (a0 + a1) + (b0 + b1);
       }
       tmem_wait_st();
       tc_fence_before();
