@@ -184,19 +184,44 @@ topk_kernel(const float *__restrict__ scores, int score_stride, int n, int budge
     for (int shift = 24; shift >= 0; shift -= 8) {
       if (tid < 256) hist[tid] = 0;
       __syncthreads();
-      for (int i = tid; i < rest; i += TK_THREADS) {
-        uint32_t key = key_at(i);
-        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+      // warp-aggregated histogram: lanes that hit the same bin elect one atomic
+      for (int i0 = 0; i0 < rest; i0 += TK_THREADS) {
+        const int i = i0 + tid;
+        uint32_t key = 0;
+        bool in = false;
+        if (i < rest) {
+          key = key_at(i);
+          in = (key & mask) == prefix;
+        }
+        const unsigned active = __ballot_sync(0xffffffffu, in);
+        if (in) {
+          const uint32_t bin = (key >> shift) & 255u;
+          const unsigned peers = __match_any_sync(active, bin);
+          if ((tid & 31) == __ffs(peers) - 1) atomicAdd(&hist[bin], __popc(peers));
+        }
       }
       __syncthreads();
-      if (tid == 0) {
-        int acc = 0, b = 255;
-        for (; b > 0; b--) {
-          if (acc + hist[b] >= need) break;
-          acc += hist[b];
+      if (tid < 32) {
+        // lane l owns bins [8l, 8l+8); suffix sums over lanes locate the bin of the need-th key
+        int loc[8], sum = 0;
+#pragma unroll
+        for (int b = 0; b < 8; b++) { loc[b] = hist[tid * 8 + b]; sum += loc[b]; }
+        int above = 0;  // keys in the bins of higher lanes
+#pragma unroll
+        for (int l2 = 0; l2 < 32; l2++) {
+          const int v = __shfl_sync(0xffffffffu, sum, l2);
+          if (l2 > (int)tid) above += v;
         }
-        s_prefix = prefix | ((uint32_t)b << shift);
-        s_need = need - acc;
+        const bool mine = (above < need) && (above + sum >= need);
+        if (mine) {
+          int acc = above, b = 7;
+          for (; b > 0; b--) {
+            if (acc + loc[b] >= need) break;
+            acc += loc[b];
+          }
+          s_prefix = prefix | ((uint32_t)(tid * 8 + b) << shift);
+          s_need = need - acc;
+        }
       }
       __syncthreads();
       prefix = s_prefix;

@@ -66,6 +66,13 @@ using namespace tc;
 constexpr int BM = 128, BK = 64, GT_THREADS = 192;
 constexpr int MAX_HKV = 32;
 
+// sigma of the retaining head with the fast division / exponential intrinsics (relative error
+// ~1e-6, far inside the score tolerance)
+__device__ __forceinline__ float fast_act(float x, int act) {
+  if (act == 0) return __fdividef(x, 1.0f + __expf(-x));
+  return apply_act(x, act);
+}
+
 template <int BN>
 struct GemmCfg {
   static constexpr int STAGES = BN == 256 ? 4 : 6;
@@ -193,23 +200,41 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           uint32_t r[32];
           tmem_ld32(taddr + c0, r);
           tmem_wait_ld();
-          if (h_kv <= 8) {
+          // activation of the 32 columns first (independent, so the special-function unit
+          // pipelines them), then the thin GEMM with W2 as broadcast 16-byte loads
+          float a[32];
+#pragma unroll
+          for (int i = 0; i < 32; i++) a[i] = fast_act(__uint_as_float(r[i]), act);
+          if (h_kv == 8) {
 #pragma unroll
             for (int i = 0; i < 32; i++) {
-              const float a = apply_act(__uint_as_float(r[i]), act);
-              const float *w = sW2 + (c0 + i) * h_kv;
+              const float4 w0 = *reinterpret_cast<const float4 *>(sW2 + (c0 + i) * 8);
+              const float4 w1 = *reinterpret_cast<const float4 *>(sW2 + (c0 + i) * 8 + 4);
+              sc[0] = fmaf(a[i], w0.x, sc[0]); sc[1] = fmaf(a[i], w0.y, sc[1]);
+              sc[2] = fmaf(a[i], w0.z, sc[2]); sc[3] = fmaf(a[i], w0.w, sc[3]);
+              sc[4] = fmaf(a[i], w1.x, sc[4]); sc[5] = fmaf(a[i], w1.y, sc[5]);
+              sc[6] = fmaf(a[i], w1.z, sc[6]); sc[7] = fmaf(a[i], w1.w, sc[7]);
+            }
+          } else if (h_kv == 32) {
 #pragma unroll
-              for (int m = 0; m < 8; m++)
-                if (m < h_kv) sc[m] = fmaf(a, w[m], sc[m]);
+            for (int i = 0; i < 32; i++) {
+              const float4 *w = reinterpret_cast<const float4 *>(sW2 + (c0 + i) * 32);
+#pragma unroll
+              for (int m4 = 0; m4 < 8; m4++) {
+                const float4 wv = w[m4];
+                sc[4 * m4 + 0] = fmaf(a[i], wv.x, sc[4 * m4 + 0]);
+                sc[4 * m4 + 1] = fmaf(a[i], wv.y, sc[4 * m4 + 1]);
+                sc[4 * m4 + 2] = fmaf(a[i], wv.z, sc[4 * m4 + 2]);
+                sc[4 * m4 + 3] = fmaf(a[i], wv.w, sc[4 * m4 + 3]);
+              }
             }
           } else {
 #pragma unroll
             for (int i = 0; i < 32; i++) {
-              const float a = apply_act(__uint_as_float(r[i]), act);
               const float *w = sW2 + (c0 + i) * h_kv;
 #pragma unroll
               for (int m = 0; m < MAX_HKV; m++)
-                if (m < h_kv) sc[m] = fmaf(a, w[m], sc[m]);
+                if (m < h_kv) sc[m] = fmaf(a[i], w[m], sc[m]);
             }
           }
         }
@@ -293,12 +318,16 @@ cudaError_t launch_gemm_tc(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16
   return launch_t<128, 0>(A, lda, Bt, ldb, C, ldc, M, N, K, nullptr, nullptr, 0, 0, status, st);
 }
 
-int rh_tc_num_tiles(int d_R) { return (d_R + 127) / 128; }
+// 128 x 256 tiles whenever d_R allows: a 128-wide tile needs twice the operand traffic per flop.
+static int rh_tile_n(int d_R) { return d_R % 256 == 0 ? 256 : 128; }
+int rh_tc_num_tiles(int d_R) { return (d_R + rh_tile_n(d_R) - 1) / rh_tile_n(d_R); }
 
 cudaError_t launch_rh_gemm_tc(const bf16 *A, int lda, const bf16 *W1t, const float *W2, float *partial,
                               int M, int d_R, int K, int h_kv, int act, int *n_tiles, int *status,
                               cudaStream_t st) {
   *n_tiles = rh_tc_num_tiles(d_R);
+  if (rh_tile_n(d_R) == 256)
+    return launch_t<256, 1>(A, lda, W1t, K, nullptr, 0, M, d_R, K, W2, partial, h_kv, act, status, st);
   return launch_t<128, 1>(A, lda, W1t, K, nullptr, 0, M, d_R, K, W2, partial, h_kv, act, status, st);
 }
 
