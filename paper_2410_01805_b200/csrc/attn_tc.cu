@@ -1,4 +1,5 @@
-// Eq. 1 on tcgen05 tensor cores with TMEM accumulators, head_dim 128.
+// Eq. 1 on tcgen05 tensor cores with TMEM accumulators, head_dim 64, 96 or 128 (tiles are laid
+// out for 128 columns; narrower heads load and multiply only their own columns).
 //
 // One CTA owns two 128-row query tiles that share a KV head (two query heads of one GQA
 // group over the same rows, or two consecutive row blocks of one head) and streams the
@@ -23,7 +24,7 @@ using namespace tc;
 
 constexpr int AT_THREADS = 384;  // 3 warpgroups: softmax 0, softmax 1, {TMA, MMA, 2 idle warps}
 constexpr int TILE = 128;               // query rows per tile and keys per tile
-constexpr int HD = 128;                 // head_dim
+constexpr int HD = 128;                 // column pitch of a head in shared and tensor memory
 constexpr int HALF_BYTES = TILE * 128;  // one 64-column swizzled box of 128 rows: 16 KB
 constexpr int TILE_BYTES = 2 * HALF_BYTES;
 constexpr int AT_SMEM = 1024 + 6 * TILE_BYTES + 256;  // Q0,Q1,K0,K1,V0,V1 + barriers
@@ -62,7 +63,7 @@ __device__ __forceinline__ void setmaxnreg_dec() {
 
 struct AttnParams {
   bf16 *out;
-  int n_tok, h, h_kv, len, pair_heads;
+  int n_tok, h, h_kv, d, len, pair_heads;
   float scale_log2;
   int *status;
 };
@@ -138,21 +139,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   } else if (warp == 8) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      mbar_expect_tx(q_full, 2 * TILE_BYTES);
+      const int nbox = (p.d + 63) / 64;  // 64-column boxes per head vector
+      mbar_expect_tx(q_full, 2 * nbox * HALF_BYTES);
       for (int t = 0; t < 2; t++)
-        for (int hh = 0; hh < 2; hh++)
-          tma_load_2d(sQ + t * TILE_BYTES + hh * HALF_BYTES, &map_q, head[t] * HD + hh * 64, row0[t],
+        for (int hh = 0; hh < nbox; hh++)
+          tma_load_2d(sQ + t * TILE_BYTES + hh * HALF_BYTES, &map_q, head[t] * p.d + hh * 64, row0[t],
                       q_full);
       for (int j = 0; j < NK; j++) {
         const int s = j & 1;
         const uint32_t ph = (j >> 1) & 1;
         if (!mbar_wait(&k_empty[s], ph ^ 1, abort_flag, p.status)) break;
-        mbar_expect_tx(&k_full[s], TILE_BYTES);
-        for (int hh = 0; hh < 2; hh++)
+        mbar_expect_tx(&k_full[s], nbox * HALF_BYTES);
+        for (int hh = 0; hh < nbox; hh++)
           tma_load_3d(sK + s * TILE_BYTES + hh * HALF_BYTES, &map_k, hh * 64, j * TILE, kvh, &k_full[s]);
         if (!mbar_wait(&v_empty[s], ph ^ 1, abort_flag, p.status)) break;
-        mbar_expect_tx(&v_full[s], TILE_BYTES);
-        for (int hh = 0; hh < 2; hh++)
+        mbar_expect_tx(&v_full[s], nbox * HALF_BYTES);
+        for (int hh = 0; hh < nbox; hh++)
           tma_load_3d(sV + s * TILE_BYTES + hh * HALF_BYTES, &map_v, hh * 64, j * TILE, kvh, &v_full[s]);
       }
     }
@@ -160,11 +162,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc_qk = idesc_bf16(TILE, TILE, 0, 0);
-      constexpr uint32_t idesc_pv = idesc_bf16(TILE, HD, 0, 1);
+      const uint32_t idesc_pv = idesc_bf16(TILE, p.d, 0, 1);
+      const int ksteps = p.d / 16;
       auto issue_s = [&](int t, int ks) {
         const unsigned char *q = sQ + t * TILE_BYTES, *k = sK + ks * TILE_BYTES;
-#pragma unroll
-        for (int kk = 0; kk < HD / 16; kk++) {
+#pragma unroll 1
+        for (int kk = 0; kk < ksteps; kk++) {
           const int off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
           mma_ss(tmem_base + t * TILE, desc_kmajor_sw128(q + off), desc_kmajor_sw128(k + off), idesc_qk,
                  kk != 0);
@@ -267,7 +270,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           if (need) { alpha = exp2f(m_used - tmax); m_used = tmax; }
           l *= alpha;
 #pragma unroll 1
-          for (int q = 0; q < 4; q++) {
+          for (int q = 0; q < p.d / 32; q++) {
             uint32_t o[32];
             tmem_ld32(o_addr + q * 32, o);
             tmem_wait_ld();
@@ -315,9 +318,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     tc_fence_after();
     if (ok) {
       const float inv = 1.0f / l;
-      bf16 *dst = p.out + (size_t)row * p.h * HD + (size_t)head[t] * HD;
+      bf16 *dst = p.out + (size_t)row * p.h * p.d + (size_t)head[t] * p.d;
 #pragma unroll 1
-      for (int q = 0; q < 4; q++) {
+      for (int q = 0; q < p.d / 32; q++) {
         uint32_t o[32];
         tmem_ld32(o_addr + q * 32, o);
         tmem_wait_ld();
@@ -348,13 +351,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 }  // namespace
 
 bool attention_tc_supported(int n_tok, int h, int h_kv, int d) {
-  return d == HD && n_tok >= 64 && h % h_kv == 0;
+  return (d == 64 || d == 96 || d == 128) && n_tok >= 64 && h % h_kv == 0;
 }
 
 // map_k / map_v: 3-D maps {d, cap, h_kv} with box {64, 128, 1}; map_q: 2-D {h*d, rows} box {64, 128}.
 cudaError_t launch_attention_tc(const CUtensorMap *map_q, const CUtensorMap *map_k,
-                                const CUtensorMap *map_v, bf16 *out, int n_tok, int h, int h_kv, int len,
-                                int *status, cudaStream_t st) {
+                                const CUtensorMap *map_v, bf16 *out, int n_tok, int h, int h_kv, int d,
+                                int len, int *status, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -363,9 +366,9 @@ cudaError_t launch_attention_tc(const CUtensorMap *map_q, const CUtensorMap *map
     attr_set = true;
   }
   AttnParams p;
-  p.out = out; p.n_tok = n_tok; p.h = h; p.h_kv = h_kv; p.len = len;
+  p.out = out; p.n_tok = n_tok; p.h = h; p.h_kv = h_kv; p.d = d; p.len = len;
   p.pair_heads = ((h / h_kv) % 2 == 0) ? 1 : 0;
-  p.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
+  p.scale_log2 = 1.4426950408889634f / sqrtf((float)d);
   p.status = status;
   const int n_rb = (n_tok + TILE - 1) / TILE;
   const int grid = p.pair_heads ? n_rb * (h / 2) : ((n_rb + 1) / 2) * h;

@@ -239,7 +239,7 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
 
   // tensor maps of the cache for the tcgen05 attention kernel
   L->map_q_base = nullptr;
-  L->tc_attn = L->use_tc && d == 128 &&
+  L->tc_attn = L->use_tc &&
                tmap_encode_3d_bf16(&L->map_k, L->k_rot, d, L->cap, hk, (uint64_t)d * 2,
                                    (uint64_t)L->cap * d * 2, 64, 128, 1) &&
                tmap_encode_3d_bf16(&L->map_v[0], L->v[0], d, L->cap, hk, (uint64_t)d * 2,
@@ -310,7 +310,7 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
     }
     if (tc_ok)
       CK(launch_attention_tc(&L->map_q, &L->map_k, &L->map_v[c], (bf16 *)attn_out, n_tok, L->h, L->h_kv,
-                             L->len, L->d_status, L->st));
+                             L->d, L->len, L->d_status, L->st));
     else
       CK(launch_attention_mma(P->q_rot, L->k_rot, L->v[c], (bf16 *)attn_out, n_tok, L->h, L->h_kv,
                               L->d, L->cap, L->len, L->st));
