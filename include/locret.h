@@ -59,6 +59,8 @@ enum {
   LOCRET_K_RH_REDUCE,   /* (c) sum of the retaining head's partial scores         */
   LOCRET_K_TOPK,        /* (d) per-head selection                                 */
   LOCRET_K_COMPACT,     /* (d) gather / compaction + re-RoPE of kept keys         */
+  LOCRET_K_DEQUANT,     /* 4-bit cache: expansion of the retained units to bf16   */
+  LOCRET_K_QUANT,       /* 4-bit cache: quantisation of the chunk's units         */
   LOCRET_K_COUNT
 };
 
@@ -117,9 +119,10 @@ int locret_cache_len(const locret_layer *layer, int32_t *len);
 
 /*
  * Copy the retained state to HOST buffers (any may be NULL to skip it): K and V as bf16
- * [h_kv × len × d] (K pre-RoPE; for an int4 cache the dequantised values rounded to
- * bf16), scores fp32 [h_kv × len], token_ids int64 [h_kv × len] (index of the token in
- * the stream), *len, *tokens_seen.  Synchronises the stream.
+ * [h_kv × len × d] (K pre-RoPE), scores fp32 [h_kv × len], token_ids int64 [h_kv × len]
+ * (index of the token in the stream), *len, *tokens_seen.  Synchronises the stream.
+ * A layer with a 4-bit cache returns LOCRET_ERR_INVALID if K or V is asked for (its state
+ * is exchanged exactly through locret_export_state_int4).
  */
 int locret_export_state(locret_layer *layer, void *K, void *V, float *scores,
                         int64_t *token_ids, int32_t *len, int64_t *tokens_seen);
@@ -127,11 +130,25 @@ int locret_export_state(locret_layer *layer, void *K, void *V, float *scores,
 /*
  * Replace the retained state from HOST buffers laid out as in locret_export_state
  * (all four required), 0 <= len <= budget + chunk + reserve.  Rebuilds the rotated-key
- * scratch at positions 0..len-1.  For an int4 cache the given K, V are quantised on
- * entry.  Synchronises the stream.
+ * scratch at positions 0..len-1.  LOCRET_ERR_INVALID for a layer with a 4-bit cache.
+ * Synchronises the stream.
  */
 int locret_import_state(locret_layer *layer, const void *K, const void *V, const float *scores,
                         const int64_t *token_ids, int32_t len, int64_t tokens_seen);
+
+/*
+ * The same two calls for a layer created with kv_dtype = 1 (the 4-bit cache that Appendix H
+ * combines with the method): codes uint8 [h_kv × len × d/2], two symmetric 4-bit codes in
+ * [-8, 7] per byte with the even element in the low nibble; scales IEEE half [h_kv × len], one
+ * per head vector (scale = half(absmax / 7), 1 if that is zero; element = code · scale).
+ * HOST buffers; both synchronise the stream.
+ */
+int locret_export_state_int4(locret_layer *layer, void *k_codes, void *k_scales, void *v_codes,
+                             void *v_scales, float *scores, int64_t *token_ids, int32_t *len,
+                             int64_t *tokens_seen);
+int locret_import_state_int4(locret_layer *layer, const void *k_codes, const void *k_scales,
+                             const void *v_codes, const void *v_scales, const float *scores,
+                             const int64_t *token_ids, int32_t len, int64_t tokens_seen);
 
 /* Synchronise the stream; return the sticky device status (0, or LOCRET_ERR_*). */
 int locret_sync_status(locret_layer *layer);

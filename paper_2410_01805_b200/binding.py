@@ -13,7 +13,7 @@ lib_path = os.path.join(_HERE, "liblocret.so")
 
 NO_EVICT = 1
 LAST_CHUNK = 2
-K_NAMES = ["qkv", "rope", "attn", "rh", "rh_reduce", "topk", "compact"]
+K_NAMES = ["qkv", "rope", "attn", "rh", "rh_reduce", "topk", "compact", "dequant", "quant"]
 
 
 class LocretError(RuntimeError):
@@ -47,6 +47,8 @@ def _load():
     l.locret_cache_len.argtypes = [P, C.POINTER(C.c_int32)]
     l.locret_export_state.argtypes = [P, P, P, P, P, C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
     l.locret_import_state.argtypes = [P, P, P, P, P, C.c_int32, C.c_int64]
+    l.locret_export_state_int4.argtypes = [P, P, P, P, P, P, P, C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
+    l.locret_import_state_int4.argtypes = [P, P, P, P, P, P, P, C.c_int32, C.c_int64]
     l.locret_sync_status.argtypes = [P]
     l.locret_reset.argtypes = [P]
     l.locret_set_timing.argtypes = [P, C.c_int32]
@@ -108,8 +110,13 @@ class LocretLayer:
         return n.value
 
     def export_state(self):
-        """dict(K, V [h_kv, len, d] float32 holding bf16 values; S [h_kv, len]; T int64; seen)."""
+        """dict(K, V [h_kv, len, d] float32 holding bf16 values; S [h_kv, len]; T int64; seen).
+
+        For a 4-bit cache: Kc, Vc int8 codes [h_kv, len, d], Ks, Vs float32 scales [h_kv, len],
+        and K, V = codes * scales."""
         n = self.cache_len
+        if self.shape.kv_dtype == 1:
+            return self._export_int4(n)
         K = torch.empty((self.h_kv, n, self.d), dtype=torch.bfloat16)
         V = torch.empty_like(K)
         S = np.empty((self.h_kv, n), dtype=np.float32)
@@ -118,6 +125,40 @@ class LocretLayer:
         _check(lib.locret_export_state(self._h, K.data_ptr(), V.data_ptr(), S.ctypes.data,
                                        T.ctypes.data, C.byref(ln), C.byref(seen)), "locret_export_state")
         return dict(K=K.float().numpy(), V=V.float().numpy(), S=S, T=T, seen=seen.value)
+
+    def _export_int4(self, n):
+        half = self.d // 2
+        kc = np.empty((self.h_kv, n, half), dtype=np.uint8); vc = np.empty_like(kc)
+        ks = np.empty((self.h_kv, n), dtype=np.float16); vs = np.empty_like(ks)
+        S = np.empty((self.h_kv, n), dtype=np.float32)
+        T = np.empty((self.h_kv, n), dtype=np.int64)
+        ln, seen = C.c_int32(), C.c_int64()
+        _check(lib.locret_export_state_int4(self._h, kc.ctypes.data, ks.ctypes.data, vc.ctypes.data,
+                                            vs.ctypes.data, S.ctypes.data, T.ctypes.data,
+                                            C.byref(ln), C.byref(seen)), "locret_export_state_int4")
+
+        def unpack(b):
+            lo = (b & 0xF).astype(np.int8); hi = (b >> 4).astype(np.int8)
+            lo = np.where(lo > 7, lo - 16, lo); hi = np.where(hi > 7, hi - 16, hi)
+            return np.stack([lo, hi], axis=-1).reshape(b.shape[0], b.shape[1], -1).astype(np.int8)
+
+        Kc, Vc = unpack(kc), unpack(vc)
+        Ks, Vs = ks.astype(np.float32), vs.astype(np.float32)
+        return dict(Kc=Kc, Vc=Vc, Ks=Ks, Vs=Vs, K=Kc * Ks[..., None], V=Vc * Vs[..., None],
+                    S=S, T=T, seen=seen.value)
+
+    def import_state_int4(self, Kc, Ks, Vc, Vs, S, T, seen: int):
+        """Codes int8 [h_kv, len, d] in [-8, 7]; scales [h_kv, len] (values exact in fp16)."""
+        def pack(c):
+            c = np.ascontiguousarray(c).astype(np.int16) & 0xF
+            return np.ascontiguousarray((c[..., 0::2] | (c[..., 1::2] << 4)).astype(np.uint8))
+
+        kc, vc = pack(Kc), pack(Vc)
+        ks = np.ascontiguousarray(Ks, dtype=np.float16); vs = np.ascontiguousarray(Vs, dtype=np.float16)
+        Sb = np.ascontiguousarray(S, dtype=np.float32); Tb = np.ascontiguousarray(T, dtype=np.int64)
+        _check(lib.locret_import_state_int4(self._h, kc.ctypes.data, ks.ctypes.data, vc.ctypes.data,
+                                            vs.ctypes.data, Sb.ctypes.data, Tb.ctypes.data,
+                                            kc.shape[1], int(seen)), "locret_import_state_int4")
 
     def import_state(self, K, V, S, T, seen: int):
         Kb = torch.from_numpy(np.ascontiguousarray(K, dtype=np.float32)).to(torch.bfloat16).contiguous()

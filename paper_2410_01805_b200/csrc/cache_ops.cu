@@ -60,7 +60,7 @@ __global__ void rope_append_kernel(RopeAppendArgs a) {
     } else {
       const int m = hd - a.h;
       size_t off = ((size_t)m * a.cap + slot) * a.d + c;
-      *reinterpret_cast<uint4 *>(a.k_pre + off) = self.raw;
+      if (a.k_pre) *reinterpret_cast<uint4 *>(a.k_pre + off) = self.raw;  // null for a 4-bit cache
       *reinterpret_cast<uint4 *>(a.k_rot + off) = rot;
       if (threadIdx.x == 0) a.tid[(size_t)m * a.cap + slot] = a.seen + t;
     }

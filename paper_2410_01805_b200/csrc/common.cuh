@@ -135,6 +135,23 @@ cudaError_t launch_compact(const CompactArgs &a, cudaStream_t st);
 cudaError_t launch_rerope(const bf16 *k_pre, bf16 *k_rot, const float2 *cs, int h_kv, int d, int cap,
                           int len, cudaStream_t st);
 
+// ---- 4-bit cache (int4_cache.cu).  One half of the ping-pong pair:
+struct Int4Half {
+  uint8_t *kq, *vq;  // [h_kv][cap][d/2] two codes per byte, even element in the low nibble
+  __half *ks, *vs;   // [h_kv][cap] one scale per head vector
+};
+// Expand slots [0, len) into bf16: keys rotated at position = slot when `rotate`, values plain.
+cudaError_t launch_dequant(const Int4Half &q, bf16 *k_out, bf16 *v_out, const float2 *cs, int h_kv, int d,
+                           int cap, int len, bool rotate, cudaStream_t st);
+// Quantise n_tok vectors per KV head into slots [slot0, slot0 + n_tok).  Vector (t, m) of K is at
+// k_src + t * tok_stride + m * head_stride (elements), likewise V.
+cudaError_t launch_quantize(const bf16 *k_src, const bf16 *v_src, long long tok_stride,
+                            long long head_stride, const Int4Half &q, int n_tok, int h_kv, int d, int cap,
+                            int slot0, cudaStream_t st);
+cudaError_t launch_compact_int4(const Int4Half &src, const Int4Half &dst, const float *s_src,
+                                const int64_t *t_src, float *s_dst, int64_t *t_dst, const int32_t *keep,
+                                int h_kv, int d, int cap, int budget, cudaStream_t st);
+
 // dst[c][r] = src[r][c]  (weight repack at create)
 cudaError_t launch_transpose_bf16(const bf16 *src, bf16 *dst, int rows, int cols, cudaStream_t st);
 cudaError_t launch_bf16_to_f32(const bf16 *src, float *dst, int n, cudaStream_t st);

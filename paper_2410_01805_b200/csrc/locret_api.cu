@@ -22,8 +22,9 @@ namespace {
 struct ScratchPool {
   cudaStream_t st = nullptr;
   int refs = 0;
-  size_t staging_b = 0, qrot_b = 0, zpost_b = 0, partial_b = 0, keep_b = 0;
+  size_t staging_b = 0, qrot_b = 0, zpost_b = 0, partial_b = 0, keep_b = 0, kexp_b = 0, vexp_b = 0;
   bf16 *staging = nullptr, *q_rot = nullptr, *z_post = nullptr;
+  bf16 *k_exp = nullptr, *v_exp = nullptr;  // 4-bit caches: bf16 expansion of the layer in flight
   float *partial = nullptr;
   int32_t *keep = nullptr;
   struct CsTable { float theta; int d, cap; float2 *ptr; };
@@ -55,7 +56,10 @@ struct locret_layer {
   ScratchPool *pool;
   bf16 *wqkv_t, *w1_t;
   float *w2f;
-  bf16 *k_pre[2], *v[2], *k_rot;
+  bf16 *k_pre[2], *v[2], *k_rot;  // bf16 cache (null for a 4-bit cache)
+  bool int4;
+  Int4Half q4[2];                 // 4-bit cache
+  const void *map_kv_base;
   float *s[2];
   int64_t *tid[2];
   int cur;
@@ -77,7 +81,10 @@ namespace {
 
 void free_layer_memory(locret_layer *L) {
   cudaFree(L->wqkv_t); cudaFree(L->w1_t); cudaFree(L->w2f);
-  for (int i = 0; i < 2; i++) { cudaFree(L->k_pre[i]); cudaFree(L->v[i]); cudaFree(L->s[i]); cudaFree(L->tid[i]); }
+  for (int i = 0; i < 2; i++) {
+    cudaFree(L->k_pre[i]); cudaFree(L->v[i]); cudaFree(L->s[i]); cudaFree(L->tid[i]);
+    cudaFree(L->q4[i].kq); cudaFree(L->q4[i].vq); cudaFree(L->q4[i].ks); cudaFree(L->q4[i].vs);
+  }
   cudaFree(L->k_rot); cudaFree(L->d_status);
   for (auto &e : L->events) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
   cudaGetLastError();
@@ -88,6 +95,7 @@ void release_pool(ScratchPool *p) {
   if (!p) return;
   if (--p->refs > 0) return;
   cudaFree(p->staging); cudaFree(p->q_rot); cudaFree(p->z_post); cudaFree(p->partial); cudaFree(p->keep);
+  cudaFree(p->k_exp); cudaFree(p->v_exp);
   for (auto &t : p->cs) cudaFree(t.ptr);
   g_pools.erase(p->st);
   delete p;
@@ -169,7 +177,7 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   if (d != 64 && d != 96 && d != 128) return LOCRET_ERR_INVALID;
   if (D < 32 || D % 32 != 0 || dR < 8 || dR % 8 != 0) return LOCRET_ERR_INVALID;
   if (cfg->act < 0 || cfg->act > 2 || cfg->rh_input < 0 || cfg->rh_input > 1) return LOCRET_ERR_INVALID;
-  if (cfg->kv_dtype != 0) return LOCRET_ERR_INVALID;
+  if (cfg->kv_dtype != 0 && cfg->kv_dtype != 1) return LOCRET_ERR_INVALID;
   if (!(cfg->rope_theta > 1.0f) || cfg->reserve < 0) return LOCRET_ERR_INVALID;
   if (budget < 1 || chunk < 1 || n_stab < 0 || n_stab > budget) return LOCRET_ERR_INVALID;
   if (!cfg->w_qkv || !cfg->w1 || !cfg->w2) return LOCRET_ERR_INVALID;
@@ -194,7 +202,10 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
     L->use_tc = !(e && e[0] == '1');
   }
 
+  L->int4 = cfg->kv_dtype == 1;
+  L->map_kv_base = nullptr;
   const size_t kv_b = (size_t)hk * L->cap * d * sizeof(bf16);
+  const size_t code_b = (size_t)hk * L->cap * (d / 2), scale_b = (size_t)hk * L->cap * sizeof(__half);
   const size_t sc_b = (size_t)hk * L->cap * sizeof(float);
   const size_t td_b = (size_t)hk * L->cap * sizeof(int64_t);
   bool ok = true;
@@ -202,12 +213,19 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   ok = ok && cudaMalloc(&L->w1_t, (size_t)dR * L->d_in * sizeof(bf16)) == cudaSuccess;
   ok = ok && cudaMalloc(&L->w2f, (size_t)dR * hk * sizeof(float)) == cudaSuccess;
   for (int i = 0; i < 2 && ok; i++) {
-    ok = ok && cudaMalloc(&L->k_pre[i], kv_b) == cudaSuccess;
-    ok = ok && cudaMalloc(&L->v[i], kv_b) == cudaSuccess;
+    if (L->int4) {
+      ok = ok && cudaMalloc(&L->q4[i].kq, code_b) == cudaSuccess;
+      ok = ok && cudaMalloc(&L->q4[i].vq, code_b) == cudaSuccess;
+      ok = ok && cudaMalloc(&L->q4[i].ks, scale_b) == cudaSuccess;
+      ok = ok && cudaMalloc(&L->q4[i].vs, scale_b) == cudaSuccess;
+    } else {
+      ok = ok && cudaMalloc(&L->k_pre[i], kv_b) == cudaSuccess;
+      ok = ok && cudaMalloc(&L->v[i], kv_b) == cudaSuccess;
+    }
     ok = ok && cudaMalloc(&L->s[i], sc_b) == cudaSuccess;
     ok = ok && cudaMalloc(&L->tid[i], td_b) == cudaSuccess;
   }
-  ok = ok && cudaMalloc(&L->k_rot, kv_b) == cudaSuccess;
+  if (!L->int4) ok = ok && cudaMalloc(&L->k_rot, kv_b) == cudaSuccess;
   ok = ok && cudaMalloc(&L->d_status, sizeof(int)) == cudaSuccess;
   if (!ok) { cudaGetLastError(); free_layer_memory(L); delete L; return LOCRET_ERR_ALLOC; }
 
@@ -229,6 +247,14 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
         g = g && grow(&p->partial, &p->partial_b, (size_t)nt * chunk * hk * sizeof(float), L->st);
       }
       g = g && grow(&p->keep, &p->keep_b, (size_t)hk * budget * sizeof(int32_t), L->st);
+      if (L->int4) {
+        const size_t before_k = p->kexp_b, before_v = p->vexp_b;
+        g = g && grow(&p->k_exp, &p->kexp_b, kv_b, L->st);
+        g = g && grow(&p->v_exp, &p->vexp_b, kv_b, L->st);
+        // rows past the live range are multiplied by zero probabilities: they must stay finite
+        if (g && p->kexp_b != before_k) g = cudaMemsetAsync(p->k_exp, 0, p->kexp_b, L->st) == cudaSuccess;
+        if (g && p->vexp_b != before_v) g = cudaMemsetAsync(p->v_exp, 0, p->vexp_b, L->st) == cudaSuccess;
+      }
       if (g) L->cs = get_cs_table(p, cfg->rope_theta, d, L->cap, L->st);
       ok = g && L->cs;
     } else {
@@ -239,13 +265,16 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
 
   // tensor maps of the cache for the tcgen05 attention kernel
   L->map_q_base = nullptr;
-  L->tc_attn = L->use_tc &&
-               tmap_encode_3d_bf16(&L->map_k, L->k_rot, d, L->cap, hk, (uint64_t)d * 2,
-                                   (uint64_t)L->cap * d * 2, 64, 128, 1) &&
-               tmap_encode_3d_bf16(&L->map_v[0], L->v[0], d, L->cap, hk, (uint64_t)d * 2,
-                                   (uint64_t)L->cap * d * 2, 64, 128, 1) &&
-               tmap_encode_3d_bf16(&L->map_v[1], L->v[1], d, L->cap, hk, (uint64_t)d * 2,
-                                   (uint64_t)L->cap * d * 2, 64, 128, 1);
+  if (L->int4)
+    L->tc_attn = L->use_tc;  // maps point at the shared expansion scratch; encoded on first use
+  else
+    L->tc_attn = L->use_tc &&
+                 tmap_encode_3d_bf16(&L->map_k, L->k_rot, d, L->cap, hk, (uint64_t)d * 2,
+                                     (uint64_t)L->cap * d * 2, 64, 128, 1) &&
+                 tmap_encode_3d_bf16(&L->map_v[0], L->v[0], d, L->cap, hk, (uint64_t)d * 2,
+                                     (uint64_t)L->cap * d * 2, 64, 128, 1) &&
+                 tmap_encode_3d_bf16(&L->map_v[1], L->v[1], d, L->cap, hk, (uint64_t)d * 2,
+                                     (uint64_t)L->cap * d * 2, 64, 128, 1);
 
   // repack the weights: K-major copies for both GEMMs, W2 in fp32
   cudaError_t e = cudaSuccess;
@@ -253,12 +282,19 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   if (e == cudaSuccess) e = launch_transpose_bf16((const bf16 *)cfg->w1, L->w1_t, L->d_in, dR, L->st);
   if (e == cudaSuccess) e = launch_bf16_to_f32((const bf16 *)cfg->w2, L->w2f, dR * hk, L->st);
   for (int i = 0; i < 2 && e == cudaSuccess; i++) {
-    e = cudaMemsetAsync(L->k_pre[i], 0, kv_b, L->st);
-    if (e == cudaSuccess) e = cudaMemsetAsync(L->v[i], 0, kv_b, L->st);
+    if (L->int4) {
+      e = cudaMemsetAsync(L->q4[i].kq, 0, code_b, L->st);
+      if (e == cudaSuccess) e = cudaMemsetAsync(L->q4[i].vq, 0, code_b, L->st);
+      if (e == cudaSuccess) e = cudaMemsetAsync(L->q4[i].ks, 0, scale_b, L->st);
+      if (e == cudaSuccess) e = cudaMemsetAsync(L->q4[i].vs, 0, scale_b, L->st);
+    } else {
+      e = cudaMemsetAsync(L->k_pre[i], 0, kv_b, L->st);
+      if (e == cudaSuccess) e = cudaMemsetAsync(L->v[i], 0, kv_b, L->st);
+    }
     if (e == cudaSuccess) e = cudaMemsetAsync(L->s[i], 0, sc_b, L->st);
     if (e == cudaSuccess) e = cudaMemsetAsync(L->tid[i], 0, td_b, L->st);
   }
-  if (e == cudaSuccess) e = cudaMemsetAsync(L->k_rot, 0, kv_b, L->st);
+  if (e == cudaSuccess && !L->int4) e = cudaMemsetAsync(L->k_rot, 0, kv_b, L->st);
   if (e == cudaSuccess) e = cudaMemsetAsync(L->d_status, 0, sizeof(int), L->st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(L->st);
   if (e != cudaSuccess) {
@@ -290,19 +326,39 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
       CK(launch_gemm_bf16((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, P->staging, L->d_in, n_tok,
                           L->d_in, L->D, L->st));
   }
+  // a 4-bit cache is expanded into bf16 scratch first: keys rotated at position = slot
+  bf16 *const k_att = L->int4 ? P->k_exp : L->k_rot;
+  bf16 *const v_att = L->int4 ? P->v_exp : L->v[c];
+  if (L->int4 && L->len > 0) {
+    Timed t(L, LOCRET_K_DEQUANT);
+    CK(launch_dequant(L->q4[c], P->k_exp, P->v_exp, L->cs, L->h_kv, L->d, L->cap, L->len, true, L->st));
+  }
   {  // positions, RoPE, append of the chunk's units at slots [len, len + n_tok)
     Timed t(L, LOCRET_K_ROPE);
     RopeAppendArgs a;
     a.staging = P->staging; a.q_rot = P->q_rot;
     a.z_post = L->cfg.rh_input == 1 ? P->z_post : nullptr;
-    a.k_pre = L->k_pre[c]; a.k_rot = L->k_rot; a.v = L->v[c]; a.tid = L->tid[c]; a.cs = L->cs;
+    a.k_pre = L->int4 ? nullptr : L->k_pre[c]; a.k_rot = k_att; a.v = v_att; a.tid = L->tid[c]; a.cs = L->cs;
     a.n_tok = n_tok; a.h = L->h; a.h_kv = L->h_kv; a.d = L->d; a.cap = L->cap; a.len = L->len;
     a.seen = L->seen;
     CK(launch_rope_append(a, L->st));
   }
+  if (L->int4) {  // the chunk's units enter the cache quantised (keys pre-RoPE)
+    Timed t(L, LOCRET_K_QUANT);
+    const bf16 *ks = P->staging + (size_t)L->h * L->d, *vs = ks + (size_t)L->h_kv * L->d;
+    CK(launch_quantize(ks, vs, L->d_in, L->d, L->q4[c], n_tok, L->h_kv, L->d, L->cap, L->len, L->st));
+  }
   {  // (b) Eq. 1
     Timed t(L, LOCRET_K_ATTN);
     bool tc_ok = L->tc_attn && attention_tc_supported(n_tok, L->h, L->h_kv, L->d);
+    if (tc_ok && L->int4 && L->map_kv_base != P->k_exp) {
+      tc_ok = tmap_encode_3d_bf16(&L->map_k, P->k_exp, L->d, L->cap, L->h_kv, (uint64_t)L->d * 2,
+                                  (uint64_t)L->cap * L->d * 2, 64, 128, 1) &&
+              tmap_encode_3d_bf16(&L->map_v[0], P->v_exp, L->d, L->cap, L->h_kv, (uint64_t)L->d * 2,
+                                  (uint64_t)L->cap * L->d * 2, 64, 128, 1);
+      L->map_v[1] = L->map_v[0];
+      L->map_kv_base = tc_ok ? P->k_exp : nullptr;
+    }
     if (tc_ok && L->map_q_base != P->q_rot) {
       tc_ok = tmap_encode_2d_bf16(&L->map_q, P->q_rot, (uint64_t)L->h * L->d, (uint64_t)L->chunk,
                                   (uint64_t)L->h * L->d * 2, 64, 128);
@@ -312,7 +368,7 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
       CK(launch_attention_tc(&L->map_q, &L->map_k, &L->map_v[c], (bf16 *)attn_out, n_tok, L->h, L->h_kv,
                              L->d, L->len, L->d_status, L->st));
     else
-      CK(launch_attention_mma(P->q_rot, L->k_rot, L->v[c], (bf16 *)attn_out, n_tok, L->h, L->h_kv,
+      CK(launch_attention_mma(P->q_rot, k_att, v_att, (bf16 *)attn_out, n_tok, L->h, L->h_kv,
                               L->d, L->cap, L->len, L->st));
   }
   int n_tiles = 0;
@@ -337,7 +393,11 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
       Timed t(L, LOCRET_K_TOPK);
       CK(launch_topk(L->s[c], L->cap, L->h_kv, n, L->budget, n_prot, P->keep, L->st));
     }
-    {
+    if (L->int4) {
+      Timed t(L, LOCRET_K_COMPACT);
+      CK(launch_compact_int4(L->q4[c], L->q4[c ^ 1], L->s[c], L->tid[c], L->s[c ^ 1], L->tid[c ^ 1],
+                             P->keep, L->h_kv, L->d, L->cap, L->budget, L->st));
+    } else {
       Timed t(L, LOCRET_K_COMPACT);
       CompactArgs a;
       a.k_src = L->k_pre[c]; a.v_src = L->v[c]; a.s_src = L->s[c]; a.t_src = L->tid[c];
@@ -368,6 +428,7 @@ int locret_cache_len(const locret_layer *L, int32_t *len) {
 int locret_export_state(locret_layer *L, void *K, void *V, float *scores, int64_t *token_ids,
                         int32_t *len, int64_t *tokens_seen) {
   if (!L) return LOCRET_ERR_INVALID;
+  if (L->int4 && (K || V)) return LOCRET_ERR_INVALID;  // use locret_export_state_int4
   const int c = L->cur, n = L->len;
   if (len) *len = n;
   if (tokens_seen) *tokens_seen = L->seen;
@@ -389,6 +450,7 @@ int locret_export_state(locret_layer *L, void *K, void *V, float *scores, int64_
 int locret_import_state(locret_layer *L, const void *K, const void *V, const float *scores,
                         const int64_t *token_ids, int32_t len, int64_t tokens_seen) {
   if (!L || len < 0 || len > L->cap || tokens_seen < 0) return LOCRET_ERR_INVALID;
+  if (L->int4) return LOCRET_ERR_INVALID;  // use locret_import_state_int4
   if (len > 0 && (!K || !V || !scores || !token_ids)) return LOCRET_ERR_INVALID;
   const int c = L->cur;
   if (len > 0) {
@@ -401,6 +463,50 @@ int locret_import_state(locret_layer *L, const void *K, const void *V, const flo
                          L->h_kv, cudaMemcpyHostToDevice, L->st));
     L->launches++;
     CK(launch_rerope(L->k_pre[c], L->k_rot, L->cs, L->h_kv, L->d, L->cap, len, L->st));
+  }
+  CK(cudaStreamSynchronize(L->st));
+  L->len = len;
+  L->seen = tokens_seen;
+  return LOCRET_OK;
+}
+
+int locret_export_state_int4(locret_layer *L, void *k_codes, void *k_scales, void *v_codes,
+                             void *v_scales, float *scores, int64_t *token_ids, int32_t *len,
+                             int64_t *tokens_seen) {
+  if (!L || !L->int4) return LOCRET_ERR_INVALID;
+  const int c = L->cur, n = L->len;
+  if (len) *len = n;
+  if (tokens_seen) *tokens_seen = L->seen;
+  if (n > 0) {
+    const size_t crow = (size_t)n * (L->d / 2), cpitch = (size_t)L->cap * (L->d / 2);
+    const Int4Half &q = L->q4[c];
+    if (k_codes) CK(cudaMemcpy2DAsync(k_codes, crow, q.kq, cpitch, crow, L->h_kv, cudaMemcpyDeviceToHost, L->st));
+    if (v_codes) CK(cudaMemcpy2DAsync(v_codes, crow, q.vq, cpitch, crow, L->h_kv, cudaMemcpyDeviceToHost, L->st));
+    if (k_scales) CK(cudaMemcpy2DAsync(k_scales, (size_t)n * 2, q.ks, (size_t)L->cap * 2, (size_t)n * 2, L->h_kv, cudaMemcpyDeviceToHost, L->st));
+    if (v_scales) CK(cudaMemcpy2DAsync(v_scales, (size_t)n * 2, q.vs, (size_t)L->cap * 2, (size_t)n * 2, L->h_kv, cudaMemcpyDeviceToHost, L->st));
+    if (scores) CK(cudaMemcpy2DAsync(scores, (size_t)n * 4, L->s[c], (size_t)L->cap * 4, (size_t)n * 4, L->h_kv, cudaMemcpyDeviceToHost, L->st));
+    if (token_ids) CK(cudaMemcpy2DAsync(token_ids, (size_t)n * 8, L->tid[c], (size_t)L->cap * 8, (size_t)n * 8, L->h_kv, cudaMemcpyDeviceToHost, L->st));
+  }
+  CK(cudaStreamSynchronize(L->st));
+  return LOCRET_OK;
+}
+
+int locret_import_state_int4(locret_layer *L, const void *k_codes, const void *k_scales,
+                             const void *v_codes, const void *v_scales, const float *scores,
+                             const int64_t *token_ids, int32_t len, int64_t tokens_seen) {
+  if (!L || !L->int4 || len < 0 || len > L->cap || tokens_seen < 0) return LOCRET_ERR_INVALID;
+  if (len > 0 && (!k_codes || !k_scales || !v_codes || !v_scales || !scores || !token_ids))
+    return LOCRET_ERR_INVALID;
+  const int c = L->cur;
+  if (len > 0) {
+    const size_t crow = (size_t)len * (L->d / 2), cpitch = (size_t)L->cap * (L->d / 2);
+    const Int4Half &q = L->q4[c];
+    CK(cudaMemcpy2DAsync(q.kq, cpitch, k_codes, crow, crow, L->h_kv, cudaMemcpyHostToDevice, L->st));
+    CK(cudaMemcpy2DAsync(q.vq, cpitch, v_codes, crow, crow, L->h_kv, cudaMemcpyHostToDevice, L->st));
+    CK(cudaMemcpy2DAsync(q.ks, (size_t)L->cap * 2, k_scales, (size_t)len * 2, (size_t)len * 2, L->h_kv, cudaMemcpyHostToDevice, L->st));
+    CK(cudaMemcpy2DAsync(q.vs, (size_t)L->cap * 2, v_scales, (size_t)len * 2, (size_t)len * 2, L->h_kv, cudaMemcpyHostToDevice, L->st));
+    CK(cudaMemcpy2DAsync(L->s[c], (size_t)L->cap * 4, scores, (size_t)len * 4, (size_t)len * 4, L->h_kv, cudaMemcpyHostToDevice, L->st));
+    CK(cudaMemcpy2DAsync(L->tid[c], (size_t)L->cap * 8, token_ids, (size_t)len * 8, (size_t)len * 8, L->h_kv, cudaMemcpyHostToDevice, L->st));
   }
   CK(cudaStreamSynchronize(L->st));
   L->len = len;

@@ -82,6 +82,13 @@ def check_keep_band(kept_slots, s_ref, budget, n_prot, oracle_keep, what=""):
     return exact
 
 
+def import_oracle_state(gpu, st, int4: bool):
+    if int4:
+        gpu.import_state_int4(st["Kc"], st["Ks"], st["Vc"], st["Vs"], st["S"], st["T"], st["seen"])
+    else:
+        gpu.import_state(st["K"], st["V"], st["S"], st["T"], st["seen"])
+
+
 def lockstep_chunk(ora, gpu, x: np.ndarray, flags: int = 0, rows=None, what=""):
     """Import the oracle's state, run one chunk on both, compare everything.  Advances the oracle."""
     shape = ora.s
@@ -94,12 +101,13 @@ def lockstep_chunk(ora, gpu, x: np.ndarray, flags: int = 0, rows=None, what=""):
     out_b = torch.zeros_like(out_a)
 
     # pass 1: append only, to read the chunk's K, V and scores before compaction
-    gpu.import_state(st["K"], st["V"], st["S"], st["T"], st["seen"])
+    int4 = bool(ora.int4)
+    import_oracle_state(gpu, st, int4)
     gpu.prefill_chunk(xd, out_a, O.NO_EVICT)
     pre = gpu.export_state()
     assert gpu.sync_status() == 0
     # pass 2: the step as asked
-    gpu.import_state(st["K"], st["V"], st["S"], st["T"], st["seen"])
+    import_oracle_state(gpu, st, int4)
     gpu.prefill_chunk(xd, out_b, flags)
     post = gpu.export_state()
     assert gpu.sync_status() == 0
@@ -114,12 +122,25 @@ def lockstep_chunk(ora, gpu, x: np.ndarray, flags: int = 0, rows=None, what=""):
     assert pre["K"].shape[1] == n and pre["seen"] == st["seen"] + n_tok
     # imported part untouched, token ids appended
     assert np.array_equal(pre["K"][:, :ln], st["K"].astype(np.float32))
+    state_keys = ("Kc", "Vc", "Ks", "Vs") if int4 else ("K", "V")
     assert np.array_equal(pre["T"][:, ln:], np.broadcast_to(st["seen"] + np.arange(n_tok), (hk, n_tok)))
     # chunk K, V as stored (bf16 of fp32 accumulation vs bf16 of fp64: rare one-ulp flips allowed)
     qkv = O.round_bf16(O.project_qkv(x, ora.w_qkv, h, hk, d))
     _, Kc, Vc = O.split_qkv(qkv, h, hk, d)
-    for name, got, ref in (("K", pre["K"][:, ln:], np.transpose(Kc, (1, 0, 2))),
-                           ("V", pre["V"][:, ln:], np.transpose(Vc, (1, 0, 2)))):
+    if int4:
+        # the chunk's units are stored quantised; a one-ulp difference in a staged bf16 value can
+        # move a code by one step (or the scale by one fp16 ulp when it hits the absmax element)
+        for name, src in (("K", Kc), ("V", Vc)):
+            codes, scale = O.quantize_int4(np.transpose(src, (1, 0, 2)))
+            got_c, got_s = pre[name + "c"][:, ln:], pre[name + "s"][:, ln:]
+            assert np.array_equal(pre[name + "c"][:, :ln], st[name + "c"]), f"{what}: imported {name} codes changed"
+            assert np.array_equal(pre[name + "s"][:, :ln], st[name + "s"].astype(np.float32))
+            assert np.mean(got_s != scale.astype(np.float32)) < 0.01, f"{what}: {name} scales differ"
+            assert np.mean(got_c != codes) < 0.01, f"{what}: {name} codes differ"
+            deq_err = np.abs(got_c * got_s[..., None] - codes * scale[..., None])
+            assert np.all(deq_err <= 1.001 * np.maximum(got_s, scale)[..., None]), f"{what}: {name} off by more than a step"
+    for name, got, ref in (() if int4 else (("K", pre["K"][:, ln:], np.transpose(Kc, (1, 0, 2))),
+                                            ("V", pre["V"][:, ln:], np.transpose(Vc, (1, 0, 2))))):
         diff = np.abs(got - ref)
         # one bf16 ulp of the value, plus the absolute error of an fp32 accumulation (matters
         # only for results that cancel to nearly zero)
@@ -139,12 +160,12 @@ def lockstep_chunk(ora, gpu, x: np.ndarray, flags: int = 0, rows=None, what=""):
             assert np.all(np.diff(pos) > 0), f"{what}: temporal order lost"
             exact &= check_keep_band(pos, s_ref[m], ora.budget, n_prot, ora.last_keep[m], f"{what} head {m}")
             # compaction is a bit-exact gather of the pre-compaction arrays
-            assert np.array_equal(post["K"][m], pre["K"][m][pos])
-            assert np.array_equal(post["V"][m], pre["V"][m][pos])
+            for key in state_keys:
+                assert np.array_equal(post[key][m], pre[key][m][pos]), f"{what}: {key} not a bit-exact gather"
             assert np.array_equal(post["S"][m].view(np.uint32), pre["S"][m][pos].view(np.uint32))
         stats["sets_identical"] = exact
     else:
-        for key in ("K", "V", "T"):
+        for key in state_keys + ("T",):
             assert np.array_equal(post[key], pre[key])
     assert gpu.cache_len == ora.len
     return stats

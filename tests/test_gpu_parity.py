@@ -133,6 +133,26 @@ def test_no_stabilizers_and_other_activations():
         gpu.destroy()
 
 
+@pytest.mark.parametrize("d,heads", [(128, (8, 2)), (96, (3, 3)), (64, (4, 1))])
+def test_int4_cache_lockstep(d, heads):
+    """4-bit cache: quantise on append, attention over the dequantised units, codes move unchanged."""
+    from parity_util import lockstep_chunk, make_pair
+    sh = small_shape(h=heads[0], hk=heads[1], d=d, D=128, dR=64, rope_theta=500000.0, kv_dtype=1)
+    ora, gpu = make_pair(sh, weights_for(sh, 40 + d), budget=300, chunk=160, n_stab=50, reserve=16)
+    for i, n_tok in enumerate([160, 160, 77, 160, 1, 130]):
+        x = hidden(n_tok, sh.d_model, seed=300 + i)
+        if i == 3:
+            x[[7, 90]] = W.to_bf16_grid(x[[7, 90]] * 5.0)
+        lockstep_chunk(ora, gpu, x, 0, what=f"int4 d{d} chunk {i}")
+    lockstep_chunk(ora, gpu, hidden(10, sh.d_model, 399), O.NO_EVICT, what="int4 tail")
+    # the generic exchange refuses a 4-bit layer
+    import paper_2410_01805_b200 as P
+    buf = np.zeros(8, dtype=np.float32)
+    assert P.lib.locret_import_state(gpu._h, buf.ctypes.data, buf.ctypes.data, buf.ctypes.data,
+                                     buf.ctypes.data, 1, 1) == -1
+    gpu.destroy()
+
+
 def test_selection_with_ties_nan_and_signed_zero():
     """Crafted imported scores put the cut inside a group of equal scores: ties prefer the
     recent unit, NaN ranks with -inf, -0 equals +0."""
