@@ -101,7 +101,8 @@ def rope(x, pos, theta: float):
     return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
 
 
-def attention_rows(Qr, Kr_cache, V_cache, Kr_chunk, V_chunk, group: int, rows=None, abs_out=None):
+def attention_rows(Qr, Kr_cache, V_cache, Kr_chunk, V_chunk, group: int, rows=None, abs_out=None,
+                   flip_sens=None):
     """Eq. 1 for the chunk's query rows.
 
     Qr [n, h, d] (roped); Kr_cache/V_cache [h_kv, len, d]; Kr_chunk/V_chunk [n, h_kv, d].
@@ -109,6 +110,9 @@ def attention_rows(Qr, Kr_cache, V_cache, Kr_chunk, V_chunk, group: int, rows=No
     Returns out [n, h*d]; rows not listed in `rows` are NaN.
     If `abs_out` (same shape) is given it receives sum_i p_i |V_i|, the magnitude of the
     terms the output sums, which error bounds of reduced-precision kernels scale with.
+    If `flip_sens` (same shape) is given it receives the first-order change of the output when
+    every key has one stored element moved by one bf16 ulp at its most influential position:
+    sum_i p_i delta_i |V_i - out|, delta_i = 2^-7 max_c |q_c k_ic| / sqrt(d).
     """
     n, h, d = Qr.shape
     ln = Kr_cache.shape[1]
@@ -129,6 +133,11 @@ def attention_rows(Qr, Kr_cache, V_cache, Kr_chunk, V_chunk, group: int, rows=No
         out[rows, j * d:(j + 1) * d] = p @ Vall
         if abs_out is not None:
             abs_out[rows, j * d:(j + 1) * d] = p @ np.abs(Vall)
+        if flip_sens is not None:
+            o = out[rows, j * d:(j + 1) * d]
+            for a, t in enumerate(rows):
+                delta = 2.0 ** -7 * np.max(np.abs(Qr[t, j, :][None, :] * Kall), axis=1) * scale
+                flip_sens[t, j * d:(j + 1) * d] = (p[a] * delta) @ np.abs(Vall - o[a][None, :])
     return out
 
 
@@ -225,6 +234,7 @@ class OracleLayer:
         self.last_scores = None
         self.last_keep = None
         self.last_abs_out = None
+        self.last_flip_sens = None
 
     @property
     def len(self) -> int:
@@ -273,7 +283,9 @@ class OracleLayer:
 
         # (b) Eq. 1
         self.last_abs_out = np.full((n_tok, h * d), np.nan)
-        out = attention_rows(Qr, Kr_cache, V_cache, Kr_chunk, V, g, rows, self.last_abs_out)
+        self.last_flip_sens = np.full((n_tok, h * d), np.nan) if self.mirror else None
+        out = attention_rows(Qr, Kr_cache, V_cache, Kr_chunk, V, g, rows, self.last_abs_out,
+                             self.last_flip_sens)
 
         # (c) retaining head on the token's concatenated [Q ‖ K ‖ V]
         if self.s.rh_input == 0:

@@ -1,0 +1,75 @@
+"""Parity at the benchmark's full layer shapes and launch configuration.
+
+Full-size chunks (the sizes bench.py times) are run in lock-step with the oracle; attention
+is compared on sampled query rows (the oracle computes those rows one by one), scores on every
+token, the kept set by the band rule, compaction bit-exactly.
+"""
+
+import numpy as np
+import pytest
+
+import workloads as W
+from oracle import locret_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+
+def sampled_rows(n_tok, seed):
+    g = np.random.default_rng(seed)
+    rows = set(g.integers(0, n_tok, size=6).tolist()) | {0, n_tok - 1, min(127, n_tok - 1), min(128, n_tok - 1)}
+    return sorted(rows)
+
+
+def run_workload_chunks(name, n_chunks, layer=0, extra_rows=()):
+    from parity_util import lockstep_chunk, make_pair
+    w = W.get_workload(name)
+    ora, gpu = make_pair(w.shape, W.layer_weights(w.shape, layer), w.budget, w.chunk, w.n_stab)
+    start, stats = 0, []
+    for i, n_tok in enumerate(w.chunk_sizes()[:n_chunks]):
+        x = W.hidden_states(w, start, n_tok)
+        rows = sampled_rows(n_tok, i)
+        # always include the outlier tokens of the chunk: they are the ill-conditioned rows
+        norms = np.linalg.norm(x, axis=1)
+        rows = sorted(set(rows) | set(np.flatnonzero(norms > 5 * np.median(norms)).tolist()[:4]) | set(extra_rows))
+        stats.append(lockstep_chunk(ora, gpu, x, 0, rows=rows, what=f"{name} chunk {i}"))
+        start += n_tok
+    assert gpu.sync_status() == 0
+    gpu.destroy()
+    return w, ora, stats
+
+
+def test_c3_llama_shape_first_chunks_through_steady_state():
+    w, ora, stats = run_workload_chunks("c3_llama_128k", 4)
+    assert ora.len == w.budget
+    assert all("sets_identical" in s for s in stats[1:])
+
+
+def test_c2_llama_shape_small_stabilizer_window():
+    w, ora, stats = run_workload_chunks("c2_llama_32k", 3, layer=31)
+    assert ora.len == w.budget
+
+
+def test_c5_llama_shape_int4_cache():
+    w, ora, stats = run_workload_chunks("c5_llama_stream_int4", 3)
+    assert ora.len == w.budget and ora.int4
+
+
+def test_c4_phi3_shape_until_the_cache_is_full():
+    # 16 chunks fill the 16384-unit budget; chunks 17 and 18 evict
+    w, ora, stats = run_workload_chunks("c4_phi3_128k", 18)
+    assert ora.len == w.budget and "sets_identical" in stats[-1]
+
+
+def test_partial_last_chunk_of_the_headline_run():
+    """The 128K run ends with a 2048-token chunk (shorter than the 2500 stabilizers)."""
+    from parity_util import lockstep_chunk, make_pair
+    w = W.get_workload("c3_llama_128k")
+    ora, gpu = make_pair(w.shape, W.layer_weights(w.shape, 0), w.budget, w.chunk, w.n_stab)
+    start = 0
+    for i, n_tok in enumerate([3072, 3072, 2048]):
+        x = W.hidden_states(w, start, n_tok)
+        st = lockstep_chunk(ora, gpu, x, 0, rows=sampled_rows(n_tok, 50 + i), what=f"tail chunk {i}")
+        start += n_tok
+    # Algorithm 1's reading: the protected units are the last 2500 entries of cache + chunk
+    assert set(range(start - w.n_stab, start)) <= set(ora.T[0])
+    gpu.destroy()
