@@ -159,6 +159,24 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
+# ----------------------------------------------------------------------------- multi-rank bookkeeping
+
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def job_throughput(world: int, tokens_per_rank: int, ms: float) -> float:
+    """Replicas only: every rank prefills its own request; whole-job tokens over the slowest rank's time."""
+    return world * tokens_per_rank / (ms * 1e-3)
+
+
 # ----------------------------------------------------------------------------- our arm
 
 def run_ours(args, w):
@@ -259,12 +277,9 @@ def run_ours(args, w):
     barrier()
 
     t_ms = float(np.mean(ms)); t_e2e = float(np.mean(ms_e2e))
-    if world > 1:
-        tt = torch.tensor([t_ms, t_e2e], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        t_ms, t_e2e = tt.tolist()
-    value = world * w.context / (t_ms * 1e-3)
-    e2e = world * w.context / (t_e2e * 1e-3)
+    t_ms, t_e2e = max_over_ranks([t_ms, t_e2e], dev)
+    value = job_throughput(world, w.context, t_ms)
+    e2e = job_throughput(world, w.context, t_e2e)
 
     # ---- roofline of the dominant kernel (attention: a dense contraction -> tensor peak)
     fl = step_flops(w) * args.steps                       # [qkv, attn, rh] flops over the timed region
