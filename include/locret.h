@@ -23,8 +23,12 @@
  *     passes; the library owns the cache, scores, token ids, scratch and its own
  *     repacked copy of the weights (taken at create; the caller's weights may be
  *     freed afterwards).
- *   - All device work of a layer is enqueued on the stream given at create, without
- *     host synchronisation unless stated.  A handle is bound to that stream and is
+ *   - All device work of a layer is enqueued without host synchronisation unless stated:
+ *     projection, RoPE/append and attention (everything attn_out depends on) on the stream
+ *     given at create; the retaining head, selection and compaction, which nothing downstream
+ *     in a decoder layer waits for, on a second stream owned by the library, ordered against
+ *     the first by events (set LOCRET_SERIAL=1 to keep everything on one stream).  Every call
+ *     that reads or replaces state waits for both.  A handle is bound to its stream and is
  *     not thread-safe.  Layers created on the same stream share scratch.
  *   - There is no CPU fallback: without a CUDA device every call that needs one
  *     returns LOCRET_ERR_CUDA.

@@ -22,8 +22,14 @@ namespace {
 struct ScratchPool {
   cudaStream_t st = nullptr;
   int refs = 0;
-  size_t staging_b = 0, qrot_b = 0, zpost_b = 0, partial_b = 0, keep_b = 0, kexp_b = 0, vexp_b = 0;
-  bf16 *staging = nullptr, *q_rot = nullptr, *z_post = nullptr;
+  // Second stream for the work that is off the critical path of a decoder layer (retaining
+  // head, selection, compaction): it overlaps the tail of the attention kernel and the next
+  // layer's projection.  staging / z_post are double-buffered because that work reads them.
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_stage_free[2] = {nullptr, nullptr};
+  int flip = 0;
+  size_t staging_b[2] = {0, 0}, qrot_b = 0, zpost_b[2] = {0, 0}, partial_b = 0, keep_b = 0, kexp_b = 0, vexp_b = 0;
+  bf16 *staging[2] = {nullptr, nullptr}, *q_rot = nullptr, *z_post[2] = {nullptr, nullptr};
   bf16 *k_exp = nullptr, *v_exp = nullptr;  // 4-bit caches: bf16 expansion of the layer in flight
   float *partial = nullptr;
   int32_t *keep = nullptr;
@@ -70,6 +76,9 @@ struct locret_layer {
   int64_t launches;
   bool timing;
   bool use_tc;  // tcgen05 kernels (default); LOCRET_LEGACY_MMA=1 keeps the mma.sync kernels for A/B runs
+  bool use_side;  // off-critical-path kernels go to the pool's second stream (LOCRET_SERIAL=1 disables)
+  bool side_pending;
+  cudaEvent_t ev_ready, ev_attn, ev_side;
   bool tc_attn;  // tensor maps for the tcgen05 attention kernel are valid
   CUtensorMap map_k, map_v[2], map_q;
   const void *map_q_base;
@@ -87,6 +96,9 @@ void free_layer_memory(locret_layer *L) {
   }
   cudaFree(L->k_rot); cudaFree(L->d_status);
   for (auto &e : L->events) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
+  if (L->ev_ready) cudaEventDestroy(L->ev_ready);
+  if (L->ev_attn) cudaEventDestroy(L->ev_attn);
+  if (L->ev_side) cudaEventDestroy(L->ev_side);
   cudaGetLastError();
 }
 
@@ -94,7 +106,12 @@ void release_pool(ScratchPool *p) {
   std::lock_guard<std::mutex> lk(g_mu);
   if (!p) return;
   if (--p->refs > 0) return;
-  cudaFree(p->staging); cudaFree(p->q_rot); cudaFree(p->z_post); cudaFree(p->partial); cudaFree(p->keep);
+  if (p->side) { cudaStreamSynchronize(p->side); cudaStreamDestroy(p->side); }
+  for (int i = 0; i < 2; i++) {
+    cudaFree(p->staging[i]); cudaFree(p->z_post[i]);
+    if (p->ev_stage_free[i]) cudaEventDestroy(p->ev_stage_free[i]);
+  }
+  cudaFree(p->q_rot); cudaFree(p->partial); cudaFree(p->keep);
   cudaFree(p->k_exp); cudaFree(p->v_exp);
   for (auto &t : p->cs) cudaFree(t.ptr);
   g_pools.erase(p->st);
@@ -126,8 +143,8 @@ const float2 *get_cs_table(ScratchPool *p, float theta, int d, int cap, cudaStre
 
 // Bracket one launch with events when timing is on; count it.
 struct Timed {
-  locret_layer *L; int kind; TimedEvent *ev = nullptr;
-  Timed(locret_layer *l, int k) : L(l), kind(k) {
+  locret_layer *L; int kind; cudaStream_t st; TimedEvent *ev = nullptr;
+  Timed(locret_layer *l, int k, cudaStream_t stream = nullptr) : L(l), kind(k), st(stream ? stream : l->st) {
     L->launches++;
     if (!L->timing) return;
     if (L->events_used == L->events.size()) {
@@ -137,9 +154,9 @@ struct Timed {
     }
     ev = &L->events[L->events_used++];
     ev->kind = k;
-    cudaEventRecord(ev->a, L->st);
+    cudaEventRecord(ev->a, st);
   }
-  ~Timed() { if (ev) cudaEventRecord(ev->b, L->st); }
+  ~Timed() { if (ev) cudaEventRecord(ev->b, st); }
 };
 
 #define CK(call)                                         \
@@ -149,6 +166,13 @@ struct Timed {
   } while (0)
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Wait for everything this layer has in flight, on both streams.
+cudaError_t sync_all(locret_layer *L) {
+  cudaError_t e = cudaStreamSynchronize(L->st);
+  if (e == cudaSuccess && L->use_side && L->pool && L->pool->side) e = cudaStreamSynchronize(L->pool->side);
+  return e;
+}
 
 }  // namespace
 
@@ -200,6 +224,10 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   {
     const char *e = getenv("LOCRET_LEGACY_MMA");
     L->use_tc = !(e && e[0] == '1');
+    const char *ser = getenv("LOCRET_SERIAL");
+    L->use_side = !(ser && ser[0] == '1');
+    L->side_pending = false;
+    L->ev_ready = L->ev_attn = L->ev_side = nullptr;
   }
 
   L->int4 = cfg->kv_dtype == 1;
@@ -238,10 +266,20 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
       p->refs++;
       L->pool = p;
       bool g = true;
-      g = g && grow(&p->staging, &p->staging_b, (size_t)chunk * L->d_in * sizeof(bf16), L->st);
+      if (L->use_side && !p->side) {
+        int lo = 0, hi = 0;
+        cudaDeviceGetStreamPriorityRange(&lo, &hi);
+        g = g && cudaStreamCreateWithPriority(&p->side, cudaStreamNonBlocking, lo) == cudaSuccess;
+        for (int i = 0; i < 2 && g; i++)
+          g = cudaEventCreateWithFlags(&p->ev_stage_free[i], cudaEventDisableTiming) == cudaSuccess;
+      }
+      if (p->side) cudaStreamSynchronize(p->side);  // buffers may be replaced below
+      for (int i = 0; i < 2; i++) {
+        g = g && grow(&p->staging[i], &p->staging_b[i], (size_t)chunk * L->d_in * sizeof(bf16), L->st);
+        if (cfg->rh_input == 1)
+          g = g && grow(&p->z_post[i], &p->zpost_b[i], (size_t)chunk * L->d_in * sizeof(bf16), L->st);
+      }
       g = g && grow(&p->q_rot, &p->qrot_b, (size_t)chunk * h * d * sizeof(bf16), L->st);
-      if (cfg->rh_input == 1)
-        g = g && grow(&p->z_post, &p->zpost_b, (size_t)chunk * L->d_in * sizeof(bf16), L->st);
       {
         int nt = rh_num_tiles(dR) > rh_tc_num_tiles(dR) ? rh_num_tiles(dR) : rh_tc_num_tiles(dR);
         g = g && grow(&p->partial, &p->partial_b, (size_t)nt * chunk * hk * sizeof(float), L->st);
@@ -262,6 +300,13 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
     }
   }
   if (!ok) { ScratchPool *p = L->pool; free_layer_memory(L); delete L; release_pool(p); return LOCRET_ERR_ALLOC; }
+
+  if (L->use_side) {
+    ok = cudaEventCreateWithFlags(&L->ev_ready, cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&L->ev_attn, cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&L->ev_side, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); ScratchPool *p = L->pool; free_layer_memory(L); delete L; release_pool(p); return LOCRET_ERR_CUDA; }
+  }
 
   // tensor maps of the cache for the tcgen05 attention kernel
   L->map_q_base = nullptr;
@@ -316,14 +361,26 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
   if (n > L->cap) return LOCRET_ERR_CAPACITY;
   ScratchPool *P = L->pool;
   const int c = L->cur;
+  const bool side = L->use_side;
+  cudaStream_t S = side ? P->side : L->st;  // stream of the off-critical-path kernels
+  const int sb = P->flip;                    // staging buffer of this call
+  P->flip ^= 1;
+  bf16 *const staging = P->staging[sb];
+  bf16 *const z_post = P->z_post[sb];
+  if (side) {
+    // the staging buffer is free once the retaining head that last read it has run, and this
+    // layer's cache once its previous selection / compaction has finished
+    CK(cudaStreamWaitEvent(L->st, P->ev_stage_free[sb], 0));
+    if (L->side_pending) CK(cudaStreamWaitEvent(L->st, L->ev_side, 0));
+  }
 
   {  // (a) projections
     Timed t(L, LOCRET_K_QKV);
     if (L->use_tc && n_tok >= 32 && gemm_tc_supported(n_tok, L->d_in, L->D, L->D, L->D))
-      CK(launch_gemm_tc((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, P->staging, L->d_in, n_tok,
+      CK(launch_gemm_tc((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, staging, L->d_in, n_tok,
                         L->d_in, L->D, L->d_status, L->st));
     else
-      CK(launch_gemm_bf16((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, P->staging, L->d_in, n_tok,
+      CK(launch_gemm_bf16((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, staging, L->d_in, n_tok,
                           L->d_in, L->D, L->st));
   }
   // a 4-bit cache is expanded into bf16 scratch first: keys rotated at position = slot
@@ -336,8 +393,8 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
   {  // positions, RoPE, append of the chunk's units at slots [len, len + n_tok)
     Timed t(L, LOCRET_K_ROPE);
     RopeAppendArgs a;
-    a.staging = P->staging; a.q_rot = P->q_rot;
-    a.z_post = L->cfg.rh_input == 1 ? P->z_post : nullptr;
+    a.staging = staging; a.q_rot = P->q_rot;
+    a.z_post = L->cfg.rh_input == 1 ? z_post : nullptr;
     a.k_pre = L->int4 ? nullptr : L->k_pre[c]; a.k_rot = k_att; a.v = v_att; a.tid = L->tid[c]; a.cs = L->cs;
     a.n_tok = n_tok; a.h = L->h; a.h_kv = L->h_kv; a.d = L->d; a.cap = L->cap; a.len = L->len;
     a.seen = L->seen;
@@ -345,9 +402,10 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
   }
   if (L->int4) {  // the chunk's units enter the cache quantised (keys pre-RoPE)
     Timed t(L, LOCRET_K_QUANT);
-    const bf16 *ks = P->staging + (size_t)L->h * L->d, *vs = ks + (size_t)L->h_kv * L->d;
+    const bf16 *ks = staging + (size_t)L->h * L->d, *vs = ks + (size_t)L->h_kv * L->d;
     CK(launch_quantize(ks, vs, L->d_in, L->d, L->q4[c], n_tok, L->h_kv, L->d, L->cap, L->len, L->st));
   }
+  if (side) CK(cudaEventRecord(L->ev_ready, L->st));
   {  // (b) Eq. 1
     Timed t(L, LOCRET_K_ATTN);
     bool tc_ok = L->tc_attn && attention_tc_supported(n_tok, L->h, L->h_kv, L->d);
@@ -371,45 +429,56 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
       CK(launch_attention_mma(P->q_rot, k_att, v_att, (bf16 *)attn_out, n_tok, L->h, L->h_kv,
                               L->d, L->cap, L->len, L->st));
   }
+  if (side) {
+    CK(cudaEventRecord(L->ev_attn, L->st));
+    CK(cudaStreamWaitEvent(S, L->ev_ready, 0));
+  }
   int n_tiles = 0;
-  {  // (c) retaining head
-    Timed t(L, LOCRET_K_RH);
-    const bf16 *z = L->cfg.rh_input == 1 ? P->z_post : P->staging;
+  {  // (c) retaining head: launched after the attention kernel, so its CTAs fill that kernel's tail
+    Timed t(L, LOCRET_K_RH, S);
+    const bf16 *z = L->cfg.rh_input == 1 ? z_post : staging;
     if (L->use_tc && n_tok >= 32 && gemm_tc_supported(n_tok, L->d_R, L->d_in, L->d_in, L->d_in))
       CK(launch_rh_gemm_tc(z, L->d_in, L->w1_t, L->w2f, P->partial, n_tok, L->d_R, L->d_in, L->h_kv,
-                           L->cfg.act, &n_tiles, L->d_status, L->st));
+                           L->cfg.act, &n_tiles, L->d_status, S));
     else
       CK(launch_rh_gemm(z, L->d_in, L->w1_t, L->w2f, P->partial, n_tok, L->d_R, L->d_in, L->h_kv,
-                        L->cfg.act, &n_tiles, L->st));
+                        L->cfg.act, &n_tiles, S));
   }
   {
-    Timed t(L, LOCRET_K_RH_REDUCE);
-    CK(launch_rh_reduce(P->partial, n_tiles, n_tok, L->h_kv, L->s[c], L->cap, L->len, L->st));
+    Timed t(L, LOCRET_K_RH_REDUCE, S);
+    CK(launch_rh_reduce(P->partial, n_tiles, n_tok, L->h_kv, L->s[c], L->cap, L->len, S));
   }
+  if (side) CK(cudaEventRecord(P->ev_stage_free[sb], S));
   // (d) protect, top-b, gather
   if (!(flags & LOCRET_NO_EVICT) && n > L->budget) {
     const int n_prot = (flags & LOCRET_LAST_CHUNK) ? 0 : (L->n_stab < n ? L->n_stab : n);
     {
-      Timed t(L, LOCRET_K_TOPK);
-      CK(launch_topk(L->s[c], L->cap, L->h_kv, n, L->budget, n_prot, P->keep, L->st));
+      Timed t(L, LOCRET_K_TOPK, S);
+      CK(launch_topk(L->s[c], L->cap, L->h_kv, n, L->budget, n_prot, P->keep, S));
     }
+    // compaction rewrites the rotated keys the attention kernel reads
+    if (side) CK(cudaStreamWaitEvent(S, L->ev_attn, 0));
     if (L->int4) {
-      Timed t(L, LOCRET_K_COMPACT);
+      Timed t(L, LOCRET_K_COMPACT, S);
       CK(launch_compact_int4(L->q4[c], L->q4[c ^ 1], L->s[c], L->tid[c], L->s[c ^ 1], L->tid[c ^ 1],
-                             P->keep, L->h_kv, L->d, L->cap, L->budget, L->st));
+                             P->keep, L->h_kv, L->d, L->cap, L->budget, S));
     } else {
-      Timed t(L, LOCRET_K_COMPACT);
+      Timed t(L, LOCRET_K_COMPACT, S);
       CompactArgs a;
       a.k_src = L->k_pre[c]; a.v_src = L->v[c]; a.s_src = L->s[c]; a.t_src = L->tid[c];
       a.k_dst = L->k_pre[c ^ 1]; a.v_dst = L->v[c ^ 1]; a.s_dst = L->s[c ^ 1]; a.t_dst = L->tid[c ^ 1];
       a.k_rot = L->k_rot; a.keep = P->keep; a.cs = L->cs;
       a.h_kv = L->h_kv; a.d = L->d; a.cap = L->cap; a.budget = L->budget;
-      CK(launch_compact(a, L->st));
+      CK(launch_compact(a, S));
     }
     L->cur = c ^ 1;
     L->len = L->budget;
   } else {
     L->len = n;
+  }
+  if (side) {
+    CK(cudaEventRecord(L->ev_side, S));
+    L->side_pending = true;
   }
   L->seen += n_tok;
   return LOCRET_OK;
@@ -429,6 +498,7 @@ int locret_export_state(locret_layer *L, void *K, void *V, float *scores, int64_
                         int32_t *len, int64_t *tokens_seen) {
   if (!L) return LOCRET_ERR_INVALID;
   if (L->int4 && (K || V)) return LOCRET_ERR_INVALID;  // use locret_export_state_int4
+  CK(sync_all(L));
   const int c = L->cur, n = L->len;
   if (len) *len = n;
   if (tokens_seen) *tokens_seen = L->seen;
@@ -452,6 +522,7 @@ int locret_import_state(locret_layer *L, const void *K, const void *V, const flo
   if (!L || len < 0 || len > L->cap || tokens_seen < 0) return LOCRET_ERR_INVALID;
   if (L->int4) return LOCRET_ERR_INVALID;  // use locret_import_state_int4
   if (len > 0 && (!K || !V || !scores || !token_ids)) return LOCRET_ERR_INVALID;
+  CK(sync_all(L));
   const int c = L->cur;
   if (len > 0) {
     const size_t row = (size_t)len * L->d * sizeof(bf16), pitch = (size_t)L->cap * L->d * sizeof(bf16);
@@ -474,6 +545,7 @@ int locret_export_state_int4(locret_layer *L, void *k_codes, void *k_scales, voi
                              void *v_scales, float *scores, int64_t *token_ids, int32_t *len,
                              int64_t *tokens_seen) {
   if (!L || !L->int4) return LOCRET_ERR_INVALID;
+  CK(sync_all(L));
   const int c = L->cur, n = L->len;
   if (len) *len = n;
   if (tokens_seen) *tokens_seen = L->seen;
@@ -497,6 +569,7 @@ int locret_import_state_int4(locret_layer *L, const void *k_codes, const void *k
   if (!L || !L->int4 || len < 0 || len > L->cap || tokens_seen < 0) return LOCRET_ERR_INVALID;
   if (len > 0 && (!k_codes || !k_scales || !v_codes || !v_scales || !scores || !token_ids))
     return LOCRET_ERR_INVALID;
+  CK(sync_all(L));
   const int c = L->cur;
   if (len > 0) {
     const size_t crow = (size_t)len * (L->d / 2), cpitch = (size_t)L->cap * (L->d / 2);
@@ -517,6 +590,7 @@ int locret_import_state_int4(locret_layer *L, const void *k_codes, const void *k
 int locret_sync_status(locret_layer *L) {
   if (!L) return LOCRET_ERR_INVALID;
   int host = 0;
+  CK(sync_all(L));
   CK(cudaMemcpyAsync(&host, L->d_status, sizeof(int), cudaMemcpyDeviceToHost, L->st));
   CK(cudaStreamSynchronize(L->st));
   CK(cudaGetLastError());
@@ -539,7 +613,7 @@ int locret_set_timing(locret_layer *L, int32_t enable) {
 int locret_read_timing(locret_layer *L, float *ms, int64_t *launches) {
   if (!L || !ms || !launches) return LOCRET_ERR_INVALID;
   for (int i = 0; i < LOCRET_K_COUNT; i++) { ms[i] = 0.f; launches[i] = 0; }
-  CK(cudaStreamSynchronize(L->st));
+  CK(sync_all(L));
   for (size_t i = 0; i < L->events_used; i++) {
     float t = 0.f;
     CK(cudaEventElapsedTime(&t, L->events[i].a, L->events[i].b));
@@ -558,7 +632,7 @@ int locret_launch_count(const locret_layer *L, int64_t *count) {
 
 void locret_destroy(locret_layer *L) {
   if (!L) return;
-  cudaStreamSynchronize(L->st);
+  sync_all(L);
   ScratchPool *p = L->pool;
   free_layer_memory(L);
   delete L;
