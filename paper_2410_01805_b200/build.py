@@ -45,7 +45,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
                                                 *[os.path.getmtime(p) for p in glob.glob(os.path.join(CSRC, "*.cuh"))],
                                                 os.path.getmtime(os.path.join(HERE, "..", "include", "locret.h")))):
             continue
-        cmd = [nvcc, *NVCC_FLAGS, "-c", src, "-o", obj]
+        cmd = [nvcc, *NVCC_FLAGS, *os.environ.get("LOCRET_EXTRA_NVCC", "").split(), "-c", src, "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas"); cmd.insert(2, "-v")
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
