@@ -32,6 +32,9 @@ import workloads as W  # noqa: E402
 METRIC = "chunked-prefill tokens/sec at 128K ctx (1 B200); % tensor/HBM roofline per kernel"
 UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "c3_llama_128k"
+# dram__bytes_read.sum + dram__bytes_write.sum of one steady-state attention launch, from the ncu
+# capture summarised in profiles/attn_tc_kernel_c3_steady_chunk.md (same launch shape as here)
+NCU_ATTN_TRAFFIC_BYTES = {"c3_llama_128k": 71.5e6, "c2_llama_32k": 71.5e6}
 
 
 def measured_peaks():
@@ -281,28 +284,48 @@ def run_ours(args, w):
     value = job_throughput(world, w.context, t_ms)
     e2e = job_throughput(world, w.context, t_e2e)
 
-    # ---- roofline of the dominant kernel (attention: a dense contraction -> tensor peak)
-    fl = step_flops(w) * args.steps                       # [qkv, attn, rh] flops over the timed region
-    ia = K_NAMES.index("attn")
+    # ---- per-kernel rates.  In the timed region the retaining head, selection and compaction run
+    # on the library's second stream and overlap attention / the next projection, so their event
+    # times (and attention's) include the time they share the SMs; one extra pass with every
+    # kernel on one stream gives each kernel's rate when it runs alone.
+    def summarise(k_ms, k_cnt, steps):
+        fl = step_flops(w) * steps
+        out_k = {}
+        tot = float(k_ms.sum())
+        for i, name in enumerate(K_NAMES):
+            if k_cnt[i]:
+                out_k[name] = {"launches": int(k_cnt[i]), "ms_total": float(k_ms[i]), "share": float(k_ms[i] / tot)}
+        for name, f in (("qkv", fl[0]), ("attn", fl[1]), ("rh", fl[2])):
+            out_k[name]["tflops"] = float(f / (k_ms[K_NAMES.index(name)] * 1e-3) / 1e12)
+        ic = K_NAMES.index("compact")
+        if k_cnt[ic]:
+            if s.kv_dtype == 1:
+                unit_b = 2 * (s.head_dim // 2) * 2 + 2 * 2 * 2 + 2 * (4 + 8)   # codes, scales, score, id: read + write
+            else:
+                unit_b = 2 * s.head_dim * 2 * 2 + 2 * (4 + 8) + s.head_dim * 2   # K, V read + write; score, id; rotated K
+            out_k["compact"]["gbs"] = float(k_cnt[ic] * s.n_kv_heads * w.budget * unit_b / (k_ms[ic] * 1e-3) / 1e9)
+        return out_k
+
+    per_kernel = summarise(k_ms, k_cnt, args.steps)
+    for L in layers:
+        L.set_timing(2)
+    flush.zero_()
+    prefill_resident()
+    iso_ms = np.zeros(len(K_NAMES)); iso_cnt = np.zeros(len(K_NAMES), dtype=np.int64)
+    for L in layers:
+        a, c = L.read_timing(); iso_ms += a; iso_cnt += c
+        L.set_timing(0)
+    isolated = summarise(iso_ms, iso_cnt, 1)
+    attn_tf = per_kernel["attn"]["tflops"]
     dom = int(np.argmax(k_ms))
-    attn_tf = fl[1] / (k_ms[ia] * 1e-3) / 1e12 if k_ms[ia] > 0 else 0.0
-    per_kernel = {}
-    for i, name in enumerate(K_NAMES):
-        if k_cnt[i]:
-            per_kernel[name] = {"launches": int(k_cnt[i]), "ms_total": float(k_ms[i]),
-                                "share": float(k_ms[i] / k_ms.sum())}
-    per_kernel["qkv"]["tflops"] = float(fl[0] / (k_ms[0] * 1e-3) / 1e12)
-    per_kernel["attn"]["tflops"] = float(attn_tf)
-    per_kernel["rh"]["tflops"] = float(fl[2] / (k_ms[K_NAMES.index("rh")] * 1e-3) / 1e12)
-    ic = K_NAMES.index("compact")
-    if k_cnt[ic]:
-        unit_b = 2 * s.head_dim * 2 * 2 + 2 * (4 + 8)        # K, V read + write; score, token id
-        rope_b = s.head_dim * 2                               # rotated key written for the next step
-        bytes_c = k_cnt[ic] * s.n_kv_heads * w.budget * (unit_b + rope_b)
-        per_kernel["compact"]["gbs"] = float(bytes_c / (k_ms[ic] * 1e-3) / 1e9)
     roofline = {"kernel": "attn", "bound": "tensor", "achieved": float(attn_tf), "peak": peaks["tf_sustained"],
-                "unit": "TFLOP/s", "frac": float(attn_tf / peaks["tf_sustained"]), "traffic": None,
-                "peak_source": f"bf16 sustained, {peaks['source']}", "dominant_by_time": K_NAMES[dom]}
+                "unit": "TFLOP/s", "frac": float(attn_tf / peaks["tf_sustained"]),
+                "traffic": NCU_ATTN_TRAFFIC_BYTES.get(w.name) if not (args.layers or args.context) else None,
+                "traffic_unit": "bytes per steady-state launch (ncu)",
+                "peak_source": f"bf16 sustained, {peaks['source']}", "dominant_by_time": K_NAMES[dom],
+                "isolated": {"achieved": isolated["attn"]["tflops"],
+                             "frac": isolated["attn"]["tflops"] / peaks["tf_sustained"],
+                             "note": "same kernel in a pass with every kernel on one stream"}}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -318,7 +341,8 @@ def run_ours(args, w):
         "clocks": clk.summary(),
         "roofline": roofline,
         "kernels": per_kernel,
-        "tflops_step": float(fl.sum() / args.steps / (t_ms * 1e-3) / 1e12),
+        "kernels_isolated": isolated,
+        "tflops_step": float(step_flops(w).sum() / (t_ms * 1e-3) / 1e12),
         "setup_s": gen_s,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -217,6 +217,7 @@ class OracleLayer:
         self.budget, self.chunk, self.n_stab = budget, chunk, n_stab
         self.cap = budget + chunk + reserve
         self.mirror = mirror
+        self.want_flip_sens = False   # tests switch this on: an error-propagation aid, not part of the method
         self.int4 = shape.kv_dtype == 1
         self.reset()
 
@@ -283,7 +284,7 @@ class OracleLayer:
 
         # (b) Eq. 1
         self.last_abs_out = np.full((n_tok, h * d), np.nan)
-        self.last_flip_sens = np.full((n_tok, h * d), np.nan) if self.mirror else None
+        self.last_flip_sens = np.full((n_tok, h * d), np.nan) if self.want_flip_sens else None
         out = attention_rows(Qr, Kr_cache, V_cache, Kr_chunk, V, g, rows, self.last_abs_out,
                              self.last_flip_sens)
 

@@ -176,8 +176,9 @@ class LocretLayer:
         _check(lib.locret_reset(self._h), "locret_reset")
 
     # -- measurement
-    def set_timing(self, on: bool):
-        _check(lib.locret_set_timing(self._h, int(on)), "locret_set_timing")
+    def set_timing(self, mode):
+        """0 off, 1 time every kernel, 2 time every kernel and run them on one stream."""
+        _check(lib.locret_set_timing(self._h, int(mode)), "locret_set_timing")
 
     def read_timing(self):
         ms = np.zeros(len(K_NAMES), dtype=np.float32)

@@ -75,6 +75,7 @@ struct locret_layer {
   int64_t seen;
   int64_t launches;
   bool timing;
+  bool serialize;  // timing mode 2: keep every kernel on the main stream (clean per-kernel times)
   bool use_tc;  // tcgen05 kernels (default); LOCRET_LEGACY_MMA=1 keeps the mma.sync kernels for A/B runs
   bool use_side;  // off-critical-path kernels go to the pool's second stream (LOCRET_SERIAL=1 disables)
   bool side_pending;
@@ -219,7 +220,7 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   L->h = h; L->h_kv = hk; L->d = d; L->D = D; L->d_R = dR;
   L->d_in = (h + 2 * hk) * d;
   L->st = (cudaStream_t)cfg->stream;
-  L->cur = 0; L->len = 0; L->seen = 0; L->launches = 0; L->timing = false; L->events_used = 0;
+  L->cur = 0; L->len = 0; L->seen = 0; L->launches = 0; L->timing = false; L->serialize = false; L->events_used = 0;
   L->pool = nullptr;
   {
     const char *e = getenv("LOCRET_LEGACY_MMA");
@@ -361,17 +362,18 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
   if (n > L->cap) return LOCRET_ERR_CAPACITY;
   ScratchPool *P = L->pool;
   const int c = L->cur;
-  const bool side = L->use_side;
+  const bool side = L->use_side && !L->serialize;
   cudaStream_t S = side ? P->side : L->st;  // stream of the off-critical-path kernels
   const int sb = P->flip;                    // staging buffer of this call
   P->flip ^= 1;
   bf16 *const staging = P->staging[sb];
   bf16 *const z_post = P->z_post[sb];
-  if (side) {
+  if (L->use_side) {
     // the staging buffer is free once the retaining head that last read it has run, and this
     // layer's cache once its previous selection / compaction has finished
     CK(cudaStreamWaitEvent(L->st, P->ev_stage_free[sb], 0));
     if (L->side_pending) CK(cudaStreamWaitEvent(L->st, L->ev_side, 0));
+    L->side_pending = false;
   }
 
   {  // (a) projections
@@ -607,6 +609,7 @@ int locret_reset(locret_layer *L) {
 int locret_set_timing(locret_layer *L, int32_t enable) {
   if (!L) return LOCRET_ERR_INVALID;
   L->timing = enable != 0;
+  L->serialize = enable == 2;
   return LOCRET_OK;
 }
 

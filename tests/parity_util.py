@@ -27,6 +27,7 @@ def make_pair(shape, weights, budget, chunk, n_stab, reserve=0):
     from paper_2410_01805_b200 import LocretLayer
     wqkv, w1, w2 = weights
     ora = O.OracleLayer(shape, wqkv, w1, w2, budget, chunk, n_stab, reserve=reserve, mirror=True)
+    ora.want_flip_sens = True
     gpu = LocretLayer(shape, bf16_dev(wqkv), bf16_dev(w1), bf16_dev(w2), budget, chunk, n_stab,
                       reserve=reserve)
     return ora, gpu
