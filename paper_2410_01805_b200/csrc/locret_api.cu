@@ -31,6 +31,8 @@ struct ScratchPool {
   size_t staging_b[2] = {0, 0}, qrot_b = 0, zpost_b[2] = {0, 0}, partial_b = 0, keep_b = 0, kexp_b = 0, vexp_b = 0;
   bf16 *staging[2] = {nullptr, nullptr}, *q_rot = nullptr, *z_post[2] = {nullptr, nullptr};
   bf16 *k_exp = nullptr, *v_exp = nullptr;  // 4-bit caches: bf16 expansion of the layer in flight
+  float *dec_o = nullptr, *dec_ml = nullptr;  // decode attention: per-split partial results
+  size_t deco_b = 0, decml_b = 0;
   float *partial = nullptr;
   int32_t *keep = nullptr;
   struct CsTable { float theta; int d, cap; float2 *ptr; };
@@ -112,7 +114,7 @@ void release_pool(ScratchPool *p) {
     cudaFree(p->staging[i]); cudaFree(p->z_post[i]);
     if (p->ev_stage_free[i]) cudaEventDestroy(p->ev_stage_free[i]);
   }
-  cudaFree(p->q_rot); cudaFree(p->partial); cudaFree(p->keep);
+  cudaFree(p->q_rot); cudaFree(p->partial); cudaFree(p->keep); cudaFree(p->dec_o); cudaFree(p->dec_ml);
   cudaFree(p->k_exp); cudaFree(p->v_exp);
   for (auto &t : p->cs) cudaFree(t.ptr);
   g_pools.erase(p->st);
@@ -283,7 +285,12 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
       g = g && grow(&p->q_rot, &p->qrot_b, (size_t)chunk * h * d * sizeof(bf16), L->st);
       {
         int nt = rh_num_tiles(dR) > rh_tc_num_tiles(dR) ? rh_num_tiles(dR) : rh_tc_num_tiles(dR);
-        g = g && grow(&p->partial, &p->partial_b, (size_t)nt * chunk * hk * sizeof(float), L->st);
+        size_t pb = (size_t)nt * chunk * hk * sizeof(float);
+        const size_t pb_dec = (size_t)rh_gemv_blocks(dR) * hk * sizeof(float);
+        if (pb < pb_dec) pb = pb_dec;
+        g = g && grow(&p->partial, &p->partial_b, pb, L->st);
+        g = g && grow(&p->dec_o, &p->deco_b, (size_t)h * 64 * d * sizeof(float), L->st);
+        g = g && grow(&p->dec_ml, &p->decml_b, (size_t)h * 64 * 2 * sizeof(float), L->st);
       }
       g = g && grow(&p->keep, &p->keep_b, (size_t)hk * budget * sizeof(int32_t), L->st);
       if (L->int4) {
@@ -376,9 +383,12 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
     L->side_pending = false;
   }
 
+  const bool decode = n_tok == 1 && L->use_tc;  // one token: bandwidth-bound kernels of decode.cu
   {  // (a) projections
     Timed t(L, LOCRET_K_QKV);
-    if (L->use_tc && n_tok >= 32 && gemm_tc_supported(n_tok, L->d_in, L->D, L->D, L->D))
+    if (decode)
+      CK(launch_gemv((const bf16 *)hidden_in, L->wqkv_t, L->d_in, L->D, staging, L->st));
+    else if (L->use_tc && n_tok >= 32 && gemm_tc_supported(n_tok, L->d_in, L->D, L->D, L->D))
       CK(launch_gemm_tc((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, staging, L->d_in, n_tok,
                         L->d_in, L->D, L->d_status, L->st));
     else
@@ -424,7 +434,10 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
                                   (uint64_t)L->h * L->d * 2, 64, 128);
       L->map_q_base = tc_ok ? P->q_rot : nullptr;
     }
-    if (tc_ok)
+    if (decode)
+      CK(launch_attention_decode(P->q_rot, k_att, v_att, (bf16 *)attn_out, P->dec_o, P->dec_ml, L->h, L->h_kv,
+                                 L->d, L->cap, n, decode_attn_splits(L->h_kv, n), L->st));
+    else if (tc_ok)
       CK(launch_attention_tc(&L->map_q, &L->map_k, &L->map_v[c], (bf16 *)attn_out, n_tok, L->h, L->h_kv,
                              L->d, L->len, L->d_status, L->st));
     else
@@ -439,7 +452,9 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
   {  // (c) retaining head: launched after the attention kernel, so its CTAs fill that kernel's tail
     Timed t(L, LOCRET_K_RH, S);
     const bf16 *z = L->cfg.rh_input == 1 ? z_post : staging;
-    if (L->use_tc && n_tok >= 32 && gemm_tc_supported(n_tok, L->d_R, L->d_in, L->d_in, L->d_in))
+    if (decode)
+      CK(launch_rh_gemv(z, L->w1_t, L->w2f, P->partial, L->d_R, L->d_in, L->h_kv, L->cfg.act, &n_tiles, S));
+    else if (L->use_tc && n_tok >= 32 && gemm_tc_supported(n_tok, L->d_R, L->d_in, L->d_in, L->d_in))
       CK(launch_rh_gemm_tc(z, L->d_in, L->w1_t, L->w2f, P->partial, n_tok, L->d_R, L->d_in, L->h_kv,
                            L->cfg.act, &n_tiles, L->d_status, S));
     else

@@ -73,3 +73,30 @@ def test_partial_last_chunk_of_the_headline_run():
     # Algorithm 1's reading: the protected units are the last 2500 entries of cache + chunk
     assert set(range(start - w.n_stab, start)) <= set(ora.T[0])
     gpu.destroy()
+
+
+@pytest.mark.parametrize("name", ["c3_llama_128k", "c5_llama_stream_int4"])
+def test_decode_steps_after_prefill_at_the_llama_shape(name):
+    """Prefill two full chunks (cache at its budget), then decode: the B = 1 case of Eq. 1."""
+    import torch
+    from parity_util import bf16_dev, check_attention, import_oracle_state, lockstep_chunk, make_pair
+    w = W.get_workload(name)
+    ora, gpu = make_pair(w.shape, W.layer_weights(w.shape, 3), w.budget, w.chunk, w.n_stab, reserve=16)
+    start = 0
+    for i in range(2):
+        lockstep_chunk(ora, gpu, W.hidden_states(w, start, w.chunk), 0, rows=[0, w.chunk - 1], what=f"{name} fill {i}")
+        start += w.chunk
+    st = ora.export_state()
+    import_oracle_state(gpu, st, bool(ora.int4))
+    out = torch.zeros((1, w.shape.n_q_heads * w.shape.head_dim), dtype=torch.bfloat16, device="cuda")
+    for t in range(6):
+        x = W.hidden_states(w, start + t, 1)
+        gpu.decode_step(bf16_dev(x), out)
+        ref = ora.decode_step(x[0])
+        check_attention(out.float().cpu().numpy().astype(np.float64), ref, f"{name} decode {t}",
+                        ora.last_abs_out, ora.last_flip_sens)
+        got = gpu.export_state()["S"][:, -1]
+        want = ora.last_scores[0]
+        assert np.all(np.abs(got - want) <= 1e-2 * np.maximum(np.abs(want), np.sqrt(np.mean(ora.S ** 2)))), f"decode {t} score"
+    assert gpu.cache_len == w.budget + 6 and gpu.sync_status() == 0
+    gpu.destroy()
