@@ -210,7 +210,8 @@ def run_ours(args, w):
     layers = []
     for l in range(w.n_layers):
         wq, w1, w2 = (torch.from_numpy(a).to(torch.bfloat16).to(dev) for a in W.layer_weights(s, l))
-        layers.append(LocretLayer(s, wq, w1, w2, w.budget, w.chunk, w.n_stab, stream=stream))
+        layers.append(LocretLayer(s, wq, w1, w2, w.budget, w.chunk, w.n_stab, reserve=args.decode_steps,
+                                  stream=stream))
         del wq, w1, w2
     gen_s = time.perf_counter() - t0
 
@@ -327,6 +328,32 @@ def run_ours(args, w):
                              "frac": isolated["attn"]["tflops"] / peaks["tf_sustained"],
                              "note": "same kernel in a pass with every kernel on one stream"}}
 
+    # ---- decoding after the prefill (the B = 1 case): one token through every layer per step
+    decode = None
+    if args.decode_steps > 0:
+        prefill_resident()
+        xd = x_dev[:args.decode_steps]
+        od = torch.empty((1, hd), dtype=torch.bfloat16, device=dev)
+
+        def decode_all():
+            for t in range(args.decode_steps):
+                for L in layers:
+                    L.decode_step(xd[t:t + 1], od)
+
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream); decode_all(); b.record(stream)
+        torch.cuda.synchronize()
+        dms = a.elapsed_time(b) / args.decode_steps
+        ln = min(w.budget, w.context)
+        kv_bytes = 2 * s.n_kv_heads * ln * s.head_dim * 2          # rotated K + V read by attention
+        w_bytes = 2 * (s.d_model * s.d_in + s.d_in * s.d_retain)
+        step_bytes = w.n_layers * (kv_bytes + w_bytes)
+        decode = {"tokens_per_s": 1e3 / dms, "ms_per_token": dms, "steps": args.decode_steps,
+                  "algorithmic_gb_per_token": step_bytes / 1e9, "achieved_gbs": step_bytes / (dms * 1e-3) / 1e9,
+                  "frac_of_hbm_peak": step_bytes / (dms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                  "cache_units_per_head": ln, "note": "one request, all layers per token, after the prefill"}
+
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": t_ms, "higher_is_better": True, "scaling": "weak",
@@ -342,6 +369,7 @@ def run_ours(args, w):
         "roofline": roofline,
         "kernels": per_kernel,
         "kernels_isolated": isolated,
+        "decode": decode,
         "tflops_step": float(step_flops(w).sum() / (t_ms * 1e-3) / 1e12),
         "setup_s": gen_s,
     }
@@ -366,6 +394,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling only)")
     ap.add_argument("--context", type=int, default=0, help="override the context length (profiling only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--decode-steps", type=int, default=64, help="decode steps timed after the prefill (0 = none)")
     args = ap.parse_args()
     w = W.get_workload(args.workload)
     if args.layers:
