@@ -191,8 +191,7 @@ int locret_launch_count(const locret_layer *layer, int64_t *count);
  * Requires d_in % 64 == 0, d_retain % 32 == 0, 1 <= n_kv_heads <= 32, act in {0,1,2}, z and w1_t
  * 16-byte aligned.  The per-tile partial sums live in a fixed array inside the library image of
  * LOCRET_STATIC_SCRATCH_FLOATS floats (4 MiB, present on every GPU that loads the library until
- * the process exits); a call needs T * n_tok * n_kv_heads of them, T = d_retain / 256 if d_retain is
- * a multiple of 256 and ceil(d_retain / 128) otherwise, and returns
+ * the process exits); a call needs ceil(d_retain / 64) * n_tok * n_kv_heads of them and returns
  * LOCRET_ERR_CAPACITY, launching nothing, if that is more.
  * The call makes no cudaMalloc/cudaFree and uses no allocating library routine.  Its first call on
  * a device looks up the array's device address (cudaGetSymbolAddress, with that device current);

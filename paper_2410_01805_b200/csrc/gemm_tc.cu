@@ -75,7 +75,7 @@ __device__ __forceinline__ float fast_act(float x, int act) {
 
 template <int BN>
 struct GemmCfg {
-  static constexpr int STAGES = BN == 256 ? 4 : 6;
+  static constexpr int STAGES = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
   static constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int W2_BYTES = BN * MAX_HKV * 4;
@@ -318,17 +318,28 @@ cudaError_t launch_gemm_tc(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16
   return launch_t<128, 0>(A, lda, Bt, ldb, C, ldc, M, N, K, nullptr, nullptr, 0, 0, status, st);
 }
 
-// 128 x 256 tiles whenever d_R allows: a 128-wide tile needs twice the operand traffic per flop.
-static int rh_tile_n(int d_R) { return d_R % 256 == 0 ? 256 : 128; }
-int rh_tc_num_tiles(int d_R) { return (d_R + rh_tile_n(d_R) - 1) / rh_tile_n(d_R); }
+// Tile width of the retaining-head GEMM: the widest of 256 / 128 / 64 columns that still gives
+// about one CTA per SM (a 128 x 256 tile needs the least operand traffic per flop, but a chunk of
+// 1024 tokens and d_R = 1024 would make only 32 of them).
+static int rh_tile_n(int M, int d_R) {
+  const int mt = (M + BM - 1) / BM;
+  for (int bn = 256; bn > 64; bn >>= 1)
+    if (d_R % bn == 0 && mt * (d_R / bn) >= 96) return bn;
+  return d_R % 64 == 0 ? 64 : 128;
+}
+// upper bound on the number of N-tiles (scratch sizing)
+int rh_tc_num_tiles(int d_R) { return (d_R + 63) / 64; }
 
 cudaError_t launch_rh_gemm_tc(const bf16 *A, int lda, const bf16 *W1t, const float *W2, float *partial,
                               int M, int d_R, int K, int h_kv, int act, int *n_tiles, int *status,
                               cudaStream_t st) {
-  *n_tiles = rh_tc_num_tiles(d_R);
-  if (rh_tile_n(d_R) == 256)
+  const int bn = rh_tile_n(M, d_R);
+  *n_tiles = (d_R + bn - 1) / bn;
+  if (bn == 256)
     return launch_t<256, 1>(A, lda, W1t, K, nullptr, 0, M, d_R, K, W2, partial, h_kv, act, status, st);
-  return launch_t<128, 1>(A, lda, W1t, K, nullptr, 0, M, d_R, K, W2, partial, h_kv, act, status, st);
+  if (bn == 128)
+    return launch_t<128, 1>(A, lda, W1t, K, nullptr, 0, M, d_R, K, W2, partial, h_kv, act, status, st);
+  return launch_t<64, 1>(A, lda, W1t, K, nullptr, 0, M, d_R, K, W2, partial, h_kv, act, status, st);
 }
 
 }  // namespace locret
