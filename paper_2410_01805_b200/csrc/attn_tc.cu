@@ -6,15 +6,23 @@
 // keys/values of that head in tiles of 128 through shared memory with TMA.  Roles:
 //   warps 0-3 / 4-7  softmax of query tile 0 / 1: one thread per query row reads its row of
 //                    S = Q K^T from TMEM, keeps a running maximum and sum, writes
-//                    P = exp2(S - max) as bf16 back into TMEM over S, and rescales the
-//                    accumulator in TMEM only when the maximum has grown by more than 2^8;
-//   warp 8           TMA producer (Q once, then K and V tiles, two stages each);
-//   warp 9           issues S_t = Q_t K_j^T (both operands in shared memory) and
-//                    O_t += P_t V_j (P from TMEM, V from shared memory), alternating the two
-//                    tiles so that one tile's softmax overlaps the other tile's MMAs.
+//                    P = exp2(S - max) as bf16 back into TMEM over S (handed to the MMA issuer in
+//                    two halves), and rescales the accumulator in TMEM only when the maximum has
+//                    grown by more than 2^100.  The two warpgroups take strict turns, so that one
+//                    tile's softmax runs while the other tile's MMAs execute; left alone the two
+//                    tiles drift into phase and tensor pipe and softmax alternate instead of
+//                    overlapping (measured: 1.3x slower).
+//   warp 8           TMA producer: Q once, then K and V tiles (two stages each), walking the
+//                    unmasked key tiles in a per-CTA rotated order, with an L2 prefetch ahead;
+//   warps 9 / 10     issue S_t = Q_t K_j^T (both operands in shared memory) and O_t += P_t V_j
+//                    (P from TMEM, V from shared memory) for tile 0 / 1.  The tensor pipe accepts
+//                    only about two instructions ahead of execution, so each issuer builds its
+//                    descriptors once and advances them by constants, and the other issuer's MMAs
+//                    cover the time one spends polling a barrier.
 // TMEM columns: S0/P0 [0,128), S1/P1 [128,256), O0 [256,384), O1 [384,512).
 // Query row t sees keys [0, len + t]: the retained cache unmasked, the chunk causally.
 #include "tc_common.cuh"
+
 
 namespace locret {
 
@@ -22,12 +30,20 @@ namespace {
 
 using namespace tc;
 
-constexpr int AT_THREADS = 384;  // 3 warpgroups: softmax 0, softmax 1, {TMA, MMA, 2 idle warps}
+constexpr int AT_THREADS = 384;  // 3 warpgroups: softmax 0, softmax 1, {TMA, 2 MMA issuers, 1 idle warp}
 constexpr int TILE = 128;               // query rows per tile and keys per tile
 constexpr int HD = 128;                 // column pitch of a head in shared and tensor memory
 constexpr int HALF_BYTES = TILE * 128;  // one 64-column swizzled box of 128 rows: 16 KB
 constexpr int TILE_BYTES = 2 * HALF_BYTES;
 constexpr int AT_SMEM = 1024 + 6 * TILE_BYTES + 256;  // Q0,Q1,K0,K1,V0,V1 + barriers
+// The accumulator is rescaled only when a row's maximum has grown by more than 2^100 since the
+// scale in use was fixed.  P is stored as bf16 and O, l accumulate in fp32, both with an 8-bit
+// exponent, so P <= 2^100 and O <= keys * 2^100 * |v| (< 2^122 for 2^14 keys, |v| < 2^8) stay
+// finite, and relative precision does not depend on the common scale.  A small threshold would
+// trigger a rescale (a TMEM round trip on the critical path) at almost every tile that holds one
+// of the workload's 20x-norm outlier keys.
+constexpr float RESCALE_LOG2 = 100.0f;
+constexpr int PF = 6;       // key tiles prefetched into L2 ahead of the shared-memory pipeline
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
@@ -68,6 +84,7 @@ struct AttnParams {
   int *status;
 };
 
+template <int D>
 __global__ void __launch_bounds__(AT_THREADS, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, const AttnParams p) {
@@ -86,7 +103,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   uint64_t *s_full = bars + 9;      // 2
   uint64_t *p_full = bars + 11;     // 2
   uint64_t *o_full = bars + 13;     // 2
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 15);
+  uint64_t *p_half = bars + 15;     // 2: first 64 keys of P_t written (p_full: all 128)
+  uint64_t *turn = bars + 17;       // 2: the two softmax warpgroups take turns (see below)
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 19);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -111,13 +130,21 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const int kvh = head[0] / g;
   int NK = (p.len + row0[1] + TILE + TILE - 1) / TILE;
   NK = min(NK, (n + TILE - 1) / TILE);
+  // The softmax is order independent, so every CTA walks the key tiles that need no mask in its
+  // own rotated order: CTAs of one KV head start together, and in a common order they would all
+  // ask the L2 for the same K and V lines at the same moment (measured: 1.4x slower).
+  const int NF = min(NK, (p.len + row0[0] + 1) / TILE);  // tiles fully visible to every row
+  const int rot = NF > 0 ? (int)((blockIdx.x * 29u + 7u) % (unsigned)NF) : 0;
+  auto tile_of = [&](int j) { int x = j + rot; return j < NF ? (x >= NF ? x - NF : x) : j; };
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
     for (int s = 0; s < 2; s++) {
       mbar_init(&k_full[s], 1); mbar_init(&v_full[s], 1);
-      mbar_init(&k_empty[s], 1); mbar_init(&v_empty[s], 1);
+      mbar_init(&k_empty[s], 2); mbar_init(&v_empty[s], 2);  // released by both MMA issuers
       mbar_init(&s_full[s], 1); mbar_init(&p_full[s], 4); mbar_init(&o_full[s], 1);
+      mbar_init(&p_half[s], 4);
+      mbar_init(&turn[s], 4);
     }
     *abort_flag = 0;
     fence_barrier_init();
@@ -134,82 +161,106 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
   if (warp >= 8) {
     setmaxnreg_dec<56>();
-  if (warp >= 10) {
-    // idle warps of the third warpgroup
+  if (warp == 11) {
+    // idle warp of the third warpgroup
   } else if (warp == 8) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      const int nbox = (p.d + 63) / 64;  // 64-column boxes per head vector
+      constexpr int nbox = (D + 63) / 64;  // 64-column boxes per head vector
       mbar_expect_tx(q_full, 2 * nbox * HALF_BYTES);
       for (int t = 0; t < 2; t++)
         for (int hh = 0; hh < nbox; hh++)
-          tma_load_2d(sQ + t * TILE_BYTES + hh * HALF_BYTES, &map_q, head[t] * p.d + hh * 64, row0[t],
+          tma_load_2d(sQ + t * TILE_BYTES + hh * HALF_BYTES, &map_q, head[t] * D + hh * 64, row0[t],
                       q_full);
+      // L2 prefetch PF tiles ahead: the cache of a layer is not L2 resident when its chunk step
+      // starts, and two stages of shared memory do not cover an HBM miss.
+      auto prefetch_tile = [&](int j) {
+        const int row = tile_of(j) * TILE;
+        for (int hh = 0; hh < nbox; hh++) {
+          tma_prefetch_3d(&map_k, hh * 64, row, kvh);
+          tma_prefetch_3d(&map_v, hh * 64, row, kvh);
+        }
+      };
+      for (int j = 0; j < min(PF, NK); j++) prefetch_tile(j);
       for (int j = 0; j < NK; j++) {
         const int s = j & 1;
         const uint32_t ph = (j >> 1) & 1;
+        if (j + PF < NK) prefetch_tile(j + PF);
         if (!mbar_wait(&k_empty[s], ph ^ 1, abort_flag, p.status)) break;
         mbar_expect_tx(&k_full[s], nbox * HALF_BYTES);
         for (int hh = 0; hh < nbox; hh++)
-          tma_load_3d(sK + s * TILE_BYTES + hh * HALF_BYTES, &map_k, hh * 64, j * TILE, kvh, &k_full[s]);
+          tma_load_3d(sK + s * TILE_BYTES + hh * HALF_BYTES, &map_k, hh * 64, tile_of(j) * TILE, kvh, &k_full[s]);
         if (!mbar_wait(&v_empty[s], ph ^ 1, abort_flag, p.status)) break;
         mbar_expect_tx(&v_full[s], nbox * HALF_BYTES);
         for (int hh = 0; hh < nbox; hh++)
-          tma_load_3d(sV + s * TILE_BYTES + hh * HALF_BYTES, &map_v, hh * 64, j * TILE, kvh, &v_full[s]);
+          tma_load_3d(sV + s * TILE_BYTES + hh * HALF_BYTES, &map_v, hh * 64, tile_of(j) * TILE, kvh, &v_full[s]);
       }
     }
-  } else if (warp == 9) {
-    // ------------------------------------------------------------ MMA issuer
+  } else {
+    // ------------------------------------------------------------ MMA issuers: warp 9 for query
+    // tile 0, warp 10 for tile 1.  The tensor pipe's queue is only a couple of instructions deep,
+    // so an issuer that stops to poll a barrier starves the pipe; with one issuer per tile the
+    // other tile's MMAs cover each wait.  Descriptors are built once and advanced by constants.
     if (lane == 0) {
+      const int t = warp - 9;
       constexpr uint32_t idesc_qk = idesc_bf16(TILE, TILE, 0, 0);
-      const uint32_t idesc_pv = idesc_bf16(TILE, p.d, 0, 1);
-      const int ksteps = p.d / 16;
-      auto issue_s = [&](int t, int ks) {
-        const unsigned char *q = sQ + t * TILE_BYTES, *k = sK + ks * TILE_BYTES;
-#pragma unroll 1
+      constexpr uint32_t idesc_pv = idesc_bf16(TILE, D, 0, 1);
+      constexpr int ksteps = D / 16;
+      const uint64_t dq = desc_kmajor_sw128(sQ + t * TILE_BYTES);
+      const uint64_t dk0 = desc_kmajor_sw128(sK), dk1 = desc_kmajor_sw128(sK + TILE_BYTES);
+      const uint64_t dv0 = desc_mnmajor_sw128(sV, HALF_BYTES), dv1 = desc_mnmajor_sw128(sV + TILE_BYTES, HALF_BYTES);
+      const uint32_t s_tmem = tmem_base + t * TILE, o_tmem = tmem_base + 2 * TILE + t * HD;
+      auto issue_s = [&](int ks) {
+        const uint64_t b = ks ? dk1 : dk0;
+#pragma unroll
         for (int kk = 0; kk < ksteps; kk++) {
-          const int off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
-          mma_ss(tmem_base + t * TILE, desc_kmajor_sw128(q + off), desc_kmajor_sw128(k + off), idesc_qk,
-                 kk != 0);
+          const uint64_t off = (uint64_t)(((kk >> 2) * HALF_BYTES + (kk & 3) * 32) >> 4);
+          if (kk == 0) mma_ss_first(s_tmem, dq + off, b + off, idesc_qk);
+          else mma_ss_acc(s_tmem, dq + off, b + off, idesc_qk);
         }
         mma_commit(&s_full[t]);
+        mma_commit(&k_empty[ks]);
       };
-      auto issue_pv = [&](int t, int vs, bool acc) {
-        const unsigned char *v = sV + vs * TILE_BYTES;
+      // the first four k-steps (keys 0..63) only need the first half of P
+      auto issue_pv = [&](int vs, bool acc, int half) {
+        const uint64_t b = vs ? dv1 : dv0;
 #pragma unroll
-        for (int kk = 0; kk < TILE / 16; kk++)
-          mma_ts(tmem_base + 2 * TILE + t * HD, tmem_base + t * TILE + kk * 8,
-                 desc_mnmajor_sw128(v + kk * 16 * 128, HALF_BYTES), idesc_pv, acc || kk != 0);
-        mma_commit(&o_full[t]);
+        for (int kk = 0; kk < TILE / 16; kk++) {
+          if ((kk >> 2) != half) continue;
+          const uint64_t off = (uint64_t)((kk * 16 * 128) >> 4);
+          if (kk == 0) mma_ts(o_tmem, s_tmem, b, idesc_pv, acc);
+          else mma_ts_acc(o_tmem, s_tmem + kk * 8, b + off, idesc_pv);
+        }
+        if (half == 1) {
+          mma_commit(&o_full[t]);
+          mma_commit(&v_empty[vs]);
+        }
       };
       bool ok = mbar_wait(q_full, 0, abort_flag, p.status);
       ok = ok && mbar_wait(&k_full[0], 0, abort_flag, p.status);
       if (ok) {
         tc_fence_after();
-        issue_s(0, 0);
-        issue_s(1, 0);
-        mma_commit(&k_empty[0]);
+        issue_s(0);
       }
       for (int j = 0; j < NK && ok; j++) {
-        const int sv = j & 1;
+        const int sv = j & 1, sk = (j + 1) & 1;
+        // O_t += P_t V_j
         ok = mbar_wait(&v_full[sv], (j >> 1) & 1, abort_flag, p.status);
-        for (int t = 0; t < 2 && ok; t++) {
-          ok = mbar_wait(&p_full[t], j & 1, abort_flag, p.status);
+        ok = ok && mbar_wait(&p_half[t], j & 1, abort_flag, p.status);
+        if (!ok) break;
+        tc_fence_after();
+        issue_pv(sv, j > 0, 0);
+        ok = mbar_wait(&p_full[t], j & 1, abort_flag, p.status);
+        if (!ok) break;
+        tc_fence_after();
+        issue_pv(sv, j > 0, 1);
+        // S_t = Q_t K_{j+1}^T
+        if (j + 1 < NK) {
+          ok = mbar_wait(&k_full[sk], ((j + 1) >> 1) & 1, abort_flag, p.status);
           if (!ok) break;
           tc_fence_after();
-          issue_pv(t, sv, j > 0);
-          if (j + 1 < NK) {
-            const int sk = (j + 1) & 1;
-            if (t == 0) {
-              ok = mbar_wait(&k_full[sk], ((j + 1) >> 1) & 1, abort_flag, p.status);
-              if (!ok) break;
-              tc_fence_after();
-            }
-            issue_s(t, sk);
-            if (t == 1) mma_commit(&k_empty[sk]);
-          }
+          issue_s(sk);
         }
-        if (ok) mma_commit(&v_empty[sv]);
       }
     }
   }
@@ -226,6 +277,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const float c = p.scale_log2;
     float m_used = -INFINITY, l = 0.f;
     bool ok = true;
+    // The two softmax warpgroups alternate strictly: while one computes, the other tile's MMAs
+    // run.  Left alone the two tiles drift into phase, both warpgroups then compute at the same
+    // time (sharing issue slots and the special-function unit) and the tensor pipe idles.
+    if (t == 1) { __syncwarp(); if (lane == 0) mbar_arrive(&turn[0]); }
 
     for (int j = 0; j < NK && ok; j++) {
       ok = mbar_wait(&s_full[t], j & 1, abort_flag, p.status);
@@ -235,8 +290,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 #pragma unroll
       for (int q = 0; q < 4; q++) tmem_ld32(s_addr + q * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[q * 32]));
       tmem_wait_ld();
+      ok = mbar_wait(&turn[t], j & 1, abort_flag, p.status);
+      if (!ok) break;
 
-      const int key0 = j * TILE;
+      const int key0 = tile_of(j) * TILE;
       float tmax = -INFINITY;
       if (key0 + TILE - 1 > p.len + row0[t]) {  // a tile that crosses the causal boundary
 #pragma unroll
@@ -261,7 +318,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       if (j == 0) {
         m_used = tmax;
       } else {
-        const bool need = tmax > m_used + 8.0f;
+        const bool need = tmax > m_used + RESCALE_LOG2;
         if (__any_sync(0xffffffffu, need)) {
           // the accumulator must hold every product issued so far before it is rescaled
           ok = mbar_wait(&o_full[t], (j - 1) & 1, abort_flag, p.status);
@@ -270,7 +327,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           if (need) { alpha = exp2f(m_used - tmax); m_used = tmax; }
           l *= alpha;
 #pragma unroll 1
-          for (int q = 0; q < p.d / 32; q++) {
+          for (int q = 0; q < D / 32; q++) {
             uint32_t o[32];
             tmem_ld32(o_addr + q * 32, o);
             tmem_wait_ld();
@@ -289,18 +346,29 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         uint32_t pk[32];
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
-          float x0, x1, x2, x3;
+          float x0, x1, p2, p3;
           unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[q * 64 + 2 * i]),
                                             __uint_as_float(s[q * 64 + 2 * i + 1])), c2, nm2), x0, x1);
-          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[q * 64 + 2 * i + 2]),
-                                            __uint_as_float(s[q * 64 + 2 * i + 3])), c2, nm2), x2, x3);
-          const float p0 = ex2_approx(x0), p1 = ex2_approx(x1), p2 = ex2_approx(x2), p3 = ex2_approx(x3);
+          const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+          const uint64_t xb = fma_f32x2(pack_f32x2(__uint_as_float(s[q * 64 + 2 * i + 2]),
+                                                   __uint_as_float(s[q * 64 + 2 * i + 3])), c2, nm2);
+          {
+            float x2, x3;
+            unpack_f32x2(xb, x2, x3);
+            p2 = ex2_approx(x2); p3 = ex2_approx(x3);
+          }
           la = add_f32x2(la, pack_f32x2(p0, p1));
           lb = add_f32x2(lb, pack_f32x2(p2, p3));
           pk[i] = pack_bf16(p0, p1);
           pk[i + 1] = pack_bf16(p2, p3);
         }
         tmem_st32(s_addr + q * 32, pk);
+        if (q == 0) {
+          tmem_wait_st();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&p_half[t]);
+        }
       }
       {
         float a0, a1, b0, b1;
@@ -308,19 +376,23 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         unpack_f32x2(lb, b0, b1);
         l += (a0 + a1) + (b0 + b1);
       }
+
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&p_full[t]);
+      if (lane == 0) {
+        mbar_arrive(&p_full[t]);
+        mbar_arrive(&turn[t ^ 1]);
+      }
     }
 
     if (ok && NK > 0) ok = mbar_wait(&o_full[t], (NK - 1) & 1, abort_flag, p.status);
     tc_fence_after();
     if (ok) {
       const float inv = 1.0f / l;
-      bf16 *dst = p.out + (size_t)row * p.h * p.d + (size_t)head[t] * p.d;
+      bf16 *dst = p.out + (size_t)row * p.h * D + (size_t)head[t] * D;
 #pragma unroll 1
-      for (int q = 0; q < p.d / 32; q++) {
+      for (int q = 0; q < D / 32; q++) {
         uint32_t o[32];
         tmem_ld32(o_addr + q * 32, o);
         tmem_wait_ld();
@@ -355,16 +427,23 @@ bool attention_tc_supported(int n_tok, int h, int h_kv, int d) {
 }
 
 // map_k / map_v: 3-D maps {d, cap, h_kv} with box {64, 128, 1}; map_q: 2-D {h*d, rows} box {64, 128}.
-cudaError_t launch_attention_tc(const CUtensorMap *map_q, const CUtensorMap *map_k,
-                                const CUtensorMap *map_v, bf16 *out, int n_tok, int h, int h_kv, int d,
-                                int len, int *status, cudaStream_t st) {
+template <int D>
+static cudaError_t launch_attn_d(const CUtensorMap *map_q, const CUtensorMap *map_k, const CUtensorMap *map_v,
+                                 const AttnParams &p, int grid, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          AT_SMEM);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
+  attn_tc_kernel<D><<<grid, AT_THREADS, AT_SMEM, st>>>(*map_q, *map_k, *map_v, p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_attention_tc(const CUtensorMap *map_q, const CUtensorMap *map_k,
+                                const CUtensorMap *map_v, bf16 *out, int n_tok, int h, int h_kv, int d,
+                                int len, int *status, cudaStream_t st) {
   AttnParams p;
   p.out = out; p.n_tok = n_tok; p.h = h; p.h_kv = h_kv; p.d = d; p.len = len;
   p.pair_heads = ((h / h_kv) % 2 == 0) ? 1 : 0;
@@ -372,8 +451,12 @@ cudaError_t launch_attention_tc(const CUtensorMap *map_q, const CUtensorMap *map
   p.status = status;
   const int n_rb = (n_tok + TILE - 1) / TILE;
   const int grid = p.pair_heads ? n_rb * (h / 2) : ((n_rb + 1) / 2) * h;
-  attn_tc_kernel<<<grid, AT_THREADS, AT_SMEM, st>>>(*map_q, *map_k, *map_v, p);
-  return cudaGetLastError();
+  switch (d) {
+    case 64: return launch_attn_d<64>(map_q, map_k, map_v, p, grid, st);
+    case 96: return launch_attn_d<96>(map_q, map_k, map_v, p, grid, st);
+    case 128: return launch_attn_d<128>(map_q, map_k, map_v, p, grid, st);
+  }
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace locret
