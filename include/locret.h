@@ -164,7 +164,8 @@ int locret_reset(locret_layer *layer);
  * Per-kernel timing.  With enable != 0 every kernel launched for this layer is
  * bracketed by CUDA events on the stream it runs on (kernels on the two streams overlap, so
  * the per-kernel times of a step add up to more than its duration); enable = 2 also keeps
- * every kernel on the layer's own stream, which gives each kernel's time when it runs alone.  locret_read_timing synchronises the
+ * every kernel on the layer's own stream, which gives each kernel's time when it runs alone;
+ * enable = 3 brackets only the attention kernel (the dominant one), for the least overhead.  locret_read_timing synchronises the
  * stream, adds up the elapsed time and the number of launches per kernel family since
  * the last read into ms[LOCRET_K_COUNT] and launches[LOCRET_K_COUNT] (host arrays), and
  * clears the record.

@@ -177,7 +177,7 @@ class LocretLayer:
 
     # -- measurement
     def set_timing(self, mode):
-        """0 off, 1 time every kernel, 2 time every kernel and run them on one stream."""
+        """0 off, 1 time every kernel, 2 time every kernel and run them on one stream, 3 time attention only."""
         _check(lib.locret_set_timing(self._h, int(mode)), "locret_set_timing")
 
     def read_timing(self):

@@ -244,8 +244,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
       for (int j = 0; j < NK && ok; j++) {
         const int sv = j & 1, sk = (j + 1) & 1;
-        // O_t += P_t V_j
+        // The tiles from memory arrive long before P does: poll them first, so that nothing but
+        // the MMAs themselves stands between P and the next S.
         ok = mbar_wait(&v_full[sv], (j >> 1) & 1, abort_flag, p.status);
+        if (j + 1 < NK) ok = ok && mbar_wait(&k_full[sk], ((j + 1) >> 1) & 1, abort_flag, p.status);
+        // O_t += P_t V_j
         ok = ok && mbar_wait(&p_half[t], j & 1, abort_flag, p.status);
         if (!ok) break;
         tc_fence_after();
@@ -256,9 +259,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         issue_pv(sv, j > 0, 1);
         // S_t = Q_t K_{j+1}^T
         if (j + 1 < NK) {
-          ok = mbar_wait(&k_full[sk], ((j + 1) >> 1) & 1, abort_flag, p.status);
-          if (!ok) break;
-          tc_fence_after();
           issue_s(sk);
         }
       }
@@ -290,8 +290,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 #pragma unroll
       for (int q = 0; q < 4; q++) tmem_ld32(s_addr + q * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[q * 32]));
       tmem_wait_ld();
-      ok = mbar_wait(&turn[t], j & 1, abort_flag, p.status);
-      if (!ok) break;
 
       const int key0 = tile_of(j) * TILE;
       float tmax = -INFINITY;
@@ -339,6 +337,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
 
+      // the turn covers the exponentials and the hand-over; loading S and its maximum above
+      // overlap the other tile's turn
+      ok = mbar_wait(&turn[t], j & 1, abort_flag, p.status);
+      if (!ok) break;
       const uint64_t c2 = pack_f32x2(c, c), nm2 = pack_f32x2(-m_used, -m_used);
       uint64_t la = pack_f32x2(0.f, 0.f), lb = la;
 #pragma unroll

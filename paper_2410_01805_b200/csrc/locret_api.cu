@@ -78,6 +78,7 @@ struct locret_layer {
   int64_t launches;
   bool timing;
   bool serialize;  // timing mode 2: keep every kernel on the main stream (clean per-kernel times)
+  bool attn_only;  // timing mode 3: bracket only the attention kernel (least overhead)
   bool use_tc;  // tcgen05 kernels (default); LOCRET_LEGACY_MMA=1 keeps the mma.sync kernels for A/B runs
   bool use_side;  // off-critical-path kernels go to the pool's second stream (LOCRET_SERIAL=1 disables)
   bool side_pending;
@@ -149,7 +150,7 @@ struct Timed {
   locret_layer *L; int kind; cudaStream_t st; TimedEvent *ev = nullptr;
   Timed(locret_layer *l, int k, cudaStream_t stream = nullptr) : L(l), kind(k), st(stream ? stream : l->st) {
     L->launches++;
-    if (!L->timing) return;
+    if (!L->timing || (L->attn_only && k != LOCRET_K_ATTN)) return;
     if (L->events_used == L->events.size()) {
       TimedEvent e; e.kind = k;
       if (cudaEventCreate(&e.a) != cudaSuccess || cudaEventCreate(&e.b) != cudaSuccess) { cudaGetLastError(); return; }
@@ -222,7 +223,7 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   L->h = h; L->h_kv = hk; L->d = d; L->D = D; L->d_R = dR;
   L->d_in = (h + 2 * hk) * d;
   L->st = (cudaStream_t)cfg->stream;
-  L->cur = 0; L->len = 0; L->seen = 0; L->launches = 0; L->timing = false; L->serialize = false; L->events_used = 0;
+  L->cur = 0; L->len = 0; L->seen = 0; L->launches = 0; L->timing = false; L->serialize = false; L->attn_only = false; L->events_used = 0;
   L->pool = nullptr;
   {
     const char *e = getenv("LOCRET_LEGACY_MMA");
@@ -625,6 +626,7 @@ int locret_set_timing(locret_layer *L, int32_t enable) {
   if (!L) return LOCRET_ERR_INVALID;
   L->timing = enable != 0;
   L->serialize = enable == 2;
+  L->attn_only = enable == 3;
   return LOCRET_OK;
 }
 
