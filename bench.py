@@ -105,33 +105,47 @@ def step_flops(w: W.Workload):
 
 # ----------------------------------------------------------------------------- reference arm (oracle on CPU)
 
+class OracleSampler:
+    """The oracle, as it stands, brought to the workload's steady state once; every sample() then
+    times `n_chunks` steady-state chunk-layers of layer 0 on the host cores."""
+
+    def __init__(self, w: W.Workload):
+        from oracle import locret_oracle as O
+        self.w = w
+        self.ora = O.OracleLayer(w.shape, *W.layer_weights(w.shape, 0), w.budget, w.chunk, w.n_stab, mirror=True)
+        self.sizes = w.chunk_sizes()
+        self.start, self.fill = 0, 0
+        # fill the cache without paying for attention (one query row per chunk)
+        while self.ora.len < min(w.budget, w.context - w.chunk) and self.fill < len(self.sizes) - 1:
+            self.ora.prefill_chunk(W.hidden_states(w, self.start, self.sizes[self.fill]), 0, rows=[0])
+            self.start += self.sizes[self.fill]; self.fill += 1
+
+    def sample(self, n_chunks: int = 1):
+        from threadpoolctl import threadpool_info
+        w, times, toks = self.w, [], 0
+        for _ in range(n_chunks):
+            idx = min(self.fill, len(self.sizes) - 2)          # a full-size chunk
+            if self.start + self.sizes[idx] > w.context:
+                self.start = self.fill_start()
+            x = W.hidden_states(w, self.start, self.sizes[idx])
+            t0 = time.perf_counter()
+            self.ora.prefill_chunk(x, 0)
+            times.append(time.perf_counter() - t0)
+            toks += self.sizes[idx]; self.start += self.sizes[idx]
+        cores = max([p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"] + [1])
+        sec = float(np.sum(times))
+        # one chunk-layer handles n_tok tokens of ONE layer; the whole job does n_layers of them per chunk
+        tok_s = toks / sec / w.n_layers
+        sample = (f"{n_chunks} steady-state chunk-layer(s) of layer 0 ({toks} tokens, cache {self.ora.len} units/head), "
+                  f"{sec:.1f} s; tokens/s = tokens / time / {w.n_layers} layers")
+        return tok_s, cores, sample, sec
+
+    def fill_start(self):
+        return sum(self.sizes[:self.fill])
+
+
 def oracle_sample(w: W.Workload, n_chunks: int):
-    """Time the oracle, as it stands, on `n_chunks` steady-state chunk-layers of layer 0."""
-    from threadpoolctl import threadpool_info
-    from oracle import locret_oracle as O
-    wts = W.layer_weights(w.shape, 0)
-    ora = O.OracleLayer(w.shape, *wts, w.budget, w.chunk, w.n_stab, mirror=True)
-    # bring the cache to its steady size without paying for attention: NO-rows calls
-    start, sizes = 0, w.chunk_sizes()
-    fill = 0
-    while ora.len < min(w.budget, w.context - w.chunk) and fill < len(sizes) - 1:
-        ora.prefill_chunk(W.hidden_states(w, start, sizes[fill]), 0, rows=[0])
-        start += sizes[fill]; fill += 1
-    times, toks = [], 0
-    for i in range(n_chunks):
-        idx = min(fill + i, len(sizes) - 1)
-        x = W.hidden_states(w, start, sizes[idx])
-        t0 = time.perf_counter()
-        ora.prefill_chunk(x, 0)
-        times.append(time.perf_counter() - t0)
-        toks += sizes[idx]; start += sizes[idx]
-    cores = max([p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"] + [1])
-    sec = float(np.sum(times))
-    # one chunk-layer handles n_tok tokens of ONE layer; the whole job does n_layers of them per chunk
-    tok_s = toks / sec / w.n_layers
-    sample = (f"{n_chunks} steady-state chunk-layer(s) of layer 0 ({toks} tokens, cache {ora.len} units/head), "
-              f"{sec:.1f} s; tokens/s = tokens / time / {w.n_layers} layers")
-    return tok_s, cores, sample, sec
+    return OracleSampler(w).sample(n_chunks)
 
 
 def run_reference(args, w):
@@ -144,8 +158,9 @@ def run_reference(args, w):
     n_per = 1
     sample = ""
     cores = 1
+    sampler = OracleSampler(w)
     for i in range(total):
-        v, cores, sample, _ = oracle_sample(w, n_per)
+        v, cores, sample, _ = sampler.sample(n_per)
         if i >= args.warmup:
             vals.append(v)
     value = float(np.mean(vals))

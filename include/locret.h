@@ -157,6 +157,14 @@ int locret_import_state_int4(locret_layer *layer, const void *k_codes, const voi
 /* Synchronise the stream; return the sticky device status (0, or LOCRET_ERR_*). */
 int locret_sync_status(locret_layer *layer);
 
+/*
+ * Self-test of the bounded device-side waits: launches a one-warp kernel whose mbarrier wait
+ * can never complete, with a limit of a few thousand polls, and returns the status word that
+ * kernel leaves.  The expected return value is LOCRET_ERR_DEVICE_TIMEOUT; the context stays
+ * usable.  (Diagnostic only; nothing on the hot path calls it.)  Synchronises `stream`.
+ */
+int locret_selftest_wait_timeout(void *stream);
+
 /* Forget all units: len = 0, tokens_seen = 0.  Asynchronous. */
 int locret_reset(locret_layer *layer);
 

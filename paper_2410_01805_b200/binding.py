@@ -49,6 +49,7 @@ def _load():
     l.locret_import_state.argtypes = [P, P, P, P, P, C.c_int32, C.c_int64]
     l.locret_export_state_int4.argtypes = [P, P, P, P, P, P, P, C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
     l.locret_import_state_int4.argtypes = [P, P, P, P, P, P, P, C.c_int32, C.c_int64]
+    l.locret_selftest_wait_timeout.argtypes = [P]
     l.locret_sync_status.argtypes = [P]
     l.locret_reset.argtypes = [P]
     l.locret_set_timing.argtypes = [P, C.c_int32]

@@ -255,3 +255,17 @@ def test_reset_and_launch_accounting():
     for k in ("K", "V", "S", "T"):
         assert np.array_equal(s1[k], s2[k])
     L.destroy()
+
+
+def test_bounded_wait_reports_a_timeout_and_the_context_survives():
+    """A device-side wait that cannot complete gives up, leaves LOCRET_ERR_DEVICE_TIMEOUT in the status
+    word and the kernel ends normally; the next step on the same context is still correct."""
+    import paper_2410_01805_b200 as P
+    from parity_util import lockstep_chunk, make_pair
+    assert P.lib.locret_selftest_wait_timeout(torch.cuda.current_stream().cuda_stream) == -5
+    assert b"timed out" in P.lib.locret_strerror(-5)
+    sh = small_shape(d=128, D=128, dR=64)
+    ora, gpu = make_pair(sh, weights_for(sh, 21), budget=200, chunk=128, n_stab=8)
+    lockstep_chunk(ora, gpu, hidden(128, sh.d_model, 5), 0, what="after the timed-out wait")
+    assert gpu.sync_status() == 0
+    gpu.destroy()
