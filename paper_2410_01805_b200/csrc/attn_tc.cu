@@ -301,15 +301,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           tmax = fmaxf(tmax, x);
         }
       } else {
-        float t0 = -INFINITY, t1 = -INFINITY, t2 = -INFINITY, t3 = -INFINITY;
+        float tm[8];
 #pragma unroll
-        for (int i = 0; i < TILE; i += 8) {
-          t0 = fmaxf(t0, fmaxf(__uint_as_float(s[i]), __uint_as_float(s[i + 1])));
-          t1 = fmaxf(t1, fmaxf(__uint_as_float(s[i + 2]), __uint_as_float(s[i + 3])));
-          t2 = fmaxf(t2, fmaxf(__uint_as_float(s[i + 4]), __uint_as_float(s[i + 5])));
-          t3 = fmaxf(t3, fmaxf(__uint_as_float(s[i + 6]), __uint_as_float(s[i + 7])));
-        }
-        tmax = fmaxf(fmaxf(t0, t1), fmaxf(t2, t3));
+        for (int a = 0; a < 8; a++) tm[a] = fmaxf(__uint_as_float(s[2 * a]), __uint_as_float(s[2 * a + 1]));
+#pragma unroll
+        for (int i = 16; i < TILE; i += 16)
+#pragma unroll
+          for (int a = 0; a < 8; a++)
+            tm[a] = fmaxf(tm[a], fmaxf(__uint_as_float(s[i + 2 * a]), __uint_as_float(s[i + 2 * a + 1])));
+        tmax = fmaxf(fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3])), fmaxf(fmaxf(tm[4], tm[5]), fmaxf(tm[6], tm[7])));
       }
       tmax *= c;
 

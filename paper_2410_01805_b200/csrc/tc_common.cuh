@@ -44,11 +44,27 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// Non-suspending test of a phase: returns at once (try_wait may park the thread for a while even
+// when the phase has already completed).
+__device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.b32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 // Bounded wait.  `abort_flag` (shared memory) is set by whoever gives up first so that the
 // other roles stop waiting as well.  Returns false if the wait was abandoned.
 template <int BACKOFF_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
                                           int *status) {
+  if (mbar_test_wait(bar, parity)) return true;
   for (uint32_t i = 0; i < WAIT_LIMIT; i++) {
     if (mbar_try_wait(bar, parity)) return true;
     if (BACKOFF_NS > 0) __nanosleep(BACKOFF_NS);  // leave the issue slots to the warps that have work
