@@ -90,6 +90,9 @@ __global__ void __launch_bounds__(GT_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                bf16 *__restrict__ C, int ldc, int M, int N, int K, const float *__restrict__ W2,
                float *__restrict__ partial, int h_kv, int act, int *status) {
+  // Persistent: CTA b computes tiles b, b + gridDim.x, ... (row-block major, so that concurrent
+  // CTAs share the A row block in L2).  The accumulator is double-buffered in TMEM: the epilogue
+  // of one tile overlaps the main loop of the next.
   using Cfg = GemmCfg<BN>;
   constexpr int STAGES = Cfg::STAGES;
   extern __shared__ unsigned char smem_raw[];
@@ -100,31 +103,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   unsigned char *tail = tiles + STAGES * Cfg::STAGE_BYTES + (MODE == 1 ? Cfg::W2_BYTES : 0);
   uint64_t *full = reinterpret_cast<uint64_t *>(tail);
   uint64_t *empty = full + STAGES;
-  uint64_t *acc_full = empty + STAGES;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+  uint64_t *acc_full = empty + STAGES;   // [2]
+  uint64_t *acc_empty = acc_full + 2;    // [2]
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
   const int KB = K / BK;
+  const int tiles_n = (N + BN - 1) / BN;
+  const int total = ((M + BM - 1) / BM) * tiles_n;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; s++) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    mbar_init(acc_full, 1);
+    for (int i = 0; i < 2; i++) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 4); }
     *abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&map_a);
     prefetch_tmap(&map_b);
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, BN);
+    tmem_alloc(tmem_slot, 2 * BN);
     tmem_relinquish();
-  }
-  if (MODE == 1) {
-    for (int v = threadIdx.x; v < BN * h_kv; v += GT_THREADS) {
-      int c = v / h_kv;
-      sW2[v] = (n0 + c < N) ? W2[(size_t)(n0 + c) * h_kv + (v - c * h_kv)] : 0.f;
-    }
   }
   tc_fence_before();
   __syncthreads();
@@ -133,125 +132,165 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   if (warp == 0) {
     if (lane == 0) {
-      for (int kb = 0; kb < KB; kb++) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, status)) break;
-        mbar_expect_tx(&full[s], Cfg::STAGE_BYTES);
-        unsigned char *a_dst = tiles + s * Cfg::STAGE_BYTES;
-        tma_load_2d(a_dst, &map_a, kb * BK, m0, &full[s]);
-        tma_load_2d(a_dst + Cfg::A_BYTES, &map_b, kb * BK, n0, &full[s]);
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
+        const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+        for (int kb = 0; kb < KB; kb++, it++) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          ok = mbar_wait(&empty[s], ph ^ 1, abort_flag, status);
+          if (!ok) break;
+          mbar_expect_tx(&full[s], Cfg::STAGE_BYTES);
+          unsigned char *a_dst = tiles + s * Cfg::STAGE_BYTES;
+          tma_load_2d(a_dst, &map_a, kb * BK, m0, &full[s]);
+          tma_load_2d(a_dst + Cfg::A_BYTES, &map_b, kb * BK, n0, &full[s]);
+        }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc = idesc_bf16(BM, BN, 0, 0);
+      uint32_t it = 0, lt = 0;
       bool ok = true;
-      for (int kb = 0; kb < KB && ok; kb++) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        ok = mbar_wait(&full[s], ph, abort_flag, status);
+      for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, lt++) {
+        const uint32_t buf = lt & 1;
+        ok = mbar_wait(&acc_empty[buf], ((lt >> 1) & 1) ^ 1, abort_flag, status);
         if (!ok) break;
         tc_fence_after();
-        unsigned char *a_src = tiles + s * Cfg::STAGE_BYTES;
-        const uint64_t da = desc_kmajor_sw128(a_src), db = desc_kmajor_sw128(a_src + Cfg::A_BYTES);
+        const uint32_t d_tmem = tmem_base + buf * BN;
+        for (int kb = 0; kb < KB; kb++, it++) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          ok = mbar_wait(&full[s], ph, abort_flag, status);
+          if (!ok) break;
+          tc_fence_after();
+          unsigned char *a_src = tiles + s * Cfg::STAGE_BYTES;
+          const uint64_t da = desc_kmajor_sw128(a_src), db = desc_kmajor_sw128(a_src + Cfg::A_BYTES);
 #pragma unroll
-        for (int k = 0; k < BK / 16; k++)
-          mma_ss(tmem_base, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) != 0);
-        mma_commit(&empty[s]);  // frees the stage once these MMAs have read it
+          for (int k = 0; k < BK / 16; k++) {
+            if (kb == 0 && k == 0) mma_ss_first(d_tmem, da, db, idesc);
+            else mma_ss_acc(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc);
+          }
+          mma_commit(&empty[s]);  // frees the stage once these MMAs have read it
+        }
+        if (ok) mma_commit(&acc_full[buf]);
       }
-      mma_commit(acc_full);
     }
   } else {
     // epilogue warps 2..5: TMEM lane quarter = warp % 4
     const int quarter = warp & 3;
-    const int row = m0 + quarter * 32 + lane;
-    const bool ok = mbar_wait(acc_full, 0, abort_flag, status);
-    tc_fence_after();
-    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    if (MODE == 0) {
-      if (ok) {
-#pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 32) {
-          uint32_t r[32];
-          tmem_ld32(taddr + c0, r);
-          tmem_wait_ld();
-          if (row < M && n0 + c0 < N) {
-            uint4 *dst = reinterpret_cast<uint4 *>(C + (size_t)row * ldc + n0 + c0);
-#pragma unroll
-            for (int v = 0; v < 4; v++) {
-              uint4 o;
-              o.x = pack_bf16(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1]));
-              o.y = pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
-              o.z = pack_bf16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]));
-              o.w = pack_bf16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]));
-              dst[v] = o;
-            }
-          }
+    const int etid = threadIdx.x - 64;  // 0..127 among the epilogue threads
+    uint32_t lt = 0;
+    bool ok = true;
+    // (no early exit: after a timed-out wait the warps still meet at the named barrier)
+    for (int tile = blockIdx.x; tile < total; tile += gridDim.x, lt++) {
+      const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+      const uint32_t buf = lt & 1;
+      const int row = m0 + quarter * 32 + lane;
+      if (MODE == 1) {
+        // this tile's slice of W2; the named barrier keeps the four warps together around it
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        for (int v = etid; v < BN * h_kv; v += 128) {
+          int c = v / h_kv;
+          sW2[v] = (n0 + c < N) ? W2[(size_t)(n0 + c) * h_kv + (v - c * h_kv)] : 0.f;
         }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
       }
-    } else {
-      float sc[MAX_HKV];
-#pragma unroll
-      for (int m = 0; m < MAX_HKV; m++) sc[m] = 0.f;
-      if (ok) {
+      if (ok) ok = mbar_wait(&acc_full[buf], (lt >> 1) & 1, abort_flag, status);
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
+      if (MODE == 0) {
+        if (ok) {
 #pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 32) {
-          uint32_t r[32];
-          tmem_ld32(taddr + c0, r);
-          tmem_wait_ld();
-          // activation of the 32 columns first (independent, so the special-function unit
-          // pipelines them), then the thin GEMM with W2 as broadcast 16-byte loads
-          float a[32];
+          for (int c0 = 0; c0 < BN; c0 += 32) {
+            uint32_t r[32];
+            tmem_ld32(taddr + c0, r);
+            tmem_wait_ld();
+            if (row < M && n0 + c0 < N) {
+              uint4 *dst = reinterpret_cast<uint4 *>(C + (size_t)row * ldc + n0 + c0);
 #pragma unroll
-          for (int i = 0; i < 32; i++) a[i] = fast_act(__uint_as_float(r[i]), act);
-          if (h_kv == 8) {
-#pragma unroll
-            for (int i = 0; i < 32; i++) {
-              const float4 w0 = *reinterpret_cast<const float4 *>(sW2 + (c0 + i) * 8);
-              const float4 w1 = *reinterpret_cast<const float4 *>(sW2 + (c0 + i) * 8 + 4);
-              sc[0] = fmaf(a[i], w0.x, sc[0]); sc[1] = fmaf(a[i], w0.y, sc[1]);
-              sc[2] = fmaf(a[i], w0.z, sc[2]); sc[3] = fmaf(a[i], w0.w, sc[3]);
-              sc[4] = fmaf(a[i], w1.x, sc[4]); sc[5] = fmaf(a[i], w1.y, sc[5]);
-              sc[6] = fmaf(a[i], w1.z, sc[6]); sc[7] = fmaf(a[i], w1.w, sc[7]);
-            }
-          } else if (h_kv == 32) {
-#pragma unroll
-            for (int i = 0; i < 32; i++) {
-              const float4 *w = reinterpret_cast<const float4 *>(sW2 + (c0 + i) * 32);
-#pragma unroll
-              for (int m4 = 0; m4 < 8; m4++) {
-                const float4 wv = w[m4];
-                sc[4 * m4 + 0] = fmaf(a[i], wv.x, sc[4 * m4 + 0]);
-                sc[4 * m4 + 1] = fmaf(a[i], wv.y, sc[4 * m4 + 1]);
-                sc[4 * m4 + 2] = fmaf(a[i], wv.z, sc[4 * m4 + 2]);
-                sc[4 * m4 + 3] = fmaf(a[i], wv.w, sc[4 * m4 + 3]);
+              for (int v = 0; v < 4; v++) {
+                uint4 o;
+                o.x = pack_bf16(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1]));
+                o.y = pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
+                o.z = pack_bf16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]));
+                o.w = pack_bf16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]));
+                dst[v] = o;
               }
             }
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; i++) {
-              const float *w = sW2 + (c0 + i) * h_kv;
-#pragma unroll
-              for (int m = 0; m < MAX_HKV; m++)
-                if (m < h_kv) sc[m] = fmaf(a[i], w[m], sc[m]);
-            }
           }
         }
-        if (row < M) {
-          float *dst = partial + ((size_t)blockIdx.x * M + row) * h_kv;
+      } else {
+        float sc[MAX_HKV];
 #pragma unroll
-          for (int m = 0; m < MAX_HKV; m++)
-            if (m < h_kv) dst[m] = sc[m];
+        for (int m = 0; m < MAX_HKV; m++) sc[m] = 0.f;
+        if (ok) {
+#pragma unroll 1
+          for (int c0 = 0; c0 < BN; c0 += 32) {
+            uint32_t r[32];
+            tmem_ld32(taddr + c0, r);
+            tmem_wait_ld();
+            // activation of the 32 columns first (independent, so the special-function unit
+            // pipelines them), then the thin GEMM with W2 as broadcast 16-byte loads
+            float a[32];
+#pragma unroll
+            for (int i = 0; i < 32; i++) a[i] = fast_act(__uint_as_float(r[i]), act);
+            if (h_kv == 8) {
+#pragma unroll
+              for (int i = 0; i < 32; i++) {
+                const float4 w0 = *reinterpret_cast<const float4 *>(sW2 + (c0 + i) * 8);
+                const float4 w1 = *reinterpret_cast<const float4 *>(sW2 + (c0 + i) * 8 + 4);
+                sc[0] = fmaf(a[i], w0.x, sc[0]); sc[1] = fmaf(a[i], w0.y, sc[1]);
+                sc[2] = fmaf(a[i], w0.z, sc[2]); sc[3] = fmaf(a[i], w0.w, sc[3]);
+                sc[4] = fmaf(a[i], w1.x, sc[4]); sc[5] = fmaf(a[i], w1.y, sc[5]);
+                sc[6] = fmaf(a[i], w1.z, sc[6]); sc[7] = fmaf(a[i], w1.w, sc[7]);
+              }
+            } else if (h_kv == 32) {
+#pragma unroll
+              for (int i = 0; i < 32; i++) {
+                const float4 *w = reinterpret_cast<const float4 *>(sW2 + (c0 + i) * 32);
+#pragma unroll
+                for (int m4 = 0; m4 < 8; m4++) {
+                  const float4 wv = w[m4];
+                  sc[4 * m4 + 0] = fmaf(a[i], wv.x, sc[4 * m4 + 0]);
+                  sc[4 * m4 + 1] = fmaf(a[i], wv.y, sc[4 * m4 + 1]);
+                  sc[4 * m4 + 2] = fmaf(a[i], wv.z, sc[4 * m4 + 2]);
+                  sc[4 * m4 + 3] = fmaf(a[i], wv.w, sc[4 * m4 + 3]);
+                }
+              }
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; i++) {
+                const float *w = sW2 + (c0 + i) * h_kv;
+#pragma unroll
+                for (int m = 0; m < MAX_HKV; m++)
+                  if (m < h_kv) sc[m] = fmaf(a[i], w[m], sc[m]);
+              }
+            }
+          }
+          if (row < M) {
+            float *dst = partial + ((size_t)(tile % tiles_n) * M + row) * h_kv;
+#pragma unroll
+            for (int m = 0; m < MAX_HKV; m++)
+              if (m < h_kv) dst[m] = sc[m];
+          }
         }
       }
+      // every tcgen05.ld of this warp has completed (wait::ld above): the buffer may be reused
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[buf]);
     }
   }
 
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  if (warp == 1) tmem_dealloc(tmem_base, BN);
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc(tmem_base, 2 * BN);
+  }
 }
 
 struct MapCache {
@@ -299,7 +338,17 @@ cudaError_t launch_t(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, i
   const CUtensorMap *ma = cached_map(A, K, M, (uint64_t)lda * 2, BM);
   const CUtensorMap *mb = cached_map(Bt, K, N, (uint64_t)ldb * 2, BN);
   if (!ma || !mb) return cudaErrorInvalidValue;
-  dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM);
+  static int num_sms = 0;
+  if (num_sms == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0) {
+      cudaGetLastError();
+      num_sms = 148;
+    }
+  }
+  const int total = ((N + BN - 1) / BN) * ((M + BM - 1) / BM);
+  const int grid = total < num_sms ? total : num_sms;
   gemm_tc_kernel<BN, MODE><<<grid, GT_THREADS, Cfg::smem_bytes(MODE), st>>>(
       *ma, *mb, C, ldc, M, N, K, W2, partial, h_kv, act, status);
   return cudaGetLastError();
