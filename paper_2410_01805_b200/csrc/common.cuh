@@ -108,6 +108,10 @@ struct RopeAppendArgs {
   int64_t seen;
 };
 cudaError_t launch_rope_append(const RopeAppendArgs &a, cudaStream_t st);
+// The projection GEMM with rope_append's work done in its epilogue (a.staging is written, not read).
+bool qkv_rope_tc_supported(int M, int N, int K, int lda, int ldb, int d);
+cudaError_t launch_qkv_rope_tc(const bf16 *X, int ldx, const bf16 *Wt, int ldw, bf16 *staging, int M,
+                               int N, int K, const RopeAppendArgs &a, int *status, cudaStream_t st);
 
 // Attention (Eq. 1): query row t of head j sees keys [0, len + t] of KV head j / g.
 cudaError_t launch_attention_mma(const bf16 *q_rot, const bf16 *k_rot, const bf16 *v, bf16 *out,

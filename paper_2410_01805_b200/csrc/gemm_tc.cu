@@ -65,6 +65,7 @@ using namespace tc;
 
 constexpr int BM = 128, BK = 64, GT_THREADS = 192;
 constexpr int MAX_HKV = 32;
+constexpr int EPI_WARP_BYTES = 32 * 128 * 2;  // 32 rows of a head of up to 128 bf16
 
 // sigma of the retaining head with the fast division / exponential intrinsics (relative error
 // ~1e-6, far inside the score tolerance)
@@ -79,17 +80,18 @@ struct GemmCfg {
   static constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int W2_BYTES = BN * MAX_HKV * 4;
+  static constexpr int EPI_BYTES = 4 * EPI_WARP_BYTES;  // MODE 2: one staged head of 32 rows per warp
   // 1024 for alignment slack, barriers + tmem pointer in a small tail
   static constexpr int smem_bytes(int mode) {
-    return 1024 + STAGES * STAGE_BYTES + (mode == 1 ? W2_BYTES : 0) + 256;
+    return 1024 + STAGES * STAGE_BYTES + (mode == 1 ? W2_BYTES : (mode == 2 ? EPI_BYTES : 0)) + 256;
   }
 };
 
-template <int BN, int MODE>
+template <int BN, int MODE, int HD = 0>
 __global__ void __launch_bounds__(GT_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                bf16 *__restrict__ C, int ldc, int M, int N, int K, const float *__restrict__ W2,
-               float *__restrict__ partial, int h_kv, int act, int *status) {
+               float *__restrict__ partial, int h_kv, int act, const RopeAppendArgs ra, int *status) {
   // Persistent: CTA b computes tiles b, b + gridDim.x, ... (row-block major, so that concurrent
   // CTAs share the A row block in L2).  The accumulator is double-buffered in TMEM: the epilogue
   // of one tile overlaps the main loop of the next.
@@ -100,7 +102,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   unsigned char *tiles = smem;
   float *sW2 = reinterpret_cast<float *>(tiles + STAGES * Cfg::STAGE_BYTES);
-  unsigned char *tail = tiles + STAGES * Cfg::STAGE_BYTES + (MODE == 1 ? Cfg::W2_BYTES : 0);
+  unsigned char *sEpi = tiles + STAGES * Cfg::STAGE_BYTES;
+  unsigned char *tail = tiles + STAGES * Cfg::STAGE_BYTES +
+                        (MODE == 1 ? Cfg::W2_BYTES : (MODE == 2 ? Cfg::EPI_BYTES : 0));
   uint64_t *full = reinterpret_cast<uint64_t *>(tail);
   uint64_t *empty = full + STAGES;
   uint64_t *acc_full = empty + STAGES;   // [2]
@@ -197,6 +201,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
       }
+      // MODE 2: (cos, sin) of this thread's position for every rotation pair, fetched while the
+      // tile's MMAs are still running
+      float4 csr[MODE == 2 ? HD / 4 : 1];
+      if (MODE == 2) {
+        const float4 *cs4 = reinterpret_cast<const float4 *>(ra.cs + (size_t)(ra.len + row) * (HD / 2));
+#pragma unroll
+        for (int i = 0; i < HD / 4; i++) csr[i] = row < M ? __ldg(cs4 + i) : make_float4(1.f, 0.f, 1.f, 0.f);
+      }
       if (ok) ok = mbar_wait(&acc_full[buf], (lt >> 1) & 1, abort_flag, status);
       tc_fence_after();
       const uint32_t taddr = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
@@ -219,6 +231,100 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 dst[v] = o;
               }
             }
+          }
+        }
+      } else if (MODE == 2) {
+        // QKV projection with the chunk's positions, RoPE and cache append in the epilogue: a
+        // tile holds BN / HD whole heads, so both halves (i, i + HD/2) of every rotation pair
+        // are in this thread's TMEM row.  The rotation starts from the bf16-rounded projection,
+        // the value the pre-RoPE cache stores.  Each warp stages its 32 rows of one head in
+        // shared memory (16-byte pieces XOR-swizzled by row) and writes them out as whole rows,
+        // so the global stores are full lines.
+        if (ok) {
+          constexpr int HALF = HD / 2, VPR = HD / 8, VMASK = VPR - 1, ROW_B = HD * 2;
+          const int d_in = (ra.h + 2 * ra.h_kv) * HD;
+          const int wrow0 = m0 + quarter * 32;  // first row of this warp
+          unsigned char *buf_w = sEpi + quarter * EPI_WARP_BYTES;
+          unsigned char *my_row = buf_w + lane * ROW_B;
+          // rows [wrow0, wrow0 + 32) of the staged head -> dst + r * stride (elements)
+          auto copy_out = [&](bf16 *dst, size_t stride) {
+#pragma unroll 4
+            for (int i = 0; i < VPR; i++) {
+              const int idx = lane + 32 * i, r = idx / VPR, j = idx % VPR;
+              if (wrow0 + r < M)
+                *reinterpret_cast<uint4 *>(dst + (size_t)r * stride + j * 8) =
+                    *reinterpret_cast<const uint4 *>(buf_w + r * ROW_B + ((j ^ (r & VMASK)) << 4));
+            }
+          };
+#pragma unroll 1
+          for (int hc = 0; hc < BN; hc += HD) {
+            const int col0 = n0 + hc;
+            if (col0 >= N) break;
+            const int hd = col0 / HD;
+            const bool is_v = hd >= ra.h + ra.h_kv, is_k = !is_v && hd >= ra.h;
+            const int m = is_v ? hd - ra.h - ra.h_kv : hd - ra.h;
+            const size_t cache_off = ((size_t)m * ra.cap + ra.len + wrow0) * HD;
+            // pass A: the projection as stored (staging, pre-RoPE key cache, value cache)
+#pragma unroll 1
+            for (int c0 = 0; c0 < HD; c0 += 32) {
+              uint32_t r[32];
+              tmem_ld32(taddr + hc + c0, r);
+              tmem_wait_ld();
+#pragma unroll
+              for (int v = 0; v < 4; v++) {
+                uint4 o;
+                o.x = pack_bf16(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1]));
+                o.y = pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
+                o.z = pack_bf16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]));
+                o.w = pack_bf16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]));
+                *reinterpret_cast<uint4 *>(my_row + ((((c0 >> 3) + v) ^ (lane & VMASK)) << 4)) = o;
+              }
+            }
+            __syncwarp();
+            copy_out(C + (size_t)wrow0 * ldc + col0, ldc);
+            if (is_v) {
+              copy_out(ra.v + cache_off, HD);
+              if (ra.z_post) copy_out(ra.z_post + (size_t)wrow0 * d_in + col0, d_in);
+            } else if (is_k && ra.k_pre) {
+              copy_out(ra.k_pre + cache_off, HD);
+            }
+            __syncwarp();
+            if (is_v) continue;
+            // pass B: rotated at position = slot
+#pragma unroll
+            for (int c0 = 0; c0 < HALF; c0 += 32) {
+              uint32_t lo[32], hi[32];
+              tmem_ld32(taddr + hc + c0, lo);
+              tmem_ld32(taddr + hc + HALF + c0, hi);
+              tmem_wait_ld();
+#pragma unroll
+              for (int v = 0; v < 4; v++) {
+                uint32_t ol[4], oh[4];
+#pragma unroll
+                for (int q = 0; q < 4; q++) {
+                  const float4 t = csr[(c0 >> 1) + 4 * v + q];  // (cos, sin) of two pairs
+                  const uint32_t wl = pack_bf16(__uint_as_float(lo[8 * v + 2 * q]), __uint_as_float(lo[8 * v + 2 * q + 1]));
+                  const uint32_t wh = pack_bf16(__uint_as_float(hi[8 * v + 2 * q]), __uint_as_float(hi[8 * v + 2 * q + 1]));
+                  const float x0 = __uint_as_float(wl << 16), x1 = __uint_as_float(wl & 0xffff0000u);
+                  const float y0 = __uint_as_float(wh << 16), y1 = __uint_as_float(wh & 0xffff0000u);
+                  // lower half: x cos − y sin ; upper half: y cos + x sin
+                  ol[q] = pack_bf16(x0 * t.x - y0 * t.y, x1 * t.z - y1 * t.w);
+                  oh[q] = pack_bf16(y0 * t.x + x0 * t.y, y1 * t.z + x1 * t.w);
+                }
+                const int jl = (c0 >> 3) + v, jh = jl + (HALF >> 3);
+                *reinterpret_cast<uint4 *>(my_row + ((jl ^ (lane & VMASK)) << 4)) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+                *reinterpret_cast<uint4 *>(my_row + ((jh ^ (lane & VMASK)) << 4)) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
+              }
+            }
+            __syncwarp();
+            if (is_k) {
+              copy_out(ra.k_rot + cache_off, HD);
+              if (row < M) ra.tid[(size_t)m * ra.cap + ra.len + row] = ra.seen + row;
+            } else {
+              copy_out(ra.q_rot + (size_t)wrow0 * ra.h * HD + (size_t)hd * HD, (size_t)ra.h * HD);
+            }
+            if (ra.z_post) copy_out(ra.z_post + (size_t)wrow0 * d_in + col0, d_in);
+            __syncwarp();
           }
         }
       } else {
@@ -322,14 +428,14 @@ const CUtensorMap *cached_map(const void *base, uint64_t inner, uint64_t outer, 
   return &c.map;
 }
 
-template <int BN, int MODE>
+template <int BN, int MODE, int HD = 0>
 cudaError_t launch_t(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, int ldc, int M, int N,
-                     int K, const float *W2, float *partial, int h_kv, int act, int *status,
-                     cudaStream_t st) {
+                     int K, const float *W2, float *partial, int h_kv, int act, const RopeAppendArgs &ra,
+                     int *status, cudaStream_t st) {
   using Cfg = GemmCfg<BN>;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, MODE>,
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, MODE, HD>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          Cfg::smem_bytes(MODE));
     if (e != cudaSuccess) return e;
@@ -349,8 +455,8 @@ cudaError_t launch_t(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, i
   }
   const int total = ((N + BN - 1) / BN) * ((M + BM - 1) / BM);
   const int grid = total < num_sms ? total : num_sms;
-  gemm_tc_kernel<BN, MODE><<<grid, GT_THREADS, Cfg::smem_bytes(MODE), st>>>(
-      *ma, *mb, C, ldc, M, N, K, W2, partial, h_kv, act, status);
+  gemm_tc_kernel<BN, MODE, HD><<<grid, GT_THREADS, Cfg::smem_bytes(MODE), st>>>(
+      *ma, *mb, C, ldc, M, N, K, W2, partial, h_kv, act, ra, status);
   return cudaGetLastError();
 }
 
@@ -363,8 +469,22 @@ bool gemm_tc_supported(int M, int N, int K, int lda, int ldb) {
 cudaError_t launch_gemm_tc(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, int ldc, int M,
                            int N, int K, int *status, cudaStream_t st) {
   if (N >= 256)
-    return launch_t<256, 0>(A, lda, Bt, ldb, C, ldc, M, N, K, nullptr, nullptr, 0, 0, status, st);
-  return launch_t<128, 0>(A, lda, Bt, ldb, C, ldc, M, N, K, nullptr, nullptr, 0, 0, status, st);
+    return launch_t<256, 0>(A, lda, Bt, ldb, C, ldc, M, N, K, nullptr, nullptr, 0, 0, RopeAppendArgs{}, status, st);
+  return launch_t<128, 0>(A, lda, Bt, ldb, C, ldc, M, N, K, nullptr, nullptr, 0, 0, RopeAppendArgs{}, status, st);
+}
+
+// QKV projection whose epilogue also assigns positions, rotates Q and K and appends K, V to the
+// cache (what rope_append_kernel does in a pass of its own): head_dim 64 or 128, so that a
+// 256-column tile holds whole heads.
+bool qkv_rope_tc_supported(int M, int N, int K, int lda, int ldb, int d) {
+  return gemm_tc_supported(M, N, K, lda, ldb) && N >= 256 && (d == 64 || d == 128) && N % d == 0;
+}
+
+cudaError_t launch_qkv_rope_tc(const bf16 *X, int ldx, const bf16 *Wt, int ldw, bf16 *staging, int M,
+                               int N, int K, const RopeAppendArgs &ra, int *status, cudaStream_t st) {
+  if (ra.d == 128)
+    return launch_t<256, 2, 128>(X, ldx, Wt, ldw, staging, N, M, N, K, nullptr, nullptr, 0, 0, ra, status, st);
+  return launch_t<256, 2, 64>(X, ldx, Wt, ldw, staging, N, M, N, K, nullptr, nullptr, 0, 0, ra, status, st);
 }
 
 // Tile width of the retaining-head GEMM: the widest of 256 / 128 / 64 columns that still gives
@@ -385,10 +505,10 @@ cudaError_t launch_rh_gemm_tc(const bf16 *A, int lda, const bf16 *W1t, const flo
   const int bn = rh_tile_n(M, d_R);
   *n_tiles = (d_R + bn - 1) / bn;
   if (bn == 256)
-    return launch_t<256, 1>(A, lda, W1t, K, nullptr, 0, M, d_R, K, W2, partial, h_kv, act, status, st);
+    return launch_t<256, 1>(A, lda, W1t, K, nullptr, 0, M, d_R, K, W2, partial, h_kv, act, RopeAppendArgs{}, status, st);
   if (bn == 128)
-    return launch_t<128, 1>(A, lda, W1t, K, nullptr, 0, M, d_R, K, W2, partial, h_kv, act, status, st);
-  return launch_t<64, 1>(A, lda, W1t, K, nullptr, 0, M, d_R, K, W2, partial, h_kv, act, status, st);
+    return launch_t<128, 1>(A, lda, W1t, K, nullptr, 0, M, d_R, K, W2, partial, h_kv, act, RopeAppendArgs{}, status, st);
+  return launch_t<64, 1>(A, lda, W1t, K, nullptr, 0, M, d_R, K, W2, partial, h_kv, act, RopeAppendArgs{}, status, st);
 }
 
 }  // namespace locret

@@ -80,6 +80,7 @@ struct locret_layer {
   bool serialize;  // timing mode 2: keep every kernel on the main stream (clean per-kernel times)
   bool attn_only;  // timing mode 3: bracket only the attention kernel (least overhead)
   bool use_tc;  // tcgen05 kernels (default); LOCRET_LEGACY_MMA=1 keeps the mma.sync kernels for A/B runs
+  bool fuse_rope;  // RoPE + append in the projection's epilogue (LOCRET_UNFUSED_ROPE=1 disables)
   bool use_side;  // off-critical-path kernels go to the pool's second stream (LOCRET_SERIAL=1 disables)
   bool side_pending;
   cudaEvent_t ev_ready, ev_attn, ev_side;
@@ -230,6 +231,8 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
     L->use_tc = !(e && e[0] == '1');
     const char *ser = getenv("LOCRET_SERIAL");
     L->use_side = !(ser && ser[0] == '1');
+    const char *unf = getenv("LOCRET_UNFUSED_ROPE");
+    L->fuse_rope = !(unf && unf[0] == '1');
     L->side_pending = false;
     L->ev_ready = L->ev_attn = L->ev_side = nullptr;
   }
@@ -385,10 +388,30 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
   }
 
   const bool decode = n_tok == 1 && L->use_tc;  // one token: bandwidth-bound kernels of decode.cu
+  // a 4-bit cache is expanded into bf16 scratch first: keys rotated at position = slot
+  bf16 *const k_att = L->int4 ? P->k_exp : L->k_rot;
+  bf16 *const v_att = L->int4 ? P->v_exp : L->v[c];
+  RopeAppendArgs ra;  // positions, RoPE, append of the chunk's units at slots [len, len + n_tok)
+  ra.staging = staging; ra.q_rot = P->q_rot;
+  ra.z_post = L->cfg.rh_input == 1 ? z_post : nullptr;
+  ra.k_pre = L->int4 ? nullptr : L->k_pre[c]; ra.k_rot = k_att; ra.v = v_att; ra.tid = L->tid[c]; ra.cs = L->cs;
+  ra.n_tok = n_tok; ra.h = L->h; ra.h_kv = L->h_kv; ra.d = L->d; ra.cap = L->cap; ra.len = L->len;
+  ra.seen = L->seen;
+  // with a tensor-core projection and head_dim 64 / 128 the epilogue of the GEMM does the RoPE pass
+  const bool fused_rope = !decode && L->fuse_rope && L->use_tc && n_tok >= 32 &&
+                          qkv_rope_tc_supported(n_tok, L->d_in, L->D, L->D, L->D, L->d);
+  if (L->int4 && L->len > 0) {
+    // the expansion writes slots [0, len) of the scratch the chunk's units are appended to
+    Timed t(L, LOCRET_K_DEQUANT);
+    CK(launch_dequant(L->q4[c], P->k_exp, P->v_exp, L->cs, L->h_kv, L->d, L->cap, L->len, true, L->st));
+  }
   {  // (a) projections
     Timed t(L, LOCRET_K_QKV);
     if (decode)
       CK(launch_gemv((const bf16 *)hidden_in, L->wqkv_t, L->d_in, L->D, staging, L->st));
+    else if (fused_rope)
+      CK(launch_qkv_rope_tc((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, staging, n_tok, L->d_in, L->D,
+                            ra, L->d_status, L->st));
     else if (L->use_tc && n_tok >= 32 && gemm_tc_supported(n_tok, L->d_in, L->D, L->D, L->D))
       CK(launch_gemm_tc((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, staging, L->d_in, n_tok,
                         L->d_in, L->D, L->d_status, L->st));
@@ -396,22 +419,9 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
       CK(launch_gemm_bf16((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, staging, L->d_in, n_tok,
                           L->d_in, L->D, L->st));
   }
-  // a 4-bit cache is expanded into bf16 scratch first: keys rotated at position = slot
-  bf16 *const k_att = L->int4 ? P->k_exp : L->k_rot;
-  bf16 *const v_att = L->int4 ? P->v_exp : L->v[c];
-  if (L->int4 && L->len > 0) {
-    Timed t(L, LOCRET_K_DEQUANT);
-    CK(launch_dequant(L->q4[c], P->k_exp, P->v_exp, L->cs, L->h_kv, L->d, L->cap, L->len, true, L->st));
-  }
-  {  // positions, RoPE, append of the chunk's units at slots [len, len + n_tok)
+  if (!fused_rope) {
     Timed t(L, LOCRET_K_ROPE);
-    RopeAppendArgs a;
-    a.staging = staging; a.q_rot = P->q_rot;
-    a.z_post = L->cfg.rh_input == 1 ? z_post : nullptr;
-    a.k_pre = L->int4 ? nullptr : L->k_pre[c]; a.k_rot = k_att; a.v = v_att; a.tid = L->tid[c]; a.cs = L->cs;
-    a.n_tok = n_tok; a.h = L->h; a.h_kv = L->h_kv; a.d = L->d; a.cap = L->cap; a.len = L->len;
-    a.seen = L->seen;
-    CK(launch_rope_append(a, L->st));
+    CK(launch_rope_append(ra, L->st));
   }
   if (L->int4) {  // the chunk's units enter the cache quantised (keys pre-RoPE)
     Timed t(L, LOCRET_K_QUANT);
