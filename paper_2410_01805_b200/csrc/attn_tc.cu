@@ -4,14 +4,15 @@
 // One CTA owns two 128-row query tiles that share a KV head (two query heads of one GQA
 // group over the same rows, or two consecutive row blocks of one head) and streams the
 // keys/values of that head in tiles of 128 through shared memory with TMA.  Roles:
-//   warps 0-3 / 4-7  softmax of query tile 0 / 1: one thread per query row reads its row of
-//                    S = Q K^T from TMEM, keeps a running maximum and sum, writes
-//                    P = exp2(S - max) as bf16 back into TMEM over S (handed to the MMA issuer in
-//                    two halves), and rescales the accumulator in TMEM only when the maximum has
-//                    grown by more than 2^100.  The two warpgroups take strict turns, so that one
-//                    tile's softmax runs while the other tile's MMAs execute; left alone the two
-//                    tiles drift into phase and tensor pipe and softmax alternate instead of
-//                    overlapping (measured: 1.3x slower).
+//   warps 0-7        softmax, one query tile at a time (tile 0 and tile 1 alternately, so one
+//                    tile's softmax runs while the other tile's MMAs execute).  A warp may only
+//                    touch TMEM lanes 32 (w % 4) .. +31, so warps q and 4 + q share the 32 rows of
+//                    quarter q and split the tile's 128 keys in halves: each thread reads half a
+//                    row of S = Q K^T from TMEM, the pair exchanges its half maxima through shared
+//                    memory, and each writes P = exp2(S - max) as bf16 back into TMEM over S (the
+//                    first half releases the first four k-steps of P V, the second the rest).
+//                    The accumulator is rescaled in TMEM only when the maximum has grown by more
+//                    than 2^100.
 //   warp 8           TMA producer: Q once, then K and V tiles (two stages each), walking the
 //                    unmasked key tiles in a per-CTA rotated order, with an L2 prefetch ahead;
 //   warps 9 / 10     issue S_t = Q_t K_j^T (both operands in shared memory) and O_t += P_t V_j
@@ -30,12 +31,12 @@ namespace {
 
 using namespace tc;
 
-constexpr int AT_THREADS = 384;  // 3 warpgroups: softmax 0, softmax 1, {TMA, 2 MMA issuers, 1 idle warp}
+constexpr int AT_THREADS = 384;  // 3 warpgroups: softmax (two), {TMA, 2 MMA issuers, 1 idle warp}
 constexpr int TILE = 128;               // query rows per tile and keys per tile
 constexpr int HD = 128;                 // column pitch of a head in shared and tensor memory
 constexpr int HALF_BYTES = TILE * 128;  // one 64-column swizzled box of 128 rows: 16 KB
 constexpr int TILE_BYTES = 2 * HALF_BYTES;
-constexpr int AT_SMEM = 1024 + 6 * TILE_BYTES + 256;  // Q0,Q1,K0,K1,V0,V1 + barriers
+constexpr int AT_SMEM = 1024 + 6 * TILE_BYTES + 256 + 2048;  // Q0,Q1,K0,K1,V0,V1 + barriers + softmax exchange
 // The accumulator is rescaled only when a row's maximum has grown by more than 2^100 since the
 // scale in use was fixed.  P is stored as bf16 and O, l accumulate in fp32, both with an 8-bit
 // exponent, so P <= 2^100 and O <= keys * 2^100 * |v| (< 2^122 for 2^14 keys, |v| < 2^8) stay
@@ -104,8 +105,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   uint64_t *p_full = bars + 11;     // 2
   uint64_t *o_full = bars + 13;     // 2
   uint64_t *p_half = bars + 15;     // 2: first 64 keys of P_t written (p_full: all 128)
-  uint64_t *turn = bars + 17;       // 2: the two softmax warpgroups take turns (see below)
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 19);
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 17);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -144,7 +144,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(&k_empty[s], 2); mbar_init(&v_empty[s], 2);  // released by both MMA issuers
       mbar_init(&s_full[s], 1); mbar_init(&p_full[s], 4); mbar_init(&o_full[s], 1);
       mbar_init(&p_half[s], 4);
-      mbar_init(&turn[s], 4);
     }
     *abort_flag = 0;
     fence_barrier_init();
@@ -265,148 +264,145 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     }
   }
   } else {
-    // ------------------------------------------------------------ softmax, one row per thread
+    // ------------------------------------------------------------ softmax: all eight warps work
+    // on one query tile at a time, tile 0 and tile 1 alternately.  Warp w may only touch TMEM
+    // lanes 32 (w % 4) .. +31, so warps q and 4 + q share the 32 rows of quarter q and split
+    // the tile's 128 keys in halves: two warps per scheduler interleave their exponentials,
+    // while the other tile's MMAs run.  The pair exchanges its half maxima through shared
+    // memory around a 64-thread named barrier; that barrier also orders the first warp's read
+    // of S columns [32, 64) before the second warp's P (keys 64..127) overwrites them.
     setmaxnreg_inc<224>();
-    const int t = warp >> 2, quarter = warp & 3;
+    const int hf = warp >> 2, quarter = warp & 3;
     const int r = quarter * 32 + lane;
-    const int row = row0[t] + r;
-    const int limit = p.len + row;  // last visible key
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
-    const uint32_t s_addr = tmem_base + lane_off + t * TILE;
-    const uint32_t o_addr = tmem_base + lane_off + 2 * TILE + t * HD;
+    float *xch = reinterpret_cast<float *>(smem + 6 * TILE_BYTES + 256);  // [tile][half][128 rows]
     const float c = p.scale_log2;
-    float m_used = -INFINITY, l = 0.f;
+    float m_used[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
     bool ok = true;
-    // The two softmax warpgroups alternate strictly: while one computes, the other tile's MMAs
-    // run.  Left alone the two tiles drift into phase, both warpgroups then compute at the same
-    // time (sharing issue slots and the special-function unit) and the tensor pipe idles.
-    if (t == 1) { __syncwarp(); if (lane == 0) mbar_arrive(&turn[0]); }
+    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + quarter) : "memory"); };
 
-    for (int j = 0; j < NK && ok; j++) {
-      ok = mbar_wait(&s_full[t], j & 1, abort_flag, p.status);
-      if (!ok) break;
-      tc_fence_after();
-      uint32_t s[TILE];
+    for (int j = 0; j < NK; j++) {
+      // (no early exit: after a timed-out wait the pair still meets at its named barrier)
 #pragma unroll
-      for (int q = 0; q < 4; q++) tmem_ld32(s_addr + q * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[q * 32]));
-      tmem_wait_ld();
+      for (int t = 0; t < 2; t++) {
+        const int row = row0[t] + r;
+        const int limit = p.len + row;  // last visible key
+        const uint32_t s_addr = tmem_base + lane_off + t * TILE;
+        const uint32_t o_addr = tmem_base + lane_off + 2 * TILE + t * HD;
+        if (ok) ok = mbar_wait(&s_full[t], j & 1, abort_flag, p.status);
+        tc_fence_after();
+        uint32_t s[64];
+        tmem_ld32(s_addr + hf * 64, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+        tmem_ld32(s_addr + hf * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+        tmem_wait_ld();
 
-      const int key0 = tile_of(j) * TILE;
-      float tmax = -INFINITY;
-      if (key0 + TILE - 1 > p.len + row0[t]) {  // a tile that crosses the causal boundary
+        const int key0 = tile_of(j) * TILE;
+        float tmax;
+        if (key0 + TILE - 1 > p.len + row0[t]) {  // a tile that crosses the causal boundary
+          tmax = -INFINITY;
 #pragma unroll
-        for (int i = 0; i < TILE; i++) {
-          float x = (key0 + i <= limit) ? __uint_as_float(s[i]) : -INFINITY;
-          s[i] = __float_as_uint(x);
-          tmax = fmaxf(tmax, x);
-        }
-      } else {
-        float tm[8];
-#pragma unroll
-        for (int a = 0; a < 8; a++) tm[a] = fmaxf(__uint_as_float(s[2 * a]), __uint_as_float(s[2 * a + 1]));
-#pragma unroll
-        for (int i = 16; i < TILE; i += 16)
-#pragma unroll
-          for (int a = 0; a < 8; a++)
-            tm[a] = fmaxf(tm[a], fmaxf(__uint_as_float(s[i + 2 * a]), __uint_as_float(s[i + 2 * a + 1])));
-        tmax = fmaxf(fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3])), fmaxf(fmaxf(tm[4], tm[5]), fmaxf(tm[6], tm[7])));
-      }
-      tmax *= c;
-
-      if (j == 0) {
-        m_used = tmax;
-      } else {
-        const bool need = tmax > m_used + RESCALE_LOG2;
-        if (__any_sync(0xffffffffu, need)) {
-          // the accumulator must hold every product issued so far before it is rescaled
-          ok = mbar_wait(&o_full[t], (j - 1) & 1, abort_flag, p.status);
-          tc_fence_after();
-          float alpha = 1.0f;
-          if (need) { alpha = exp2f(m_used - tmax); m_used = tmax; }
-          l *= alpha;
-#pragma unroll 1
-          for (int q = 0; q < D / 32; q++) {
-            uint32_t o[32];
-            tmem_ld32(o_addr + q * 32, o);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; i++) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-            tmem_st32(o_addr + q * 32, o);
+          for (int i = 0; i < 64; i++) {
+            float x = (key0 + hf * 64 + i <= limit) ? __uint_as_float(s[i]) : -INFINITY;
+            s[i] = __float_as_uint(x);
+            tmax = fmaxf(tmax, x);
           }
-          tmem_wait_st();
-        }
-      }
-
-      // the turn covers the exponentials and the hand-over; loading S and its maximum above
-      // overlap the other tile's turn
-      ok = mbar_wait(&turn[t], j & 1, abort_flag, p.status);
-      if (!ok) break;
-      const uint64_t c2 = pack_f32x2(c, c), nm2 = pack_f32x2(-m_used, -m_used);
-      uint64_t la = pack_f32x2(0.f, 0.f), lb = la;
+        } else {
+          float tm[8];
 #pragma unroll
-      for (int q = 0; q < 2; q++) {
+          for (int a = 0; a < 8; a++) tm[a] = fmaxf(__uint_as_float(s[2 * a]), __uint_as_float(s[2 * a + 1]));
+#pragma unroll
+          for (int i = 16; i < 64; i += 16)
+#pragma unroll
+            for (int a = 0; a < 8; a++)
+              tm[a] = fmaxf(tm[a], fmaxf(__uint_as_float(s[i + 2 * a]), __uint_as_float(s[i + 2 * a + 1])));
+          tmax = fmaxf(fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3])), fmaxf(fmaxf(tm[4], tm[5]), fmaxf(tm[6], tm[7])));
+        }
+        xch[(t * 2 + hf) * TILE + r] = tmax;
+        pair_sync();
+        tmax = fmaxf(tmax, xch[(t * 2 + (hf ^ 1)) * TILE + r]) * c;
+
+        if (j == 0) {
+          m_used[t] = tmax;
+        } else {
+          // both warps of the pair see the same maxima, hence take the same branch
+          const bool need = tmax > m_used[t] + RESCALE_LOG2;
+          if (__any_sync(0xffffffffu, need)) {
+            // the accumulator must hold every product issued so far before it is rescaled
+            if (ok) ok = mbar_wait(&o_full[t], (j - 1) & 1, abort_flag, p.status);
+            tc_fence_after();
+            float alpha = 1.0f;
+            if (need) { alpha = exp2f(m_used[t] - tmax); m_used[t] = tmax; }
+            l[t] *= alpha;
+#pragma unroll 1
+            for (int q = hf; q < D / 32; q += 2) {  // the pair shares the accumulator's columns
+              uint32_t o[32];
+              tmem_ld32(o_addr + q * 32, o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; i++) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+              tmem_st32(o_addr + q * 32, o);
+            }
+            tmem_wait_st();
+            // the next product touches every column: both halves must be rescaled before either
+            // warp hands over its P
+            pair_sync();
+          }
+        }
+
+        const uint64_t c2 = pack_f32x2(c, c), nm2 = pack_f32x2(-m_used[t], -m_used[t]);
+        uint64_t la = pack_f32x2(0.f, 0.f), lb = la;
         uint32_t pk[32];
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
-          float x0, x1, p2, p3;
-          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[q * 64 + 2 * i]),
-                                            __uint_as_float(s[q * 64 + 2 * i + 1])), c2, nm2), x0, x1);
-          const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
-          const uint64_t xb = fma_f32x2(pack_f32x2(__uint_as_float(s[q * 64 + 2 * i + 2]),
-                                                   __uint_as_float(s[q * 64 + 2 * i + 3])), c2, nm2);
-          {
-            float x2, x3;
-            unpack_f32x2(xb, x2, x3);
-            p2 = ex2_approx(x2); p3 = ex2_approx(x3);
-          }
+          float x0, x1, x2, x3;
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), c2, nm2), x0, x1);
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[2 * i + 2]), __uint_as_float(s[2 * i + 3])), c2, nm2), x2, x3);
+          const float p0 = ex2_approx(x0), p1 = ex2_approx(x1), p2 = ex2_approx(x2), p3 = ex2_approx(x3);
           la = add_f32x2(la, pack_f32x2(p0, p1));
           lb = add_f32x2(lb, pack_f32x2(p2, p3));
           pk[i] = pack_bf16(p0, p1);
           pk[i + 1] = pack_bf16(p2, p3);
         }
-        tmem_st32(s_addr + q * 32, pk);
-        if (q == 0) {
-          tmem_wait_st();
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&p_half[t]);
+        tmem_st32(s_addr + hf * 32, pk);
+        {
+          float a0, a1, b0, b1;
+          unpack_f32x2(la, a0, a1);
+          unpack_f32x2(lb, b0, b1);
+          l[t] += (a0 + a1) + (b0 + b1);
         }
-      }
-      {
-        float a0, a1, b0, b1;
-        unpack_f32x2(la, a0, a1);
-        unpack_f32x2(lb, b0, b1);
-        l += (a0 + a1) + (b0 + b1);
-      }
-
-      tmem_wait_st();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(&p_full[t]);
-        mbar_arrive(&turn[t ^ 1]);
+        tmem_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(hf == 0 ? &p_half[t] : &p_full[t]);
       }
     }
 
-    if (ok && NK > 0) ok = mbar_wait(&o_full[t], (NK - 1) & 1, abort_flag, p.status);
-    tc_fence_after();
-    if (ok) {
-      const float inv = 1.0f / l;
-      bf16 *dst = p.out + (size_t)row * p.h * D + (size_t)head[t] * D;
-#pragma unroll 1
-      for (int q = 0; q < D / 32; q++) {
-        uint32_t o[32];
-        tmem_ld32(o_addr + q * 32, o);
-        tmem_wait_ld();
-        if (row < p.n_tok) {
 #pragma unroll
-          for (int v = 0; v < 4; v++) {
-            uint4 w;
-            w.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
-            w.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
-            w.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
-            w.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
-            *reinterpret_cast<uint4 *>(dst + q * 32 + v * 8) = w;
+    for (int t = 0; t < 2; t++) {
+      const int row = row0[t] + r;
+      const uint32_t o_addr = tmem_base + lane_off + 2 * TILE + t * HD;
+      if (ok && NK > 0) ok = mbar_wait(&o_full[t], (NK - 1) & 1, abort_flag, p.status);
+      tc_fence_after();
+      xch[(t * 2 + hf) * TILE + r] = l[t];
+      pair_sync();
+      const float inv = 1.0f / (l[t] + xch[(t * 2 + (hf ^ 1)) * TILE + r]);
+      if (ok) {
+        bf16 *dst = p.out + (size_t)row * p.h * D + (size_t)head[t] * D;
+#pragma unroll 1
+        for (int q = hf; q < D / 32; q += 2) {
+          uint32_t o[32];
+          tmem_ld32(o_addr + q * 32, o);
+          tmem_wait_ld();
+          if (row < p.n_tok) {
+#pragma unroll
+            for (int v = 0; v < 4; v++) {
+              uint4 w;
+              w.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
+              w.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
+              w.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
+              w.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
+              *reinterpret_cast<uint4 *>(dst + q * 32 + v * 8) = w;
+            }
           }
         }
       }
