@@ -34,7 +34,7 @@ UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "c3_llama_128k"
 # dram__bytes_read.sum + dram__bytes_write.sum of one steady-state attention launch, from the ncu
 # capture summarised in profiles/attn_tc_kernel_c3_steady_chunk.md (same launch shape as here)
-NCU_ATTN_TRAFFIC_BYTES = {"c3_llama_128k": 71.5e6, "c2_llama_32k": 71.5e6}
+NCU_ATTN_TRAFFIC_BYTES = {"c3_llama_128k": 67.5e6, "c2_llama_32k": 67.5e6}
 
 
 def measured_peaks():
