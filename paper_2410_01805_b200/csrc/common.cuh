@@ -158,14 +158,21 @@ cudaError_t launch_compact_int4(const Int4Half &src, const Int4Half &dst, const 
 
 // ---- decoding (decode.cu): one token
 cudaError_t launch_gemv(const bf16 *x, const bf16 *Wt, int N, int K, bf16 *y, cudaStream_t st);
+// projection + positions + RoPE + cache append of one token (a.staging is not used: `staging` is written)
+cudaError_t launch_gemv_rope(const bf16 *x, const bf16 *Wt, int K, bf16 *staging, const RopeAppendArgs &a,
+                             cudaStream_t st);
+// retaining head of one token; the last block sums the per-block partials into
+// score_out[m * score_stride]; counter: one zeroed word, left at zero
 cudaError_t launch_rh_gemv(const bf16 *z, const bf16 *W1t, const float *W2, float *partial, int d_R, int K,
-                           int h_kv, int act, int *n_blocks, cudaStream_t st);
+                           int h_kv, int act, unsigned *counter, float *score_out, int score_stride,
+                           cudaStream_t st);
 int rh_gemv_blocks(int d_R);
 int decode_attn_splits(int h_kv, int n);
-// part_o: fp32 [h][n_splits][d]; part_ml: fp32 [h][n_splits][2]
+// part_o: fp32 [h][n_splits][d]; part_ml: fp32 [h][n_splits][2]; counters: one zeroed word per
+// (KV head, group of 8 query heads), left at zero (the last split merges the partial results)
 cudaError_t launch_attention_decode(const bf16 *q_rot, const bf16 *k_rot, const bf16 *v, bf16 *out,
-                                    float *part_o, float *part_ml, int h, int h_kv, int d, int cap, int n,
-                                    int n_splits, cudaStream_t st);
+                                    float *part_o, float *part_ml, unsigned *counters, int h, int h_kv, int d,
+                                    int cap, int n, int n_splits, cudaStream_t st);
 
 // dst[c][r] = src[r][c]  (weight repack at create)
 cudaError_t launch_transpose_bf16(const bf16 *src, bf16 *dst, int rows, int cols, cudaStream_t st);

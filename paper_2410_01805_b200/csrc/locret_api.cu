@@ -27,12 +27,20 @@ struct ScratchPool {
   // layer's projection.  staging / z_post are double-buffered because that work reads them.
   cudaStream_t side = nullptr;
   cudaEvent_t ev_stage_free[2] = {nullptr, nullptr};
+  bool stage_busy[2] = {false, false};  // recorded and not yet waited for
   int flip = 0;
   size_t staging_b[2] = {0, 0}, qrot_b = 0, zpost_b[2] = {0, 0}, partial_b = 0, keep_b = 0, kexp_b = 0, vexp_b = 0;
   bf16 *staging[2] = {nullptr, nullptr}, *q_rot = nullptr, *z_post[2] = {nullptr, nullptr};
   bf16 *k_exp = nullptr, *v_exp = nullptr;  // 4-bit caches: bf16 expansion of the layer in flight
   float *dec_o = nullptr, *dec_ml = nullptr;  // decode attention: per-split partial results
   size_t deco_b = 0, decml_b = 0;
+  // decode kernels whose last block merges the partial results: zeroed words that each launch
+  // leaves at zero (word 0: retaining head; words 1..: attention, one per KV head x head group)
+  unsigned *dec_cnt = nullptr;
+  // recorded after the last second-stream kernel of every chunk step: a decode step, which runs
+  // on the caller's stream alone, waits for it before it reuses the shared scratch
+  cudaEvent_t ev_side_tail = nullptr;
+  bool side_tail_pending = false;
   float *partial = nullptr;
   int32_t *keep = nullptr;
   struct CsTable { float theta; int d, cap; float2 *ptr; };
@@ -54,6 +62,7 @@ bool grow(T **p, size_t *have, size_t want, cudaStream_t st) {
 }
 
 struct TimedEvent { cudaEvent_t a, b; int kind; };
+constexpr int DEC_CNT_WORDS = 1 + 32 * 16;  // retaining head + (KV head, head group) pairs
 
 }  // namespace
 
@@ -116,7 +125,8 @@ void release_pool(ScratchPool *p) {
     cudaFree(p->staging[i]); cudaFree(p->z_post[i]);
     if (p->ev_stage_free[i]) cudaEventDestroy(p->ev_stage_free[i]);
   }
-  cudaFree(p->q_rot); cudaFree(p->partial); cudaFree(p->keep); cudaFree(p->dec_o); cudaFree(p->dec_ml);
+  cudaFree(p->q_rot); cudaFree(p->partial); cudaFree(p->keep); cudaFree(p->dec_o); cudaFree(p->dec_ml); cudaFree(p->dec_cnt);
+  if (p->ev_side_tail) cudaEventDestroy(p->ev_side_tail);
   cudaFree(p->k_exp); cudaFree(p->v_exp);
   for (auto &t : p->cs) cudaFree(t.ptr);
   g_pools.erase(p->st);
@@ -279,6 +289,12 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
         g = g && cudaStreamCreateWithPriority(&p->side, cudaStreamNonBlocking, lo) == cudaSuccess;
         for (int i = 0; i < 2 && g; i++)
           g = cudaEventCreateWithFlags(&p->ev_stage_free[i], cudaEventDisableTiming) == cudaSuccess;
+        g = g && cudaEventCreateWithFlags(&p->ev_side_tail, cudaEventDisableTiming) == cudaSuccess;
+      }
+      if (g && !p->dec_cnt) {
+        g = cudaMalloc(&p->dec_cnt, DEC_CNT_WORDS * sizeof(unsigned)) == cudaSuccess &&
+            cudaMemsetAsync(p->dec_cnt, 0, DEC_CNT_WORDS * sizeof(unsigned), L->st) == cudaSuccess;
+        if (!g) cudaGetLastError();
       }
       if (p->side) cudaStreamSynchronize(p->side);  // buffers may be replaced below
       for (int i = 0; i < 2; i++) {
@@ -373,7 +389,8 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
   if (n > L->cap) return LOCRET_ERR_CAPACITY;
   ScratchPool *P = L->pool;
   const int c = L->cur;
-  const bool side = L->use_side && !L->serialize;
+  const bool decode = n_tok == 1 && L->use_tc;  // one token: bandwidth-bound kernels of decode.cu
+  const bool side = L->use_side && !L->serialize && !decode;
   cudaStream_t S = side ? P->side : L->st;  // stream of the off-critical-path kernels
   const int sb = P->flip;                    // staging buffer of this call
   P->flip ^= 1;
@@ -382,12 +399,16 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
   if (L->use_side) {
     // the staging buffer is free once the retaining head that last read it has run, and this
     // layer's cache once its previous selection / compaction has finished
-    CK(cudaStreamWaitEvent(L->st, P->ev_stage_free[sb], 0));
+    if (P->stage_busy[sb]) CK(cudaStreamWaitEvent(L->st, P->ev_stage_free[sb], 0));
+    P->stage_busy[sb] = false;
     if (L->side_pending) CK(cudaStreamWaitEvent(L->st, L->ev_side, 0));
     L->side_pending = false;
+    if (decode && P->side_tail_pending) {
+      CK(cudaStreamWaitEvent(L->st, P->ev_side_tail, 0));
+      P->side_tail_pending = false;
+    }
   }
 
-  const bool decode = n_tok == 1 && L->use_tc;  // one token: bandwidth-bound kernels of decode.cu
   // a 4-bit cache is expanded into bf16 scratch first: keys rotated at position = slot
   bf16 *const k_att = L->int4 ? P->k_exp : L->k_rot;
   bf16 *const v_att = L->int4 ? P->v_exp : L->v[c];
@@ -407,8 +428,8 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
   }
   {  // (a) projections
     Timed t(L, LOCRET_K_QKV);
-    if (decode)
-      CK(launch_gemv((const bf16 *)hidden_in, L->wqkv_t, L->d_in, L->D, staging, L->st));
+    if (decode)  // projection, positions, RoPE and append of the one token in one kernel
+      CK(launch_gemv_rope((const bf16 *)hidden_in, L->wqkv_t, L->D, staging, ra, L->st));
     else if (fused_rope)
       CK(launch_qkv_rope_tc((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, staging, n_tok, L->d_in, L->D,
                             ra, L->d_status, L->st));
@@ -419,7 +440,7 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
       CK(launch_gemm_bf16((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, staging, L->d_in, n_tok,
                           L->d_in, L->D, L->st));
   }
-  if (!fused_rope) {
+  if (!fused_rope && !decode) {
     Timed t(L, LOCRET_K_ROPE);
     CK(launch_rope_append(ra, L->st));
   }
@@ -446,8 +467,8 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
       L->map_q_base = tc_ok ? P->q_rot : nullptr;
     }
     if (decode)
-      CK(launch_attention_decode(P->q_rot, k_att, v_att, (bf16 *)attn_out, P->dec_o, P->dec_ml, L->h, L->h_kv,
-                                 L->d, L->cap, n, decode_attn_splits(L->h_kv, n), L->st));
+      CK(launch_attention_decode(P->q_rot, k_att, v_att, (bf16 *)attn_out, P->dec_o, P->dec_ml, P->dec_cnt + 1,
+                                 L->h, L->h_kv, L->d, L->cap, n, decode_attn_splits(L->h_kv, n), L->st));
     else if (tc_ok)
       CK(launch_attention_tc(&L->map_q, &L->map_k, &L->map_v[c], (bf16 *)attn_out, n_tok, L->h, L->h_kv,
                              L->d, L->len, L->d_status, L->st));
@@ -464,7 +485,8 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
     Timed t(L, LOCRET_K_RH, S);
     const bf16 *z = L->cfg.rh_input == 1 ? z_post : staging;
     if (decode)
-      CK(launch_rh_gemv(z, L->w1_t, L->w2f, P->partial, L->d_R, L->d_in, L->h_kv, L->cfg.act, &n_tiles, S));
+      CK(launch_rh_gemv(z, L->w1_t, L->w2f, P->partial, L->d_R, L->d_in, L->h_kv, L->cfg.act, P->dec_cnt,
+                        L->s[c] + L->len, L->cap, S));
     else if (L->use_tc && n_tok >= 32 && gemm_tc_supported(n_tok, L->d_R, L->d_in, L->d_in, L->d_in))
       CK(launch_rh_gemm_tc(z, L->d_in, L->w1_t, L->w2f, P->partial, n_tok, L->d_R, L->d_in, L->h_kv,
                            L->cfg.act, &n_tiles, L->d_status, S));
@@ -472,11 +494,14 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
       CK(launch_rh_gemm(z, L->d_in, L->w1_t, L->w2f, P->partial, n_tok, L->d_R, L->d_in, L->h_kv,
                         L->cfg.act, &n_tiles, S));
   }
-  {
+  if (!decode) {  // (the one-token kernel sums its own partial scores)
     Timed t(L, LOCRET_K_RH_REDUCE, S);
     CK(launch_rh_reduce(P->partial, n_tiles, n_tok, L->h_kv, L->s[c], L->cap, L->len, S));
   }
-  if (side) CK(cudaEventRecord(P->ev_stage_free[sb], S));
+  if (side) {
+    CK(cudaEventRecord(P->ev_stage_free[sb], S));
+    P->stage_busy[sb] = true;
+  }
   // (d) protect, top-b, gather
   if (!(flags & LOCRET_NO_EVICT) && n > L->budget) {
     const int n_prot = (flags & LOCRET_LAST_CHUNK) ? 0 : (L->n_stab < n ? L->n_stab : n);
@@ -507,6 +532,8 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
   if (side) {
     CK(cudaEventRecord(L->ev_side, S));
     L->side_pending = true;
+    CK(cudaEventRecord(P->ev_side_tail, S));
+    P->side_tail_pending = true;
   }
   L->seen += n_tok;
   return LOCRET_OK;
