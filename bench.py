@@ -393,7 +393,7 @@ def run_ours(args, w):
         "setup_s": gen_s,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, cores, sample, _ = oracle_sample(w, 1)
+        v, cores, sample, _ = oracle_sample(w, 2)  # two steady-state chunk-layers: about 15 s of host work
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
     if rank == 0:
         print(json.dumps(line), flush=True)

@@ -123,6 +123,22 @@ def test_flags_and_decode_lockstep():
     gpu.destroy()
 
 
+@pytest.mark.parametrize("d,heads,n_stab", [(128, (8, 2), 0), (64, (4, 4), 9), (96, (3, 3), 5)])
+def test_single_token_steps_that_evict(d, heads, n_stab):
+    """Decode-time eviction (a multi-turn stream with a small budget): once the cache is full every
+    one-token step with flags = 0 scores the new unit, drops one and compacts, through the
+    one-token kernels."""
+    from parity_util import lockstep_chunk, make_pair
+    sh = small_shape(h=heads[0], hk=heads[1], d=d, D=128, dR=64, rope_theta=500000.0)
+    ora, gpu = make_pair(sh, weights_for(sh, 11), budget=96, chunk=64, n_stab=n_stab)
+    lockstep_chunk(ora, gpu, hidden(64, sh.d_model, 70), 0, what="fill 1")
+    lockstep_chunk(ora, gpu, hidden(64, sh.d_model, 71), 0, what="fill 2 (evicts)")
+    for t in range(6):
+        lockstep_chunk(ora, gpu, hidden(1, sh.d_model, 80 + t), 0, what=f"evicting token {t}")
+        assert gpu.cache_len == 96 and ora.len == 96
+    gpu.destroy()
+
+
 def test_no_stabilizers_and_other_activations():
     from parity_util import lockstep_chunk, make_pair
     for act in (1, 2):
