@@ -16,6 +16,7 @@ What each function follows:
                              GQA map ceil(j/g), scale 1/sqrt(d_m).
 * ``retaining_scores``     – S~ = sigma([Q, K, V] W1) W2 (Section 3.3).
 * ``select_keep``          – Algorithm 1: last n_s scores set to +inf, top-b, gather
+                            (+ the protected prefix of the query-aware variant, Section 4.4)
                              (stated without infinities: protected ∪ top-(b − n_prot) of the rest).
 * ``OracleLayer.prefill_chunk`` – one iteration of Algorithm 1's loop body for one layer.
 * ``quantize_int4`` / ``dequantize_int4`` – the 4-bit cache variant (Appendix H combines
@@ -157,23 +158,28 @@ def retaining_scores(z, w1, w2, act: int = 0):
     return hidden @ np.asarray(w2, np.float64)
 
 
-def select_keep(scores, budget: int, n_prot: int):
+def select_keep(scores, budget: int, n_prot: int, n_prefix: int = 0):
     """Slots kept by one head: the last n_prot, plus the best (budget − n_prot) of the rest.
 
     Order among the rest: higher score first; equal scores: more recent slot first;
     NaN ranks as −inf.  Returns ascending slot indices (temporal order).
+
+    n_prefix > 0 (the query-aware variant of Section 4.4: the query sits at the start of the
+    sequence and has to stay visible across every eviction) also keeps slots [0, n_prefix);
+    the choice is then among the slots between the two protected ends.
     """
     s = np.array(scores, dtype=np.float64)
     n = s.shape[0]
     if n <= budget:
         return np.arange(n, dtype=np.int64)
     n_prot = min(n_prot, n, budget)
+    n_prefix = min(n_prefix, budget - n_prot)
     rest = n - n_prot
-    sr = np.where(np.isnan(s[:rest]), -np.inf, s[:rest])
-    idx = np.arange(rest, dtype=np.int64)
+    sr = np.where(np.isnan(s[n_prefix:rest]), -np.inf, s[n_prefix:rest])
+    idx = np.arange(n_prefix, rest, dtype=np.int64)
     order = np.lexsort((-idx, -sr))          # primary: score desc; secondary: slot desc
-    chosen = order[: budget - n_prot]
-    keep = np.concatenate([chosen, np.arange(rest, n, dtype=np.int64)])
+    chosen = idx[order[: budget - n_prot - n_prefix]]
+    keep = np.concatenate([np.arange(n_prefix, dtype=np.int64), chosen, np.arange(rest, n, dtype=np.int64)])
     return np.sort(keep)
 
 
@@ -219,7 +225,15 @@ class OracleLayer:
         self.mirror = mirror
         self.want_flip_sens = False   # tests switch this on: an error-propagation aid, not part of the method
         self.int4 = shape.kv_dtype == 1
+        self.n_prefix = 0             # Section 4.4 variant: slots [0, n_prefix) are never evicted
         self.reset()
+
+    def set_protected_prefix(self, n_prefix: int):
+        """Section 4.4 variant: the first n_prefix slots of the cache (the query placed at the start
+        of the sequence) are kept by every eviction, besides the last n_stab."""
+        if n_prefix < 0 or n_prefix + self.n_stab > self.budget:
+            raise ValueError("need 0 <= n_prefix and n_prefix + n_stab <= budget")
+        self.n_prefix = int(n_prefix)
 
     # ---- state
     def reset(self):
@@ -317,7 +331,7 @@ class OracleLayer:
         self.last_keep = None
         if not (flags & NO_EVICT) and n > self.budget:
             n_prot = 0 if (flags & LAST_CHUNK) else min(self.n_stab, n)
-            keep = np.stack([select_keep(self.S[m], self.budget, n_prot) for m in range(hk)])
+            keep = np.stack([select_keep(self.S[m], self.budget, n_prot, self.n_prefix) for m in range(hk)])
             self.last_keep = keep
             take = lambda a: np.stack([a[m][keep[m]] for m in range(hk)])
             self.K, self.V, self.S, self.T = take(self.K), take(self.V), take(self.S), take(self.T)

@@ -455,9 +455,14 @@ cudaError_t launch_attention_decode(const bf16 *q_rot, const bf16 *k_rot, const 
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)d);
   const int smem = 2 * DA_THREADS * d * (int)sizeof(bf16);
   auto launch = [&](auto kern) -> cudaError_t {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         2 * DA_THREADS * 128 * (int)sizeof(bf16));
-    if (e != cudaSuccess) return e;
+    static bool attr_set[4][3] = {};  // per (G, d) instantiation: the kernels share one pointer type
+    bool &done = attr_set[G == 1 ? 0 : (G == 2 ? 1 : (G == 4 ? 2 : 3))][d == 64 ? 0 : (d == 96 ? 1 : 2)];
+    if (!done) {
+      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           2 * DA_THREADS * 128 * (int)sizeof(bf16));
+      if (e != cudaSuccess) return e;
+      done = true;
+    }
     kern<<<grid, DA_THREADS, smem, st>>>(q_rot, k_rot, v, part_o, part_ml, h, h_kv, d, cap, n, n_splits,
                                          scale_log2, counters, out);
     return cudaGetLastError();

@@ -262,6 +262,66 @@ def test_select_keep_ties_prefer_recent_and_nan_ranks_last():
     assert list(O.select_keep([np.nan, np.nan, -np.inf], 2, 0)) == [1, 2]
 
 
+def literal_selection_with_prefix(scores, b, n_s, n_q):
+    """The same overwrite-and-sort statement with both protected ends at +inf."""
+    s = np.array(scores, dtype=np.float64)
+    n = len(s)
+    s = np.where(np.isnan(s), -np.inf, s)
+    if n_s > 0:
+        s[max(0, n - n_s):] = np.inf
+    s[:min(n_q, n)] = np.inf
+    order = sorted(range(n), key=lambda i: (-s[i], -i))
+    return sorted(order[:b])
+
+
+def test_protected_prefix_equals_overwrite_and_sort_bruteforce():
+    """Section 4.4 (query at the start of the sequence, visible across every eviction)."""
+    g = np.random.default_rng(160)
+    for n, b, n_s, n_q in itertools.product([6, 9, 14, 23], [3, 5, 8], [0, 1, 3], [0, 1, 2, 4]):
+        if n_s + n_q > b or n <= b:
+            continue
+        for trial in range(4):
+            s = g.standard_normal(n)
+            if trial == 1:
+                s = np.round(s)                       # many ties
+            if trial == 2:
+                s[g.integers(0, n, 2)] = np.nan
+            got = list(O.select_keep(s, b, n_s, n_q))
+            assert got == literal_selection_with_prefix(s, b, n_s, n_q), (n, b, n_s, n_q, s)
+            assert len(got) == b and got[:n_q] == list(range(n_q))
+            assert got[b - n_s:] == list(range(n - n_s, n))
+    # no prefix: the statement of Algorithm 1 itself
+    s = g.standard_normal(12)
+    assert list(O.select_keep(s, 5, 2, 0)) == list(O.select_keep(s, 5, 2))
+
+
+@pytest.mark.parametrize("n_stab,n_q", [(0, 4), (6, 3), (9, 11)])
+def test_protected_prefix_closed_form_and_chunk_size_invariance(n_stab, n_q):
+    """With a protected prefix the final cache is Prefix ∪ Last_{n_s} ∪ Top_{b − n_s − l_q}(between),
+    whatever the chunk size: the induction of the cache-problem argument (Appendix N) with both
+    ends fixed."""
+    sh = shape()
+    b, ctx = 30, 131
+    X = np.random.default_rng(190).standard_normal((ctx, sh.d_model))
+    finals = []
+    for B in [1, 7, 30, 50]:
+        layer, (wqkv, w1, w2) = rand_layer(sh, budget=b, chunk=B, n_stab=n_stab, seed=200)
+        layer.set_protected_prefix(n_q)
+        run_chunks(layer, X, B)
+        t = torch.from_numpy
+        s_all = (torch.nn.functional.silu(t(X @ wqkv) @ t(w1)) @ t(w2)).numpy()   # [ctx, hk]
+        for m in range(sh.n_kv_heads):
+            mid = list(range(n_q, ctx - n_stab))
+            order = sorted(mid, key=lambda i: (-s_all[i, m], -i))
+            want = sorted(list(range(n_q)) + order[: b - n_stab - n_q] + list(range(ctx - n_stab, ctx)))
+            assert list(layer.T[m]) == want
+        finals.append(layer.T.copy())
+    for f in finals[1:]:
+        assert np.array_equal(f, finals[0])
+    with pytest.raises(ValueError):
+        layer.set_protected_prefix(b - n_stab + 1)
+
+
 # ------------------------------------------------------------------ Pin 2 / Pin 3
 
 @pytest.mark.parametrize("n_stab", [0, 3, 11, 40])
