@@ -169,6 +169,20 @@ int locret_selftest_wait_timeout(void *stream);
 int locret_reset(locret_layer *layer);
 
 /*
+ * Query-aware variant (Section 4.4; Appendix "Evaluating Locret-Q on RULER"): the query is
+ * placed at the start of the sequence and has to stay visible across every eviction.  After
+ * this call every evicting step keeps cache slots [0, n_prefix) besides the last n_stab
+ * units, and chooses budget - n_stab - n_prefix units among the slots between them (with
+ * LOCRET_LAST_CHUNK: budget - n_prefix).  Slots are in temporal order, so set before the
+ * first evicting step the prefix is tokens 0 .. n_prefix-1 for the life of the stream; set
+ * later it is whatever then occupies the first slots.  n_prefix = 0 (the default, and the
+ * state after create) is Algorithm 1 unchanged.  Host-side state only: nothing is launched
+ * and nothing on the device changes.  Requires 0 <= n_prefix and n_prefix + n_stab <= budget,
+ * else LOCRET_ERR_INVALID and the previous value stays.  locret_reset keeps the value.
+ */
+int locret_set_protected_prefix(locret_layer *layer, int32_t n_prefix);
+
+/*
  * Per-kernel timing.  With enable != 0 every kernel launched for this layer is
  * bracketed by CUDA events on the stream it runs on (kernels on the two streams overlap, so
  * the per-kernel times of a step add up to more than its duration); enable = 2 also keeps

@@ -52,6 +52,7 @@ def _load():
     l.locret_selftest_wait_timeout.argtypes = [P]
     l.locret_sync_status.argtypes = [P]
     l.locret_reset.argtypes = [P]
+    l.locret_set_protected_prefix.argtypes = [P, C.c_int32]
     l.locret_set_timing.argtypes = [P, C.c_int32]
     l.locret_read_timing.argtypes = [P, P, P]
     l.locret_launch_count.argtypes = [P, C.POINTER(C.c_int64)]
@@ -177,6 +178,9 @@ class LocretLayer:
         _check(lib.locret_reset(self._h), "locret_reset")
 
     # -- measurement
+    def set_protected_prefix(self, n_prefix: int):
+        _check(lib.locret_set_protected_prefix(self._h, int(n_prefix)), "locret_set_protected_prefix")
+
     def set_timing(self, mode):
         """0 off, 1 time every kernel, 2 time every kernel and run them on one stream, 3 time attention only."""
         _check(lib.locret_set_timing(self._h, int(mode)), "locret_set_timing")

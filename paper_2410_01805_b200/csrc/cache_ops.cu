@@ -157,7 +157,7 @@ __device__ __forceinline__ int block_exclusive_scan(int val, int *warp_sums, int
 }
 
 __global__ void __launch_bounds__(TK_THREADS)
-topk_kernel(const float *__restrict__ scores, int score_stride, int n, int budget, int n_prot,
+topk_kernel(const float *__restrict__ scores, int score_stride, int n, int budget, int n_prot, int n_pre,
             int32_t *__restrict__ keep, int smem_keys) {
   extern __shared__ uint32_t skeys[];  // [rest] when it fits (smem_keys != 0)
   __shared__ int hist[256];
@@ -170,7 +170,8 @@ topk_kernel(const float *__restrict__ scores, int score_stride, int n, int budge
   int32_t *out = keep + (size_t)m * budget;
   const int tid = threadIdx.x;
   const int rest = n - n_prot;
-  const int k = budget - n_prot;  // 0 <= k < rest (the caller guarantees n > budget)
+  // slots [0, n_pre) and [rest, n) are kept unconditionally; k of the slots between them are chosen
+  const int k = budget - n_prot - n_pre;  // 0 <= k < rest - n_pre (the caller guarantees n > budget)
 
   auto key_at = [&](int i) -> uint32_t { return smem_keys ? skeys[i] : score_key(sc[i]); };
 
@@ -191,7 +192,7 @@ topk_kernel(const float *__restrict__ scores, int score_stride, int n, int budge
         bool in = false;
         if (i < rest) {
           key = key_at(i);
-          in = (key & mask) == prefix;
+          in = i >= n_pre && (key & mask) == prefix;
         }
         const unsigned active = __ballot_sync(0xffffffffu, in);
         if (in) {
@@ -237,7 +238,7 @@ topk_kernel(const float *__restrict__ scores, int score_stride, int n, int budge
   const int lo = min(tid * per, n), hi = min(lo + per, n);
   int cnt_eq = 0;
   if (k > 0)
-    for (int i = lo; i < hi && i < rest; i++) cnt_eq += (key_at(i) == tau);
+    for (int i = max(lo, n_pre); i < hi && i < rest; i++) cnt_eq += (key_at(i) == tau);
   int total_eq;
   int eq_before = block_exclusive_scan(cnt_eq, warp_sums, &total_eq);
   const int eq_skip = total_eq - need;  // equal units with rank-from-start < eq_skip are dropped
@@ -247,7 +248,7 @@ topk_kernel(const float *__restrict__ scores, int score_stride, int n, int budge
     int eqr = eq_before;
     for (int i = lo; i < hi; i++) {
       bool kp;
-      if (i >= rest) kp = true;
+      if (i >= rest || i < n_pre) kp = true;
       else if (k == 0) kp = false;
       else {
         uint32_t key = key_at(i);
@@ -263,7 +264,7 @@ topk_kernel(const float *__restrict__ scores, int score_stride, int n, int budge
     int eqr = eq_before;
     for (int i = lo; i < hi; i++) {
       bool kp;
-      if (i >= rest) kp = true;
+      if (i >= rest || i < n_pre) kp = true;
       else if (k == 0) kp = false;
       else {
         uint32_t key = key_at(i);
@@ -333,7 +334,7 @@ cudaError_t launch_rerope(const bf16 *k_pre, bf16 *k_rot, const float2 *cs, int 
 }
 
 cudaError_t launch_topk(const float *scores, int score_stride, int h_kv, int n, int budget,
-                        int n_prot, int32_t *keep, cudaStream_t st) {
+                        int n_prot, int n_pre, int32_t *keep, cudaStream_t st) {
   const int rest = n - n_prot;
   const size_t bytes = (size_t)rest * 4;
   const size_t max_dyn = 200 * 1024;
@@ -346,7 +347,7 @@ cudaError_t launch_topk(const float *scores, int score_stride, int h_kv, int n, 
   }
   int use_smem = bytes <= max_dyn;
   topk_kernel<<<h_kv, TK_THREADS, use_smem ? bytes : 0, st>>>(scores, score_stride, n, budget, n_prot,
-                                                              keep, use_smem);
+                                                              n_pre, keep, use_smem);
   return cudaGetLastError();
 }
 

@@ -118,9 +118,10 @@ cudaError_t launch_attention_mma(const bf16 *q_rot, const bf16 *k_rot, const bf1
                                  int n_tok, int h, int h_kv, int d, int cap, int len,
                                  cudaStream_t st);
 
-// keep[m][0..budget) = ascending slots kept among n candidates (the last n_prot protected).
+// keep[m][0..budget) = ascending slots kept among n candidates (the first n_pre and the last n_prot
+// protected).
 cudaError_t launch_topk(const float *scores, int score_stride, int h_kv, int n, int budget,
-                        int n_prot, int32_t *keep, cudaStream_t st);
+                        int n_prot, int n_pre, int32_t *keep, cudaStream_t st);
 
 struct CompactArgs {
   const bf16 *k_src, *v_src;

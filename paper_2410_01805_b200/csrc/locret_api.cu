@@ -69,6 +69,7 @@ constexpr int DEC_CNT_WORDS = 1 + 32 * 16;  // retaining head + (KV head, head g
 struct locret_layer {
   locret_layer_cfg cfg;
   int budget, chunk, n_stab, cap, d_in, h, h_kv, d, D, d_R;
+  int n_prefix;  // Section 4.4 variant: cache slots [0, n_prefix) are never evicted
   cudaStream_t st;
   ScratchPool *pool;
   bf16 *wqkv_t, *w1_t;
@@ -234,6 +235,7 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   L->h = h; L->h_kv = hk; L->d = d; L->D = D; L->d_R = dR;
   L->d_in = (h + 2 * hk) * d;
   L->st = (cudaStream_t)cfg->stream;
+  L->n_prefix = 0;
   L->cur = 0; L->len = 0; L->seen = 0; L->launches = 0; L->timing = false; L->serialize = false; L->attn_only = false; L->events_used = 0;
   L->pool = nullptr;
   {
@@ -507,7 +509,8 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
     const int n_prot = (flags & LOCRET_LAST_CHUNK) ? 0 : (L->n_stab < n ? L->n_stab : n);
     {
       Timed t(L, LOCRET_K_TOPK, S);
-      CK(launch_topk(L->s[c], L->cap, L->h_kv, n, L->budget, n_prot, P->keep, S));
+      // (n_prefix + n_stab <= budget < n, so the prefix never reaches into the protected tail)
+      CK(launch_topk(L->s[c], L->cap, L->h_kv, n, L->budget, n_prot, L->n_prefix, P->keep, S));
     }
     // compaction rewrites the rotated keys the attention kernel reads
     if (side) CK(cudaStreamWaitEvent(S, L->ev_attn, 0));
@@ -656,6 +659,12 @@ int locret_reset(locret_layer *L) {
   if (!L) return LOCRET_ERR_INVALID;
   L->len = 0;
   L->seen = 0;
+  return LOCRET_OK;
+}
+
+int locret_set_protected_prefix(locret_layer *L, int32_t n_prefix) {
+  if (!L || n_prefix < 0 || n_prefix + L->n_stab > L->budget) return LOCRET_ERR_INVALID;
+  L->n_prefix = n_prefix;
   return LOCRET_OK;
 }
 

@@ -61,27 +61,29 @@ def check_scores(got: np.ndarray, ref: np.ndarray, what=""):
     return worst
 
 
-def check_keep_band(kept_slots, s_ref, budget, n_prot, oracle_keep, what=""):
-    """kept_slots: ascending slot indices (into cache ‖ chunk) kept by the CUDA path for one head."""
+def check_keep_band(kept_slots, s_ref, budget, n_prot, oracle_keep, what="", n_pre=0):
+    """kept_slots: ascending slot indices (into cache ‖ chunk) kept by the CUDA path for one head.
+    n_pre: protected prefix of the query-aware variant (0 = Algorithm 1)."""
     n = len(s_ref)
     kept = np.zeros(n, dtype=bool)
     kept[kept_slots] = True
     assert kept.sum() == min(budget, n), f"{what}: kept {kept.sum()} units"
     assert kept[n - n_prot:].all(), f"{what}: a protected unit was evicted"
+    assert kept[:n_pre].all(), f"{what}: a unit of the protected prefix was evicted"
     rest = n - n_prot
-    k = budget - n_prot
+    k = budget - n_prot - n_pre
     if k == 0:
-        assert not kept[:rest].any()
+        assert not kept[n_pre:rest].any()
         return True
-    if k >= rest:
+    if k >= rest - n_pre:
         return True
-    sr = np.where(np.isnan(s_ref[:rest]), -np.inf, s_ref[:rest])
+    sr = np.where(np.isnan(s_ref[n_pre:rest]), -np.inf, s_ref[n_pre:rest])
     srt = np.sort(sr)[::-1]
     tau_hi, tau_lo = srt[k - 1], srt[k]
     must = sr >= tau_hi + BAND
     never = sr <= tau_lo - BAND
-    assert kept[:rest][must].all(), f"{what}: a unit above the band was evicted"
-    assert not kept[:rest][never].any(), f"{what}: a unit below the band was kept"
+    assert kept[n_pre:rest][must].all(), f"{what}: a unit above the band was evicted"
+    assert not kept[n_pre:rest][never].any(), f"{what}: a unit below the band was kept"
     exact = np.array_equal(np.flatnonzero(kept), np.asarray(oracle_keep))
     if tau_hi - tau_lo > BAND:
         assert exact, f"{what}: index set differs although the gap is {tau_hi - tau_lo:.3g}"
@@ -165,7 +167,7 @@ def lockstep_chunk(ora, gpu, x: np.ndarray, flags: int = 0, rows=None, what=""):
             pos = np.searchsorted(pre["T"][m], post["T"][m])
             assert np.array_equal(pre["T"][m][pos], post["T"][m]), f"{what}: unknown token id after compaction"
             assert np.all(np.diff(pos) > 0), f"{what}: temporal order lost"
-            exact &= check_keep_band(pos, s_ref[m], ora.budget, n_prot, ora.last_keep[m], f"{what} head {m}")
+            exact &= check_keep_band(pos, s_ref[m], ora.budget, n_prot, ora.last_keep[m], f"{what} head {m}", n_pre=ora.n_prefix)
             # compaction is a bit-exact gather of the pre-compaction arrays
             for key in state_keys:
                 assert np.array_equal(post[key][m], pre[key][m][pos]), f"{what}: {key} not a bit-exact gather"

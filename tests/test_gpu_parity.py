@@ -139,6 +139,44 @@ def test_single_token_steps_that_evict(d, heads, n_stab):
     gpu.destroy()
 
 
+@pytest.mark.parametrize("kv_dtype", [0, 1])
+def test_protected_prefix_lockstep_and_crafted_scores(kv_dtype):
+    """Query-aware variant (Section 4.4): the first l_q slots survive every eviction."""
+    from parity_util import import_oracle_state, lockstep_chunk, make_pair
+    sh = small_shape(h=4, hk=2, d=128, D=128, dR=64, rope_theta=500000.0, kv_dtype=kv_dtype)
+    ora, gpu = make_pair(sh, weights_for(sh, 21), budget=160, chunk=96, n_stab=20)
+    ora.set_protected_prefix(24)
+    gpu.set_protected_prefix(24)
+    for i, n_tok in enumerate([96, 96, 50, 96, 1, 96]):
+        lockstep_chunk(ora, gpu, hidden(n_tok, sh.d_model, 90 + i), 0, what=f"prefix chunk {i}")
+        if ora.seen > 160:
+            assert list(ora.T[0][:24]) == list(range(24))
+    lockstep_chunk(ora, gpu, hidden(40, sh.d_model, 99), O.LAST_CHUNK, what="prefix, last chunk")
+    post = gpu.export_state()
+    assert list(post["T"][1][:24]) == list(range(24))
+    # crafted scores: the prefix holds the worst scores of all and still stays; ties next to the cut
+    if kv_dtype == 0:
+        st = ora.export_state()
+        S = st["S"].copy()
+        S[:, :24] = -1e30
+        S[:, 24:60] = 0.25
+        S[0, 30] = np.nan
+        st["S"] = S
+        ora.import_state(st)
+        x = hidden(96, sh.d_model, 123)
+        stats = lockstep_chunk(ora, gpu, x, 0, what="prefix, crafted")
+        assert list(ora.T[0][:24]) == list(range(24))
+        assert stats["sets_identical"]          # ties resolved alike (most recent first), NaN last
+    # argument checks: prefix + stabilizers must fit the budget
+    from paper_2410_01805_b200 import LocretError
+    with pytest.raises(LocretError):
+        gpu.set_protected_prefix(141)
+    with pytest.raises(LocretError):
+        gpu.set_protected_prefix(-1)
+    gpu.set_protected_prefix(140)
+    gpu.destroy()
+
+
 def test_no_stabilizers_and_other_activations():
     from parity_util import lockstep_chunk, make_pair
     for act in (1, 2):
