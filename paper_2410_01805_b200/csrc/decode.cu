@@ -70,7 +70,7 @@ gemv_kernel(const bf16 *__restrict__ x, const bf16 *__restrict__ Wt, int N, int 
       if (n < N) {
         const uint4 *row = reinterpret_cast<const uint4 *>(Wt + (size_t)n * K) + hf * kv2;
         const uint4 *xs = sx + hf * kv2;
-#pragma unroll 4
+#pragma unroll 12
         for (int v = lane; v < kv2; v += 32) s += dot8(__ldg(row + v), xs[v]);
       }
       s = warp_sum(s);
@@ -171,193 +171,195 @@ gemv_rope_kernel(const bf16 *__restrict__ x, const bf16 *__restrict__ Wt, int K,
   }
 }
 
-// ---- decode attention: grid (h_kv, splits, head groups of <= 8).  128 threads: a tile of 128
-// keys and values is brought into shared memory with 16-byte loads (all of a thread's loads in
-// flight together; key rows rotated by their index so that thread = key reads without bank
-// conflicts); in the score phase thread = key, in the value phase thread = column.
-constexpr int DA_THREADS = 128, DA_MAXG = 8;
+// ---- decode attention on warp-level tensor-core instructions.  grid (h_kv, splits, head groups
+// of <= 16).  The rows of the m16n8k16 tiles are the query heads of one GQA group (all of them read
+// the same keys), padded to 16; keys and values of the split stream through shared memory in
+// tiles of 64 (cp.async, two stages).  Each of the four warps takes 16 keys of a tile and keeps
+// its own running maximum, sum and output, so the tile loop has no block-wide reduction; the
+// four states meet in shared memory at the end, the block writes one partial result per head,
+// and the split that finishes last for its (KV head, head group) merges all splits in split
+// order (a wrapping atomic counter, left at zero for the next step).
+constexpr int DA_THREADS = 128, DA_G = 16, DA_KT = 64;
 
-// G: query heads per block (a power of two up to DA_MAXG; the launcher picks the GQA group size);
-// D: head_dim (= d), compile-time so that the tile indexing needs no divisions
-template <int G, int D>
+template <int D>
 __global__ void __launch_bounds__(DA_THREADS)
 attn_decode_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_rot,
                    const bf16 *__restrict__ v, float *__restrict__ part_o, float *__restrict__ part_ml,
-                   int h, int h_kv, int d, int cap, int n, int n_splits, float scale_log2,
+                   int h, int h_kv, int cap, int n, int n_splits, float scale_log2,
                    unsigned *__restrict__ counters, bf16 *__restrict__ out) {
-  extern __shared__ uint4 da_smem[];  // K tile [128][d/8], V tile [128][d/8]
-  __shared__ __align__(16) float sq[DA_MAXG][128];
-  __shared__ __align__(16) float sp[DA_THREADS * DA_MAXG];  // p[key][head]; reused for the final column sums
-  __shared__ float sred[DA_MAXG][4];
+  constexpr int LD = D + 8;
+  constexpr int VPR = D / 8;  // 16-byte vectors per row
+  extern __shared__ __align__(16) unsigned char da_smem[];
+  bf16 *sQ = reinterpret_cast<bf16 *>(da_smem);  // [16][LD]
+  bf16 *sK = sQ + DA_G * LD;                     // [2][64][LD]
+  bf16 *sV = sK + 2 * DA_KT * LD;                // [2][64][LD]
+  __shared__ float wm[4][DA_G], wl[4][DA_G];     // per-warp running maximum and sum of every head
+  __shared__ float sm[DA_G][64], sl[DA_G][64], sinv[DA_G];
+  __shared__ bool last;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g4 = lane >> 2, q = lane & 3;
   const int g = h / h_kv;
   const int m = blockIdx.x, split = blockIdx.y, hg = blockIdx.z;
-  const int h0 = m * g + hg * G;
-  const int gh = min(G, g - hg * G);  // heads handled here
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  for (int i = tid; i < gh * D; i += DA_THREADS) sq[i / D][i % D] = __bfloat162float(q_rot[(size_t)(h0 + i / D) * D + i % D]);
-  __syncthreads();
+  const int h0 = m * g + hg * DA_G;
+  const int gh = min(DA_G, g - hg * DA_G);  // heads handled here
   const int per = (n + n_splits - 1) / n_splits;
   const int k0 = split * per, k1 = min(n, k0 + per);
-  const bf16 *kb = k_rot + (size_t)m * cap * D, *vb = v + (size_t)m * cap * D;
-  constexpr int vpr = D / 8;  // 16-byte vectors per row: 8, 12 or 16
-  constexpr int HC = D / 2;   // value phase: thread = column pair, two key halves of the tile
-  const int cp = tid % HC, kh = tid / HC;
-  uint4 *sK = da_smem, *sV = da_smem + DA_THREADS * vpr;
+  const int NKT = k1 > k0 ? (k1 - k0 + DA_KT - 1) / DA_KT : 0;
+  const bf16 *kbase = k_rot + (size_t)m * cap * D;
+  const bf16 *vbase = v + (size_t)m * cap * D;
 
-  float mrun[G], lrun[G], acc[G][2];
-#pragma unroll
-  for (int i = 0; i < G; i++) { mrun[i] = -INFINITY; lrun[i] = 0.f; acc[i][0] = acc[i][1] = 0.f; }
+  auto load_kv = [&](int buf, int kt) {
+    for (int x = tid; x < DA_KT * VPR; x += DA_THREADS) {
+      const int r = x / VPR, c = (x - r * VPR) * 8;
+      const int key = k0 + kt * DA_KT + r;
+      const bool ok = key < k1;
+      const size_t off = (size_t)min(key, n - 1) * D + c;
+      cp_async16(sK + (buf * DA_KT + r) * LD + c, kbase + off, ok);
+      cp_async16(sV + (buf * DA_KT + r) * LD + c, vbase + off, ok);
+    }
+  };
+  for (int x = tid; x < DA_G * VPR; x += DA_THREADS) {
+    const int r = x / VPR, c = (x - r * VPR) * 8;
+    cp_async16(sQ + r * LD + c, q_rot + (size_t)(h0 + min(r, gh - 1)) * D + c, r < gh);
+  }
+  if (NKT > 0) load_kv(0, 0);
+  cp_async_commit();
 
-  for (int t0 = k0; t0 < k1; t0 += DA_THREADS) {
-    {  // the tile: row r of K at vectors (c + r) % vpr, V row-major
-      uint4 kreg[16], vreg[16];
+  uint32_t qf[D / 16][4];
+  float o[D / 8][4];
 #pragma unroll
-      for (int it = 0; it < 16; it++) {
-        const int idx = tid + it * DA_THREADS, r = idx / vpr, c = idx - r * vpr;
-        if (it < vpr && t0 + r < k1) {
-          kreg[it] = __ldg(reinterpret_cast<const uint4 *>(kb + (size_t)(t0 + r) * D) + c);
-          vreg[it] = __ldg(reinterpret_cast<const uint4 *>(vb + (size_t)(t0 + r) * D) + c);
-        }
-      }
+  for (int i = 0; i < D / 8; i++)
 #pragma unroll
-      for (int it = 0; it < 16; it++) {
-        const int idx = tid + it * DA_THREADS, r = idx / vpr, c = idx - r * vpr;
-        if (it < vpr && t0 + r < k1) {
-          int cr = c + r % vpr;
-          if (cr >= vpr) cr -= vpr;
-          sK[r * vpr + cr] = kreg[it];
-          sV[idx] = vreg[it];
-        }
-      }
-    }
+    for (int e = 0; e < 4; e++) o[i][e] = 0.f;
+  float mrow[2] = {-INFINITY, -INFINITY}, lrow[2] = {0.f, 0.f};  // heads g4 and g4 + 8
+
+  for (int kt = 0; kt < NKT; kt++) {
+    if (kt + 1 < NKT) load_kv((kt + 1) & 1, kt + 1);
+    cp_async_commit();
+    cp_async_wait<1>();
     __syncthreads();
-    const int key = t0 + tid;
-    float s[G];
+    if (kt == 0) {
 #pragma unroll
-    for (int i = 0; i < G; i++) s[i] = -INFINITY;
-    if (key < k1) {
+      for (int kk = 0; kk < D / 16; kk++)
+        ldmatrix_x4(qf[kk][0], qf[kk][1], qf[kk][2], qf[kk][3],
+                    sQ + (lane & 15) * LD + kk * 16 + (lane >> 4) * 8);
+    }
+    const bf16 *k_s = sK + ((kt & 1) * DA_KT + warp * 16) * LD;  // this warp's 16 keys
+    const bf16 *v_s = sV + ((kt & 1) * DA_KT + warp * 16) * LD;
+
+    float s[2][4];
 #pragma unroll
-      for (int i = 0; i < G; i++) s[i] = 0.f;
-      const uint4 *kr = sK + tid * vpr;
-      const int rot = tid % vpr;
-      for (int c = 0; c < vpr; c++) {
-        int cr = c + rot;
-        if (cr >= vpr) cr -= vpr;
-        const uint4 kv = kr[cr];
-        float kf[8];
-        {
-          const __nv_bfloat162 *kp = reinterpret_cast<const __nv_bfloat162 *>(&kv);
+    for (int i = 0; i < 2; i++)
 #pragma unroll
-          for (int e = 0; e < 4; e++) {
-            const float2 f = __bfloat1622float2(kp[e]);
-            kf[2 * e] = f.x; kf[2 * e + 1] = f.y;
-          }
-        }
+      for (int e = 0; e < 4; e++) s[i][e] = 0.f;
 #pragma unroll
-        for (int i = 0; i < G; i++) {
-          if (i < gh) {
-            const float4 q0 = *reinterpret_cast<const float4 *>(&sq[i][c * 8]);
-            const float4 q1 = *reinterpret_cast<const float4 *>(&sq[i][c * 8 + 4]);
-            s[i] = fmaf(kf[0], q0.x, s[i]); s[i] = fmaf(kf[1], q0.y, s[i]);
-            s[i] = fmaf(kf[2], q0.z, s[i]); s[i] = fmaf(kf[3], q0.w, s[i]);
-            s[i] = fmaf(kf[4], q1.x, s[i]); s[i] = fmaf(kf[5], q1.y, s[i]);
-            s[i] = fmaf(kf[6], q1.z, s[i]); s[i] = fmaf(kf[7], q1.w, s[i]);
-          }
-        }
+    for (int kk = 0; kk < D / 16; kk++) {
+      uint32_t b0, b1, b2, b3;
+      const int id = lane >> 3;
+      const int r = (id >> 1) * 8 + (lane & 7);
+      const int c = kk * 16 + (id & 1) * 8;
+      ldmatrix_x4(b0, b1, b2, b3, k_s + r * LD + c);
+      mma_bf16_16816(s[0], qf[kk], b0, b1);
+      mma_bf16_16816(s[1], qf[kk], b2, b3);
+    }
+
+    // scale, mask the keys past the split's end, online softmax of this warp's 16 keys
+    const int key0 = k0 + kt * DA_KT + warp * 16;
+    float tmax[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int i = 0; i < 2; i++)
+#pragma unroll
+      for (int e = 0; e < 4; e++) {
+        float val = s[i][e] * scale_log2;
+        if (key0 + i * 8 + q * 2 + (e & 1) >= k1) val = -INFINITY;
+        s[i][e] = val;
+        tmax[e >> 1] = fmaxf(tmax[e >> 1], val);
       }
+    float alpha[2];
 #pragma unroll
-      for (int i = 0; i < G; i++) s[i] = (i < gh) ? s[i] * scale_log2 : -INFINITY;
-    }
-    // tile maximum per head
-#pragma unroll
-    for (int i = 0; i < G; i++) {
-      float mx = warp_max(s[i]);
-      if (lane == 0) sred[i][warp] = mx;
-    }
-    __syncthreads();
-    float alpha[G];
-#pragma unroll
-    for (int i = 0; i < G; i++) {
-      const float tmax = fmaxf(fmaxf(sred[i][0], sred[i][1]), fmaxf(sred[i][2], sred[i][3]));
-      const float mnew = fmaxf(mrun[i], tmax);
+    for (int r = 0; r < 2; r++) {
+      tmax[r] = fmaxf(tmax[r], __shfl_xor_sync(0xffffffffu, tmax[r], 1));
+      tmax[r] = fmaxf(tmax[r], __shfl_xor_sync(0xffffffffu, tmax[r], 2));
+      const float mnew = fmaxf(mrow[r], tmax[r]);
       const float muse = (mnew == -INFINITY) ? 0.f : mnew;
-      alpha[i] = exp2f(mrun[i] - muse);
-      mrun[i] = mnew;
-      const float p = exp2f(s[i] - muse);
-      sp[tid * G + i] = p;
-      s[i] = p;
-    }
-    __syncthreads();  // sred is reused below, sp is complete
+      alpha[r] = exp2f(mrow[r] - muse);
+      mrow[r] = mnew;
+      float psum = 0.f;
 #pragma unroll
-    for (int i = 0; i < G; i++) {
-      float sm = warp_sum(s[i]);
-      if (lane == 0) sred[i][warp] = sm;
-    }
-    __syncthreads();
-#pragma unroll
-    for (int i = 0; i < G; i++)
-      lrun[i] = lrun[i] * alpha[i] + (sred[i][0] + sred[i][1]) + (sred[i][2] + sred[i][3]);
-    // values: thread = column pair cp, keys [64 kh, 64 kh + 64) of the tile
-    if (kh < 2) {
-#pragma unroll
-      for (int i = 0; i < G; i++) { acc[i][0] *= alpha[i]; acc[i][1] *= alpha[i]; }
-      const int cnt = min(DA_THREADS, k1 - t0);
-      const uint32_t *sv = reinterpret_cast<const uint32_t *>(sV);
-      const int kend = min(cnt, kh * 64 + 64);
-#pragma unroll 4
-      for (int kk = kh * 64; kk < kend; kk++) {
-        const uint32_t v2 = sv[kk * HC + cp];
-        const float v0 = __uint_as_float(v2 << 16), v1 = __uint_as_float(v2 & 0xffff0000u);
-        float pr[G];
-        if (G % 4 == 0) {
-#pragma unroll
-          for (int i4 = 0; i4 < G / 4; i4++) {
-            const float4 t = *reinterpret_cast<const float4 *>(&sp[kk * G + 4 * i4]);
-            pr[4 * i4] = t.x; pr[4 * i4 + 1] = t.y; pr[4 * i4 + 2] = t.z; pr[4 * i4 + 3] = t.w;
-          }
-        } else {
-#pragma unroll
-          for (int i = 0; i < G; i++) pr[i] = sp[kk * G + i];
-        }
-#pragma unroll
-        for (int i = 0; i < G; i++) {
-          acc[i][0] = fmaf(pr[i], v0, acc[i][0]);
-          acc[i][1] = fmaf(pr[i], v1, acc[i][1]);
-        }
+      for (int i = 0; i < 2; i++) {
+        const float p0 = exp2f(s[i][2 * r] - muse), p1 = exp2f(s[i][2 * r + 1] - muse);
+        s[i][2 * r] = p0;
+        s[i][2 * r + 1] = p1;
+        psum += p0 + p1;
       }
+      lrow[r] = lrow[r] * alpha[r] + psum;
+    }
+#pragma unroll
+    for (int i = 0; i < D / 8; i++) {
+      o[i][0] *= alpha[0]; o[i][1] *= alpha[0];
+      o[i][2] *= alpha[1]; o[i][3] *= alpha[1];
+    }
+    // O += P V over this warp's 16 keys
+    uint32_t pf[4];
+    pf[0] = pack_bf16(s[0][0], s[0][1]);
+    pf[1] = pack_bf16(s[0][2], s[0][3]);
+    pf[2] = pack_bf16(s[1][0], s[1][1]);
+    pf[3] = pack_bf16(s[1][2], s[1][3]);
+#pragma unroll
+    for (int dn = 0; dn < D / 16; dn++) {
+      uint32_t b0, b1, b2, b3;
+      const int id = lane >> 3;
+      const int r = (id & 1) * 8 + (lane & 7);
+      const int c = dn * 16 + (id >> 1) * 8;
+      ldmatrix_x4_trans(b0, b1, b2, b3, v_s + r * LD + c);
+      mma_bf16_16816(o[2 * dn], pf, b0, b1);
+      mma_bf16_16816(o[2 * dn + 1], pf, b2, b3);
     }
     __syncthreads();
   }
-  // the two key halves of every column pair meet in shared memory
-  if (kh == 1) {
+  cp_async_wait<0>();
+
+  // ---- the four warps' states meet: fo[warp][head][column] in the tile buffers
 #pragma unroll
-    for (int i = 0; i < G; i++) { sp[(i * HC + cp) * 2] = acc[i][0]; sp[(i * HC + cp) * 2 + 1] = acc[i][1]; }
+  for (int r = 0; r < 2; r++) {
+    lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 1);
+    lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 2);
+    if (q == 0) { wm[warp][g4 + 8 * r] = mrow[r]; wl[warp][g4 + 8 * r] = lrow[r]; }
   }
+  float *fo = reinterpret_cast<float *>(sK);  // [4][16][D] floats = 32 KB at D = 128 <= the tile buffers
   __syncthreads();
-  // partial results: o [h][split][d], (m, l) [h][split][2]
 #pragma unroll
-  for (int i = 0; i < G; i++) {
-    if (i < gh) {
-      const size_t hs = (size_t)(h0 + i) * n_splits + split;
-      if (kh == 0) {
-        part_o[hs * D + 2 * cp] = acc[i][0] + sp[(i * HC + cp) * 2];
-        part_o[hs * D + 2 * cp + 1] = acc[i][1] + sp[(i * HC + cp) * 2 + 1];
-      }
-      if (tid == 0) { part_ml[hs * 2] = mrun[i]; part_ml[hs * 2 + 1] = lrun[i]; }
+  for (int r = 0; r < 2; r++)
+#pragma unroll
+    for (int i = 0; i < D / 8; i++) {
+      float2 val = make_float2(o[i][2 * r], o[i][2 * r + 1]);
+      *reinterpret_cast<float2 *>(fo + ((size_t)(warp * DA_G + g4 + 8 * r)) * D + i * 8 + q * 2) = val;
     }
+  __syncthreads();
+  // partial result of this split: o [h][split][D] (not normalised), (m, l) [h][split][2]
+  for (int idx = tid; idx < gh * D; idx += DA_THREADS) {
+    const int i = idx / D, c = idx - i * D;
+    const float mx = fmaxf(fmaxf(wm[0][i], wm[1][i]), fmaxf(wm[2][i], wm[3][i]));
+    float acc = 0.f, l = 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; w++) {
+      const float wgt = (wm[w][i] == -INFINITY) ? 0.f : exp2f(wm[w][i] - mx);
+      acc = fmaf(wgt, fo[((size_t)(w * DA_G + i)) * D + c], acc);
+      l = fmaf(wgt, wl[w][i], l);
+    }
+    const size_t hs = (size_t)(h0 + i) * n_splits + split;
+    part_o[hs * D + c] = acc;
+    if (c == 0) { part_ml[hs * 2] = mx; part_ml[hs * 2 + 1] = l; }
   }
-  // the split that finishes last for this (KV head, head group) merges the partial results, in
-  // split order; the wrapping atomic leaves the counter at zero for the next step
-  __shared__ bool last;
+
+  // ---- the split that finishes last merges the partial results of all splits
   __threadfence();
   __syncthreads();
   if (tid == 0) last = atomicInc(&counters[m * gridDim.z + hg], n_splits - 1) == (unsigned)(n_splits - 1);
   __syncthreads();
   if (!last) return;
   __threadfence();
-  // sm / sl: running maximum and sum of every split; then one thread per head turns them into
-  // weights; then thread = column adds the weighted partial outputs, four loads in flight
-  __shared__ float sm[DA_MAXG][64], sl[DA_MAXG][64], sinv[DA_MAXG];
   for (int idx = tid; idx < gh * n_splits; idx += DA_THREADS) {
     const int i = idx / n_splits, s2 = idx - i * n_splits;
     const size_t hs = (size_t)(h0 + i) * n_splits + s2;
@@ -365,7 +367,7 @@ attn_decode_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_ro
     sl[i][s2] = __ldcg(part_ml + hs * 2 + 1);
   }
   __syncthreads();
-  if (tid < gh) {
+  if (tid < gh) {  // weights of the splits of head tid
     float mx = -INFINITY;
     for (int s2 = 0; s2 < n_splits; s2++) mx = fmaxf(mx, sm[tid][s2]);
     float l = 0.f;
@@ -378,28 +380,34 @@ attn_decode_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_ro
     sinv[tid] = 1.0f / l;
   }
   __syncthreads();
-  if (tid < D) {
-    // all heads of this column together, four splits at a time: 4 G loads in flight per thread
-    float o[G];
+  // thread = (head, column) items, four at a time with eight splits each in flight
+  for (int base = 0; base < gh * D; base += 4 * DA_THREADS) {
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    int hi[4];
+    const float *po[4];
 #pragma unroll
-    for (int i = 0; i < G; i++) o[i] = 0.f;
-    const float *po = part_o + (size_t)h0 * n_splits * D + tid;
-    for (int s2 = 0; s2 < n_splits; s2 += 4) {
-      float a[G][4];
+    for (int t = 0; t < 4; t++) {
+      const int idx = min(base + t * DA_THREADS + tid, gh * D - 1);
+      hi[t] = idx / D;
+      po[t] = part_o + (size_t)(h0 + hi[t]) * n_splits * D + (idx - hi[t] * D);
+    }
+    for (int s2 = 0; s2 < n_splits; s2 += 8) {
+      float a[4][8];
 #pragma unroll
-      for (int i = 0; i < G; i++)
+      for (int t = 0; t < 4; t++)
 #pragma unroll
-        for (int u = 0; u < 4; u++)
-          a[i][u] = (i < gh && s2 + u < n_splits) ? __ldcg(po + ((size_t)i * n_splits + s2 + u) * D) : 0.f;
+        for (int u = 0; u < 8; u++) a[t][u] = (s2 + u < n_splits) ? __ldcg(po[t] + (size_t)(s2 + u) * D) : 0.f;
 #pragma unroll
-      for (int i = 0; i < G; i++)
+      for (int t = 0; t < 4; t++)
 #pragma unroll
-        for (int u = 0; u < 4; u++)
-          if (s2 + u < n_splits) o[i] = fmaf(sm[i][s2 + u], a[i][u], o[i]);
+        for (int u = 0; u < 8; u++)
+          if (s2 + u < n_splits) acc[t] = fmaf(sm[hi[t]][s2 + u], a[t][u], acc[t]);
     }
 #pragma unroll
-    for (int i = 0; i < G; i++)
-      if (i < gh) out[(size_t)(h0 + i) * D + tid] = __float2bfloat16_rn(o[i] * sinv[i]);
+    for (int t = 0; t < 4; t++) {
+      const int idx = base + t * DA_THREADS + tid;
+      if (idx < gh * D) out[(size_t)(h0 + hi[t]) * D + (idx - hi[t] * D)] = __float2bfloat16_rn(acc[t] * sinv[hi[t]]);
+    }
   }
 }
 
@@ -449,38 +457,26 @@ cudaError_t launch_attention_decode(const bf16 *q_rot, const bf16 *k_rot, const 
                                     float *part_o, float *part_ml, unsigned *counters, int h, int h_kv, int d,
                                     int cap, int n, int n_splits, cudaStream_t st) {
   const int g = h / h_kv;
-  const int G = g >= 8 ? 8 : (g > 2 ? (g == 4 ? 4 : 8) : g);  // 1, 2, 4 exactly; otherwise blocks of 8
-  dim3 grid(h_kv, n_splits, (g + G - 1) / G);
-  if ((int)grid.x * (int)grid.z > 32 * 16) return cudaErrorInvalidValue;  // counters: one per (x, z)
+  dim3 grid(h_kv, n_splits, (g + DA_G - 1) / DA_G);
+  if ((int)grid.x * (int)grid.z > 32 * 16 || n_splits > 64) return cudaErrorInvalidValue;
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)d);
-  const int smem = 2 * DA_THREADS * d * (int)sizeof(bf16);
-  auto launch = [&](auto kern) -> cudaError_t {
-    static bool attr_set[4][3] = {};  // per (G, d) instantiation: the kernels share one pointer type
-    bool &done = attr_set[G == 1 ? 0 : (G == 2 ? 1 : (G == 4 ? 2 : 3))][d == 64 ? 0 : (d == 96 ? 1 : 2)];
-    if (!done) {
-      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           2 * DA_THREADS * 128 * (int)sizeof(bf16));
+  auto launch = [&](auto kern, int smem, bool &attr_set) -> cudaError_t {
+    if (!attr_set) {
+      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
       if (e != cudaSuccess) return e;
-      done = true;
+      attr_set = true;
     }
-    kern<<<grid, DA_THREADS, smem, st>>>(q_rot, k_rot, v, part_o, part_ml, h, h_kv, d, cap, n, n_splits,
+    kern<<<grid, DA_THREADS, smem, st>>>(q_rot, k_rot, v, part_o, part_ml, h, h_kv, cap, n, n_splits,
                                          scale_log2, counters, out);
     return cudaGetLastError();
   };
-#define LOCRET_DA_CASE(GG)                                           \
-  switch (d) {                                                       \
-    case 64: return launch(attn_decode_kernel<GG, 64>);              \
-    case 96: return launch(attn_decode_kernel<GG, 96>);              \
-    case 128: return launch(attn_decode_kernel<GG, 128>);            \
-    default: return cudaErrorInvalidValue;                           \
+  static bool set64 = false, set96 = false, set128 = false;
+  switch (d) {
+    case 64: return launch(attn_decode_kernel<64>, (DA_G + 4 * DA_KT) * (64 + 8) * 2, set64);
+    case 96: return launch(attn_decode_kernel<96>, (DA_G + 4 * DA_KT) * (96 + 8) * 2, set96);
+    case 128: return launch(attn_decode_kernel<128>, (DA_G + 4 * DA_KT) * (128 + 8) * 2, set128);
   }
-  switch (G) {
-    case 1: LOCRET_DA_CASE(1)
-    case 2: LOCRET_DA_CASE(2)
-    case 4: LOCRET_DA_CASE(4)
-    default: LOCRET_DA_CASE(8)
-  }
-#undef LOCRET_DA_CASE
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace locret
