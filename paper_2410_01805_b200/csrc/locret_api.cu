@@ -37,10 +37,6 @@ struct ScratchPool {
   // decode kernels whose last block merges the partial results: zeroed words that each launch
   // leaves at zero (word 0: retaining head; words 1..: attention, one per KV head x head group)
   unsigned *dec_cnt = nullptr;
-  // recorded after the last second-stream kernel of every chunk step: a decode step, which runs
-  // on the caller's stream alone, waits for it before it reuses the shared scratch
-  cudaEvent_t ev_side_tail = nullptr;
-  bool side_tail_pending = false;
   float *partial = nullptr;
   int32_t *keep = nullptr;
   struct CsTable { float theta; int d, cap; float2 *ptr; };
@@ -127,7 +123,6 @@ void release_pool(ScratchPool *p) {
     if (p->ev_stage_free[i]) cudaEventDestroy(p->ev_stage_free[i]);
   }
   cudaFree(p->q_rot); cudaFree(p->partial); cudaFree(p->keep); cudaFree(p->dec_o); cudaFree(p->dec_ml); cudaFree(p->dec_cnt);
-  if (p->ev_side_tail) cudaEventDestroy(p->ev_side_tail);
   cudaFree(p->k_exp); cudaFree(p->v_exp);
   for (auto &t : p->cs) cudaFree(t.ptr);
   g_pools.erase(p->st);
@@ -291,7 +286,6 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
         g = g && cudaStreamCreateWithPriority(&p->side, cudaStreamNonBlocking, lo) == cudaSuccess;
         for (int i = 0; i < 2 && g; i++)
           g = cudaEventCreateWithFlags(&p->ev_stage_free[i], cudaEventDisableTiming) == cudaSuccess;
-        g = g && cudaEventCreateWithFlags(&p->ev_side_tail, cudaEventDisableTiming) == cudaSuccess;
       }
       if (g && !p->dec_cnt) {
         g = cudaMalloc(&p->dec_cnt, DEC_CNT_WORDS * sizeof(unsigned)) == cudaSuccess &&
@@ -392,7 +386,7 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
   ScratchPool *P = L->pool;
   const int c = L->cur;
   const bool decode = n_tok == 1 && L->use_tc;  // one token: bandwidth-bound kernels of decode.cu
-  const bool side = L->use_side && !L->serialize && !decode;
+  const bool side = L->use_side && !L->serialize;
   cudaStream_t S = side ? P->side : L->st;  // stream of the off-critical-path kernels
   const int sb = P->flip;                    // staging buffer of this call
   P->flip ^= 1;
@@ -405,10 +399,6 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
     P->stage_busy[sb] = false;
     if (L->side_pending) CK(cudaStreamWaitEvent(L->st, L->ev_side, 0));
     L->side_pending = false;
-    if (decode && P->side_tail_pending) {
-      CK(cudaStreamWaitEvent(L->st, P->ev_side_tail, 0));
-      P->side_tail_pending = false;
-    }
   }
 
   // a 4-bit cache is expanded into bf16 scratch first: keys rotated at position = slot
@@ -535,8 +525,6 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
   if (side) {
     CK(cudaEventRecord(L->ev_side, S));
     L->side_pending = true;
-    CK(cudaEventRecord(P->ev_side_tail, S));
-    P->side_tail_pending = true;
   }
   L->seen += n_tok;
   return LOCRET_OK;
