@@ -170,10 +170,14 @@ cudaError_t launch_rh_gemv(const bf16 *z, const bf16 *W1t, const float *W2, floa
 int rh_gemv_blocks(int d_R);
 int decode_attn_splits(int h_kv, int n);
 // part_o: fp32 [h][n_splits][d]; part_ml: fp32 [h][n_splits][2]; counters: one zeroed word per
-// (KV head, group of 8 query heads), left at zero (the last split merges the partial results)
+// (KV head, group of 16 query heads), left at zero (the last split merges the partial results).
+// q4 != nullptr: keys [0, n - 1) are read from the 4-bit cache (expanded and rotated with `cs` on the
+// way into shared memory) and only key n - 1, the token of this step, from k_rot / v.
+struct Int4Half;
 cudaError_t launch_attention_decode(const bf16 *q_rot, const bf16 *k_rot, const bf16 *v, bf16 *out,
                                     float *part_o, float *part_ml, unsigned *counters, int h, int h_kv, int d,
-                                    int cap, int n, int n_splits, cudaStream_t st);
+                                    int cap, int n, int n_splits, const Int4Half *q4, const float2 *cs,
+                                    cudaStream_t st);
 
 // dst[c][r] = src[r][c]  (weight repack at create)
 cudaError_t launch_transpose_bf16(const bf16 *src, bf16 *dst, int rows, int cols, cudaStream_t st);

@@ -171,6 +171,23 @@ gemv_rope_kernel(const bf16 *__restrict__ x, const bf16 *__restrict__ Wt, int K,
   }
 }
 
+// 4-bit codes -> floats, the arithmetic of the cache's expansion pre-pass (two codes per byte, even
+// element in the low nibble, value = code * scale)
+__device__ __forceinline__ void dequant8(uint32_t w, float s, float (&x)[8]) {
+#pragma unroll
+  for (int b = 0; b < 4; b++) {
+    const uint32_t byte = (w >> (8 * b)) & 0xFFu;
+    x[2 * b] = (float)((int)(byte << 28) >> 28) * s;
+    x[2 * b + 1] = (float)((int)(byte << 24) >> 28) * s;
+  }
+}
+__device__ __forceinline__ uint4 to_bf16x8(const float (&x)[8]) {
+  uint4 o;
+  o.x = pack_bf16(x[0], x[1]); o.y = pack_bf16(x[2], x[3]);
+  o.z = pack_bf16(x[4], x[5]); o.w = pack_bf16(x[6], x[7]);
+  return o;
+}
+
 // ---- decode attention on warp-level tensor-core instructions.  grid (h_kv, splits, head groups
 // of <= 16).  The rows of the m16n8k16 tiles are the query heads of one GQA group (all of them read
 // the same keys), padded to 16; keys and values of the split stream through shared memory in
@@ -181,12 +198,17 @@ gemv_rope_kernel(const bf16 *__restrict__ x, const bf16 *__restrict__ Wt, int K,
 // order (a wrapping atomic counter, left at zero for the next step).
 constexpr int DA_THREADS = 128, DA_G = 16, DA_KT = 64;
 
-template <int D>
+// INT4: keys [0, n - 1) come from the 4-bit cache (codes and scales expanded, keys rotated at
+// position = slot, with the arithmetic of the expansion pre-pass, as the tile is brought into shared
+// memory); key n - 1, the token of this step, comes from the bf16 arrays k_rot / v like every key of
+// a bf16 cache.
+template <int D, bool INT4>
 __global__ void __launch_bounds__(DA_THREADS)
 attn_decode_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_rot,
                    const bf16 *__restrict__ v, float *__restrict__ part_o, float *__restrict__ part_ml,
                    int h, int h_kv, int cap, int n, int n_splits, float scale_log2,
-                   unsigned *__restrict__ counters, bf16 *__restrict__ out) {
+                   unsigned *__restrict__ counters, bf16 *__restrict__ out, Int4Half q4,
+                   const float2 *__restrict__ cs) {
   constexpr int LD = D + 8;
   constexpr int VPR = D / 8;  // 16-byte vectors per row
   extern __shared__ __align__(16) unsigned char da_smem[];
@@ -219,11 +241,46 @@ attn_decode_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_ro
       cp_async16(sV + (buf * DA_KT + r) * LD + c, vbase + off, ok);
     }
   };
+  // 4-bit cache: one thread expands elements [c, c+8) and [c+half, c+half+8) of K and V of one key
+  auto load_kv_q4 = [&](int buf, int kt) {
+    constexpr int HALF = D / 2, HV = D / 16;
+    for (int x = tid; x < DA_KT * HV; x += DA_THREADS) {
+      const int r = x / HV, c = (x - r * HV) * 8;
+      const int key = k0 + kt * DA_KT + r;
+      bf16 *kd = sK + (buf * DA_KT + r) * LD, *vd = sV + (buf * DA_KT + r) * LD;
+      uint4 ka = make_uint4(0, 0, 0, 0), kb = ka, va = ka, vb = ka;
+      if (key < n - 1) {
+        const size_t u = (size_t)m * cap + key;
+        const uint8_t *kc = q4.kq + u * HALF, *vc = q4.vq + u * HALF;
+        const float ks = __half2float(q4.ks[u]), vs = __half2float(q4.vs[u]);
+        float a[8], b[8];
+        dequant8(*reinterpret_cast<const uint32_t *>(kc + c / 2), ks, a);
+        dequant8(*reinterpret_cast<const uint32_t *>(kc + (c + HALF) / 2), ks, b);
+        const float2 *t = cs + (size_t)key * HALF + c;
+#pragma unroll
+        for (int e = 0; e < 8; e++) {
+          const float x1 = a[e], x2 = b[e];
+          a[e] = x1 * t[e].x - x2 * t[e].y;
+          b[e] = x2 * t[e].x + x1 * t[e].y;
+        }
+        ka = to_bf16x8(a); kb = to_bf16x8(b);
+        dequant8(*reinterpret_cast<const uint32_t *>(vc + c / 2), vs, a);
+        dequant8(*reinterpret_cast<const uint32_t *>(vc + (c + HALF) / 2), vs, b);
+        va = to_bf16x8(a); vb = to_bf16x8(b);
+      } else if (key < k1) {  // the token of this step
+        const size_t off = ((size_t)m * cap + key) * D + c;
+        ka = *reinterpret_cast<const uint4 *>(k_rot + off); kb = *reinterpret_cast<const uint4 *>(k_rot + off + HALF);
+        va = *reinterpret_cast<const uint4 *>(v + off); vb = *reinterpret_cast<const uint4 *>(v + off + HALF);
+      }
+      *reinterpret_cast<uint4 *>(kd + c) = ka; *reinterpret_cast<uint4 *>(kd + c + HALF) = kb;
+      *reinterpret_cast<uint4 *>(vd + c) = va; *reinterpret_cast<uint4 *>(vd + c + HALF) = vb;
+    }
+  };
   for (int x = tid; x < DA_G * VPR; x += DA_THREADS) {
     const int r = x / VPR, c = (x - r * VPR) * 8;
     cp_async16(sQ + r * LD + c, q_rot + (size_t)(h0 + min(r, gh - 1)) * D + c, r < gh);
   }
-  if (NKT > 0) load_kv(0, 0);
+  if (!INT4 && NKT > 0) load_kv(0, 0);
   cp_async_commit();
 
   uint32_t qf[D / 16][4];
@@ -235,9 +292,14 @@ attn_decode_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_ro
   float mrow[2] = {-INFINITY, -INFINITY}, lrow[2] = {0.f, 0.f};  // heads g4 and g4 + 8
 
   for (int kt = 0; kt < NKT; kt++) {
-    if (kt + 1 < NKT) load_kv((kt + 1) & 1, kt + 1);
-    cp_async_commit();
-    cp_async_wait<1>();
+    if (INT4) {
+      load_kv_q4(kt & 1, kt);  // (the other buffer may still be read by a slower warp)
+      cp_async_wait<0>();
+    } else {
+      if (kt + 1 < NKT) load_kv((kt + 1) & 1, kt + 1);
+      cp_async_commit();
+      cp_async_wait<1>();
+    }
     __syncthreads();
     if (kt == 0) {
 #pragma unroll
@@ -455,11 +517,13 @@ int decode_attn_splits(int h_kv, int n) {
 
 cudaError_t launch_attention_decode(const bf16 *q_rot, const bf16 *k_rot, const bf16 *v, bf16 *out,
                                     float *part_o, float *part_ml, unsigned *counters, int h, int h_kv, int d,
-                                    int cap, int n, int n_splits, cudaStream_t st) {
+                                    int cap, int n, int n_splits, const Int4Half *q4, const float2 *cs,
+                                    cudaStream_t st) {
   const int g = h / h_kv;
   dim3 grid(h_kv, n_splits, (g + DA_G - 1) / DA_G);
   if ((int)grid.x * (int)grid.z > 32 * 16 || n_splits > 64) return cudaErrorInvalidValue;
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)d);
+  const Int4Half qq = q4 ? *q4 : Int4Half{nullptr, nullptr, nullptr, nullptr};
   auto launch = [&](auto kern, int smem, bool &attr_set) -> cudaError_t {
     if (!attr_set) {
       cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -467,14 +531,21 @@ cudaError_t launch_attention_decode(const bf16 *q_rot, const bf16 *k_rot, const 
       attr_set = true;
     }
     kern<<<grid, DA_THREADS, smem, st>>>(q_rot, k_rot, v, part_o, part_ml, h, h_kv, cap, n, n_splits,
-                                         scale_log2, counters, out);
+                                         scale_log2, counters, out, qq, cs);
     return cudaGetLastError();
   };
-  static bool set64 = false, set96 = false, set128 = false;
+  static bool set_done[2][3] = {};
+  const int qi = q4 ? 1 : 0;
   switch (d) {
-    case 64: return launch(attn_decode_kernel<64>, (DA_G + 4 * DA_KT) * (64 + 8) * 2, set64);
-    case 96: return launch(attn_decode_kernel<96>, (DA_G + 4 * DA_KT) * (96 + 8) * 2, set96);
-    case 128: return launch(attn_decode_kernel<128>, (DA_G + 4 * DA_KT) * (128 + 8) * 2, set128);
+    case 64:
+      return q4 ? launch(attn_decode_kernel<64, true>, (DA_G + 4 * DA_KT) * (64 + 8) * 2, set_done[qi][0])
+                : launch(attn_decode_kernel<64, false>, (DA_G + 4 * DA_KT) * (64 + 8) * 2, set_done[qi][0]);
+    case 96:
+      return q4 ? launch(attn_decode_kernel<96, true>, (DA_G + 4 * DA_KT) * (96 + 8) * 2, set_done[qi][1])
+                : launch(attn_decode_kernel<96, false>, (DA_G + 4 * DA_KT) * (96 + 8) * 2, set_done[qi][1]);
+    case 128:
+      return q4 ? launch(attn_decode_kernel<128, true>, (DA_G + 4 * DA_KT) * (128 + 8) * 2, set_done[qi][2])
+                : launch(attn_decode_kernel<128, false>, (DA_G + 4 * DA_KT) * (128 + 8) * 2, set_done[qi][2]);
   }
   return cudaErrorInvalidValue;
 }

@@ -413,8 +413,9 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
   // with a tensor-core projection and head_dim 64 / 128 the epilogue of the GEMM does the RoPE pass
   const bool fused_rope = !decode && L->fuse_rope && L->use_tc && n_tok >= 32 &&
                           qkv_rope_tc_supported(n_tok, L->d_in, L->D, L->D, L->D, L->d);
-  if (L->int4 && L->len > 0) {
+  if (L->int4 && L->len > 0 && !decode) {
     // the expansion writes slots [0, len) of the scratch the chunk's units are appended to
+    // (a one-token step reads the codes inside its attention kernel instead)
     Timed t(L, LOCRET_K_DEQUANT);
     CK(launch_dequant(L->q4[c], P->k_exp, P->v_exp, L->cs, L->h_kv, L->d, L->cap, L->len, true, L->st));
   }
@@ -460,7 +461,8 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
     }
     if (decode)
       CK(launch_attention_decode(P->q_rot, k_att, v_att, (bf16 *)attn_out, P->dec_o, P->dec_ml, P->dec_cnt + 1,
-                                 L->h, L->h_kv, L->d, L->cap, n, decode_attn_splits(L->h_kv, n), L->st));
+                                 L->h, L->h_kv, L->d, L->cap, n, decode_attn_splits(L->h_kv, n),
+                                 L->int4 ? &L->q4[c] : nullptr, L->cs, L->st));
     else if (tc_ok)
       CK(launch_attention_tc(&L->map_q, &L->map_k, &L->map_v[c], (bf16 *)attn_out, n_tok, L->h, L->h_kv,
                              L->d, L->len, L->d_status, L->st));

@@ -123,13 +123,14 @@ def test_flags_and_decode_lockstep():
     gpu.destroy()
 
 
-@pytest.mark.parametrize("d,heads,n_stab", [(128, (8, 2), 0), (64, (4, 4), 9), (96, (3, 3), 5)])
-def test_single_token_steps_that_evict(d, heads, n_stab):
+@pytest.mark.parametrize("d,heads,n_stab,kv_dtype", [(128, (8, 2), 0, 0), (64, (4, 4), 9, 0), (96, (3, 3), 5, 0),
+                                                      (128, (8, 2), 7, 1), (64, (4, 1), 0, 1)])
+def test_single_token_steps_that_evict(d, heads, n_stab, kv_dtype):
     """Decode-time eviction (a multi-turn stream with a small budget): once the cache is full every
     one-token step with flags = 0 scores the new unit, drops one and compacts, through the
     one-token kernels."""
     from parity_util import lockstep_chunk, make_pair
-    sh = small_shape(h=heads[0], hk=heads[1], d=d, D=128, dR=64, rope_theta=500000.0)
+    sh = small_shape(h=heads[0], hk=heads[1], d=d, D=128, dR=64, rope_theta=500000.0, kv_dtype=kv_dtype)
     ora, gpu = make_pair(sh, weights_for(sh, 11), budget=96, chunk=64, n_stab=n_stab)
     lockstep_chunk(ora, gpu, hidden(64, sh.d_model, 70), 0, what="fill 1")
     lockstep_chunk(ora, gpu, hidden(64, sh.d_model, 71), 0, what="fill 2 (evicts)")
