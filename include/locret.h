@@ -56,11 +56,14 @@ extern "C" {
 
 /* kernel families, indices into locret_read_timing's arrays */
 enum {
-  LOCRET_K_QKV = 0,     /* (a) projection GEMM                                   */
-  LOCRET_K_ROPE,        /* position assignment + RoPE + append of the chunk       */
+  LOCRET_K_QKV = 0,     /* (a) projection GEMM (head_dim 64 / 128 and one-token   */
+                        /*     steps: positions, RoPE and append in the same kernel) */
+  LOCRET_K_ROPE,        /* position assignment + RoPE + append of the chunk, where */
+                        /*     it is a kernel of its own (head_dim 96, fallbacks)  */
   LOCRET_K_ATTN,        /* (b) attention                                          */
   LOCRET_K_RH,          /* (c) retaining head GEMM -> activation -> GEMM          */
-  LOCRET_K_RH_REDUCE,   /* (c) sum of the retaining head's partial scores         */
+  LOCRET_K_RH_REDUCE,   /* (c) sum of the retaining head's partial scores (a      */
+                        /*     one-token step sums them inside LOCRET_K_RH)        */
   LOCRET_K_TOPK,        /* (d) per-head selection                                 */
   LOCRET_K_COMPACT,     /* (d) gather / compaction + re-RoPE of kept keys         */
   LOCRET_K_DEQUANT,     /* 4-bit cache: expansion of the retained units to bf16   */
