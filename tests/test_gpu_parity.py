@@ -124,7 +124,8 @@ def test_flags_and_decode_lockstep():
 
 
 @pytest.mark.parametrize("d,heads,n_stab,kv_dtype", [(128, (8, 2), 0, 0), (64, (4, 4), 9, 0), (96, (3, 3), 5, 0),
-                                                      (128, (8, 2), 7, 1), (64, (4, 1), 0, 1)])
+                                                      (128, (8, 2), 7, 1), (64, (4, 1), 0, 1),
+                                                      (64, (40, 1), 3, 0)])  # 40 heads on one KV head: three head groups
 def test_single_token_steps_that_evict(d, heads, n_stab, kv_dtype):
     """Decode-time eviction (a multi-turn stream with a small budget): once the cache is full every
     one-token step with flags = 0 scores the new unit, drops one and compacts, through the
