@@ -35,7 +35,7 @@ class locret_layer_cfg(C.Structure):
 def _load():
     if not os.path.exists(lib_path):
         raise ImportError(
-            f"{lib_path} is missing: build it with `python -m paper_2410_01805_b200.build` "
+            f"{lib_path} is missing: build it with `python paper_2410_01805_b200/build.py` "
             "(there is no CPU fallback)")
     l = C.CDLL(lib_path)
     P = C.c_void_p
