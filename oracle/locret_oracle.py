@@ -343,3 +343,60 @@ class OracleLayer:
     def decode_step(self, x):
         """The B = 1 case of Eq. 1: append without eviction."""
         return self.prefill_chunk(np.asarray(x, np.float64).reshape(1, -1), NO_EVICT)
+
+
+# --------------------------------------------------------------------------- the rest of the decoder layer
+#
+# Section 3.1 writes the layer as A = [A_1 .. A_h] W^O followed by H = FFN(A) and leaves the
+# normalisation, the residual connections and the form of the FFN to the backbone.  Both
+# backbones of the paper (Llama-3.1, Phi-3) are pre-norm decoders with a gated SiLU FFN, which
+# is the reading taken here:
+#     h1 = RMSNorm(x; g1)            -> the attention block above (its hidden_in is h1)
+#     x1 = x + attn_out W_o
+#     h2 = RMSNorm(x1; g2)
+#     y  = x1 + (silu(h2 W_gate) * (h2 W_up)) W_down
+
+RMS_EPS = 1e-5
+
+
+def rmsnorm(x, gain, eps: float = RMS_EPS):
+    """Row-wise x / sqrt(mean(x^2) + eps) * gain."""
+    x = np.asarray(x, np.float64)
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x / np.sqrt(ms + eps) * np.asarray(gain, np.float64)
+
+
+def gated_ffn(h, w_gate, w_up, w_down, rnd=None):
+    """(silu(h W_gate) * (h W_up)) W_down; `rnd` rounds the gated product where it is stored."""
+    h = np.asarray(h, np.float64)
+    a = activation(h @ np.asarray(w_gate, np.float64), 0) * (h @ np.asarray(w_up, np.float64))
+    if rnd is not None:
+        a = rnd(a)
+    return a @ np.asarray(w_down, np.float64)
+
+
+class OracleBlock:
+    """One decoder layer: RMSNorm -> attention block with eviction (OracleLayer) -> W_o + residual
+    -> RMSNorm -> gated FFN + residual.  In mirror mode values are rounded to bf16 where the CUDA
+    path stores them: h1, x1, h2, the gated product, y."""
+
+    def __init__(self, attn: "OracleLayer", w_o, w_gate, w_up, w_down, g1, g2):
+        self.attn = attn
+        self.w_o = np.asarray(w_o, np.float64)
+        self.w_gate, self.w_up = np.asarray(w_gate, np.float64), np.asarray(w_up, np.float64)
+        self.w_down = np.asarray(w_down, np.float64)
+        self.g1, self.g2 = np.asarray(g1, np.float64), np.asarray(g2, np.float64)
+        self.last_h1 = None
+
+    def _r(self, x):
+        return round_bf16(x) if self.attn.mirror else x
+
+    def prefill_chunk(self, X, flags: int = 0, rows=None):
+        X = np.asarray(X, np.float64)
+        h1 = self._r(rmsnorm(X, self.g1))
+        self.last_h1 = h1
+        att = self.attn.prefill_chunk(h1, flags, rows=rows)        # NaN rows where not computed
+        att = self._r(att)
+        x1 = self._r(X + att @ self.w_o)
+        h2 = self._r(rmsnorm(x1, self.g2))
+        return self._r(x1 + gated_ffn(h2, self.w_gate, self.w_up, self.w_down, rnd=self._r))

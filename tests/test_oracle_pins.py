@@ -471,3 +471,67 @@ def test_mirror_mode_rounds_only_storage_points():
     a, b = lp.prefill_chunk(X), lm.prefill_chunk(X)
     assert np.array_equal(lm.K, O.round_bf16(lm.K))            # cached K is on the bf16 grid
     assert np.max(np.abs(a - b)) < 0.05 and not np.array_equal(a, b)
+
+
+# ------------------------------------------------------------------ the rest of the decoder layer
+
+def test_rmsnorm_matches_library_and_its_invariants():
+    g = np.random.default_rng(300)
+    x = g.standard_normal((9, 24)) * 3.0
+    gain = 1.0 + 0.1 * g.standard_normal(24)
+    want = torch.nn.functional.rms_norm(torch.from_numpy(x), (24,), torch.from_numpy(gain), eps=O.RMS_EPS).numpy()
+    assert np.allclose(O.rmsnorm(x, gain), want, rtol=0, atol=1e-13)
+    # unit gain: every row has mean square 1 (up to eps); scaling a row by c > 0 changes nothing
+    y = O.rmsnorm(x, np.ones(24), eps=0.0)
+    assert np.allclose(np.mean(y * y, axis=1), 1.0, atol=1e-12)
+    assert np.allclose(O.rmsnorm(7.5 * x, gain, eps=0.0), O.rmsnorm(x, gain, eps=0.0), atol=1e-12)
+    # a hand case: x = (3, 4) has mean square 12.5
+    assert np.allclose(O.rmsnorm(np.array([[3.0, 4.0]]), np.array([1.0, 2.0]), eps=0.0),
+                       [[3.0 / math.sqrt(12.5), 8.0 / math.sqrt(12.5)]])
+
+
+def test_gated_ffn_matches_library_ops():
+    g = np.random.default_rng(301)
+    h = g.standard_normal((7, 10))
+    wg, wu, wd = g.standard_normal((10, 14)), g.standard_normal((10, 14)), g.standard_normal((14, 10))
+    t = torch.from_numpy
+    want = ((torch.nn.functional.silu(t(h) @ t(wg)) * (t(h) @ t(wu))) @ t(wd)).numpy()
+    assert np.allclose(O.gated_ffn(h, wg, wu, wd), want, rtol=0, atol=1e-12)
+    # gate and up are not interchangeable, and a zero gate input gives zero (silu(0) = 0)
+    assert not np.allclose(O.gated_ffn(h, wu, wg, wd), want)
+    assert np.allclose(O.gated_ffn(h, np.zeros_like(wg), wu, wd), 0.0)
+
+
+def test_decoder_block_equals_library_composition_when_nothing_is_evicted():
+    """Budget >= context: the block is an ordinary pre-norm decoder layer, written here with the
+    library's rms_norm / scaled_dot_product_attention / silu, in any chunking."""
+    sh = shape(n_q_heads=4, n_kv_heads=2, head_dim=16, d_model=24)
+    ctx, F = 41, 40
+    h, hk, d, D = 4, 2, 16, 24
+    g = np.random.default_rng(302)
+    w_o = g.standard_normal((h * d, D)) / math.sqrt(h * d)
+    wg, wu = g.standard_normal((D, F)) / math.sqrt(D), g.standard_normal((D, F)) / math.sqrt(D)
+    wd = g.standard_normal((F, D)) / math.sqrt(F)
+    g1, g2 = 1.0 + 0.1 * g.standard_normal(D), 1.0 + 0.1 * g.standard_normal(D)
+    X = g.standard_normal((ctx, D)) * 2.0
+    t = torch.from_numpy
+    F_ = torch.nn.functional
+    outs = []
+    for B in (1, 6, 41):
+        layer, (wqkv, _, _) = rand_layer(sh, budget=64, chunk=B, n_stab=0, seed=303)
+        blk = O.OracleBlock(layer, w_o, wg, wu, wd, g1, g2)
+        outs.append(np.concatenate([blk.prefill_chunk(X[s:s + B]) for s in range(0, ctx, B)], axis=0))
+    h1 = F_.rms_norm(t(X), (D,), t(g1), eps=O.RMS_EPS)
+    proj = h1 @ t(wqkv)
+    pos = np.arange(ctx)[:, None]
+    Q = t(O.rope(proj[:, : h * d].reshape(ctx, h, d).numpy(), pos, sh.rope_theta))
+    K = t(O.rope(proj[:, h * d:(h + hk) * d].reshape(ctx, hk, d).numpy(), pos, sh.rope_theta))
+    V = proj[:, (h + hk) * d:].reshape(ctx, hk, d)
+    K, V = K.repeat_interleave(h // hk, dim=1), V.repeat_interleave(h // hk, dim=1)
+    att = F_.scaled_dot_product_attention(Q.transpose(0, 1), K.transpose(0, 1), V.transpose(0, 1), is_causal=True)
+    att = att.transpose(0, 1).reshape(ctx, h * d)
+    x1 = t(X) + att @ t(w_o)
+    h2 = F_.rms_norm(x1, (D,), t(g2), eps=O.RMS_EPS)
+    want = (x1 + (F_.silu(h2 @ t(wg)) * (h2 @ t(wu))) @ t(wd)).numpy()
+    for got in outs:
+        assert np.allclose(got, want, rtol=0, atol=1e-10)

@@ -9,6 +9,7 @@ float32 values.
 from .configs import CONFIGS, LayerShape, Workload, get_workload  # noqa: F401
 from .generate import (  # noqa: F401
     BASE_SEED,
+    block_weights,
     hidden_block_tokens,
     hidden_states,
     layer_weights,

@@ -22,6 +22,7 @@ class LayerShape:
     act: int = 0          # 0 SiLU, 1 GELU(tanh), 2 ReLU
     rh_input: int = 0     # 0: retaining head sees pre-RoPE [Q;K;V], 1: post-RoPE Q,K
     kv_dtype: int = 0     # 0 bf16 cache, 1 int4 (group = head vector) + fp16 scale
+    d_ff: int = 0         # hidden size of the gated FFN that closes the decoder layer (0: none given)
 
     @property
     def d_in(self) -> int:
@@ -54,15 +55,15 @@ class Workload:
 
 
 _LLAMA = LayerShape(d_model=4096, n_q_heads=32, n_kv_heads=8, head_dim=128,
-                    d_retain=1024, rope_theta=500000.0)
+                    d_retain=1024, rope_theta=500000.0, d_ff=14336)
 _PHI3 = LayerShape(d_model=3072, n_q_heads=32, n_kv_heads=32, head_dim=96,
-                   d_retain=1024, rope_theta=10000.0)
+                   d_retain=1024, rope_theta=10000.0, d_ff=8192)
 
 CONFIGS = {
     # configs[0]: the small case the oracle runs in full within seconds.
     "c1_small_gqa": Workload(
         "c1_small_gqa",
-        LayerShape(d_model=512, n_q_heads=8, n_kv_heads=2, head_dim=64, d_retain=256),
+        LayerShape(d_model=512, n_q_heads=8, n_kv_heads=2, head_dim=64, d_retain=256, d_ff=1536),
         n_layers=1, context=4096, chunk=512, budget=1024, n_stab=64, hidden="normal"),
     # configs[1]
     "c2_llama_32k": Workload(

@@ -23,6 +23,11 @@ _S_TOPIC_MEAN = 4
 _S_WQKV = 1000
 _S_W1 = 2000
 _S_W2 = 3000
+_S_WO = 4000
+_S_WGATE = 5000
+_S_WUP = 6000
+_S_WDOWN = 7000
+_S_NORM = 8000
 
 hidden_block_tokens = 1024
 
@@ -53,6 +58,24 @@ def layer_weights(shape: LayerShape, layer: int, seed: int = BASE_SEED):
     w2 = _rng(seed, _S_W2 + layer).standard_normal((d_R, hk), dtype=np.float32)
     w2 *= np.float32(1.0 / np.sqrt(d_R))
     return to_bf16_grid(wqkv), to_bf16_grid(w1), to_bf16_grid(w2)
+
+
+def block_weights(shape: LayerShape, layer: int, seed: int = BASE_SEED):
+    """Weights that close the decoder layer around the attention block: W_o [h*d x D],
+    W_gate, W_up [D x d_ff], W_down [d_ff x D], each ~ N(0, 1/fan_in), and the two RMSNorm gains
+    (1 + N(0, 0.1^2)), all on the bfloat16 grid."""
+    D, hd, F = shape.d_model, shape.n_q_heads * shape.head_dim, shape.d_ff
+    if F <= 0:
+        raise ValueError("the shape has no d_ff")
+    def w(stream, rows, cols):
+        a = _rng(seed, stream + layer).standard_normal((rows, cols), dtype=np.float32)
+        a *= np.float32(1.0 / np.sqrt(rows))
+        return to_bf16_grid(a)
+    g = _rng(seed, _S_NORM + layer)
+    g1 = to_bf16_grid(1.0 + 0.1 * g.standard_normal(D, dtype=np.float32))
+    g2 = to_bf16_grid(1.0 + 0.1 * g.standard_normal(D, dtype=np.float32))
+    return {"w_o": w(_S_WO, hd, D), "w_gate": w(_S_WGATE, D, F), "w_up": w(_S_WUP, D, F),
+            "w_down": w(_S_WDOWN, F, D), "g1": g1, "g2": g2}
 
 
 def _topic_sequence(context: int, seed: int, n_topics: int = 64, mean_len: int = 512):
