@@ -202,6 +202,53 @@ int locret_read_timing(locret_layer *layer, float *ms, int64_t *launches);
 int locret_launch_count(const locret_layer *layer, int64_t *count);
 
 /*
+ * ---- The rest of the decoder layer (beyond the scope of the chunk step itself) ----
+ *
+ * Section 3.1 writes a layer as A = [A_1 .. A_h] W^O followed by H = FFN(A) and leaves
+ * normalisation, residual connections and the form of the FFN to the backbone; both backbones
+ * of the paper are pre-norm decoders with a gated SiLU FFN, which is what a block computes:
+ *     h1 = RMSNorm(x; g1)   ->   the attention block above (hidden_in = h1), with eviction
+ *     x1 = x + attn_out W_o
+ *     h2 = RMSNorm(x1; g2)
+ *     y  = x1 + (silu(h2 W_gate) * (h2 W_up)) W_down
+ * so that a stack of blocks can be fed real hidden states, layer after layer.  bf16 storage of
+ * h1, attn_out, x1, h2, the gated product and y; fp32 accumulation everywhere.
+ */
+typedef struct locret_block locret_block;
+
+typedef struct {
+  locret_layer_cfg attn;  /* the attention block (its w_qkv multiplies h1)                       */
+  int32_t d_ff;           /* FFN hidden size; a multiple of 128                                   */
+  float   rms_eps;        /* epsilon of both RMSNorms (1e-5 if <= 0)                              */
+  const void *w_o;        /* device bf16 [h·d × d_model] row-major; borrowed until create returns */
+  const void *w_gate;     /* device bf16 [d_model × d_ff]                                         */
+  const void *w_up;       /* device bf16 [d_model × d_ff]                                         */
+  const void *w_down;     /* device bf16 [d_ff × d_model]                                         */
+  const void *g1, *g2;    /* device bf16 [d_model]: gains of the two RMSNorms                     */
+} locret_block_cfg;
+
+/*
+ * Create a block: the attention layer (locret_create with the same budget, chunk, n_stab) plus
+ * repacked copies of the four weight matrices and scratch shared by the blocks of one stream.
+ * On failure *out is NULL and nothing stays allocated.
+ */
+int locret_block_create(const locret_block_cfg *cfg, int32_t budget, int32_t chunk, int32_t n_stab,
+                        locret_block **out);
+
+/*
+ * One chunk through the whole layer.  x_in, y_out: device bf16 [n_tok × d_model], 16-byte
+ * aligned, 1 <= n_tok <= chunk; they may be the same buffer.  flags as for
+ * locret_prefill_chunk.  Asynchronous on the stream of cfg.attn.
+ */
+int locret_block_prefill_chunk(locret_block *block, const void *x_in, int32_t n_tok, uint32_t flags,
+                               void *y_out);
+
+/* The block's attention layer, for state export/import, status, timing (owned by the block). */
+locret_layer *locret_block_attention(locret_block *block);
+
+void locret_block_destroy(locret_block *block);
+
+/*
  * Retaining-head scores without any allocation.  (The paper has no counterpart: this entry
  * point exists for hosts that may not allocate device memory where they need scores, e.g. code
  * that runs inside a pool owning the whole device, or under an allocator that is locked while

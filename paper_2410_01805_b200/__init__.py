@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     K_NAMES,
     LAST_CHUNK,
     NO_EVICT,
+    LocretBlock,
     LocretError,
     LocretLayer,
     lib,

@@ -32,6 +32,14 @@ class locret_layer_cfg(C.Structure):
     ]
 
 
+class locret_block_cfg(C.Structure):
+    _fields_ = [
+        ("attn", locret_layer_cfg), ("d_ff", C.c_int32), ("rms_eps", C.c_float),
+        ("w_o", C.c_void_p), ("w_gate", C.c_void_p), ("w_up", C.c_void_p), ("w_down", C.c_void_p),
+        ("g1", C.c_void_p), ("g2", C.c_void_p),
+    ]
+
+
 def _load():
     if not os.path.exists(lib_path):
         raise ImportError(
@@ -59,6 +67,12 @@ def _load():
     l.locret_rh_scores_static.argtypes = [P, C.c_int32, C.c_int32, P, C.c_int32, P, C.c_int32, C.c_int32, P, P]
     l.locret_destroy.argtypes = [P]
     l.locret_destroy.restype = None
+    l.locret_block_create.argtypes = [C.POINTER(locret_block_cfg), C.c_int32, C.c_int32, C.c_int32, C.POINTER(P)]
+    l.locret_block_prefill_chunk.argtypes = [P, P, C.c_int32, C.c_uint32, P]
+    l.locret_block_attention.argtypes = [P]
+    l.locret_block_attention.restype = P
+    l.locret_block_destroy.argtypes = [P]
+    l.locret_block_destroy.restype = None
     return l
 
 
@@ -201,6 +215,54 @@ class LocretLayer:
         if self._h:
             lib.locret_destroy(self._h)
             self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+class LocretBlock:
+    """A whole decoder layer (RMSNorm, attention block with eviction, W_o, gated FFN); methods
+    mirror the locret_block_* entry points.  `attn` is the block's attention layer (owned by the
+    block), with the state / status / timing methods of LocretLayer."""
+
+    def __init__(self, shape, w_qkv, w1, w2, w_o, w_gate, w_up, w_down, g1, g2,
+                 budget: int, chunk: int, n_stab: int, reserve: int = 0, rms_eps: float = 1e-5, stream=None):
+        for w in (w_qkv, w1, w2, w_o, w_gate, w_up, w_down, g1, g2):
+            if not (w.is_cuda and w.dtype == torch.bfloat16 and w.is_contiguous()):
+                raise ValueError("weights must be contiguous CUDA bfloat16 tensors")
+        self.shape, self.chunk = shape, chunk
+        self.stream = stream if stream is not None else torch.cuda.current_stream()
+        cfg = locret_block_cfg(
+            locret_layer_cfg(
+                shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.d_retain,
+                shape.act, float(shape.rope_theta), shape.rh_input, shape.kv_dtype, reserve,
+                w_qkv.data_ptr(), w1.data_ptr(), w2.data_ptr(), self.stream.cuda_stream),
+            shape.d_ff, float(rms_eps), w_o.data_ptr(), w_gate.data_ptr(), w_up.data_ptr(), w_down.data_ptr(),
+            g1.data_ptr(), g2.data_ptr())
+        self._b = C.c_void_p()
+        _check(lib.locret_block_create(C.byref(cfg), budget, chunk, n_stab, C.byref(self._b)), "locret_block_create")
+        # a non-owning view of the attention layer
+        self.attn = LocretLayer.__new__(LocretLayer)
+        self.attn.shape = shape
+        self.attn.h, self.attn.h_kv, self.attn.d = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+        self.attn.chunk, self.attn.budget, self.attn.n_stab = chunk, budget, n_stab
+        self.attn.stream = self.stream
+        self.attn._h = C.c_void_p(lib.locret_block_attention(self._b))
+        self.attn.destroy = lambda: None
+
+    def prefill_chunk(self, x_in: torch.Tensor, y_out: torch.Tensor, flags: int = 0, n_tok: int | None = None):
+        n_tok = x_in.shape[0] if n_tok is None else n_tok
+        _check(lib.locret_block_prefill_chunk(self._b, x_in.data_ptr(), n_tok, flags, y_out.data_ptr()),
+               "locret_block_prefill_chunk")
+
+    def destroy(self):
+        if self._b:
+            self.attn._h = C.c_void_p()
+            lib.locret_block_destroy(self._b)
+            self._b = C.c_void_p()
 
     def __del__(self):
         try:

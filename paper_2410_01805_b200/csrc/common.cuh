@@ -84,6 +84,14 @@ int rh_num_tiles(int d_R);
 // The same two GEMMs on tcgen05 tensor cores (TMA-fed, TMEM accumulators); `status` is the
 // layer's device status word (set if a bounded wait gives up).
 bool gemm_tc_supported(int M, int N, int K, int lda, int ldb);
+// the same GEMM with a residual added before the one rounding: C = A Bt^T + R
+cudaError_t launch_gemm_tc_resid(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, int ldc, int M,
+                                 int N, int K, const bf16 *R, int ldr, int *status, cudaStream_t st);
+// first half of a gated FFN: C[M x N/2] = silu(A Wg) * (A Wu); Bt [N x K] interleaves, per block of
+// 128 outputs, 128 rows of Wg^T and 128 rows of Wu^T
+bool gemm_tc_gated_supported(int M, int N, int K, int lda, int ldb);
+cudaError_t launch_gemm_tc_gated(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, int ldc, int M,
+                                 int N, int K, int *status, cudaStream_t st);
 cudaError_t launch_gemm_tc(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, int ldc, int M,
                            int N, int K, int *status, cudaStream_t st);
 cudaError_t launch_rh_gemm_tc(const bf16 *A, int lda, const bf16 *W1t, const float *W2, float *partial,

@@ -91,7 +91,8 @@ template <int BN, int MODE, int HD = 0>
 __global__ void __launch_bounds__(GT_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                bf16 *__restrict__ C, int ldc, int M, int N, int K, const float *__restrict__ W2,
-               float *__restrict__ partial, int h_kv, int act, const RopeAppendArgs ra, int *status) {
+               float *__restrict__ partial, int h_kv, int act, const RopeAppendArgs ra,
+               const bf16 *__restrict__ resid, int ldr, int *status) {
   // Persistent: CTA b computes tiles b, b + gridDim.x, ... (row-block major, so that concurrent
   // CTAs share the A row block in L2).  The accumulator is double-buffered in TMEM: the epilogue
   // of one tile overlaps the main loop of the next.
@@ -221,13 +222,51 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             tmem_wait_ld();
             if (row < M && n0 + c0 < N) {
               uint4 *dst = reinterpret_cast<uint4 *>(C + (size_t)row * ldc + n0 + c0);
+              const uint4 *rs = resid ? reinterpret_cast<const uint4 *>(resid + (size_t)row * ldr + n0 + c0) : nullptr;
 #pragma unroll
               for (int v = 0; v < 4; v++) {
+                float f[8];
+#pragma unroll
+                for (int e = 0; e < 8; e++) f[e] = __uint_as_float(r[8 * v + e]);
+                if (rs) {  // C = A B^T + R (a residual connection), rounded once
+                  const uint4 rv = rs[v];
+                  const uint32_t w[4] = {rv.x, rv.y, rv.z, rv.w};
+#pragma unroll
+                  for (int e = 0; e < 4; e++) {
+                    f[2 * e] += __uint_as_float(w[e] << 16);
+                    f[2 * e + 1] += __uint_as_float(w[e] & 0xffff0000u);
+                  }
+                }
                 uint4 o;
-                o.x = pack_bf16(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1]));
-                o.y = pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
-                o.z = pack_bf16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]));
-                o.w = pack_bf16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]));
+                o.x = pack_bf16(f[0], f[1]); o.y = pack_bf16(f[2], f[3]);
+                o.z = pack_bf16(f[4], f[5]); o.w = pack_bf16(f[6], f[7]);
+                dst[v] = o;
+              }
+            }
+          }
+        }
+      } else if (MODE == 3) {
+        // Gated FFN: a 256-column tile holds 128 gate columns followed by the 128 up columns
+        // of the same outputs (the weight rows are laid out that way when the block is
+        // created); the epilogue stores silu(gate) * up, 128 outputs per tile.
+        if (ok) {
+#pragma unroll 1
+          for (int c0 = 0; c0 < BN / 2; c0 += 32) {
+            uint32_t gt[32], up[32];
+            tmem_ld32(taddr + c0, gt);
+            tmem_ld32(taddr + BN / 2 + c0, up);
+            tmem_wait_ld();
+            if (row < M && n0 + c0 < N) {
+              uint4 *dst = reinterpret_cast<uint4 *>(C + (size_t)row * ldc + n0 / 2 + c0);
+#pragma unroll
+              for (int v = 0; v < 4; v++) {
+                float f[8];
+#pragma unroll
+                for (int e = 0; e < 8; e++)
+                  f[e] = fast_act(__uint_as_float(gt[8 * v + e]), 0) * __uint_as_float(up[8 * v + e]);
+                uint4 o;
+                o.x = pack_bf16(f[0], f[1]); o.y = pack_bf16(f[2], f[3]);
+                o.z = pack_bf16(f[4], f[5]); o.w = pack_bf16(f[6], f[7]);
                 dst[v] = o;
               }
             }
@@ -431,7 +470,7 @@ const CUtensorMap *cached_map(const void *base, uint64_t inner, uint64_t outer, 
 template <int BN, int MODE, int HD = 0>
 cudaError_t launch_t(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, int ldc, int M, int N,
                      int K, const float *W2, float *partial, int h_kv, int act, const RopeAppendArgs &ra,
-                     int *status, cudaStream_t st) {
+                     int *status, cudaStream_t st, const bf16 *resid = nullptr, int ldr = 0) {
   using Cfg = GemmCfg<BN>;
   static bool attr_set = false;
   if (!attr_set) {
@@ -456,7 +495,7 @@ cudaError_t launch_t(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, i
   const int total = ((N + BN - 1) / BN) * ((M + BM - 1) / BM);
   const int grid = total < num_sms ? total : num_sms;
   gemm_tc_kernel<BN, MODE, HD><<<grid, GT_THREADS, Cfg::smem_bytes(MODE), st>>>(
-      *ma, *mb, C, ldc, M, N, K, W2, partial, h_kv, act, ra, status);
+      *ma, *mb, C, ldc, M, N, K, W2, partial, h_kv, act, ra, resid, ldr, status);
   return cudaGetLastError();
 }
 
@@ -471,6 +510,26 @@ cudaError_t launch_gemm_tc(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16
   if (N >= 256)
     return launch_t<256, 0>(A, lda, Bt, ldb, C, ldc, M, N, K, nullptr, nullptr, 0, 0, RopeAppendArgs{}, status, st);
   return launch_t<128, 0>(A, lda, Bt, ldb, C, ldc, M, N, K, nullptr, nullptr, 0, 0, RopeAppendArgs{}, status, st);
+}
+
+// C = A Bt^T + R: a projection with its residual connection (R [M x N] bf16, leading dimension ldr)
+cudaError_t launch_gemm_tc_resid(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, int ldc, int M,
+                                 int N, int K, const bf16 *R, int ldr, int *status, cudaStream_t st) {
+  if (N >= 256)
+    return launch_t<256, 0>(A, lda, Bt, ldb, C, ldc, M, N, K, nullptr, nullptr, 0, 0, RopeAppendArgs{}, status,
+                            st, R, ldr);
+  return launch_t<128, 0>(A, lda, Bt, ldb, C, ldc, M, N, K, nullptr, nullptr, 0, 0, RopeAppendArgs{}, status, st,
+                          R, ldr);
+}
+
+// Gated FFN first half: C[M x N/2] = silu(A Wg) * (A Wu), where Bt [N x K] holds, for every block
+// of 128 outputs, the 128 rows of Wg^T followed by the 128 rows of Wu^T (N = 2 d_ff, d_ff % 128 == 0)
+bool gemm_tc_gated_supported(int M, int N, int K, int lda, int ldb) {
+  return gemm_tc_supported(M, N, K, lda, ldb) && N % 256 == 0;
+}
+cudaError_t launch_gemm_tc_gated(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, int ldc, int M,
+                                 int N, int K, int *status, cudaStream_t st) {
+  return launch_t<256, 3>(A, lda, Bt, ldb, C, ldc, M, N, K, nullptr, nullptr, 0, 0, RopeAppendArgs{}, status, st);
 }
 
 // QKV projection whose epilogue also assigns positions, rotates Q and K and appends K, V to the
