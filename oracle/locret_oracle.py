@@ -396,7 +396,11 @@ class OracleBlock:
         h1 = self._r(rmsnorm(X, self.g1))
         self.last_h1 = h1
         att = self.attn.prefill_chunk(h1, flags, rows=rows)        # NaN rows where not computed
-        att = self._r(att)
-        x1 = self._r(X + att @ self.w_o)
+        # everything after attention is row-wise: with `rows` only those rows are computed
+        sel = np.arange(X.shape[0]) if rows is None else np.asarray(rows, dtype=np.int64)
+        a = self._r(att[sel])
+        x1 = self._r(X[sel] + a @ self.w_o)
         h2 = self._r(rmsnorm(x1, self.g2))
-        return self._r(x1 + gated_ffn(h2, self.w_gate, self.w_up, self.w_down, rnd=self._r))
+        y = np.full((X.shape[0], X.shape[1]), np.nan)
+        y[sel] = self._r(x1 + gated_ffn(h2, self.w_gate, self.w_up, self.w_down, rnd=self._r))
+        return y

@@ -83,3 +83,30 @@ def test_block_in_place_and_argument_checks():
     with pytest.raises(LocretError):
         gpu.prefill_chunk(xd, xd, 0, n_tok=65)
     gpu.destroy()
+
+
+def test_block_at_the_llama_shape_sampled_rows():
+    """Full benchmark shape (d_model 4096, 32/8 heads of 128, d_ff 14336), chunks of 3072 in the
+    launch configuration bench.py times; rows sampled (everything after attention is row-wise, the
+    oracle computes the sampled rows only)."""
+    from parity_util import bf16_dev, import_oracle_state
+    w = W.get_workload("c3_llama_128k")
+    ora, gpu = block_pair(w.shape, 0, w.budget, w.chunk, w.n_stab)
+    start = 0
+    for i, n_tok in enumerate(w.chunk_sizes()[:3]):          # the third chunk evicts at full cache
+        x = W.hidden_states(w, start, n_tok)
+        g = np.random.default_rng(700 + i)
+        rows = sorted(set(g.integers(0, n_tok, size=5).tolist()) | {0, 127, 128, n_tok - 1})
+        st = ora.attn.export_state()
+        import_oracle_state(gpu.attn, st, False)
+        xd = bf16_dev(x)
+        y = torch.zeros_like(xd)
+        gpu.prefill_chunk(xd, y, 0)
+        assert gpu.attn.sync_status() == 0
+        ref = ora.prefill_chunk(x, 0, rows=rows)
+        got = y.float().cpu().numpy().astype(np.float64)
+        ok = ~np.isnan(ref)
+        err = np.abs(got[ok] - ref[ok]) / np.maximum(1.0, np.abs(ref[ok]))
+        assert err.max() <= BLOCK_TOL, f"chunk {i}: worst err/bound {err.max() / BLOCK_TOL:.3f}"
+        start += n_tok
+    gpu.destroy()
