@@ -16,6 +16,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import subprocess
 import sys
@@ -403,8 +404,97 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+# ----------------------------------------------------------------------------- whole decoder layers
+
+def run_whole_model(args, w):
+    """Extra (not the headline metric): the same chunked prefill through whole decoder layers
+    (locret_block_*: RMSNorm, attention block with eviction, W_o, gated FFN), hidden states chained
+    from layer to layer.  Weights are drawn on the device (seeded torch generator, N(0, 1/fan_in)):
+    the host generator would need minutes for 32 layers of FFN weights."""
+    import torch
+    from paper_2410_01805_b200 import LocretBlock
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    s = w.shape
+    if s.d_ff <= 0:
+        raise SystemExit("this workload's shape has no d_ff")
+    sizes = w.chunk_sizes()
+    t0 = time.perf_counter()
+    x_dev = torch.empty((w.context, s.d_model), dtype=torch.bfloat16, device=dev)
+    pos = 0
+    for n_tok in sizes:
+        x_dev[pos:pos + n_tok] = torch.from_numpy(W.hidden_states(w, pos, n_tok)).to(torch.bfloat16).to(dev)
+        pos += n_tok
+    g = torch.Generator(device=dev)
+    g.manual_seed(W.BASE_SEED)
+    hd = s.n_q_heads * s.head_dim
+
+    def draw(rows, cols):
+        return (torch.randn((rows, cols), generator=g, device=dev, dtype=torch.float32) / math.sqrt(rows)).to(torch.bfloat16)
+
+    blocks = []
+    stream = torch.cuda.current_stream()
+    for l in range(w.n_layers):
+        gains = [(1.0 + 0.1 * torch.randn(s.d_model, generator=g, device=dev)).to(torch.bfloat16) for _ in range(2)]
+        ws = [draw(s.d_model, s.d_in), draw(s.d_in, s.d_retain), draw(s.d_retain, s.n_kv_heads),
+              draw(hd, s.d_model), draw(s.d_model, s.d_ff), draw(s.d_model, s.d_ff), draw(s.d_ff, s.d_model)]
+        blocks.append((LocretBlock(s, *ws, gains[0], gains[1], w.budget, w.chunk, w.n_stab, stream=stream), ws[:3]))
+        del ws[3:], gains
+    setup_s = time.perf_counter() - t0
+    bufs = [torch.empty((w.chunk, s.d_model), dtype=torch.bfloat16, device=dev) for _ in range(2)]
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+
+    def run():
+        for b, _ in blocks:
+            b.attn.reset()
+        p = 0
+        for n_tok in sizes:
+            src = x_dev[p:p + n_tok]
+            for i, (b, _) in enumerate(blocks):
+                dst = bufs[i & 1]
+                b.prefill_chunk(src, dst, 0, n_tok)
+                src = dst
+            p += n_tok
+
+    for _ in range(args.warmup):
+        run()
+    torch.cuda.synchronize()
+    times = []
+    with ClockSampler(local) as clk:
+        for _ in range(args.steps):
+            flush.fill_(1)
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); run(); b_.record(stream)
+            torch.cuda.synchronize()
+            times.append(a.elapsed_time(b_))
+    status = max(b.attn.sync_status() for b, _ in blocks)
+    t_ms = float(np.mean(times))
+    fl = float(step_flops(w).sum())
+    extra = w.n_layers * w.context * (2.0 * hd * s.d_model + 6.0 * s.d_model * s.d_ff)
+    finite = bool(torch.isfinite(bufs[(len(blocks) - 1) & 1][: sizes[-1]].float()).all().item())
+    line = {
+        "metric": "whole-decoder-layer chunked-prefill tokens/sec (extra; the headline metric is the attention block alone)",
+        "value": w.context / (t_ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": t_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic (hidden states from the seeded host generator, weights drawn on the device)",
+        "config": {"workload": w.name + " + W_o, RMSNorm, gated FFN (d_ff %d), hidden states chained" % s.d_ff,
+                   "layers": w.n_layers, "context": w.context, "chunk": w.chunk, "budget": w.budget,
+                   "l2": "flushed between timed iterations (256 MB write)"},
+        "tflops_step": (fl + extra) / (t_ms * 1e-3) / 1e12, "flops_attention_block": fl, "flops_rest_of_layer": extra,
+        "device_status": status, "outputs_finite": finite, "clocks": clk.summary(), "setup_s": setup_s,
+    }
+    if rank == 0:
+        print(json.dumps(line))
+    for b, _ in blocks:
+        b.destroy()
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--whole-model", action="store_true",
+                    help="extra run: whole decoder layers (attention block + W_o + gated FFN), hidden states chained")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
@@ -427,7 +517,10 @@ def main():
     else:
         import __graft_entry__ as G
         G.build()
-        run_ours(args, w)
+        if args.whole_model:
+            run_whole_model(args, w)
+        else:
+            run_ours(args, w)
 
 
 if __name__ == "__main__":
