@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(GT_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                bf16 *__restrict__ C, int ldc, int M, int N, int K, const float *__restrict__ W2,
                float *__restrict__ partial, int h_kv, int act, const RopeAppendArgs ra,
-               const bf16 *__restrict__ resid, int ldr, int *status) {
+               const bf16 *__restrict__ resid, int ldr, int n_major, int *status) {
   // Persistent: CTA b computes tiles b, b + gridDim.x, ... (row-block major, so that concurrent
   // CTAs share the A row block in L2).  The accumulator is double-buffered in TMEM: the epilogue
   // of one tile overlaps the main loop of the next.
@@ -116,7 +116,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int KB = K / BK;
   const int tiles_n = (N + BN - 1) / BN;
-  const int total = ((M + BM - 1) / BM) * tiles_n;
+  const int tiles_m = (M + BM - 1) / BM;
+  const int total = tiles_m * tiles_n;
+  // tile order: row-block major (concurrent CTAs share the A row block in L2), or, when B is the
+  // large operand and does not fit the L2, column-block major (they share the B tile and sweep M)
+  auto tile_mn = [&](int tile, int &m0, int &n0) {
+    if (n_major) { m0 = (tile % tiles_m) * BM; n0 = (tile / tiles_m) * BN; }
+    else { m0 = (tile / tiles_n) * BM; n0 = (tile % tiles_n) * BN; }
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; s++) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -140,7 +147,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       uint32_t it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
-        const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+        int m0, n0;
+        tile_mn(tile, m0, n0);
         for (int kb = 0; kb < KB; kb++, it++) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
@@ -190,7 +198,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     bool ok = true;
     // (no early exit: after a timed-out wait the warps still meet at the named barrier)
     for (int tile = blockIdx.x; tile < total; tile += gridDim.x, lt++) {
-      const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+      int m0, n0;
+      tile_mn(tile, m0, n0);
       const uint32_t buf = lt & 1;
       const int row = m0 + quarter * 32 + lane;
       if (MODE == 1) {
@@ -415,7 +424,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
           }
           if (row < M) {
-            float *dst = partial + ((size_t)(tile % tiles_n) * M + row) * h_kv;
+            float *dst = partial + ((size_t)(n0 / BN) * M + row) * h_kv;
 #pragma unroll
             for (int m = 0; m < MAX_HKV; m++)
               if (m < h_kv) dst[m] = sc[m];
@@ -494,8 +503,11 @@ cudaError_t launch_t(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, i
   }
   const int total = ((N + BN - 1) / BN) * ((M + BM - 1) / BM);
   const int grid = total < num_sms ? total : num_sms;
+  // B much larger than A and larger than half the L2: keep a B tile resident and sweep the rows
+  const size_t a_bytes = (size_t)M * K * 2, b_bytes = (size_t)N * K * 2;
+  const int n_major = (MODE == 0 || MODE == 3) && b_bytes > 2 * a_bytes && b_bytes > ((size_t)64 << 20);
   gemm_tc_kernel<BN, MODE, HD><<<grid, GT_THREADS, Cfg::smem_bytes(MODE), st>>>(
-      *ma, *mb, C, ldc, M, N, K, W2, partial, h_kv, act, ra, resid, ldr, status);
+      *ma, *mb, C, ldc, M, N, K, W2, partial, h_kv, act, ra, resid, ldr, n_major, status);
   return cudaGetLastError();
 }
 
