@@ -503,9 +503,11 @@ cudaError_t launch_t(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, i
   }
   const int total = ((N + BN - 1) / BN) * ((M + BM - 1) / BM);
   const int grid = total < num_sms ? total : num_sms;
-  // B much larger than A and larger than half the L2: keep a B tile resident and sweep the rows
+  // B is the larger operand: keep a B tile resident and sweep the rows (each B tile is then read
+  // from HBM once; in row-block-major order a B that exceeds the L2 is re-read for every row
+  // block, and even one that fits is read about three times)
   const size_t a_bytes = (size_t)M * K * 2, b_bytes = (size_t)N * K * 2;
-  const int n_major = (MODE == 0 || MODE == 3) && b_bytes > 2 * a_bytes && b_bytes > ((size_t)64 << 20);
+  const int n_major = MODE != 1 && b_bytes > a_bytes;
   gemm_tc_kernel<BN, MODE, HD><<<grid, GT_THREADS, Cfg::smem_bytes(MODE), st>>>(
       *ma, *mb, C, ldc, M, N, K, W2, partial, h_kv, act, ra, resid, ldr, n_major, status);
   return cudaGetLastError();
