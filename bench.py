@@ -469,6 +469,26 @@ def run_whole_model(args, w):
             a.record(stream); run(); b_.record(stream)
             torch.cuda.synchronize()
             times.append(a.elapsed_time(b_))
+    # decoding through the whole layers: one token at a time, appended without eviction
+    n_dec = 32
+    tok = [torch.empty((1, s.d_model), dtype=torch.bfloat16, device=dev) for _ in range(2)]
+
+    def decode_all():
+        for t in range(n_dec):
+            src = x_dev[t:t + 1]
+            for i, (b, _) in enumerate(blocks):
+                b.prefill_chunk(src, tok[i & 1], 1, 1)   # flags = NO_EVICT
+                src = tok[i & 1]
+
+    torch.cuda.synchronize()
+    a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream); decode_all(); b_.record(stream)
+    torch.cuda.synchronize()
+    dec_ms = a.elapsed_time(b_) / n_dec
+    w_bytes = 2.0 * (s.d_model * s.d_in + s.d_in * s.d_retain + hd * s.d_model + 3 * s.d_model * s.d_ff)
+    kv_bytes = 2.0 * s.n_kv_heads * min(w.budget, w.context) * s.head_dim * 2
+    dec_bytes = w.n_layers * (w_bytes + kv_bytes)
+    peaks = measured_peaks()
     status = max(b.attn.sync_status() for b, _ in blocks)
     t_ms = float(np.mean(times))
     fl = float(step_flops(w).sum())
@@ -483,6 +503,9 @@ def run_whole_model(args, w):
                    "layers": w.n_layers, "context": w.context, "chunk": w.chunk, "budget": w.budget,
                    "l2": "flushed between timed iterations (256 MB write)"},
         "tflops_step": (fl + extra) / (t_ms * 1e-3) / 1e12, "flops_attention_block": fl, "flops_rest_of_layer": extra,
+        "decode": {"tokens_per_s": 1e3 / dec_ms, "ms_per_token": dec_ms, "steps": n_dec,
+                   "algorithmic_gb_per_token": dec_bytes / 1e9, "achieved_gbs": dec_bytes / (dec_ms * 1e-3) / 1e9,
+                   "frac_of_hbm_peak": dec_bytes / (dec_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
         "device_status": status, "outputs_finite": finite, "clocks": clk.summary(), "setup_s": setup_s,
     }
     if rank == 0:

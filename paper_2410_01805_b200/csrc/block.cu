@@ -238,6 +238,8 @@ int locret_block_prefill_chunk(locret_block *B, const void *x_in, int32_t n_tok,
   const bool tc = n_tok >= 32;
   if (tc && gemm_tc_supported(n_tok, D, hd, hd, hd)) {
     BCK(launch_gemm_tc_resid(P->att, hd, B->wo_t, hd, P->x1, D, n_tok, D, hd, x, D, B->d_status, B->st));
+  } else if (n_tok == 1 && hd % 8 == 0) {  // one token: bandwidth-bound GEMV
+    BCK(launch_gemv_resid(P->att, B->wo_t, D, hd, x, P->x1, B->st));
   } else {
     gemm_resid_naive_kernel<<<dim3((D + 127) / 128, n_tok), 128, 0, B->st>>>(P->att, B->wo_t, x, P->x1, n_tok, D, hd);
     BCK(cudaGetLastError());
@@ -248,6 +250,8 @@ int locret_block_prefill_chunk(locret_block *B, const void *x_in, int32_t n_tok,
   // act = silu(h2 W_gate) * (h2 W_up)
   if (tc && gemm_tc_gated_supported(n_tok, 2 * F, D, D, D)) {
     BCK(launch_gemm_tc_gated(P->h, D, B->wgu_t, D, P->act, F, n_tok, 2 * F, D, B->d_status, B->st));
+  } else if (n_tok == 1) {
+    BCK(launch_gemv_gated(P->h, B->wgu_t, F, D, P->act, B->st));
   } else {
     {
       std::lock_guard<std::mutex> lk(b_mu);
@@ -262,6 +266,8 @@ int locret_block_prefill_chunk(locret_block *B, const void *x_in, int32_t n_tok,
   // y = x1 + act W_down
   if (tc && gemm_tc_supported(n_tok, D, F, F, F)) {
     BCK(launch_gemm_tc_resid(P->act, F, B->wd_t, F, y, D, n_tok, D, F, P->x1, D, B->d_status, B->st));
+  } else if (n_tok == 1) {
+    BCK(launch_gemv_resid(P->act, B->wd_t, D, F, P->x1, y, B->st));
   } else {
     gemm_resid_naive_kernel<<<dim3((D + 127) / 128, n_tok), 128, 0, B->st>>>(P->act, B->wd_t, P->x1, y, n_tok, D, F);
     BCK(cudaGetLastError());

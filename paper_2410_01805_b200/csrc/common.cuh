@@ -167,6 +167,12 @@ cudaError_t launch_compact_int4(const Int4Half &src, const Int4Half &dst, const 
 
 // ---- decoding (decode.cu): one token
 cudaError_t launch_gemv(const bf16 *x, const bf16 *Wt, int N, int K, bf16 *y, cudaStream_t st);
+// y = x Wt^T + r (one token; the residual is added before the one rounding)
+cudaError_t launch_gemv_resid(const bf16 *x, const bf16 *Wt, int N, int K, const bf16 *r, bf16 *y,
+                              cudaStream_t st);
+// act[c] = silu(x . Wg[:, c]) * (x . Wu[:, c]) for one token; Wt [2F x K] in the interleaved
+// layout of launch_gemm_tc_gated
+cudaError_t launch_gemv_gated(const bf16 *x, const bf16 *Wt, int F, int K, bf16 *act, cudaStream_t st);
 // projection + positions + RoPE + cache append of one token (a.staging is not used: `staging` is written)
 cudaError_t launch_gemv_rope(const bf16 *x, const bf16 *Wt, int K, bf16 *staging, const RopeAppendArgs &a,
                              cudaStream_t st);

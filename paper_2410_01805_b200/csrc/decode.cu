@@ -41,7 +41,8 @@ template <int MODE>
 __global__ void __launch_bounds__(GV_THREADS)
 gemv_kernel(const bf16 *__restrict__ x, const bf16 *__restrict__ Wt, int N, int K, bf16 *__restrict__ y,
             const float *__restrict__ W2, float *__restrict__ partial, int h_kv, int act,
-            unsigned *__restrict__ counter, float *__restrict__ score_out, int score_stride) {
+            unsigned *__restrict__ counter, float *__restrict__ score_out, int score_stride,
+            const bf16 *__restrict__ resid) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint4 *sx = reinterpret_cast<uint4 *>(smem_raw);  // K / 8 vectors
   float *swarp = reinterpret_cast<float *>(sx + K / 8);  // [8 warps][32]
@@ -57,7 +58,7 @@ gemv_kernel(const bf16 *__restrict__ x, const bf16 *__restrict__ Wt, int N, int 
 #pragma unroll 8
       for (int v = lane; v < K / 8; v += 32) s += dot8(__ldg(row + v), sx[v]);
       s = warp_sum(s);
-      if (lane == 0) y[n] = __float2bfloat16_rn(s);
+      if (lane == 0) y[n] = __float2bfloat16_rn(resid ? s + __bfloat162float(resid[n]) : s);
     }
   } else {
     // two warps per row (halves of K), four rows per block at a time: d_R rows are too few to
@@ -479,7 +480,52 @@ cudaError_t launch_gemv(const bf16 *x, const bf16 *Wt, int N, int K, bf16 *y, cu
   if (K % 8) return cudaErrorInvalidValue;
   const int smem = K * 2 + 8 * 32 * 4;
   const int blocks = min((N + 7) / 8, 148 * 4);
-  gemv_kernel<0><<<blocks, GV_THREADS, smem, st>>>(x, Wt, N, K, y, nullptr, nullptr, 0, 0, nullptr, nullptr, 0);
+  gemv_kernel<0><<<blocks, GV_THREADS, smem, st>>>(x, Wt, N, K, y, nullptr, nullptr, 0, 0, nullptr, nullptr, 0,
+                                                   nullptr);
+  return cudaGetLastError();
+}
+
+// y[n] = x . Wt[n] + r[n]: a projection of one token with its residual connection
+cudaError_t launch_gemv_resid(const bf16 *x, const bf16 *Wt, int N, int K, const bf16 *r, bf16 *y,
+                              cudaStream_t st) {
+  if (K % 8) return cudaErrorInvalidValue;
+  const int smem = K * 2 + 8 * 32 * 4;
+  const int blocks = min((N + 7) / 8, 148 * 4);
+  gemv_kernel<0><<<blocks, GV_THREADS, smem, st>>>(x, Wt, N, K, y, nullptr, nullptr, 0, 0, nullptr, nullptr, 0, r);
+  return cudaGetLastError();
+}
+
+// Gated FFN, first half, for one token: Wt [2F x K] holds, per block of 128 outputs, the 128
+// rows of W_gate^T followed by the 128 rows of W_up^T; a warp computes one gate row and the
+// matching up row and stores silu(gate) * up.
+__global__ void __launch_bounds__(GV_THREADS)
+gemv_gated_kernel(const bf16 *__restrict__ x, const bf16 *__restrict__ Wt, int F, int K, bf16 *__restrict__ act) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  uint4 *sx = reinterpret_cast<uint4 *>(smem_raw);
+  for (int i = threadIdx.x; i < K / 8; i += GV_THREADS) sx[i] = reinterpret_cast<const uint4 *>(x)[i];
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gw = blockIdx.x * (GV_THREADS / 32) + warp, nw = gridDim.x * (GV_THREADS / 32);
+  for (int c = gw; c < F; c += nw) {
+    const size_t row = (size_t)(c / 128) * 256 + (c % 128);
+    const uint4 *r0 = reinterpret_cast<const uint4 *>(Wt + row * K);
+    const uint4 *r1 = reinterpret_cast<const uint4 *>(Wt + (row + 128) * K);
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll 8
+    for (int v = lane; v < K / 8; v += 32) {
+      const uint4 xv = sx[v];
+      s0 += dot8(__ldg(r0 + v), xv);
+      s1 += dot8(__ldg(r1 + v), xv);
+    }
+    s0 = warp_sum(s0);
+    s1 = warp_sum(s1);
+    if (lane == 0) act[c] = __float2bfloat16_rn(s0 / (1.0f + __expf(-s0)) * s1);
+  }
+}
+cudaError_t launch_gemv_gated(const bf16 *x, const bf16 *Wt, int F, int K, bf16 *act, cudaStream_t st) {
+  if (K % 8) return cudaErrorInvalidValue;
+  const int blocks = min((F + 7) / 8, 148 * 8);
+  gemv_gated_kernel<<<blocks, GV_THREADS, K * 2, st>>>(x, Wt, F, K, act);
   return cudaGetLastError();
 }
 
@@ -503,7 +549,7 @@ cudaError_t launch_rh_gemv(const bf16 *z, const bf16 *W1t, const float *W2, floa
   const int smem = K * 2 + 8 * 32 * 4;
   const int blocks = rh_gemv_blocks(d_R);
   gemv_kernel<1><<<blocks, GV_THREADS, smem, st>>>(z, W1t, d_R, K, nullptr, W2, partial, h_kv, act, counter,
-                                                  score_out, score_stride);
+                                                  score_out, score_stride, nullptr);
   return cudaGetLastError();
 }
 
