@@ -404,3 +404,28 @@ class OracleBlock:
         y = np.full((X.shape[0], X.shape[1]), np.nan)
         y[sel] = self._r(x1 + gated_ffn(h2, self.w_gate, self.w_up, self.w_down, rnd=self._r))
         return y
+
+
+# --------------------------------------------------------------------------- training labels
+#
+# Section 3.3: the ground truth for the retaining head of a layer is, for prompt token k and
+# head j, the largest attention score before the softmax that any answer token gives to k:
+#     S[k]_j = max_p (Q_j K_j^T)[p, k],   n_q < p <= n_q + n_a,
+# and for grouped-query attention the maximum is also taken over the query heads that share
+# the KV head.  The passage prints the product without the 1/sqrt(d) factor of Eq. 1; `scale`
+# is left to the caller (1 = as printed).
+
+def cis_labels(q_ans, k_prompt, n_kv_heads: int, scale: float = 1.0):
+    """q_ans [n_a, h, d] (queries of the answer tokens, as they enter the attention scores),
+    k_prompt [n_q, h_kv, d] (keys of the prompt tokens) -> labels [h_kv, n_q]."""
+    q = np.asarray(q_ans, np.float64)
+    k = np.asarray(k_prompt, np.float64)
+    n_a, h, d = q.shape
+    n_q = k.shape[0]
+    g = h // n_kv_heads
+    out = np.full((n_kv_heads, n_q), -np.inf)
+    for m in range(n_kv_heads):
+        for j in range(m * g, (m + 1) * g):
+            s = (q[:, j, :] @ k[:, m, :].T) * scale          # [n_a, n_q]
+            out[m] = np.maximum(out[m], s.max(axis=0))
+    return out

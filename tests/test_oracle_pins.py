@@ -535,3 +535,37 @@ def test_decoder_block_equals_library_composition_when_nothing_is_evicted():
     want = (x1 + (F_.silu(h2 @ t(wg)) * (h2 @ t(wu))) @ t(wd)).numpy()
     for got in outs:
         assert np.allclose(got, want, rtol=0, atol=1e-10)
+
+
+# ------------------------------------------------------------------ training labels (Section 3.3)
+
+def test_cis_labels_equal_the_definition_by_brute_force():
+    g = np.random.default_rng(400)
+    for n_a, n_q, h, hk, d in [(1, 5, 2, 2, 4), (3, 7, 4, 2, 6), (5, 4, 6, 1, 3), (4, 9, 3, 3, 8)]:
+        q = g.standard_normal((n_a, h, d))
+        k = g.standard_normal((n_q, hk, d))
+        grp = h // hk
+        want = np.full((hk, n_q), -np.inf)
+        for kk in range(n_q):
+            for j in range(h):
+                for p in range(n_a):
+                    want[j // grp, kk] = max(want[j // grp, kk], float(np.dot(q[p, j], k[kk, j // grp])))
+        assert np.allclose(O.cis_labels(q, k, hk), want, rtol=0, atol=1e-12)
+        assert np.allclose(O.cis_labels(q, k, hk, scale=0.25), 0.25 * want, atol=1e-12)
+
+
+def test_cis_labels_special_cases_and_invariants():
+    g = np.random.default_rng(401)
+    q = g.standard_normal((6, 4, 8))
+    k = g.standard_normal((11, 2, 8))
+    full = O.cis_labels(q, k, 2)
+    # one answer token, no grouping: a row of the library's Q K^T
+    assert np.allclose(O.cis_labels(q[:1, :1], k[:, :1], 1)[0],
+                       (torch.from_numpy(q[0, 0]) @ torch.from_numpy(k[:, 0]).T).numpy())
+    # more answer tokens can only raise a label; order of answer tokens and of heads in a group is irrelevant
+    assert (O.cis_labels(q[:3], k, 2) <= full + 1e-15).all()
+    perm = g.permutation(6)
+    assert np.allclose(O.cis_labels(q[perm], k, 2), full)
+    assert np.allclose(O.cis_labels(q[:, [1, 0, 3, 2]], k, 2), full)
+    # an MHA model (h_kv = h) has no maximum over heads
+    assert not np.allclose(O.cis_labels(q, np.repeat(k, 2, axis=1), 4)[0], full[0])
