@@ -514,8 +514,35 @@ def run_whole_model(args, w):
         b.destroy()
 
 
+def run_cis(args, w):
+    """Extra: the training labels of Section 3.3 (locret_cis_labels) at the workload's layer shape,
+    131072 prompt tokens and 1024 answer tokens, one layer."""
+    import torch
+    from paper_2410_01805_b200 import cis_labels
+    torch.cuda.set_device(0)
+    s = w.shape
+    n_q, n_a = w.context, 1024
+    g = torch.Generator(device="cuda"); g.manual_seed(W.BASE_SEED)
+    q = torch.randn((n_a, s.n_q_heads, s.head_dim), generator=g, device="cuda").to(torch.bfloat16)
+    k = torch.randn((n_q, s.n_kv_heads, s.head_dim), generator=g, device="cuda").to(torch.bfloat16)
+    for _ in range(args.warmup):
+        cis_labels(q, k)
+    ts = []
+    for _ in range(args.steps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); out = cis_labels(q, k); b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b))
+    ms = float(np.mean(ts))
+    flops = 2.0 * n_q * n_a * s.n_q_heads * s.head_dim
+    print(json.dumps({"metric": "training labels (Section 3.3), one layer", "ms": ms, "tflops": flops / (ms * 1e-3) / 1e12,
+                      "config": {"n_prompt": n_q, "n_answer": n_a, "heads": f"{s.n_q_heads}q/{s.n_kv_heads}kv x {s.head_dim}"},
+                      "finite": bool(torch.isfinite(out).all().item())}))
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--cis", action="store_true", help="extra run: the training labels of Section 3.3")
     ap.add_argument("--whole-model", action="store_true",
                     help="extra run: whole decoder layers (attention block + W_o + gated FFN), hidden states chained")
     ap.add_argument("--gpus", type=int, default=1)
@@ -540,7 +567,9 @@ def main():
     else:
         import __graft_entry__ as G
         G.build()
-        if args.whole_model:
+        if args.cis:
+            run_cis(args, w)
+        elif args.whole_model:
             run_whole_model(args, w)
         else:
             run_ours(args, w)

@@ -249,6 +249,21 @@ locret_layer *locret_block_attention(locret_block *block);
 void locret_block_destroy(locret_block *block);
 
 /*
+ * Training labels of the retaining heads (Section 3.3): for prompt token k and KV head m the
+ * causal importance score is the largest attention score before the softmax that any answer
+ * token gives to k, over the query heads of the group:
+ *     labels[m][k] = scale * max over p < n_a, j in group m of  q_ans[p][j] . k_prompt[k][m].
+ * q_ans: device bf16 [n_a × h × d] (queries of the answer tokens as they enter the scores, i.e.
+ * after RoPE); k_prompt: device bf16 [n_q × h_kv × d]; labels: device fp32 [h_kv × n_q]
+ * (overwritten).  The passage prints the product without the 1/sqrt(d) of Eq. 1: scale = 1
+ * reproduces it as printed; scale must be > 0.  head_dim 64 or 128; pointers 16-byte aligned.
+ * One tensor-core contraction per query head whose epilogue keeps only row maxima (the
+ * n_q × n_a score matrix is never written).  Synchronises the stream before it returns.
+ */
+int locret_cis_labels(const void *q_ans, const void *k_prompt, int32_t n_a, int32_t n_q, int32_t h,
+                      int32_t h_kv, int32_t d, float scale, float *labels, void *stream);
+
+/*
  * Retaining-head scores without any allocation.  (The paper has no counterpart: this entry
  * point exists for hosts that may not allocate device memory where they need scores, e.g. code
  * that runs inside a pool owning the whole device, or under an allocator that is locked while

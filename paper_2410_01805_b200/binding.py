@@ -73,6 +73,7 @@ def _load():
     l.locret_block_attention.restype = P
     l.locret_block_destroy.argtypes = [P]
     l.locret_block_destroy.restype = None
+    l.locret_cis_labels.argtypes = [P, P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float, P, P]
     return l
 
 
@@ -269,3 +270,14 @@ class LocretBlock:
             self.destroy()
         except Exception:
             pass
+
+
+def cis_labels(q_ans: torch.Tensor, k_prompt: torch.Tensor, scale: float = 1.0) -> torch.Tensor:
+    """Training labels (Section 3.3): q_ans [n_a, h, d], k_prompt [n_q, h_kv, d] (CUDA bf16,
+    contiguous) -> fp32 [h_kv, n_q]."""
+    n_a, h, d = q_ans.shape
+    n_q, h_kv, _ = k_prompt.shape
+    out = torch.empty((h_kv, n_q), dtype=torch.float32, device=q_ans.device)
+    _check(lib.locret_cis_labels(q_ans.data_ptr(), k_prompt.data_ptr(), n_a, n_q, h, h_kv, d, float(scale),
+                                 out.data_ptr(), torch.cuda.current_stream().cuda_stream), "locret_cis_labels")
+    return out

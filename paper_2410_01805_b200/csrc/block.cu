@@ -276,3 +276,38 @@ int locret_block_prefill_chunk(locret_block *B, const void *x_in, int32_t n_tok,
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------- training labels (Section 3.3)
+namespace {
+__global__ void fill_f32_kernel(float *p, size_t n, float v) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) p[i] = v;
+}
+__device__ int g_cis_status;
+}  // namespace
+
+extern "C" int locret_cis_labels(const void *q_ans, const void *k_prompt, int32_t n_a, int32_t n_q, int32_t h,
+                                 int32_t h_kv, int32_t d, float scale, float *labels, void *stream) {
+  if (!q_ans || !k_prompt || !labels) return LOCRET_ERR_INVALID;
+  if (n_a < 1 || n_q < 1 || h < 1 || h_kv < 1 || h % h_kv || (d != 64 && d != 128) || !(scale > 0.f))
+    return LOCRET_ERR_INVALID;
+  if ((reinterpret_cast<uintptr_t>(q_ans) | reinterpret_cast<uintptr_t>(k_prompt)) & 15u) return LOCRET_ERR_INVALID;
+  cudaStream_t st = (cudaStream_t)stream;
+  int *d_status = nullptr;
+  BCK(cudaGetSymbolAddress((void **)&d_status, g_cis_status));
+  BCK(cudaMemsetAsync(d_status, 0, sizeof(int), st));
+  const size_t n = (size_t)h_kv * n_q;
+  fill_f32_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(labels, n, -INFINITY);
+  BCK(cudaGetLastError());
+  const bf16 *q = (const bf16 *)q_ans, *k = (const bf16 *)k_prompt;
+  const int g = h / h_kv;
+  for (int j = 0; j < h; j++) {  // one contraction per query head: keys of its KV head x its answer queries
+    const int m = j / g;
+    BCK(launch_gemm_tc_rowmax(k + (size_t)m * d, h_kv * d, q + (size_t)j * d, h * d, labels + (size_t)m * n_q, n_q,
+                              n_a, d, scale, d_status, st));
+  }
+  int status = 0;
+  BCK(cudaMemcpyAsync(&status, d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
+  BCK(cudaStreamSynchronize(st));
+  return status ? LOCRET_ERR_DEVICE_TIMEOUT : LOCRET_OK;
+}

@@ -89,6 +89,10 @@ cudaError_t launch_gemm_tc_resid(const bf16 *A, int lda, const bf16 *Bt, int ldb
                                  int N, int K, const bf16 *R, int ldr, int *status, cudaStream_t st);
 // first half of a gated FFN: C[M x N/2] = silu(A Wg) * (A Wu); Bt [N x K] interleaves, per block of
 // 128 outputs, 128 rows of Wg^T and 128 rows of Wu^T
+// out[m] = max(out[m], scale * max_n (A Bt^T)[m][n]): row maxima merged with atomics (out fp32,
+// initialised by the caller); K % 64 == 0, lda / ldb multiples of 8, scale > 0
+cudaError_t launch_gemm_tc_rowmax(const bf16 *A, int lda, const bf16 *Bt, int ldb, float *out, int M, int N,
+                                  int K, float scale, int *status, cudaStream_t st);
 bool gemm_tc_gated_supported(int M, int N, int K, int lda, int ldb);
 cudaError_t launch_gemm_tc_gated(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, int ldc, int M,
                                  int N, int K, int *status, cudaStream_t st);

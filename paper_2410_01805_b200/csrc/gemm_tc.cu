@@ -5,6 +5,7 @@
 //   MODE 0: bf16 store (the QKV projection);
 //   MODE 1: the retaining head's activation and its second, thin GEMM with W2, written as one
 //           partial score per (N-tile, row, KV head)                       (Section 3.3).
+#include <cstring>
 #include "tc_common.cuh"
 
 namespace locret {
@@ -252,6 +253,32 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 dst[v] = o;
               }
             }
+          }
+        }
+      } else if (MODE == 4) {
+        // Row maximum of A B^T over the valid columns, merged into out[row] with an atomic
+        // maximum on the order-preserving integer image of the float (`partial` is the output,
+        // `act` carries the bits of the scale factor): the labels of Section 3.3.
+        if (ok) {
+          const float scale = __int_as_float(act);
+          float mx = -INFINITY;
+#pragma unroll 1
+          for (int c0 = 0; c0 < BN; c0 += 32) {
+            uint32_t r[32];
+            tmem_ld32(taddr + c0, r);
+            tmem_wait_ld();
+            if (n0 + c0 < N) {
+#pragma unroll
+              for (int i = 0; i < 32; i++)
+                if (n0 + c0 + i < N) mx = fmaxf(mx, __uint_as_float(r[i]));
+            }
+          }
+          if (row < M && mx > -INFINITY) {
+            mx *= scale;
+            if (mx == 0.f) mx = 0.f;  // -0 would order below every negative as an integer
+            float *dst = partial + row;
+            if (mx >= 0.f) atomicMax(reinterpret_cast<int *>(dst), __float_as_int(mx));
+            else atomicMin(reinterpret_cast<unsigned int *>(dst), __float_as_uint(mx));
           }
         }
       } else if (MODE == 3) {
@@ -544,6 +571,15 @@ bool gemm_tc_gated_supported(int M, int N, int K, int lda, int ldb) {
 cudaError_t launch_gemm_tc_gated(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, int ldc, int M,
                                  int N, int K, int *status, cudaStream_t st) {
   return launch_t<256, 3>(A, lda, Bt, ldb, C, ldc, M, N, K, nullptr, nullptr, 0, 0, RopeAppendArgs{}, status, st);
+}
+
+// out[m] = max(out[m], scale * max_n (A Bt^T)[m][n]) for m < M (out fp32, initialised by the
+// caller, e.g. to -inf); scale > 0.  K % 64 == 0; any N.
+cudaError_t launch_gemm_tc_rowmax(const bf16 *A, int lda, const bf16 *Bt, int ldb, float *out, int M, int N,
+                                  int K, float scale, int *status, cudaStream_t st) {
+  int bits;
+  memcpy(&bits, &scale, sizeof(bits));
+  return launch_t<256, 4>(A, lda, Bt, ldb, nullptr, 0, M, N, K, nullptr, out, 0, bits, RopeAppendArgs{}, status, st);
 }
 
 // QKV projection whose epilogue also assigns positions, rotates Q and K and appends K, V to the
