@@ -429,3 +429,40 @@ def cis_labels(q_ans, k_prompt, n_kv_heads: int, scale: float = 1.0):
             s = (q[:, j, :] @ k[:, m, :].T) * scale          # [n_a, n_q]
             out[m] = np.maximum(out[m], s.max(axis=0))
     return out
+
+
+# --------------------------------------------------------------------------- training objective
+#
+# Eq. 3: per (token k, KV head m) Smooth-L1 between the predicted and the true score, plus
+# alpha times the squared difference of adjacent predictions; Eq. 2 sums it over heads and
+# prompt tokens.  Readings where the text is silent: Smooth-L1 with the usual threshold 1
+# (0.5 x^2 for |x| < 1, |x| - 0.5 beyond), the L2 term as the plain square (s~[k] - s~[k+1])^2
+# for k < n - 1, summed like the rest (no mean); alpha = 2.5e-3 (Section 4.1).  SiLU only.
+
+def smooth_l1(x):
+    ax = np.abs(x)
+    return np.where(ax < 1.0, 0.5 * x * x, ax - 0.5)
+
+
+def rh_loss_and_grads(z, labels, w1, w2, alpha: float = 2.5e-3):
+    """z [n, d_in] (the tokens' [Q ‖ K ‖ V]), labels [h_kv, n] -> (loss, dL/dW1 [d_in, d_R],
+    dL/dW2 [d_R, h_kv]); the backbone is frozen, only the retaining head gets gradients."""
+    z = np.asarray(z, np.float64)
+    w1 = np.asarray(w1, np.float64)
+    w2 = np.asarray(w2, np.float64)
+    tgt = np.asarray(labels, np.float64).T                 # [n, h_kv]
+    pre = z @ w1
+    sig = 1.0 / (1.0 + np.exp(-pre))
+    a = pre * sig                                          # SiLU
+    s = a @ w2                                             # [n, h_kv]
+    diff = s - tgt
+    adj = s[:-1] - s[1:]
+    loss = float(smooth_l1(diff).sum() + alpha * (adj * adj).sum())
+    ds = np.clip(diff, -1.0, 1.0)                          # derivative of Smooth-L1
+    ds[:-1] += 2.0 * alpha * adj
+    ds[1:] -= 2.0 * alpha * adj
+    dw2 = a.T @ ds
+    da = ds @ w2.T
+    dpre = da * (sig * (1.0 + pre * (1.0 - sig)))          # d SiLU / d pre
+    dw1 = z.T @ dpre
+    return loss, dw1, dw2

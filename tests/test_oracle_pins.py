@@ -569,3 +569,36 @@ def test_cis_labels_special_cases_and_invariants():
     assert np.allclose(O.cis_labels(q[:, [1, 0, 3, 2]], k, 2), full)
     # an MHA model (h_kv = h) has no maximum over heads
     assert not np.allclose(O.cis_labels(q, np.repeat(k, 2, axis=1), 4)[0], full[0])
+
+
+# ------------------------------------------------------------------ training objective (Eq. 2, Eq. 3)
+
+def test_rh_loss_and_gradients_match_library_autograd_and_finite_differences():
+    g = np.random.default_rng(500)
+    n, d_in, d_R, hk = 23, 12, 9, 3
+    z = g.standard_normal((n, d_in))
+    w1 = g.standard_normal((d_in, d_R)) / math.sqrt(d_in)
+    w2 = g.standard_normal((d_R, hk)) / math.sqrt(d_R)
+    labels = g.standard_normal((hk, n)) * 2.0              # |error| on both sides of the Smooth-L1 knee
+    alpha = 0.3
+    loss, dw1, dw2 = O.rh_loss_and_grads(z, labels, w1, w2, alpha)
+    t = torch.from_numpy
+    W1 = t(w1).clone().requires_grad_(True)
+    W2 = t(w2).clone().requires_grad_(True)
+    s = torch.nn.functional.silu(t(z) @ W1) @ W2
+    ref = torch.nn.functional.smooth_l1_loss(s, t(labels).T, reduction="sum", beta=1.0) \
+        + alpha * ((s[:-1] - s[1:]) ** 2).sum()
+    ref.backward()
+    assert abs(loss - ref.item()) < 1e-10
+    assert np.allclose(dw1, W1.grad.numpy(), atol=1e-10) and np.allclose(dw2, W2.grad.numpy(), atol=1e-10)
+    # central differences on a few entries
+    eps = 1e-6
+    for (i, j) in [(0, 0), (5, 3), (11, 8)]:
+        wp, wm = w1.copy(), w1.copy()
+        wp[i, j] += eps; wm[i, j] -= eps
+        fd = (O.rh_loss_and_grads(z, labels, wp, w2, alpha)[0] - O.rh_loss_and_grads(z, labels, wm, w2, alpha)[0]) / (2 * eps)
+        assert abs(fd - dw1[i, j]) < 1e-5
+    # alpha = 0 and predictions equal to the labels: zero loss, zero gradient
+    s0 = O.retaining_scores(z, w1, w2)
+    l0, g1, g2 = O.rh_loss_and_grads(z, s0.T, w1, w2, 0.0)
+    assert l0 == 0.0 and not g1.any() and not g2.any()
