@@ -535,9 +535,29 @@ def run_cis(args, w):
         ts.append(a.elapsed_time(b))
     ms = float(np.mean(ts))
     flops = 2.0 * n_q * n_a * s.n_q_heads * s.head_dim
+    # loss and gradients of the retaining head (Eq. 2, Eq. 3) for one sequence of the paper's training length
+    from paper_2410_01805_b200 import rh_loss_grad
+    n_tr = 10240
+    z = torch.randn((n_tr, s.d_in), generator=g, device="cuda").to(torch.bfloat16)
+    w1 = (torch.randn((s.d_in, s.d_retain), generator=g, device="cuda") / math.sqrt(s.d_in)).to(torch.bfloat16)
+    w2 = (torch.randn((s.d_retain, s.n_kv_heads), generator=g, device="cuda") / math.sqrt(s.d_retain)).to(torch.bfloat16)
+    lab = torch.randn((s.n_kv_heads, n_tr), generator=g, device="cuda")
+    for _ in range(args.warmup):
+        rh_loss_grad(z, lab, w1, w2)
+    tt = []
+    for _ in range(args.steps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); loss, g1, g2 = rh_loss_grad(z, lab, w1, w2); b.record()
+        torch.cuda.synchronize()
+        tt.append(a.elapsed_time(b))
+    ms_tr = float(np.mean(tt))
+    fl_tr = 4.0 * n_tr * s.d_in * s.d_retain
     print(json.dumps({"metric": "training labels (Section 3.3), one layer", "ms": ms, "tflops": flops / (ms * 1e-3) / 1e12,
                       "config": {"n_prompt": n_q, "n_answer": n_a, "heads": f"{s.n_q_heads}q/{s.n_kv_heads}kv x {s.head_dim}"},
-                      "finite": bool(torch.isfinite(out).all().item())}))
+                      "finite": bool(torch.isfinite(out).all().item()),
+                      "loss_and_gradients": {"ms": ms_tr, "tflops": fl_tr / (ms_tr * 1e-3) / 1e12, "n_tokens": n_tr,
+                                             "note": "Eq. 2/3 for one sequence and one layer, workspace allocated inside the call",
+                                             "finite": bool(torch.isfinite(g1).all().item() and torch.isfinite(loss).item())}}))
 
 
 def main():

@@ -264,6 +264,23 @@ int locret_cis_labels(const void *q_ans, const void *k_prompt, int32_t n_a, int3
                       int32_t h_kv, int32_t d, float scale, float *labels, void *stream);
 
 /*
+ * Training objective of the retaining head for one sequence (Eq. 2, Eq. 3), backbone frozen:
+ *     s~ = silu(z W1) W2,   L = sum_{k,m} SmoothL1(s~[k][m] - labels[m][k]) + alpha sum_{k<n-1,m} (s~[k][m] - s~[k+1][m])^2
+ * and its gradients dL/dW1, dL/dW2.  Readings where the text is silent: Smooth-L1 threshold 1,
+ * the L2 term as the plain square, sums rather than means; SiLU only.
+ * z: device bf16 [n × d_in] (the tokens' [Q ‖ K ‖ V]); labels: device fp32 [h_kv × n] (e.g. from
+ * locret_cis_labels); w1: device bf16 [d_in × d_R]; w2: device bf16 [d_R × h_kv]; outputs on the
+ * device: loss (one fp32), d_w1 fp32 [d_in × d_R], d_w2 fp32 [d_R × h_kv] (all overwritten).
+ * Requires n, d_in multiples of 64, d_R a multiple of 32, h_kv <= 32, alpha >= 0.  The two
+ * large contractions take bf16 operands (dpre is rounded to bf16) and accumulate in fp32.
+ * Allocates and frees its workspace (about n·(4 d_R + 2 d_in + 2 d_R) bytes) inside the call and
+ * synchronises the stream before it returns.
+ */
+int locret_rh_loss_grad(const void *z, const float *labels, const void *w1, const void *w2, int32_t n,
+                        int32_t d_in, int32_t d_R, int32_t h_kv, float alpha, float *loss, float *d_w1,
+                        float *d_w2, void *stream);
+
+/*
  * Retaining-head scores without any allocation.  (The paper has no counterpart: this entry
  * point exists for hosts that may not allocate device memory where they need scores, e.g. code
  * that runs inside a pool owning the whole device, or under an allocator that is locked while

@@ -16,4 +16,5 @@ from .binding import (  # noqa: F401
     cis_labels,
     lib,
     lib_path,
+    rh_loss_grad,
 )

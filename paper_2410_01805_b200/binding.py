@@ -73,6 +73,7 @@ def _load():
     l.locret_block_attention.restype = P
     l.locret_block_destroy.argtypes = [P]
     l.locret_block_destroy.restype = None
+    l.locret_rh_loss_grad.argtypes = [P, P, P, P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float, P, P, P, P]
     l.locret_cis_labels.argtypes = [P, P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float, P, P]
     return l
 
@@ -281,3 +282,17 @@ def cis_labels(q_ans: torch.Tensor, k_prompt: torch.Tensor, scale: float = 1.0) 
     _check(lib.locret_cis_labels(q_ans.data_ptr(), k_prompt.data_ptr(), n_a, n_q, h, h_kv, d, float(scale),
                                  out.data_ptr(), torch.cuda.current_stream().cuda_stream), "locret_cis_labels")
     return out
+
+
+def rh_loss_grad(z: torch.Tensor, labels: torch.Tensor, w1: torch.Tensor, w2: torch.Tensor, alpha: float = 2.5e-3):
+    """Eq. 2 / Eq. 3 for one sequence: z [n, d_in] bf16, labels [h_kv, n] fp32, w1 [d_in, d_R], w2 [d_R, h_kv]
+    bf16 (CUDA, contiguous) -> (loss fp32 scalar tensor, d_w1 fp32 [d_in, d_R], d_w2 fp32 [d_R, h_kv])."""
+    n, d_in = z.shape
+    d_R, h_kv = w2.shape
+    loss = torch.empty((), dtype=torch.float32, device=z.device)
+    d_w1 = torch.empty((d_in, d_R), dtype=torch.float32, device=z.device)
+    d_w2 = torch.empty((d_R, h_kv), dtype=torch.float32, device=z.device)
+    _check(lib.locret_rh_loss_grad(z.data_ptr(), labels.data_ptr(), w1.data_ptr(), w2.data_ptr(), n, d_in, d_R, h_kv,
+                                   float(alpha), loss.data_ptr(), d_w1.data_ptr(), d_w2.data_ptr(),
+                                   torch.cuda.current_stream().cuda_stream), "locret_rh_loss_grad")
+    return loss, d_w1, d_w2

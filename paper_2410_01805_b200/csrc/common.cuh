@@ -93,6 +93,9 @@ cudaError_t launch_gemm_tc_resid(const bf16 *A, int lda, const bf16 *Bt, int ldb
 // initialised by the caller); K % 64 == 0, lda / ldb multiples of 8, scale > 0
 cudaError_t launch_gemm_tc_rowmax(const bf16 *A, int lda, const bf16 *Bt, int ldb, float *out, int M, int N,
                                   int K, float scale, int *status, cudaStream_t st);
+// C (fp32, leading dimension ldc in floats) = A Bt^T
+cudaError_t launch_gemm_tc_f32(const bf16 *A, int lda, const bf16 *Bt, int ldb, float *C, int ldc, int M, int N,
+                               int K, int *status, cudaStream_t st);
 bool gemm_tc_gated_supported(int M, int N, int K, int lda, int ldb);
 cudaError_t launch_gemm_tc_gated(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, int ldc, int M,
                                  int N, int K, int *status, cudaStream_t st);

@@ -255,6 +255,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
           }
         }
+      } else if (MODE == 5) {
+        // plain GEMM with an fp32 result (gradients): C is a float array, ldc in floats
+        if (ok) {
+          float *Cf = reinterpret_cast<float *>(C);
+#pragma unroll 1
+          for (int c0 = 0; c0 < BN; c0 += 32) {
+            uint32_t r[32];
+            tmem_ld32(taddr + c0, r);
+            tmem_wait_ld();
+            if (row < M && n0 + c0 < N) {
+              float4 *dst = reinterpret_cast<float4 *>(Cf + (size_t)row * ldc + n0 + c0);
+#pragma unroll
+              for (int v = 0; v < 8; v++)
+                dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                     __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+            }
+          }
+        }
       } else if (MODE == 4) {
         // Row maximum of A B^T over the valid columns, merged into out[row] with an atomic
         // maximum on the order-preserving integer image of the float (`partial` is the output,
@@ -534,7 +552,7 @@ cudaError_t launch_t(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, i
   // from HBM once; in row-block-major order a B that exceeds the L2 is re-read for every row
   // block, and even one that fits is read about three times)
   const size_t a_bytes = (size_t)M * K * 2, b_bytes = (size_t)N * K * 2;
-  const int n_major = MODE != 1 && b_bytes > a_bytes;
+  const int n_major = MODE != 1 && b_bytes > a_bytes;  // (MODE 1 indexes its partial sums by column tile either way)
   gemm_tc_kernel<BN, MODE, HD><<<grid, GT_THREADS, Cfg::smem_bytes(MODE), st>>>(
       *ma, *mb, C, ldc, M, N, K, W2, partial, h_kv, act, ra, resid, ldr, n_major, status);
   return cudaGetLastError();
@@ -571,6 +589,15 @@ bool gemm_tc_gated_supported(int M, int N, int K, int lda, int ldb) {
 cudaError_t launch_gemm_tc_gated(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, int ldc, int M,
                                  int N, int K, int *status, cudaStream_t st) {
   return launch_t<256, 3>(A, lda, Bt, ldb, C, ldc, M, N, K, nullptr, nullptr, 0, 0, RopeAppendArgs{}, status, st);
+}
+
+// C (fp32, leading dimension ldc in floats) = A Bt^T
+cudaError_t launch_gemm_tc_f32(const bf16 *A, int lda, const bf16 *Bt, int ldb, float *C, int ldc, int M, int N,
+                               int K, int *status, cudaStream_t st) {
+  bf16 *Cb = reinterpret_cast<bf16 *>(C);
+  if (N >= 256)
+    return launch_t<256, 5>(A, lda, Bt, ldb, Cb, ldc, M, N, K, nullptr, nullptr, 0, 0, RopeAppendArgs{}, status, st);
+  return launch_t<128, 5>(A, lda, Bt, ldb, Cb, ldc, M, N, K, nullptr, nullptr, 0, 0, RopeAppendArgs{}, status, st);
 }
 
 // out[m] = max(out[m], scale * max_n (A Bt^T)[m][n]) for m < M (out fp32, initialised by the

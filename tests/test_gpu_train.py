@@ -1,0 +1,58 @@
+"""Training objective of the retaining head (Eq. 2, Eq. 3) on the GPU against the oracle."""
+
+import numpy as np
+import pytest
+import torch
+
+import workloads as W
+from oracle import locret_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+
+def case(n, d_in, d_R, hk, seed):
+    g = np.random.default_rng(7000 + seed)
+    z = W.to_bf16_grid(g.standard_normal((n, d_in)).astype(np.float32))
+    w1 = W.to_bf16_grid((g.standard_normal((d_in, d_R)) / np.sqrt(d_in)).astype(np.float32))
+    w2 = W.to_bf16_grid((g.standard_normal((d_R, hk)) / np.sqrt(d_R)).astype(np.float32))
+    labels = (g.standard_normal((hk, n)) * 1.5).astype(np.float32)      # errors on both sides of the Smooth-L1 knee
+    return z, w1, w2, labels
+
+
+@pytest.mark.parametrize("n,d_in,d_R,hk", [(128, 128, 64, 2), (1024, 768, 256, 2), (2048, 6144, 1024, 8)])
+def test_loss_and_gradients_match_the_oracle(n, d_in, d_R, hk):
+    from parity_util import bf16_dev
+    from paper_2410_01805_b200 import rh_loss_grad
+    z, w1, w2, labels = case(n, d_in, d_R, hk, n)
+    alpha = 0.05
+    loss, dw1, dw2 = O.rh_loss_and_grads(z, labels, w1, w2, alpha)
+    gl, g1, g2 = rh_loss_grad(bf16_dev(z), torch.from_numpy(labels).cuda(), bf16_dev(w1), bf16_dev(w2), alpha)
+    gl, g1, g2 = float(gl.item()), g1.cpu().numpy().astype(np.float64), g2.cpu().numpy().astype(np.float64)
+    # loss and dW2 come from fp32 arithmetic on exact bf16 products: only summation order differs
+    assert abs(gl - loss) <= 1e-4 * abs(loss)
+    assert np.abs(g2 - dw2).max() <= 1e-4 * np.abs(dw2).max()
+    # dW1 = z^T dpre with dpre rounded to bf16 for the contraction: every term carries at most 2^-9
+    # relative error, so |Δ| <= 2^-8 (|z|^T |dpre|) element-wise (twice the worst case, for the fp32 sums)
+    zf = np.asarray(z, np.float64)
+    pre = zf @ np.asarray(w1, np.float64)
+    sig = 1.0 / (1.0 + np.exp(-pre))
+    s = (pre * sig) @ np.asarray(w2, np.float64)
+    ds = np.clip(s - labels.T.astype(np.float64), -1.0, 1.0)
+    adj = s[:-1] - s[1:]
+    ds[:-1] += 2 * alpha * adj
+    ds[1:] -= 2 * alpha * adj
+    dpre = (ds @ np.asarray(w2, np.float64).T) * (sig * (1.0 + pre * (1.0 - sig)))
+    bound = 2.0 ** -8 * (np.abs(zf).T @ np.abs(dpre)) + 1e-6
+    assert (np.abs(g1 - dw1) <= bound).all(), float((np.abs(g1 - dw1) / bound).max())
+    # and in practice the errors are random: far inside the worst case
+    assert np.abs(g1 - dw1).max() <= 2e-2 * np.sqrt(np.mean(dw1 ** 2))
+
+
+def test_training_argument_checks():
+    from paper_2410_01805_b200 import LocretError, rh_loss_grad
+    z = torch.zeros((100, 128), dtype=torch.bfloat16, device="cuda")          # n not a multiple of 64
+    w1 = torch.zeros((128, 64), dtype=torch.bfloat16, device="cuda")
+    w2 = torch.zeros((64, 2), dtype=torch.bfloat16, device="cuda")
+    lab = torch.zeros((2, 100), dtype=torch.float32, device="cuda")
+    with pytest.raises(LocretError):
+        rh_loss_grad(z, lab, w1, w2)
