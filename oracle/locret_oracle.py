@@ -466,3 +466,29 @@ def rh_loss_and_grads(z, labels, w1, w2, alpha: float = 2.5e-3):
     dpre = da * (sig * (1.0 + pre * (1.0 - sig)))          # d SiLU / d pre
     dw1 = z.T @ dpre
     return loss, dw1, dw2
+
+
+# --------------------------------------------------------------------------- optimiser
+#
+# Appendix A (training): AdamW, learning rate 5e-4, linear schedule with 2000 warm-up steps, 3000
+# steps, batch size 1.  Where the text is silent the usual defaults are taken: betas (0.9,
+# 0.999), eps 1e-8, decoupled weight decay 0.01, bias correction on.
+
+def adamw_step(param, grad, m, v, step: int, lr: float, beta1: float = 0.9, beta2: float = 0.999,
+               eps: float = 1e-8, weight_decay: float = 0.01):
+    """One decoupled-weight-decay Adam update (step counts from 1).  Returns (param, m, v)."""
+    p = np.asarray(param, np.float64) * (1.0 - lr * weight_decay)
+    g = np.asarray(grad, np.float64)
+    m = beta1 * np.asarray(m, np.float64) + (1.0 - beta1) * g
+    v = beta2 * np.asarray(v, np.float64) + (1.0 - beta2) * g * g
+    mhat = m / (1.0 - beta1 ** step)
+    vhat = v / (1.0 - beta2 ** step)
+    return p - lr * mhat / (np.sqrt(vhat) + eps), m, v
+
+
+def linear_schedule(step: int, peak_lr: float = 5e-4, warmup: int = 2000, total: int = 3000):
+    """Learning rate of update number `step` (from 1): linear warm-up, then linear decay to 0."""
+    k = step - 1
+    if k < warmup:
+        return peak_lr * k / max(1, warmup)
+    return peak_lr * max(0.0, (total - k) / max(1, total - warmup))

@@ -602,3 +602,31 @@ def test_rh_loss_and_gradients_match_library_autograd_and_finite_differences():
     s0 = O.retaining_scores(z, w1, w2)
     l0, g1, g2 = O.rh_loss_and_grads(z, s0.T, w1, w2, 0.0)
     assert l0 < 1e-25 and np.abs(g1).max() < 1e-12 and np.abs(g2).max() < 1e-12
+
+
+# ------------------------------------------------------------------ optimiser (Appendix A, training)
+
+def test_adamw_step_matches_the_library_optimiser():
+    g = np.random.default_rng(600)
+    p0 = g.standard_normal((5, 7))
+    p = torch.nn.Parameter(torch.from_numpy(p0.copy()))
+    opt = torch.optim.AdamW([p], lr=5e-4, betas=(0.9, 0.999), eps=1e-8, weight_decay=0.01)
+    mine, m, v = p0.copy(), np.zeros_like(p0), np.zeros_like(p0)
+    for step in range(1, 6):
+        grad = g.standard_normal((5, 7)) * (10.0 if step == 3 else 1.0)
+        p.grad = torch.from_numpy(grad.copy())
+        opt.step()
+        mine, m, v = O.adamw_step(mine, grad, m, v, step, 5e-4)
+        assert np.allclose(mine, p.detach().numpy(), rtol=0, atol=1e-12)
+
+
+def test_linear_schedule_matches_the_library_scheduler():
+    p = torch.nn.Parameter(torch.zeros(1))
+    opt = torch.optim.SGD([p], lr=5e-4)
+    sched = torch.optim.lr_scheduler.LambdaLR(
+        opt, lambda k: k / 2000 if k < 2000 else max(0.0, (3000 - k) / 1000))
+    for step in range(1, 3001):
+        if step in (1, 2, 1000, 2000, 2001, 2500, 3000):
+            assert abs(O.linear_schedule(step) - sched.get_last_lr()[0]) < 1e-15, step
+        opt.step(); sched.step()
+    assert O.linear_schedule(1) == 0.0 and abs(O.linear_schedule(2001) - 5e-4) < 1e-18
