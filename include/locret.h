@@ -281,6 +281,18 @@ int locret_rh_loss_grad(const void *z, const float *labels, const void *w1, cons
                         float *d_w2, void *stream);
 
 /*
+ * One AdamW update of a parameter array (Appendix A: AdamW, learning rate 5e-4 with a linear
+ * warm-up schedule; the schedule is the caller's).  param: device fp32 master copy [n], updated
+ * in place; param_bf16: device bf16 [n] that receives the rounded parameters, or NULL; grad: device
+ * fp32 [n]; m, v: device fp32 [n] moment estimates (zero before the first step), updated in place.
+ * step counts from 1 (bias correction).  Decoupled weight decay: p <- p (1 - lr wd) - lr m^/(sqrt(v^) + eps).
+ * Asynchronous on the stream.
+ */
+int locret_adamw_step(float *param, void *param_bf16, const float *grad, float *m, float *v, int64_t n,
+                      int32_t step, float lr, float beta1, float beta2, float eps, float weight_decay,
+                      void *stream);
+
+/*
  * Retaining-head scores without any allocation.  (The paper has no counterpart: this entry
  * point exists for hosts that may not allocate device memory where they need scores, e.g. code
  * that runs inside a pool owning the whole device, or under an allocator that is locked while

@@ -13,6 +13,7 @@ from .binding import (  # noqa: F401
     LocretBlock,
     LocretError,
     LocretLayer,
+    adamw_step,
     cis_labels,
     lib,
     lib_path,

@@ -74,6 +74,7 @@ def _load():
     l.locret_block_destroy.argtypes = [P]
     l.locret_block_destroy.restype = None
     l.locret_rh_loss_grad.argtypes = [P, P, P, P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float, P, P, P, P]
+    l.locret_adamw_step.argtypes = [P, P, P, P, P, C.c_int64, C.c_int32, C.c_float, C.c_float, C.c_float, C.c_float, C.c_float, P]
     l.locret_cis_labels.argtypes = [P, P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float, P, P]
     return l
 
@@ -296,3 +297,13 @@ def rh_loss_grad(z: torch.Tensor, labels: torch.Tensor, w1: torch.Tensor, w2: to
                                    float(alpha), loss.data_ptr(), d_w1.data_ptr(), d_w2.data_ptr(),
                                    torch.cuda.current_stream().cuda_stream), "locret_rh_loss_grad")
     return loss, d_w1, d_w2
+
+
+def adamw_step(param: torch.Tensor, grad: torch.Tensor, m: torch.Tensor, v: torch.Tensor, step: int, lr: float,
+               param_bf16: torch.Tensor | None = None, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
+               weight_decay: float = 0.01):
+    """In-place AdamW update of a contiguous fp32 CUDA tensor (and its bf16 copy, if given)."""
+    _check(lib.locret_adamw_step(param.data_ptr(), param_bf16.data_ptr() if param_bf16 is not None else None,
+                                 grad.data_ptr(), m.data_ptr(), v.data_ptr(), param.numel(), int(step), float(lr),
+                                 float(beta1), float(beta2), float(eps), float(weight_decay),
+                                 torch.cuda.current_stream().cuda_stream), "locret_adamw_step")

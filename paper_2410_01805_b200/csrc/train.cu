@@ -182,3 +182,34 @@ extern "C" int locret_rh_loss_grad(const void *z, const float *labels, const voi
   TCK(cudaStreamSynchronize(st));
   return status ? LOCRET_ERR_DEVICE_TIMEOUT : LOCRET_OK;
 }
+
+// ---------------------------------------------------------------- AdamW (Appendix A, training)
+namespace {
+__global__ void adamw_kernel(float *__restrict__ p, bf16 *__restrict__ p_bf16, const float *__restrict__ g,
+                             float *__restrict__ m, float *__restrict__ v, size_t n, float lr, float beta1,
+                             float beta2, float eps, float wd, float bc1, float bc2) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const float gi = g[i];
+  const float mi = beta1 * m[i] + (1.0f - beta1) * gi;
+  const float vi = beta2 * v[i] + (1.0f - beta2) * gi * gi;
+  m[i] = mi;
+  v[i] = vi;
+  const float pi = p[i] * (1.0f - lr * wd) - lr * (mi / bc1) / (sqrtf(vi / bc2) + eps);
+  p[i] = pi;
+  if (p_bf16) p_bf16[i] = __float2bfloat16_rn(pi);
+}
+}  // namespace
+
+extern "C" int locret_adamw_step(float *param, void *param_bf16, const float *grad, float *m, float *v, int64_t n,
+                                 int32_t step, float lr, float beta1, float beta2, float eps, float weight_decay,
+                                 void *stream) {
+  if (!param || !grad || !m || !v || n < 1 || step < 1) return LOCRET_ERR_INVALID;
+  if (!(beta1 >= 0.f && beta1 < 1.f && beta2 >= 0.f && beta2 < 1.f) || eps <= 0.f) return LOCRET_ERR_INVALID;
+  const float bc1 = 1.0f - powf(beta1, (float)step), bc2 = 1.0f - powf(beta2, (float)step);
+  adamw_kernel<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(param, (bf16 *)param_bf16, grad, m, v,
+                                                                             (size_t)n, lr, beta1, beta2, eps,
+                                                                             weight_decay, bc1, bc2);
+  TCK(cudaGetLastError());
+  return LOCRET_OK;
+}

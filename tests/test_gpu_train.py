@@ -56,3 +56,47 @@ def test_training_argument_checks():
     lab = torch.zeros((2, 100), dtype=torch.float32, device="cuda")
     with pytest.raises(LocretError):
         rh_loss_grad(z, lab, w1, w2)
+
+
+def test_a_few_training_steps_follow_the_oracle_and_reduce_the_loss():
+    """Labels from the definition, loss and gradients, AdamW: three updates in lock-step with the
+    oracle's fp64 trajectory (the GPU's bf16 weights are fed to both sides at every step)."""
+    from parity_util import bf16_dev
+    from paper_2410_01805_b200 import adamw_step, cis_labels, rh_loss_grad
+    g = np.random.default_rng(8100)
+    n, h, hk, d, d_R, n_a = 512, 4, 2, 64, 128, 64
+    d_in = (h + 2 * hk) * d
+    qkv = W.to_bf16_grid(g.standard_normal((n + n_a, d_in)).astype(np.float32))
+    q = qkv[:, : h * d].reshape(n + n_a, h, d)
+    k = qkv[:, h * d:(h + hk) * d].reshape(n + n_a, hk, d)
+    labels = cis_labels(bf16_dev(np.ascontiguousarray(q[n:])), bf16_dev(np.ascontiguousarray(k[:n])), 1.0 / np.sqrt(d))
+    ref_labels = O.cis_labels(q[n:], k[:n], hk, 1.0 / np.sqrt(d))
+    assert np.abs(labels.cpu().numpy() - ref_labels).max() < 1e-4 * max(1.0, np.abs(ref_labels).max())
+    z = qkv[:n]
+    w1 = (g.standard_normal((d_in, d_R)) / np.sqrt(d_in)).astype(np.float32)
+    w2 = (g.standard_normal((d_R, hk)) / np.sqrt(d_R)).astype(np.float32)
+    P1, P2 = torch.from_numpy(w1).cuda(), torch.from_numpy(w2).cuda()
+    B1, B2 = P1.to(torch.bfloat16), P2.to(torch.bfloat16)
+    M1, V1, M2, V2 = (torch.zeros_like(t) for t in (P1, P1, P2, P2))
+    o1, o2 = w1.astype(np.float64), w2.astype(np.float64)
+    om1, ov1, om2, ov2 = (np.zeros_like(a) for a in (o1, o1, o2, o2))
+    zd = bf16_dev(z)
+    losses = []
+    lr = 2e-2
+    for step in range(1, 4):
+        loss, g1, g2 = rh_loss_grad(zd, labels, B1, B2, 2.5e-3)
+        # the oracle starts every step from the bf16 weights the GPU used
+        b1, b2 = B1.float().cpu().numpy().astype(np.float64), B2.float().cpu().numpy().astype(np.float64)
+        rl, r1, r2 = O.rh_loss_and_grads(z, ref_labels, b1, b2, 2.5e-3)
+        assert abs(float(loss.item()) - rl) <= 1e-3 * abs(rl)
+        assert np.abs(g2.cpu().numpy() - r2).max() <= 1e-3 * np.abs(r2).max()
+        assert np.abs(g1.cpu().numpy() - r1).max() <= 2e-2 * np.sqrt(np.mean(r1 ** 2))
+        losses.append(float(loss.item()))
+        o1, om1, ov1 = O.adamw_step(P1.cpu().numpy(), g1.cpu().numpy(), M1.cpu().numpy(), V1.cpu().numpy(), step, lr)
+        o2, om2, ov2 = O.adamw_step(P2.cpu().numpy(), g2.cpu().numpy(), M2.cpu().numpy(), V2.cpu().numpy(), step, lr)
+        adamw_step(P1, g1, M1, V1, step, lr, param_bf16=B1)
+        adamw_step(P2, g2, M2, V2, step, lr, param_bf16=B2)
+        torch.cuda.synchronize()
+        assert np.abs(P1.cpu().numpy() - o1).max() <= 1e-5 and np.abs(P2.cpu().numpy() - o2).max() <= 1e-5
+        assert torch.equal(B1, P1.to(torch.bfloat16))
+    assert losses[2] < losses[0]
