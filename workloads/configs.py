@@ -82,6 +82,10 @@ CONFIGS = {
         "c5_llama_stream_int4", replace(_LLAMA, kv_dtype=1), n_layers=32,
         context=1_000_000, chunk=3072, budget=6000, n_stab=2500,
         hidden="outlier", decode_steps=256),
+    # extra (not one of the five benchmark configurations): a soak run, 10M tokens in chunks of 10240
+    "x_llama_10m_stream": Workload(
+        "x_llama_10m_stream", _LLAMA, n_layers=32, context=10_000_000 // 10240 * 10240, chunk=10240,
+        budget=6000, n_stab=2500, hidden="outlier"),
 }
 
 
