@@ -19,6 +19,12 @@ What each function follows:
                             (+ the protected prefix of the query-aware variant, Section 4.4)
                              (stated without infinities: protected ∪ top-(b − n_prot) of the rest).
 * ``OracleLayer.prefill_chunk`` – one iteration of Algorithm 1's loop body for one layer.
+* ``shard_by_kv_head`` / ``OracleLayer.partial_preact`` / ``tp_prefill_chunk`` – the same step
+                             with the KV heads (and their query groups) divided over several
+                             workers: heads attend and evict independently (Algorithm 1 runs
+                             per head), the retaining head reads every head's [Q, K, V]
+                             (Section 3.3), so the workers exchange one thing, the sum of
+                             their partial products z_local · W1_local, before the activation.
 * ``quantize_int4`` / ``dequantize_int4`` – the 4-bit cache variant (Appendix H combines
                              a 4-bit KV cache with the method; the number format is the
                              workload's: symmetric, one fp16 scale per head vector).
@@ -274,8 +280,27 @@ class OracleLayer:
         return round_bf16(x) if self.mirror else x
 
     # ---- one chunk
-    def prefill_chunk(self, X, flags: int = 0, rows=None):
-        """One loop iteration of Algorithm 1 for this layer.  Returns attn_out [n_tok, h·d]."""
+    def _rh_input(self, X):
+        """z of the chunk's tokens, [n_tok, (h + 2 h_kv) d]: what the retaining head reads."""
+        n_tok = X.shape[0]
+        qkv = self._r(project_qkv(X, self.w_qkv, self.h, self.hk, self.d))
+        if self.s.rh_input == 0:
+            return qkv
+        Q, K, V = split_qkv(qkv, self.h, self.hk, self.d)
+        pos_chunk = (self.len + np.arange(n_tok))[:, None]
+        Qr = self._r(rope(Q, pos_chunk, self.s.rope_theta))
+        Kr = self._r(rope(K, pos_chunk, self.s.rope_theta))
+        return np.concatenate([Qr.reshape(n_tok, -1), Kr.reshape(n_tok, -1), V.reshape(n_tok, -1)], axis=1)
+
+    def partial_preact(self, X):
+        """This worker's share of the retaining head's first product, z_local · W1_local
+        [n_tok, d_R]: summed over the workers it is z · W1 of the whole layer."""
+        return self._rh_input(np.asarray(X, np.float64)) @ self.w1
+
+    def prefill_chunk(self, X, flags: int = 0, rows=None, preact=None):
+        """One loop iteration of Algorithm 1 for this layer.  Returns attn_out [n_tok, h·d].
+        preact: the summed first product of the retaining head when the heads are divided over
+        workers (this worker's own product alone is not the layer's)."""
         X = np.asarray(X, np.float64)
         n_tok = X.shape[0]
         h, hk, d, g = self.h, self.hk, self.d, self.g
@@ -308,7 +333,10 @@ class OracleLayer:
         else:
             z = np.concatenate([Qr.reshape(n_tok, -1), Kr_chunk.reshape(n_tok, -1),
                                 V.reshape(n_tok, -1)], axis=1)
-        s_chunk = retaining_scores(z, self.w1, self.w2, self.s.act)     # [n_tok, h_kv]
+        if preact is None:
+            s_chunk = retaining_scores(z, self.w1, self.w2, self.s.act)     # [n_tok, h_kv]
+        else:
+            s_chunk = activation(np.asarray(preact, np.float64), self.s.act) @ self.w2
         self.last_scores = s_chunk
 
         # (d) concat, protect, top-b, gather
@@ -343,6 +371,32 @@ class OracleLayer:
     def decode_step(self, x):
         """The B = 1 case of Eq. 1: append without eviction."""
         return self.prefill_chunk(np.asarray(x, np.float64).reshape(1, -1), NO_EVICT)
+
+
+# --------------------------------------------------------------------------- heads divided over workers
+def shard_by_kv_head(w_qkv, w1, w2, h: int, h_kv: int, d: int, rank: int, world: int):
+    """Worker rank's slices when KV heads [rank·h_kv/world, (rank+1)·h_kv/world) and the query
+    heads of their groups live on it: the matching columns of W_qkv, the matching rows of W1
+    (same order: local Q heads, local K heads, local V heads), the matching columns of W2."""
+    if h_kv % world or not 0 <= rank < world:
+        raise ValueError("n_kv_heads must divide evenly over the workers")
+    g, hk_l = h // h_kv, h_kv // world
+    q_heads = np.arange(rank * hk_l * g, (rank + 1) * hk_l * g)
+    kv_heads = np.arange(rank * hk_l, (rank + 1) * hk_l)
+    cols = np.concatenate([
+        (q_heads[:, None] * d + np.arange(d)[None, :]).ravel(),
+        ((h + kv_heads)[:, None] * d + np.arange(d)[None, :]).ravel(),
+        ((h + h_kv + kv_heads)[:, None] * d + np.arange(d)[None, :]).ravel()])
+    return (np.asarray(w_qkv)[:, cols], np.asarray(w1)[cols, :], np.asarray(w2)[:, kv_heads])
+
+
+def tp_prefill_chunk(shards, X, flags: int = 0, rows=None):
+    """One step of Algorithm 1 with the heads divided over len(shards) workers (OracleLayer
+    objects built from shard_by_kv_head slices).  The only exchange is the sum of the partial
+    products before the activation.  Returns the workers' attn_out side by side, which is the
+    undivided layer's attn_out because query heads are dealt out in order."""
+    total = sum(sh.partial_preact(X) for sh in shards)
+    return np.concatenate([sh.prefill_chunk(X, flags, rows, preact=total) for sh in shards], axis=1)
 
 
 # --------------------------------------------------------------------------- the rest of the decoder layer

@@ -630,3 +630,52 @@ def test_linear_schedule_matches_the_library_scheduler():
             assert abs(O.linear_schedule(step) - sched.get_last_lr()[0]) < 1e-15, step
         opt.step(); sched.step()
     assert O.linear_schedule(1) == 0.0 and abs(O.linear_schedule(2001) - 5e-4) < 1e-18
+
+
+# ------------------------------------------------------------------ heads divided over workers
+# Heads attend and evict independently and only the retaining head mixes them, so dividing the
+# KV heads over workers and summing the partial first products must reproduce the undivided layer.
+@pytest.mark.parametrize("world,rh_input,kv_dtype", [(2, 0, 0), (4, 0, 0), (2, 1, 0), (2, 0, 1)])
+def test_heads_divided_over_workers_reproduce_the_undivided_layer(world, rh_input, kv_dtype):
+    sh = shape(n_q_heads=8, n_kv_heads=4, head_dim=8, d_retain=12, rh_input=rh_input, kv_dtype=kv_dtype)
+    whole, (wqkv, w1, w2) = rand_layer(sh, budget=24, chunk=8, n_stab=3, seed=70 + world)
+    sh_l = shape(n_q_heads=8 // world, n_kv_heads=4 // world, head_dim=8, d_retain=12, rh_input=rh_input,
+                 kv_dtype=kv_dtype)
+    shards = [O.OracleLayer(sh_l, *O.shard_by_kv_head(wqkv, w1, w2, 8, 4, 8, r, world), 24, 8, 3)
+              for r in range(world)]
+    hk_l = 4 // world
+    X = np.random.default_rng(71).standard_normal((50, sh.d_model))
+    for s in range(0, 50, 8):
+        want = whole.prefill_chunk(X[s:s + 8])
+        got = O.tp_prefill_chunk(shards, X[s:s + 8])
+        assert np.allclose(got, want, atol=1e-12)
+        assert np.allclose(np.concatenate([sh_.last_scores for sh_ in shards], axis=1), whole.last_scores,
+                           atol=1e-12)
+        for r, sh_ in enumerate(shards):
+            assert np.array_equal(sh_.T, whole.T[r * hk_l:(r + 1) * hk_l])
+            assert np.allclose(sh_.K, whole.K[r * hk_l:(r + 1) * hk_l], atol=1e-12)
+    assert whole.len == 24 and whole.last_keep is not None
+    # the slices are what they claim: a worker's own product alone is not the layer's first product
+    part = shards[0].partial_preact(X[:8])
+    full = (X[:8] @ wqkv) @ w1 if rh_input == 0 else None
+    if full is not None:
+        assert not np.allclose(part, full, atol=1e-3)
+        shards2 = [O.OracleLayer(sh_l, *O.shard_by_kv_head(wqkv, w1, w2, 8, 4, 8, r, world), 24, 8, 3)
+                   for r in range(world)]
+        assert np.allclose(sum(s2.partial_preact(X[:8]) for s2 in shards2), full, atol=1e-12)
+
+
+def test_shard_slices_name_the_right_heads():
+    h, hk, d = 8, 4, 2
+    d_in = (h + 2 * hk) * d
+    wqkv = np.arange(3 * d_in, dtype=np.float64).reshape(3, d_in)
+    w1 = np.arange(d_in * 5, dtype=np.float64).reshape(d_in, 5)
+    w2 = np.arange(5 * hk, dtype=np.float64).reshape(5, hk)
+    a, b, c = O.shard_by_kv_head(wqkv, w1, w2, h, hk, d, rank=1, world=2)
+    # worker 1 of 2: query heads 4..7 (columns 8..15), key heads 2, 3 (columns 16+4..16+7), value heads 2, 3
+    cols = list(range(8, 16)) + list(range(20, 24)) + list(range(28, 32))
+    assert np.array_equal(a[0], np.array(cols, dtype=np.float64))
+    assert np.array_equal(b[:, 0], np.array(cols, dtype=np.float64) * 5)
+    assert np.array_equal(c[0], np.array([2.0, 3.0]))
+    with pytest.raises(ValueError):
+        O.shard_by_kv_head(wqkv, w1, w2, h, hk, d, rank=0, world=3)
