@@ -121,6 +121,33 @@ int locret_prefill_chunk(locret_layer *layer, const void *hidden_in, int32_t n_t
  */
 int locret_decode_step(locret_layer *layer, const void *hidden_in, void *attn_out);
 
+/*
+ * The same step with the KV heads (and the query heads of their groups) divided over several
+ * GPUs, one layer object per GPU.  Heads attend and evict independently (Algorithm 1 runs per
+ * head) and only the retaining head reads every head's [Q, K, V] (Section 3.3), so the GPUs
+ * exchange one thing per step: the sum of their partial first products z_local · W1_local.
+ *
+ * A GPU's layer object is created by locret_create with its share of the heads: n_q_heads and
+ * n_kv_heads are the local counts, w_qkv holds the columns of its query, key and value heads
+ * (in that order), w1 the matching rows [(h_local + 2 h_kv_local)·d x d_R], w2 the columns of
+ * its KV heads [d_R x h_kv_local].  budget, chunk and n_stab are the same on every GPU, so
+ * cache lengths and positions agree without communication.
+ *
+ * locret_prefill_chunk_tp_begin: steps (a), (b) as in locret_prefill_chunk for the local heads
+ *   (attn_out: device bf16 [n_tok x h_local·d]), then preact_partial (device fp32
+ *   [n_tok x d_R], 16-byte aligned, caller-owned) = z_local · W1_local.  Every kernel runs on the
+ *   layer's stream.  The caller sums preact_partial over the GPUs on that stream (an all-reduce)
+ *   and passes the sum to
+ * locret_prefill_chunk_tp_finish: scores = act(preact_sum) · W2_local for the chunk's units, then
+ *   step (d) as in locret_prefill_chunk (with the flags given to _begin).  preact_sum may be the
+ *   buffer given to _begin.
+ * Between the two calls the layer accepts no other step (LOCRET_ERR_INVALID); locret_reset
+ * abandons a begun step.  _finish without _begin returns LOCRET_ERR_INVALID.
+ */
+int locret_prefill_chunk_tp_begin(locret_layer *layer, const void *hidden_in, int32_t n_tok,
+                                  uint32_t flags, void *attn_out, float *preact_partial);
+int locret_prefill_chunk_tp_finish(locret_layer *layer, const float *preact_sum);
+
 /* Number of retained units per KV head (the same for every head).  No device work. */
 int locret_cache_len(const locret_layer *layer, int32_t *len);
 

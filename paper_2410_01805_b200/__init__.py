@@ -13,9 +13,11 @@ from .binding import (  # noqa: F401
     LocretBlock,
     LocretError,
     LocretLayer,
+    LocretLayerTP,
     adamw_step,
     cis_labels,
     lib,
     lib_path,
     rh_loss_grad,
+    shard_by_kv_head,
 )

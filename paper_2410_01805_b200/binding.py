@@ -52,6 +52,8 @@ def _load():
     l.locret_create.argtypes = [C.POINTER(locret_layer_cfg), C.c_int32, C.c_int32, C.c_int32, C.POINTER(P)]
     l.locret_prefill_chunk.argtypes = [P, P, C.c_int32, C.c_uint32, P]
     l.locret_decode_step.argtypes = [P, P, P]
+    l.locret_prefill_chunk_tp_begin.argtypes = [P, P, C.c_int32, C.c_uint32, P, P]
+    l.locret_prefill_chunk_tp_finish.argtypes = [P, P]
     l.locret_cache_len.argtypes = [P, C.POINTER(C.c_int32)]
     l.locret_export_state.argtypes = [P, P, P, P, P, C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
     l.locret_import_state.argtypes = [P, P, P, P, P, C.c_int32, C.c_int64]
@@ -120,6 +122,21 @@ class LocretLayer:
     def decode_step(self, hidden_in: torch.Tensor, attn_out: torch.Tensor):
         _check(lib.locret_decode_step(self._h, hidden_in.data_ptr(), attn_out.data_ptr()),
                "locret_decode_step")
+
+    # -- the same step with the heads divided over GPUs (this object holds one GPU's heads)
+    def prefill_chunk_tp_begin(self, hidden_in: torch.Tensor, attn_out: torch.Tensor,
+                               preact_partial: torch.Tensor, flags: int = 0, n_tok: int | None = None):
+        n_tok = hidden_in.shape[0] if n_tok is None else n_tok
+        if not (preact_partial.is_cuda and preact_partial.dtype == torch.float32 and preact_partial.is_contiguous()
+                and preact_partial.numel() >= n_tok * self.shape.d_retain):
+            raise ValueError("preact_partial must be a contiguous CUDA float32 tensor of n_tok x d_retain")
+        _check(lib.locret_prefill_chunk_tp_begin(self._h, hidden_in.data_ptr(), n_tok, flags, attn_out.data_ptr(),
+                                                 preact_partial.data_ptr()), "locret_prefill_chunk_tp_begin")
+
+    def prefill_chunk_tp_finish(self, preact_sum: torch.Tensor):
+        if not (preact_sum.is_cuda and preact_sum.dtype == torch.float32 and preact_sum.is_contiguous()):
+            raise ValueError("preact_sum must be a contiguous CUDA float32 tensor")
+        _check(lib.locret_prefill_chunk_tp_finish(self._h, preact_sum.data_ptr()), "locret_prefill_chunk_tp_finish")
 
     # -- state
     @property
@@ -224,6 +241,62 @@ class LocretLayer:
             self.destroy()
         except Exception:
             pass
+
+
+def shard_by_kv_head(w_qkv: torch.Tensor, w1: torch.Tensor, w2: torch.Tensor, n_q_heads: int,
+                     n_kv_heads: int, head_dim: int, rank: int, world: int):
+    """One GPU's slices of a layer's weights when KV heads [rank * n_kv_heads / world, ...) and the
+    query heads of their groups live on it: columns of w_qkv, the matching rows of w1 (local query
+    heads, local key heads, local value heads, in that order), the matching columns of w2."""
+    if n_kv_heads % world or not 0 <= rank < world:
+        raise ValueError("n_kv_heads must divide evenly over the GPUs")
+    g, hk = n_q_heads // n_kv_heads, n_kv_heads // world
+    d = head_dim
+    q0, k0, v0 = rank * hk * g * d, (n_q_heads + rank * hk) * d, (n_q_heads + n_kv_heads + rank * hk) * d
+    idx = torch.cat([torch.arange(q0, q0 + hk * g * d), torch.arange(k0, k0 + hk * d),
+                     torch.arange(v0, v0 + hk * d)]).to(w_qkv.device)
+    return (w_qkv.index_select(1, idx).contiguous(), w1.index_select(0, idx).contiguous(),
+            w2[:, rank * hk:(rank + 1) * hk].contiguous())
+
+
+class LocretLayerTP:
+    """A layer whose heads are divided over the ranks of a process group, one rank per GPU.
+
+    Each rank holds the cache of its own KV heads; a step is the library's begin call, one
+    all-reduce (sum) of the [n_tok x d_retain] float32 partial products on the current stream,
+    and the library's finish call.  The layer's stream must be torch's current stream when a step
+    is issued, so that the collective is ordered between the two calls.  ``reduce`` replaces the
+    all-reduce (a callable that sums the tensor in place across the ranks)."""
+
+    def __init__(self, shape, w_qkv, w1, w2, budget: int, chunk: int, n_stab: int, rank: int, world: int,
+                 reserve: int = 0, group=None, reduce=None, stream=None):
+        from dataclasses import replace
+        wq, wa, wb = shard_by_kv_head(w_qkv, w1, w2, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
+                                      rank, world)
+        self.rank, self.world = rank, world
+        self.local_shape = replace(shape, n_q_heads=shape.n_q_heads // world,
+                                   n_kv_heads=shape.n_kv_heads // world)
+        self._weights = (wq, wa, wb)  # the library borrows them
+        self.layer = LocretLayer(self.local_shape, wq, wa, wb, budget, chunk, n_stab, reserve, stream)
+        self.preact = torch.empty(chunk, shape.d_retain, dtype=torch.float32, device=wq.device)
+        if reduce is None:
+            import torch.distributed as dist
+
+            def reduce(t, _g=group):
+                dist.all_reduce(t, op=dist.ReduceOp.SUM, group=_g)
+        self._reduce = reduce
+
+    def prefill_chunk(self, hidden_in: torch.Tensor, attn_out_local: torch.Tensor, flags: int = 0,
+                      n_tok: int | None = None):
+        """attn_out_local: bf16 [n_tok x (n_q_heads / world) * head_dim], this rank's heads."""
+        n_tok = hidden_in.shape[0] if n_tok is None else n_tok
+        pre = self.preact[:n_tok]
+        self.layer.prefill_chunk_tp_begin(hidden_in, attn_out_local, pre, flags, n_tok)
+        self._reduce(pre)
+        self.layer.prefill_chunk_tp_finish(pre)
+
+    def destroy(self):
+        self.layer.destroy()
 
 
 class LocretBlock:

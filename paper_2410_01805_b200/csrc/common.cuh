@@ -94,6 +94,12 @@ cudaError_t launch_gemm_tc_resid(const bf16 *A, int lda, const bf16 *Bt, int ldb
 cudaError_t launch_gemm_tc_rowmax(const bf16 *A, int lda, const bf16 *Bt, int ldb, float *out, int M, int N,
                                   int K, float scale, int *status, cudaStream_t st);
 // C (fp32, leading dimension ldc in floats) = A Bt^T
+// heads divided over GPUs: this GPU's partial first product of the retaining head (fallback for
+// shapes the tensor-core GEMM does not take), and scores from the summed product
+cudaError_t launch_preact_naive(const bf16 *z, const bf16 *W1t, float *pre, int n_tok, int d_R, int d_in,
+                                cudaStream_t st);
+cudaError_t launch_rh_finish(const float *pre, const float *w2, float *s, int score_stride, int slot0,
+                             int n_tok, int d_R, int h_kv, int act, cudaStream_t st);
 cudaError_t launch_gemm_tc_f32(const bf16 *A, int lda, const bf16 *Bt, int ldb, float *C, int ldc, int M, int N,
                                int K, int *status, cudaStream_t st);
 bool gemm_tc_gated_supported(int M, int N, int K, int lda, int ldb);

@@ -89,6 +89,9 @@ struct locret_layer {
   bool fuse_rope;  // RoPE + append in the projection's epilogue (LOCRET_UNFUSED_ROPE=1 disables)
   bool use_side;  // off-critical-path kernels go to the pool's second stream (LOCRET_SERIAL=1 disables)
   bool side_pending;
+  bool tp_pending;  // a divided-heads step was begun and waits for the summed product
+  int tp_n_tok;
+  uint32_t tp_flags;
   cudaEvent_t ev_ready, ev_attn, ev_side;
   bool tc_attn;  // tensor maps for the tcgen05 attention kernel are valid
   CUtensorMap map_k, map_v[2], map_q;
@@ -375,9 +378,56 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   return LOCRET_OK;
 }
 
-int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t flags,
-                         void *attn_out) {
+}  // extern "C"
+
+namespace {
+
+// (d) of the step: protect, top-b, gather; then the bookkeeping that closes the step
+int evict_and_close(locret_layer *L, int n_tok, uint32_t flags, bool side, cudaStream_t S) {
+  ScratchPool *P = L->pool;
+  const int c = L->cur, n = L->len + n_tok;
+  if (!(flags & LOCRET_NO_EVICT) && n > L->budget) {
+    const int n_prot = (flags & LOCRET_LAST_CHUNK) ? 0 : (L->n_stab < n ? L->n_stab : n);
+    {
+      Timed t(L, LOCRET_K_TOPK, S);
+      // (n_prefix + n_stab <= budget < n, so the prefix never reaches into the protected tail)
+      CK(launch_topk(L->s[c], L->cap, L->h_kv, n, L->budget, n_prot, L->n_prefix, P->keep, S));
+    }
+    // compaction rewrites the rotated keys the attention kernel reads
+    if (side) CK(cudaStreamWaitEvent(S, L->ev_attn, 0));
+    if (L->int4) {
+      Timed t(L, LOCRET_K_COMPACT, S);
+      CK(launch_compact_int4(L->q4[c], L->q4[c ^ 1], L->s[c], L->tid[c], L->s[c ^ 1], L->tid[c ^ 1],
+                             P->keep, L->h_kv, L->d, L->cap, L->budget, S));
+    } else {
+      Timed t(L, LOCRET_K_COMPACT, S);
+      CompactArgs a;
+      a.k_src = L->k_pre[c]; a.v_src = L->v[c]; a.s_src = L->s[c]; a.t_src = L->tid[c];
+      a.k_dst = L->k_pre[c ^ 1]; a.v_dst = L->v[c ^ 1]; a.s_dst = L->s[c ^ 1]; a.t_dst = L->tid[c ^ 1];
+      a.k_rot = L->k_rot; a.keep = P->keep; a.cs = L->cs;
+      a.h_kv = L->h_kv; a.d = L->d; a.cap = L->cap; a.budget = L->budget;
+      CK(launch_compact(a, S));
+    }
+    L->cur = c ^ 1;
+    L->len = L->budget;
+  } else {
+    L->len = n;
+  }
+  if (side) {
+    CK(cudaEventRecord(L->ev_side, S));
+    L->side_pending = true;
+  }
+  L->seen += n_tok;
+  return LOCRET_OK;
+}
+
+// One step.  tp_partial == nullptr: the whole step.  Otherwise the heads of this layer object are
+// one GPU's share: the step stops after attention and this GPU's partial first product of the
+// retaining head (fp32 [n_tok x d_R], written to tp_partial), everything on the layer's stream.
+int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t flags, void *attn_out,
+               float *tp_partial) {
   if (!L || !hidden_in || !attn_out) return LOCRET_ERR_INVALID;
+  if (L->tp_pending) return LOCRET_ERR_INVALID;  // a begun step is finished first
   if (n_tok < 1 || n_tok > L->chunk) return LOCRET_ERR_INVALID;
   if (flags & ~(LOCRET_NO_EVICT | LOCRET_LAST_CHUNK)) return LOCRET_ERR_INVALID;
   if (!aligned16(hidden_in) || !aligned16(attn_out)) return LOCRET_ERR_INVALID;
@@ -385,8 +435,9 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
   if (n > L->cap) return LOCRET_ERR_CAPACITY;
   ScratchPool *P = L->pool;
   const int c = L->cur;
-  const bool decode = n_tok == 1 && L->use_tc;  // one token: bandwidth-bound kernels of decode.cu
-  const bool side = L->use_side && !L->serialize;
+  const bool tp = tp_partial != nullptr;
+  const bool decode = n_tok == 1 && L->use_tc && !tp;  // one token: bandwidth-bound kernels of decode.cu
+  const bool side = L->use_side && !L->serialize && !tp;
   cudaStream_t S = side ? P->side : L->st;  // stream of the off-critical-path kernels
   const int sb = P->flip;                    // staging buffer of this call
   P->flip ^= 1;
@@ -470,6 +521,20 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
       CK(launch_attention_mma(P->q_rot, k_att, v_att, (bf16 *)attn_out, n_tok, L->h, L->h_kv,
                               L->d, L->cap, L->len, L->st));
   }
+  if (tp) {
+    // this GPU's columns of z times its rows of W1; the caller sums the products of all GPUs
+    Timed t(L, LOCRET_K_RH);
+    const bf16 *z = L->cfg.rh_input == 1 ? z_post : staging;
+    if (L->use_tc && gemm_tc_supported(n_tok, L->d_R, L->d_in, L->d_in, L->d_in))
+      CK(launch_gemm_tc_f32(z, L->d_in, L->w1_t, L->d_in, tp_partial, L->d_R, n_tok, L->d_R, L->d_in,
+                            L->d_status, L->st));
+    else
+      CK(launch_preact_naive(z, L->w1_t, tp_partial, n_tok, L->d_R, L->d_in, L->st));
+    L->tp_pending = true;
+    L->tp_n_tok = n_tok;
+    L->tp_flags = flags;
+    return LOCRET_OK;
+  }
   if (side) {
     CK(cudaEventRecord(L->ev_attn, L->st));
     CK(cudaStreamWaitEvent(S, L->ev_ready, 0));
@@ -496,40 +561,35 @@ int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, 
     CK(cudaEventRecord(P->ev_stage_free[sb], S));
     P->stage_busy[sb] = true;
   }
-  // (d) protect, top-b, gather
-  if (!(flags & LOCRET_NO_EVICT) && n > L->budget) {
-    const int n_prot = (flags & LOCRET_LAST_CHUNK) ? 0 : (L->n_stab < n ? L->n_stab : n);
-    {
-      Timed t(L, LOCRET_K_TOPK, S);
-      // (n_prefix + n_stab <= budget < n, so the prefix never reaches into the protected tail)
-      CK(launch_topk(L->s[c], L->cap, L->h_kv, n, L->budget, n_prot, L->n_prefix, P->keep, S));
-    }
-    // compaction rewrites the rotated keys the attention kernel reads
-    if (side) CK(cudaStreamWaitEvent(S, L->ev_attn, 0));
-    if (L->int4) {
-      Timed t(L, LOCRET_K_COMPACT, S);
-      CK(launch_compact_int4(L->q4[c], L->q4[c ^ 1], L->s[c], L->tid[c], L->s[c ^ 1], L->tid[c ^ 1],
-                             P->keep, L->h_kv, L->d, L->cap, L->budget, S));
-    } else {
-      Timed t(L, LOCRET_K_COMPACT, S);
-      CompactArgs a;
-      a.k_src = L->k_pre[c]; a.v_src = L->v[c]; a.s_src = L->s[c]; a.t_src = L->tid[c];
-      a.k_dst = L->k_pre[c ^ 1]; a.v_dst = L->v[c ^ 1]; a.s_dst = L->s[c ^ 1]; a.t_dst = L->tid[c ^ 1];
-      a.k_rot = L->k_rot; a.keep = P->keep; a.cs = L->cs;
-      a.h_kv = L->h_kv; a.d = L->d; a.cap = L->cap; a.budget = L->budget;
-      CK(launch_compact(a, S));
-    }
-    L->cur = c ^ 1;
-    L->len = L->budget;
-  } else {
-    L->len = n;
+  return evict_and_close(L, n_tok, flags, side, S);
+}
+
+}  // namespace
+
+extern "C" {
+
+int locret_prefill_chunk(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t flags,
+                         void *attn_out) {
+  return chunk_step(L, hidden_in, n_tok, flags, attn_out, nullptr);
+}
+
+int locret_prefill_chunk_tp_begin(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t flags,
+                                  void *attn_out, float *preact_partial) {
+  if (!preact_partial || !aligned16(preact_partial)) return LOCRET_ERR_INVALID;
+  return chunk_step(L, hidden_in, n_tok, flags, attn_out, preact_partial);
+}
+
+int locret_prefill_chunk_tp_finish(locret_layer *L, const float *preact_sum) {
+  if (!L || !preact_sum || !aligned16(preact_sum)) return LOCRET_ERR_INVALID;
+  if (!L->tp_pending) return LOCRET_ERR_INVALID;
+  L->tp_pending = false;
+  const int n_tok = L->tp_n_tok;
+  {  // (c) finished: activation and this GPU's columns of W2, into the score cache
+    Timed t(L, LOCRET_K_RH_REDUCE);
+    CK(launch_rh_finish(preact_sum, L->w2f, L->s[L->cur], L->cap, L->len, n_tok, L->d_R, L->h_kv, L->cfg.act,
+                        L->st));
   }
-  if (side) {
-    CK(cudaEventRecord(L->ev_side, S));
-    L->side_pending = true;
-  }
-  L->seen += n_tok;
-  return LOCRET_OK;
+  return evict_and_close(L, n_tok, L->tp_flags, false, L->st);
 }
 
 int locret_decode_step(locret_layer *L, const void *hidden_in, void *attn_out) {
@@ -649,6 +709,7 @@ int locret_reset(locret_layer *L) {
   if (!L) return LOCRET_ERR_INVALID;
   L->len = 0;
   L->seen = 0;
+  L->tp_pending = false;
   return LOCRET_OK;
 }
 
