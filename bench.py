@@ -564,8 +564,82 @@ def run_cis(args, w):
                                              "finite": bool(torch.isfinite(g1).all().item() and torch.isfinite(loss).item())}}))
 
 
+def run_tp(args, w):
+    """Extra: the step with the KV heads divided over GPUs (locret_prefill_chunk_tp_begin / _finish
+    around one all-reduce per chunk-layer).  Under torchrun every rank holds its heads of every layer
+    and the exchange is NCCL's all-reduce (total work fixed: strong scaling).  In a single process it
+    times ONE rank's share at degree --tp with no exchange, and says so."""
+    import torch
+    from paper_2410_01805_b200 import LocretLayerTP
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    multi = world > 1
+    if multi:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    degree = world if multi else args.tp
+    s = w.shape
+    if s.n_kv_heads % degree:
+        raise SystemExit(f"--tp {degree} does not divide {s.n_kv_heads} KV heads")
+    g = torch.Generator(device=dev); g.manual_seed(W.BASE_SEED)
+
+    def mat(rows, cols):
+        return (torch.randn((rows, cols), generator=g, device=dev, dtype=torch.float32) / math.sqrt(rows)).to(torch.bfloat16)
+
+    layers = []
+    for _ in range(w.n_layers):
+        full = (mat(s.d_model, s.d_in), mat(s.d_in, s.d_retain), mat(s.d_retain, s.n_kv_heads))
+        layers.append(LocretLayerTP(s, *full, w.budget, w.chunk, w.n_stab, rank if multi else 0, degree,
+                                    reduce=None if multi else (lambda t: None)))
+        del full
+    sizes = w.chunk_sizes()
+    x = torch.randn((w.chunk, s.d_model), generator=g, device=dev).to(torch.bfloat16)
+    out = torch.zeros((w.chunk, (s.n_q_heads // degree) * s.head_dim), dtype=torch.bfloat16, device=dev)
+
+    def one_pass():
+        for L in layers:
+            L.layer.reset()
+        for n_tok in sizes:
+            for L in layers:
+                L.prefill_chunk(x[:n_tok], out, 0, n_tok)
+
+    for _ in range(max(1, args.warmup)):
+        one_pass()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(args.steps):
+        if multi:
+            dist.barrier()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); one_pass(); b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b))
+    ms = float(np.mean(ts))
+    if multi:
+        t = torch.tensor([ms], device=dev); dist.all_reduce(t, op=dist.ReduceOp.MAX); ms = float(t.item())
+    status = max(abs(L.layer.sync_status()) for L in layers)
+    exch = w.chunk * s.d_retain * 4
+    if rank == 0:
+        print(json.dumps({
+            "metric": "prefill tokens/s, KV heads divided over GPUs" if multi else
+                      "one rank's share of the divided step (no exchange timed)",
+            "value": w.context / (ms * 1e-3), "unit": "tokens/s", "n_gpus": world, "tp_degree": degree,
+            "ms_per_step": ms, "steps": args.steps, "warmup": max(1, args.warmup), "scaling": "strong",
+            "status": status, "data": "synthetic (device-generated weights and hidden states)",
+            "config": {"workload": w.name, "layers": w.n_layers, "heads_per_rank": f"{s.n_q_heads // degree}q/{s.n_kv_heads // degree}kv",
+                       "exchange": f"all-reduce of {exch / 1e6:.1f} MB fp32 per chunk-layer" + ("" if multi else " (not run: single process)")}}))
+    if multi:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--tp", type=int, default=0,
+                    help="extra run: KV heads divided over GPUs (degree = world size under torchrun, else this value)")
     ap.add_argument("--cis", action="store_true", help="extra run: the training labels of Section 3.3")
     ap.add_argument("--whole-model", action="store_true",
                     help="extra run: whole decoder layers (attention block + W_o + gated FFN), hidden states chained")
@@ -591,7 +665,9 @@ def main():
     else:
         import __graft_entry__ as G
         G.build()
-        if args.cis:
+        if args.tp:
+            run_tp(args, w)
+        elif args.cis:
             run_cis(args, w)
         elif args.whole_model:
             run_whole_model(args, w)
