@@ -172,6 +172,108 @@ gemv_rope_kernel(const bf16 *__restrict__ x, const bf16 *__restrict__ Wt, int K,
   }
 }
 
+// The same projection for K <= 4096 laid out for bandwidth: a block of 512 threads owns a contiguous
+// range of rotation pairs, thread t holds element group t of x in registers (no staging step before
+// the first weight load) and reads group t of both rows of four pairs at a time, so a block has
+// 64 KB of weights in flight and two blocks per SM cover each other's reductions.  The eight
+// partial sums of a batch are reduced with one butterfly that halves the number of values at each
+// step (9 shuffles instead of 40), then across the warps through shared memory.
+constexpr int GW_THREADS = 512, GW_PB = 4;
+
+__global__ void __launch_bounds__(GW_THREADS, 2)
+gemv_rope_wide_kernel(const bf16 *__restrict__ x, const bf16 *__restrict__ Wt, int K, bf16 *__restrict__ staging,
+                      RopeAppendArgs a) {
+  __shared__ float red[2][GW_THREADS / 32][2 * GW_PB];
+  __shared__ float res[2][2 * GW_PB];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int kv = K / 8;
+  const bool act = tid < kv;
+  const int half = a.d / 2, heads = a.h + 2 * a.h_kv;
+  const int n_pairs = heads * half;
+  const int p_lo = (int)((long long)blockIdx.x * n_pairs / gridDim.x);
+  const int p_hi = (int)((long long)(blockIdx.x + 1) * n_pairs / gridDim.x);
+  const uint4 *W4 = reinterpret_cast<const uint4 *>(Wt);
+  // the first batch of weights is requested before x
+  uint4 w[2 * GW_PB];
+  auto load_batch = [&](int p0) {
+#pragma unroll
+    for (int j = 0; j < GW_PB; j++) {
+      const int it = min(p0 + j, n_pairs - 1);
+      const int hd = it / half, i = it - hd * half;
+      const size_t n0 = (size_t)hd * a.d + i;
+      w[2 * j] = act ? __ldg(W4 + n0 * kv + tid) : make_uint4(0, 0, 0, 0);
+      w[2 * j + 1] = act ? __ldg(W4 + (n0 + half) * kv + tid) : make_uint4(0, 0, 0, 0);
+    }
+  };
+  load_batch(p_lo);
+  const uint4 xv = act ? __ldg(reinterpret_cast<const uint4 *>(x) + tid) : make_uint4(0, 0, 0, 0);
+  int par = 0;
+  for (int p0 = p_lo; p0 < p_hi; p0 += GW_PB, par ^= 1) {
+    float v[2 * GW_PB];
+#pragma unroll
+    for (int e = 0; e < 2 * GW_PB; e++) v[e] = dot8(w[e], xv);
+    if (p0 + GW_PB < p_hi) load_batch(p0 + GW_PB);  // in flight during the reduction
+    // eight values across 32 lanes: exchange half of them at each of three steps
+#pragma unroll
+    for (int e = 0; e < 4; e++) {
+      const float send = (lane & 16) ? v[e] : v[e + 4], keep = (lane & 16) ? v[e + 4] : v[e];
+      v[e] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+    }
+#pragma unroll
+    for (int e = 0; e < 2; e++) {
+      const float send = (lane & 8) ? v[e] : v[e + 2], keep = (lane & 8) ? v[e + 2] : v[e];
+      v[e] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+    }
+    {
+      const float send = (lane & 4) ? v[0] : v[1], keep = (lane & 4) ? v[1] : v[0];
+      v[0] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+    }
+    v[0] += __shfl_xor_sync(0xffffffffu, v[0], 2);
+    v[0] += __shfl_xor_sync(0xffffffffu, v[0], 1);
+    if ((lane & 3) == 0) red[par][warp][((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1)] = v[0];
+    __syncthreads();
+    if (tid < 2 * GW_PB) {
+      float t = 0.f;
+#pragma unroll
+      for (int q = 0; q < GW_THREADS / 32; q++) t += red[par][q][tid];
+      res[par][tid] = t;
+    }
+    __syncthreads();
+    if (tid < GW_PB && p0 + tid < p_hi) {
+      const int it = p0 + tid;
+      const int hd = it / half, i = it - hd * half;
+      const int n0 = hd * a.d + i, n1 = n0 + half;
+      const bf16 b0 = __float2bfloat16_rn(res[par][2 * tid]), b1 = __float2bfloat16_rn(res[par][2 * tid + 1]);
+      staging[n0] = b0;
+      staging[n1] = b1;
+      const int slot = a.len;
+      if (hd < a.h + a.h_kv) {
+        const float2 t = a.cs[(size_t)slot * half + i];
+        const float x0 = __bfloat162float(b0), x1 = __bfloat162float(b1);
+        const bf16 q0 = __float2bfloat16_rn(x0 * t.x - x1 * t.y), q1 = __float2bfloat16_rn(x1 * t.x + x0 * t.y);
+        if (hd < a.h) {
+          a.q_rot[n0] = q0;
+          a.q_rot[n1] = q1;
+        } else {
+          const int m = hd - a.h;
+          const size_t off = ((size_t)m * a.cap + slot) * a.d + i;
+          if (a.k_pre) { a.k_pre[off] = b0; a.k_pre[off + half] = b1; }  // null for a 4-bit cache
+          a.k_rot[off] = q0;
+          a.k_rot[off + half] = q1;
+          if (i == 0) a.tid[(size_t)m * a.cap + slot] = a.seen;
+        }
+        if (a.z_post) { a.z_post[n0] = q0; a.z_post[n1] = q1; }
+      } else {
+        const int m = hd - a.h - a.h_kv;
+        const size_t off = ((size_t)m * a.cap + slot) * a.d + i;
+        a.v[off] = b0;
+        a.v[off + half] = b1;
+        if (a.z_post) { a.z_post[n0] = b0; a.z_post[n1] = b1; }
+      }
+    }
+  }
+}
+
 // 4-bit codes -> floats, the arithmetic of the cache's expansion pre-pass (two codes per byte, even
 // element in the low nibble, value = code * scale)
 __device__ __forceinline__ void dequant8(uint32_t w, float s, float (&x)[8]) {
@@ -430,47 +532,49 @@ attn_decode_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_ro
     sl[i][s2] = __ldcg(part_ml + hs * 2 + 1);
   }
   __syncthreads();
-  if (tid < gh) {  // weights of the splits of head tid
+  // weights of the splits: one warp per head at a time, the splits across its lanes
+  for (int i = warp; i < gh; i += DA_THREADS / 32) {
     float mx = -INFINITY;
-    for (int s2 = 0; s2 < n_splits; s2++) mx = fmaxf(mx, sm[tid][s2]);
+    for (int s2 = lane; s2 < n_splits; s2 += 32) mx = fmaxf(mx, sm[i][s2]);
+#pragma unroll
+    for (int o2 = 16; o2 > 0; o2 >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o2));
     float l = 0.f;
-    for (int s2 = 0; s2 < n_splits; s2++) {
-      const float ms = sm[tid][s2];
+    for (int s2 = lane; s2 < n_splits; s2 += 32) {
+      const float ms = sm[i][s2];
       const float w = (ms == -INFINITY) ? 0.f : exp2f(ms - mx);
-      l += w * sl[tid][s2];
-      sm[tid][s2] = w;
+      l = fmaf(w, sl[i][s2], l);
+      sm[i][s2] = w;
     }
-    sinv[tid] = 1.0f / l;
+    // (fixed order of the partial sums: lanes, then the butterfly)
+#pragma unroll
+    for (int o2 = 16; o2 > 0; o2 >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o2);
+    if (lane == 0) sinv[i] = 1.0f / l;
   }
   __syncthreads();
-  // thread = (head, column) items, four at a time with eight splits each in flight
-  for (int base = 0; base < gh * D; base += 4 * DA_THREADS) {
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    int hi[4];
-    const float *po[4];
+  // thread = (head, four columns); sixteen splits in flight as 16-byte loads
+  for (int item = tid; item < gh * (D / 4); item += DA_THREADS) {
+    const int i = item / (D / 4), c = (item - i * (D / 4)) * 4;
+    const float *po = part_o + (size_t)(h0 + i) * n_splits * D + c;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s2 = 0; s2 < n_splits; s2 += 16) {
+      float4 a[16];
 #pragma unroll
-    for (int t = 0; t < 4; t++) {
-      const int idx = min(base + t * DA_THREADS + tid, gh * D - 1);
-      hi[t] = idx / D;
-      po[t] = part_o + (size_t)(h0 + hi[t]) * n_splits * D + (idx - hi[t] * D);
+      for (int u = 0; u < 16; u++)
+        a[u] = (s2 + u < n_splits) ? __ldcg(reinterpret_cast<const float4 *>(po + (size_t)(s2 + u) * D))
+                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int u = 0; u < 16; u++)
+        if (s2 + u < n_splits) {
+          const float w = sm[i][s2 + u];
+          acc.x = fmaf(w, a[u].x, acc.x); acc.y = fmaf(w, a[u].y, acc.y);
+          acc.z = fmaf(w, a[u].z, acc.z); acc.w = fmaf(w, a[u].w, acc.w);
+        }
     }
-    for (int s2 = 0; s2 < n_splits; s2 += 8) {
-      float a[4][8];
-#pragma unroll
-      for (int t = 0; t < 4; t++)
-#pragma unroll
-        for (int u = 0; u < 8; u++) a[t][u] = (s2 + u < n_splits) ? __ldcg(po[t] + (size_t)(s2 + u) * D) : 0.f;
-#pragma unroll
-      for (int t = 0; t < 4; t++)
-#pragma unroll
-        for (int u = 0; u < 8; u++)
-          if (s2 + u < n_splits) acc[t] = fmaf(sm[hi[t]][s2 + u], a[t][u], acc[t]);
-    }
-#pragma unroll
-    for (int t = 0; t < 4; t++) {
-      const int idx = base + t * DA_THREADS + tid;
-      if (idx < gh * D) out[(size_t)(h0 + hi[t]) * D + (idx - hi[t] * D)] = __float2bfloat16_rn(acc[t] * sinv[hi[t]]);
-    }
+    const float inv = sinv[i];
+    uint2 o2;
+    o2.x = pack_bf16(acc.x * inv, acc.y * inv);
+    o2.y = pack_bf16(acc.z * inv, acc.w * inv);
+    *reinterpret_cast<uint2 *>(out + (size_t)(h0 + i) * D + c) = o2;
   }
 }
 
@@ -535,6 +639,11 @@ cudaError_t launch_gemv_rope(const bf16 *x, const bf16 *Wt, int K, bf16 *staging
                              cudaStream_t st) {
   if (K % 8 || a.d % 2) return cudaErrorInvalidValue;
   const int items = (a.h + 2 * a.h_kv) * (a.d / 2);
+  if (K / 8 <= GW_THREADS) {
+    const int blocks = min((items + GW_PB - 1) / GW_PB, 148 * 2);
+    gemv_rope_wide_kernel<<<blocks, GW_THREADS, 0, st>>>(x, Wt, K, staging, a);
+    return cudaGetLastError();
+  }
   const int blocks = min((items + 7) / 8, 148 * 4);
   gemv_rope_kernel<<<blocks, GV_THREADS, K * 2, st>>>(x, Wt, K, staging, a);
   return cudaGetLastError();
