@@ -135,12 +135,14 @@ int locret_decode_step(locret_layer *layer, const void *hidden_in, void *attn_ou
  *
  * locret_prefill_chunk_tp_begin: steps (a), (b) as in locret_prefill_chunk for the local heads
  *   (attn_out: device bf16 [n_tok x h_local·d]), then preact_partial (device fp32
- *   [n_tok x d_R], 16-byte aligned, caller-owned) = z_local · W1_local.  Every kernel runs on the
- *   layer's stream.  The caller sums preact_partial over the GPUs on that stream (an all-reduce)
- *   and passes the sum to
+ *   [n_tok x d_R], 16-byte aligned, caller-owned) = z_local · W1_local.  Work enqueued on the
+ *   layer's stream after the call returns sees the finished product.  The caller sums
+ *   preact_partial over the GPUs on that stream (an all-reduce) and passes the sum to
  * locret_prefill_chunk_tp_finish: scores = act(preact_sum) · W2_local for the chunk's units, then
  *   step (d) as in locret_prefill_chunk (with the flags given to _begin).  preact_sum may be the
- *   buffer given to _begin.
+ *   buffer given to _begin.  It is read asynchronously (what was enqueued on the layer's stream
+ *   before the call is seen): leave it unchanged until this layer's next call or
+ *   locret_sync_status.
  * Between the two calls the layer accepts no other step (LOCRET_ERR_INVALID); locret_reset
  * abandons a begun step.  _finish without _begin returns LOCRET_ERR_INVALID.
  */

@@ -92,7 +92,7 @@ struct locret_layer {
   bool tp_pending;  // a divided-heads step was begun and waits for the summed product
   int tp_n_tok;
   uint32_t tp_flags;
-  cudaEvent_t ev_ready, ev_attn, ev_side;
+  cudaEvent_t ev_ready, ev_attn, ev_side, ev_tp;  // ev_tp: the divided-heads exchange (both directions)
   bool tc_attn;  // tensor maps for the tcgen05 attention kernel are valid
   CUtensorMap map_k, map_v[2], map_q;
   const void *map_q_base;
@@ -111,6 +111,7 @@ void free_layer_memory(locret_layer *L) {
   cudaFree(L->k_rot); cudaFree(L->d_status);
   for (auto &e : L->events) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
   if (L->ev_ready) cudaEventDestroy(L->ev_ready);
+  if (L->ev_tp) cudaEventDestroy(L->ev_tp);
   if (L->ev_attn) cudaEventDestroy(L->ev_attn);
   if (L->ev_side) cudaEventDestroy(L->ev_side);
   cudaGetLastError();
@@ -244,7 +245,7 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
     const char *unf = getenv("LOCRET_UNFUSED_ROPE");
     L->fuse_rope = !(unf && unf[0] == '1');
     L->side_pending = false;
-    L->ev_ready = L->ev_attn = L->ev_side = nullptr;
+    L->ev_ready = L->ev_attn = L->ev_side = L->ev_tp = nullptr;
   }
 
   L->int4 = cfg->kv_dtype == 1;
@@ -331,7 +332,8 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   if (L->use_side) {
     ok = cudaEventCreateWithFlags(&L->ev_ready, cudaEventDisableTiming) == cudaSuccess &&
          cudaEventCreateWithFlags(&L->ev_attn, cudaEventDisableTiming) == cudaSuccess &&
-         cudaEventCreateWithFlags(&L->ev_side, cudaEventDisableTiming) == cudaSuccess;
+         cudaEventCreateWithFlags(&L->ev_side, cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&L->ev_tp, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) { cudaGetLastError(); ScratchPool *p = L->pool; free_layer_memory(L); delete L; release_pool(p); return LOCRET_ERR_CUDA; }
   }
 
@@ -437,7 +439,7 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
   const int c = L->cur;
   const bool tp = tp_partial != nullptr;
   const bool decode = n_tok == 1 && L->use_tc && !tp;  // one token: bandwidth-bound kernels of decode.cu
-  const bool side = L->use_side && !L->serialize && !tp;
+  const bool side = L->use_side && !L->serialize;
   cudaStream_t S = side ? P->side : L->st;  // stream of the off-critical-path kernels
   const int sb = P->flip;                    // staging buffer of this call
   P->flip ^= 1;
@@ -522,14 +524,28 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
                               L->d, L->cap, L->len, L->st));
   }
   if (tp) {
-    // this GPU's columns of z times its rows of W1; the caller sums the products of all GPUs
-    Timed t(L, LOCRET_K_RH);
-    const bf16 *z = L->cfg.rh_input == 1 ? z_post : staging;
-    if (L->use_tc && gemm_tc_supported(n_tok, L->d_R, L->d_in, L->d_in, L->d_in))
-      CK(launch_gemm_tc_f32(z, L->d_in, L->w1_t, L->d_in, tp_partial, L->d_R, n_tok, L->d_R, L->d_in,
-                            L->d_status, L->st));
-    else
-      CK(launch_preact_naive(z, L->w1_t, tp_partial, n_tok, L->d_R, L->d_in, L->st));
+    // this GPU's columns of z times its rows of W1; the caller sums the products of all GPUs.
+    // Like the retaining head of the undivided step it runs beside the attention kernel; the
+    // layer's stream then waits for it, because the caller's all-reduce is enqueued there.
+    if (side) {
+      CK(cudaEventRecord(L->ev_attn, L->st));
+      CK(cudaStreamWaitEvent(S, L->ev_ready, 0));
+    }
+    {
+      Timed t(L, LOCRET_K_RH, S);
+      const bf16 *z = L->cfg.rh_input == 1 ? z_post : staging;
+      if (L->use_tc && gemm_tc_supported(n_tok, L->d_R, L->d_in, L->d_in, L->d_in))
+        CK(launch_gemm_tc_f32(z, L->d_in, L->w1_t, L->d_in, tp_partial, L->d_R, n_tok, L->d_R, L->d_in,
+                              L->d_status, S));
+      else
+        CK(launch_preact_naive(z, L->w1_t, tp_partial, n_tok, L->d_R, L->d_in, S));
+    }
+    if (side) {
+      CK(cudaEventRecord(P->ev_stage_free[sb], S));
+      P->stage_busy[sb] = true;
+      CK(cudaEventRecord(L->ev_tp, S));
+      CK(cudaStreamWaitEvent(L->st, L->ev_tp, 0));
+    }
     L->tp_pending = true;
     L->tp_n_tok = n_tok;
     L->tp_flags = flags;
@@ -584,12 +600,19 @@ int locret_prefill_chunk_tp_finish(locret_layer *L, const float *preact_sum) {
   if (!L->tp_pending) return LOCRET_ERR_INVALID;
   L->tp_pending = false;
   const int n_tok = L->tp_n_tok;
-  {  // (c) finished: activation and this GPU's columns of W2, into the score cache
-    Timed t(L, LOCRET_K_RH_REDUCE);
-    CK(launch_rh_finish(preact_sum, L->w2f, L->s[L->cur], L->cap, L->len, n_tok, L->d_R, L->h_kv, L->cfg.act,
-                        L->st));
+  // nothing downstream in a decoder layer waits for the scores, the selection or the compaction: they
+  // go to the second stream, after the summed product has arrived on the layer's stream
+  const bool side = L->use_side && !L->serialize;
+  cudaStream_t S = side ? L->pool->side : L->st;
+  if (side) {
+    CK(cudaEventRecord(L->ev_tp, L->st));
+    CK(cudaStreamWaitEvent(S, L->ev_tp, 0));
   }
-  return evict_and_close(L, n_tok, L->tp_flags, false, L->st);
+  {  // (c) finished: activation and this GPU's columns of W2, into the score cache
+    Timed t(L, LOCRET_K_RH_REDUCE, S);
+    CK(launch_rh_finish(preact_sum, L->w2f, L->s[L->cur], L->cap, L->len, n_tok, L->d_R, L->h_kv, L->cfg.act, S));
+  }
+  return evict_and_close(L, n_tok, L->tp_flags, side, S);
 }
 
 int locret_decode_step(locret_layer *L, const void *hidden_in, void *attn_out) {
