@@ -27,6 +27,9 @@ struct ScratchPool {
   // layer's projection.  staging / z_post are double-buffered because that work reads them.
   cudaStream_t side = nullptr;
   cudaEvent_t ev_stage_free[2] = {nullptr, nullptr};
+  // 4-bit caches: the bf16 expansion is written on the second stream while the projection runs
+  cudaEvent_t ev_exp_free = nullptr, ev_exp_ready = nullptr;
+  bool exp_busy = false;  // ev_exp_free recorded and not yet waited for
   bool stage_busy[2] = {false, false};  // recorded and not yet waited for
   int flip = 0;
   size_t staging_b[2] = {0, 0}, qrot_b = 0, zpost_b[2] = {0, 0}, partial_b = 0, keep_b = 0, kexp_b = 0, vexp_b = 0;
@@ -126,6 +129,8 @@ void release_pool(ScratchPool *p) {
     cudaFree(p->staging[i]); cudaFree(p->z_post[i]);
     if (p->ev_stage_free[i]) cudaEventDestroy(p->ev_stage_free[i]);
   }
+  if (p->ev_exp_free) cudaEventDestroy(p->ev_exp_free);
+  if (p->ev_exp_ready) cudaEventDestroy(p->ev_exp_ready);
   cudaFree(p->q_rot); cudaFree(p->partial); cudaFree(p->keep); cudaFree(p->dec_o); cudaFree(p->dec_ml); cudaFree(p->dec_cnt);
   cudaFree(p->k_exp); cudaFree(p->v_exp);
   for (auto &t : p->cs) cudaFree(t.ptr);
@@ -290,6 +295,8 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
         g = g && cudaStreamCreateWithPriority(&p->side, cudaStreamNonBlocking, lo) == cudaSuccess;
         for (int i = 0; i < 2 && g; i++)
           g = cudaEventCreateWithFlags(&p->ev_stage_free[i], cudaEventDisableTiming) == cudaSuccess;
+        g = g && cudaEventCreateWithFlags(&p->ev_exp_free, cudaEventDisableTiming) == cudaSuccess &&
+            cudaEventCreateWithFlags(&p->ev_exp_ready, cudaEventDisableTiming) == cudaSuccess;
       }
       if (g && !p->dec_cnt) {
         g = cudaMalloc(&p->dec_cnt, DEC_CNT_WORDS * sizeof(unsigned)) == cudaSuccess &&
@@ -466,11 +473,18 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
   // with a tensor-core projection and head_dim 64 / 128 the epilogue of the GEMM does the RoPE pass
   const bool fused_rope = !decode && L->fuse_rope && L->use_tc && n_tok >= 32 &&
                           qkv_rope_tc_supported(n_tok, L->d_in, L->D, L->D, L->D, L->d);
-  if (L->int4 && L->len > 0 && !decode) {
+  const bool deq = L->int4 && L->len > 0 && !decode;
+  if (deq) {
     // the expansion writes slots [0, len) of the scratch the chunk's units are appended to
-    // (a one-token step reads the codes inside its attention kernel instead)
-    Timed t(L, LOCRET_K_DEQUANT);
-    CK(launch_dequant(L->q4[c], P->k_exp, P->v_exp, L->cs, L->h_kv, L->d, L->cap, L->len, true, L->st));
+    // (a one-token step reads the codes inside its attention kernel instead).  Only attention
+    // reads it, so it runs on the second stream beside the projection; the scratch is free once
+    // the attention kernel that read it last has finished.
+    if (side && P->exp_busy) { CK(cudaStreamWaitEvent(S, P->ev_exp_free, 0)); P->exp_busy = false; }
+    {
+      Timed t(L, LOCRET_K_DEQUANT, S);
+      CK(launch_dequant(L->q4[c], P->k_exp, P->v_exp, L->cs, L->h_kv, L->d, L->cap, L->len, true, S));
+    }
+    if (side) CK(cudaEventRecord(P->ev_exp_ready, S));
   }
   {  // (a) projections
     Timed t(L, LOCRET_K_QKV);
@@ -490,12 +504,17 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
     Timed t(L, LOCRET_K_ROPE);
     CK(launch_rope_append(ra, L->st));
   }
-  if (L->int4) {  // the chunk's units enter the cache quantised (keys pre-RoPE)
-    Timed t(L, LOCRET_K_QUANT);
+  auto quantize_chunk = [&](cudaStream_t R) -> int {  // the chunk's units enter the cache quantised (keys pre-RoPE)
+    Timed t(L, LOCRET_K_QUANT, R);
     const bf16 *ks = staging + (size_t)L->h * L->d, *vs = ks + (size_t)L->h_kv * L->d;
-    CK(launch_quantize(ks, vs, L->d_in, L->d, L->q4[c], n_tok, L->h_kv, L->d, L->cap, L->len, L->st));
-  }
+    CK(launch_quantize(ks, vs, L->d_in, L->d, L->q4[c], n_tok, L->h_kv, L->d, L->cap, L->len, R));
+    return LOCRET_OK;
+  };
+  // the codes are read by the compaction of this step and by later steps, never by this step's
+  // attention (the chunk attends to its own keys and values in bf16): second stream
+  if (L->int4 && !side) { const int rc = quantize_chunk(L->st); if (rc != LOCRET_OK) return rc; }
   if (side) CK(cudaEventRecord(L->ev_ready, L->st));
+  if (side && deq) CK(cudaStreamWaitEvent(L->st, P->ev_exp_ready, 0));
   {  // (b) Eq. 1
     Timed t(L, LOCRET_K_ATTN);
     bool tc_ok = L->tc_attn && attention_tc_supported(n_tok, L->h, L->h_kv, L->d);
@@ -523,6 +542,10 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
       CK(launch_attention_mma(P->q_rot, k_att, v_att, (bf16 *)attn_out, n_tok, L->h, L->h_kv,
                               L->d, L->cap, L->len, L->st));
   }
+  if (side && L->int4) {  // the attention kernel just launched is the scratch's last reader (a one-token step reads its own token there)
+    CK(cudaEventRecord(P->ev_exp_free, L->st));
+    P->exp_busy = true;
+  }
   if (tp) {
     // this GPU's columns of z times its rows of W1; the caller sums the products of all GPUs.
     // Like the retaining head of the undivided step it runs beside the attention kernel; the
@@ -530,6 +553,7 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
     if (side) {
       CK(cudaEventRecord(L->ev_attn, L->st));
       CK(cudaStreamWaitEvent(S, L->ev_ready, 0));
+      if (L->int4) { const int rc = quantize_chunk(S); if (rc != LOCRET_OK) return rc; }
     }
     {
       Timed t(L, LOCRET_K_RH, S);
@@ -554,6 +578,7 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
   if (side) {
     CK(cudaEventRecord(L->ev_attn, L->st));
     CK(cudaStreamWaitEvent(S, L->ev_ready, 0));
+    if (L->int4) { const int rc = quantize_chunk(S); if (rc != LOCRET_OK) return rc; }
   }
   int n_tiles = 0;
   {  // (c) retaining head: launched after the attention kernel, so its CTAs fill that kernel's tail
