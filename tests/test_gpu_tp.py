@@ -52,6 +52,11 @@ class ShardsOnOneGpu:
             sl = slice(r * self.hkl, (r + 1) * self.hkl)
             L.import_state(K[sl], V[sl], S[sl], T[sl], seen)
 
+    def import_state_int4(self, Kc, Ks, Vc, Vs, S, T, seen):
+        for r, L in enumerate(self.layers):
+            sl = slice(r * self.hkl, (r + 1) * self.hkl)
+            L.import_state_int4(Kc[sl], Ks[sl], Vc[sl], Vs[sl], S[sl], T[sl], seen)
+
     @property
     def cache_len(self):
         lens = {L.cache_len for L in self.layers}
@@ -87,6 +92,20 @@ def test_divided_heads_lockstep_with_the_undivided_oracle(world, h, hk, d):
         st = lockstep_chunk(ora, gpu, x, 0, what=f"tp{world} chunk {i}")
         exact += bool(st.get("sets_identical", True))
     assert ora.len == 300 and exact >= len(sizes) - 1
+    gpu.destroy()
+
+
+def test_divided_heads_with_the_4bit_cache():
+    from parity_util import lockstep_chunk
+    sh = W.LayerShape(d_model=128, n_q_heads=8, n_kv_heads=4, head_dim=128, d_retain=96, kv_dtype=1)
+    weights = W.layer_weights(sh, 0, seed=W.BASE_SEED + 930)
+    ora = oracle_for(sh, weights, 300, 200, 17)
+    gpu = ShardsOnOneGpu(sh, weights, 300, 200, 17, 2)
+    g = np.random.default_rng(31)
+    for i, n_tok in enumerate([200, 130, 200, 1, 64]):
+        x = W.to_bf16_grid(g.standard_normal((n_tok, sh.d_model)).astype(np.float32))
+        lockstep_chunk(ora, gpu, x, 0, what=f"tp2 int4 chunk {i}")
+    assert ora.len == 300
     gpu.destroy()
 
 
