@@ -56,10 +56,10 @@ extern "C" {
 
 /* kernel families, indices into locret_read_timing's arrays */
 enum {
-  LOCRET_K_QKV = 0,     /* (a) projection GEMM (head_dim 64 / 128 and one-token   */
-                        /*     steps: positions, RoPE and append in the same kernel) */
+  LOCRET_K_QKV = 0,     /* (a) projection GEMM (positions, RoPE and append in the   */
+                        /*     same kernel)                                        */
   LOCRET_K_ROPE,        /* position assignment + RoPE + append of the chunk, where */
-                        /*     it is a kernel of its own (head_dim 96, fallbacks)  */
+                        /*     it is a kernel of its own (fallback shapes)         */
   LOCRET_K_ATTN,        /* (b) attention                                          */
   LOCRET_K_RH,          /* (c) retaining head GEMM -> activation -> GEMM          */
   LOCRET_K_RH_REDUCE,   /* (c) sum of the retaining head's partial scores (a      */

@@ -77,7 +77,8 @@ __device__ __forceinline__ float fast_act(float x, int act) {
 
 template <int BN>
 struct GemmCfg {
-  static constexpr int STAGES = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
+  static constexpr int STAGES = BN >= 192 ? 4 : (BN == 128 ? 6 : 8);
+  static constexpr int TMEM_COLS = BN == 192 ? 512 : 2 * BN;  // two accumulators; a power of two
   static constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int W2_BYTES = BN * MAX_HKV * 4;
@@ -135,7 +136,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     prefetch_tmap(&map_b);
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, 2 * BN);
+    tmem_alloc(tmem_slot, Cfg::TMEM_COLS);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -334,7 +335,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // shared memory (16-byte pieces XOR-swizzled by row) and writes them out as whole rows,
         // so the global stores are full lines.
         if (ok) {
-          constexpr int HALF = HD / 2, VPR = HD / 8, VMASK = VPR - 1, ROW_B = HD * 2;
+          // 16-byte pieces of a staged row: XOR-swizzled by row when their number is a power of
+          // two, else rows padded by one piece (an odd stride in pieces spreads the banks as well)
+          constexpr int HALF = HD / 2, VPR = HD / 8, VMASK = VPR - 1;
+          constexpr bool POW2 = (VPR & (VPR - 1)) == 0;
+          constexpr int ROW_B = POW2 ? HD * 2 : HD * 2 + 16;
+          auto piece = [&](int j, int r) { return POW2 ? ((j ^ (r & VMASK)) << 4) : (j << 4); };
           const int d_in = (ra.h + 2 * ra.h_kv) * HD;
           const int wrow0 = m0 + quarter * 32;  // first row of this warp
           unsigned char *buf_w = sEpi + quarter * EPI_WARP_BYTES;
@@ -346,7 +352,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               const int idx = lane + 32 * i, r = idx / VPR, j = idx % VPR;
               if (wrow0 + r < M)
                 *reinterpret_cast<uint4 *>(dst + (size_t)r * stride + j * 8) =
-                    *reinterpret_cast<const uint4 *>(buf_w + r * ROW_B + ((j ^ (r & VMASK)) << 4));
+                    *reinterpret_cast<const uint4 *>(buf_w + r * ROW_B + piece(j, r));
             }
           };
 #pragma unroll 1
@@ -370,7 +376,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 o.y = pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
                 o.z = pack_bf16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]));
                 o.w = pack_bf16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]));
-                *reinterpret_cast<uint4 *>(my_row + ((((c0 >> 3) + v) ^ (lane & VMASK)) << 4)) = o;
+                *reinterpret_cast<uint4 *>(my_row + piece((c0 >> 3) + v, lane)) = o;
               }
             }
             __syncwarp();
@@ -392,6 +398,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               tmem_wait_ld();
 #pragma unroll
               for (int v = 0; v < 4; v++) {
+                if (c0 + 8 * v >= HALF) break;  // head_dim 96: the second load holds 16 columns of the half
                 uint32_t ol[4], oh[4];
 #pragma unroll
                 for (int q = 0; q < 4; q++) {
@@ -405,8 +412,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                   oh[q] = pack_bf16(y0 * t.x + x0 * t.y, y1 * t.z + x1 * t.w);
                 }
                 const int jl = (c0 >> 3) + v, jh = jl + (HALF >> 3);
-                *reinterpret_cast<uint4 *>(my_row + ((jl ^ (lane & VMASK)) << 4)) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
-                *reinterpret_cast<uint4 *>(my_row + ((jh ^ (lane & VMASK)) << 4)) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
+                *reinterpret_cast<uint4 *>(my_row + piece(jl, lane)) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+                *reinterpret_cast<uint4 *>(my_row + piece(jh, lane)) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
               }
             }
             __syncwarp();
@@ -488,7 +495,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   tc_fence_after();
   if (warp == 1) {
     __syncwarp();
-    tmem_dealloc(tmem_base, 2 * BN);
+    tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
   }
 }
 
@@ -613,11 +620,14 @@ cudaError_t launch_gemm_tc_rowmax(const bf16 *A, int lda, const bf16 *Bt, int ld
 // cache (what rope_append_kernel does in a pass of its own): head_dim 64 or 128, so that a
 // 256-column tile holds whole heads.
 bool qkv_rope_tc_supported(int M, int N, int K, int lda, int ldb, int d) {
+  if (d == 96) return gemm_tc_supported(M, N, K, lda, ldb) && N % 192 == 0;
   return gemm_tc_supported(M, N, K, lda, ldb) && N >= 256 && (d == 64 || d == 128) && N % d == 0;
 }
 
 cudaError_t launch_qkv_rope_tc(const bf16 *X, int ldx, const bf16 *Wt, int ldw, bf16 *staging, int M,
                                int N, int K, const RopeAppendArgs &ra, int *status, cudaStream_t st) {
+  if (ra.d == 96)
+    return launch_t<192, 2, 96>(X, ldx, Wt, ldw, staging, N, M, N, K, nullptr, nullptr, 0, 0, ra, status, st);
   if (ra.d == 128)
     return launch_t<256, 2, 128>(X, ldx, Wt, ldw, staging, N, M, N, K, nullptr, nullptr, 0, 0, ra, status, st);
   return launch_t<256, 2, 64>(X, ldx, Wt, ldw, staging, N, M, N, K, nullptr, nullptr, 0, 0, ra, status, st);

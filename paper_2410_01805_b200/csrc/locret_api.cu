@@ -470,7 +470,7 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
   ra.k_pre = L->int4 ? nullptr : L->k_pre[c]; ra.k_rot = k_att; ra.v = v_att; ra.tid = L->tid[c]; ra.cs = L->cs;
   ra.n_tok = n_tok; ra.h = L->h; ra.h_kv = L->h_kv; ra.d = L->d; ra.cap = L->cap; ra.len = L->len;
   ra.seen = L->seen;
-  // with a tensor-core projection and head_dim 64 / 128 the epilogue of the GEMM does the RoPE pass
+  // with a tensor-core projection whose width is a whole number of tiles the epilogue of the GEMM does the RoPE pass
   const bool fused_rope = !decode && L->fuse_rope && L->use_tc && n_tok >= 32 &&
                           qkv_rope_tc_supported(n_tok, L->d_in, L->D, L->D, L->D, L->d);
   const bool deq = L->int4 && L->len > 0 && !decode;
