@@ -633,14 +633,14 @@ cudaError_t launch_qkv_rope_tc(const bf16 *X, int ldx, const bf16 *Wt, int ldw, 
   return launch_t<256, 2, 64>(X, ldx, Wt, ldw, staging, N, M, N, K, nullptr, nullptr, 0, 0, ra, status, st);
 }
 
-// Tile width of the retaining-head GEMM: the widest of 256 / 128 / 64 columns that still gives
-// about one CTA per SM (a 128 x 256 tile needs the least operand traffic per flop, but a chunk of
-// 1024 tokens and d_R = 1024 would make only 32 of them).
+// Tile width of the retaining-head GEMM: the widest of 256 / 128 / 64 columns that divides d_R.  The
+// kernel runs beside attention and the next projection, so what it costs the step is SM time, not
+// latency, and a CTA's latency is set by the length of K whatever the width (measured at 1024 tokens,
+// K = 9216: 128 / 64 / 32 CTAs for 70.6 / 76.4 / 87.7 us; the whole run is 4 % faster with the 32 wide ones).
 static int rh_tile_n(int M, int d_R) {
-  const int mt = (M + BM - 1) / BM;
-  for (int bn = 256; bn > 64; bn >>= 1)
-    if (d_R % bn == 0 && mt * (d_R / bn) >= 96) return bn;
-  return d_R % 64 == 0 ? 64 : 128;
+  (void)M;
+  if (d_R % 256 == 0) return 256;
+  return d_R % 128 == 0 ? 128 : 64;
 }
 // upper bound on the number of N-tiles (scratch sizing)
 int rh_tc_num_tiles(int d_R) { return (d_R + 63) / 64; }

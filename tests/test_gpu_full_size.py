@@ -60,6 +60,21 @@ def test_c4_phi3_shape_until_the_cache_is_full():
     assert ora.len == w.budget and "sets_identical" in stats[-1]
 
 
+def test_llama_shape_short_chunks():
+    # 512-token chunks and shorter ragged ones at the full layer width: few tiles per GEMM, a small
+    # budget that evicts from the third chunk on
+    from parity_util import lockstep_chunk, make_pair
+    w = W.get_workload("c3_llama_128k")
+    ora, gpu = make_pair(w.shape, W.layer_weights(w.shape, 3), 1024, 512, 100)
+    start = 0
+    for i, n_tok in enumerate([512, 512, 512, 300, 33]):
+        x = W.hidden_states(w, start, n_tok)
+        lockstep_chunk(ora, gpu, x, 0, rows=sampled_rows(n_tok, 40 + i), what=f"short chunk {i}")
+        start += n_tok
+    assert ora.len == 1024 and gpu.sync_status() == 0
+    gpu.destroy()
+
+
 def test_partial_last_chunk_of_the_headline_run():
     """The 128K run ends with a 2048-token chunk (shorter than the 2500 stabilizers)."""
     from parity_util import lockstep_chunk, make_pair
