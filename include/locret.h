@@ -29,7 +29,11 @@
  *     in a decoder layer waits for, on a second stream owned by the library, ordered against
  *     the first by events (set LOCRET_SERIAL=1 to keep everything on one stream).  Every call
  *     that reads or replaces state waits for both.  A handle is bound to its stream and is
- *     not thread-safe.  Layers created on the same stream share scratch.
+ *     not thread-safe.  Layers created on the same stream of the same device share scratch.
+ *   - A handle belongs to the device that was current when it was created (one process may
+ *     create layers on several devices).  Every call that takes the handle must be made with
+ *     that device current, else it returns LOCRET_ERR_INVALID and launches nothing
+ *     (locret_destroy, locret_cache_len and the other host-only calls work from any device).
  *   - There is no CPU fallback: without a CUDA device every call that needs one
  *     returns LOCRET_ERR_CUDA.
  */
@@ -197,7 +201,22 @@ int locret_sync_status(locret_layer *layer);
  */
 int locret_selftest_wait_timeout(void *stream);
 
-/* Forget all units: len = 0, tokens_seen = 0.  Asynchronous. */
+/*
+ * Self-test of the give-up path of the production wait itself (the routine every tcgen05 kernel
+ * of the library polls its mbarriers with).  Two warps of one CTA wait on barriers nothing ever
+ * arrives at: warp 0 with a limit of a few thousand polls, warp 1 with the production limit.
+ * Warp 0 gives up, sets the CTA's abort flag and the status word; warp 1 must notice the flag
+ * and stop long before its own limit.  report (HOST, 4 x int64): [0] the status word the kernel
+ * left (expected LOCRET_ERR_DEVICE_TIMEOUT), [1] 1 if warp 1's wait returned "abandoned",
+ * [2] clock cycles warp 0 waited, [3] clock cycles warp 1 waited.  Returns 0, or
+ * LOCRET_ERR_ALLOC / LOCRET_ERR_CUDA.  Nothing faults, traps or hangs; the context stays usable.
+ * Synchronises `stream`.
+ */
+int locret_selftest_wait_abort(void *stream, int64_t *report);
+
+/* Forget all units: len = 0, tokens_seen = 0.  Asynchronous: nothing is launched; the layer's
+ * stream is ordered behind any selection / compaction of this layer still in flight on the
+ * library's second stream, so work enqueued after the reset finds the cache quiescent. */
 int locret_reset(locret_layer *layer);
 
 /*
@@ -339,6 +358,9 @@ int locret_adamw_step(float *param, void *param_bf16, const float *grad, float *
  * LOCRET_STATIC_SCRATCH_FLOATS floats (4 MiB, present on every GPU that loads the library until
  * the process exits); a call needs ceil(d_retain / 64) * n_tok * n_kv_heads of them and returns
  * LOCRET_ERR_CAPACITY, launching nothing, if that is more.
+ * status: device int32 that receives LOCRET_ERR_DEVICE_TIMEOUT if a bounded wait inside the kernel
+ * gives up (the caller clears and reads it), or NULL: then such a give-up goes unreported and the
+ * scores of that call are garbage.
  * The call makes no cudaMalloc/cudaFree and uses no allocating library routine.  Its first call on
  * a device looks up the array's device address (cudaGetSymbolAddress, with that device current);
  * make that first call outside of any stream capture.  All calls share the one array, which
@@ -349,7 +371,7 @@ int locret_adamw_step(float *param, void *param_bf16, const float *grad, float *
 #define LOCRET_STATIC_SCRATCH_FLOATS (1 << 20)
 int locret_rh_scores_static(const void *z, int32_t n_tok, int32_t d_in, const void *w1_t,
                             int32_t d_retain, const float *w2, int32_t n_kv_heads, int32_t act,
-                            float *scores, void *stream);
+                            float *scores, int32_t *status, void *stream);
 
 /* Free everything the layer owns.  Synchronises the stream.  NULL is allowed. */
 void locret_destroy(locret_layer *layer);

@@ -184,13 +184,8 @@ template <int D>
 cudaError_t launch_d(const bf16 *q_rot, const bf16 *k_rot, const bf16 *v, bf16 *out, int n_tok, int h,
                      int h_kv, int cap, int len, cudaStream_t st) {
   constexpr int smem = (QT + 4 * KT_) * (D + 8) * 2;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attn_mma_kernel<D>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static PerDeviceFlag attr_set;
+  if (cudaError_t e = allow_dynamic_smem(attn_mma_kernel<D>, smem, attr_set); e != cudaSuccess) return e;
   dim3 grid((n_tok + QT - 1) / QT, h);
   float scale_log2 = 1.4426950408889634f / sqrtf((float)D);
   attn_mma_kernel<D><<<grid, ATHREADS, smem, st>>>(q_rot, k_rot, v, out, n_tok, h, h_kv, cap, len,

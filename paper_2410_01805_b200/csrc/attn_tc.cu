@@ -428,13 +428,8 @@ bool attention_tc_supported(int n_tok, int h, int h_kv, int d) {
 template <int D>
 static cudaError_t launch_attn_d(const CUtensorMap *map_q, const CUtensorMap *map_k, const CUtensorMap *map_v,
                                  const AttnParams &p, int grid, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         AT_SMEM);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static PerDeviceFlag attr_set;
+  if (cudaError_t e = allow_dynamic_smem(attn_tc_kernel<D>, AT_SMEM, attr_set); e != cudaSuccess) return e;
   attn_tc_kernel<D><<<grid, AT_THREADS, AT_SMEM, st>>>(*map_q, *map_k, *map_v, p);
   return cudaGetLastError();
 }

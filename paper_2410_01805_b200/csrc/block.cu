@@ -112,7 +112,8 @@ struct BlockScratch {
   size_t h_b = 0, att_b = 0, x1_b = 0, act_b = 0, gu_b = 0;
 };
 std::mutex b_mu;
-std::map<cudaStream_t, BlockScratch *> b_pools;
+// keyed by (device, stream): the default stream has the same handle on every device
+std::map<std::pair<int, cudaStream_t>, BlockScratch *> b_pools;
 
 bool grow_b(void **p, size_t *have, size_t want, cudaStream_t st) {
   if (want <= *have) return true;
@@ -134,6 +135,7 @@ struct locret_block {
   bf16 *wo_t, *wgu_t, *wd_t, *g1, *g2;  // repacked: [D x hd], [2F x D] gated layout, [D x F]
   int *d_status;
   BlockScratch *pool;
+  int device;
 };
 
 #define BCK(call)                                                            \
@@ -154,7 +156,7 @@ void locret_block_destroy(locret_block *B) {
     if (--B->pool->refs == 0) {
       BlockScratch *p = B->pool;
       cudaFree(p->h); cudaFree(p->att); cudaFree(p->x1); cudaFree(p->act); cudaFree(p->gu);
-      b_pools.erase(B->st);
+      b_pools.erase(std::make_pair(B->device, B->st));
       delete p;
     }
   }
@@ -185,7 +187,8 @@ int locret_block_create(const locret_block_cfg *cfg, int32_t budget, int32_t chu
   ok = ok && cudaMalloc(&B->d_status, sizeof(int)) == cudaSuccess;
   if (ok) {
     std::lock_guard<std::mutex> lk(b_mu);
-    BlockScratch *&p = b_pools[B->st];
+    if (cudaGetDevice(&B->device) != cudaSuccess) { cudaGetLastError(); B->device = 0; }
+    BlockScratch *&p = b_pools[std::make_pair(B->device, B->st)];
     if (!p) p = new (std::nothrow) BlockScratch();
     if (p) {
       p->refs++;

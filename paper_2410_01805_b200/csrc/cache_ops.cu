@@ -338,13 +338,8 @@ cudaError_t launch_topk(const float *scores, int score_stride, int h_kv, int n, 
   const int rest = n - n_prot;
   const size_t bytes = (size_t)rest * 4;
   const size_t max_dyn = 200 * 1024;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)max_dyn);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static PerDeviceFlag attr_set;
+  if (cudaError_t e = allow_dynamic_smem(topk_kernel, (int)max_dyn, attr_set); e != cudaSuccess) return e;
   int use_smem = bytes <= max_dyn;
   topk_kernel<<<h_kv, TK_THREADS, use_smem ? bytes : 0, st>>>(scores, score_stride, n, budget, n_prot,
                                                               n_pre, keep, use_smem);

@@ -67,6 +67,46 @@ __device__ __forceinline__ float apply_act(float x, int act) {
   return fmaxf(x, 0.0f);                         // ReLU
 }
 
+// ---------------------------------------------------------------- per-device launch state (host)
+// cudaFuncSetAttribute acts on the current device only, so "already done" is remembered per
+// device: one process may drive several GPUs.
+constexpr int MAX_DEVICES = 64;
+struct PerDeviceFlag { bool done[MAX_DEVICES] = {}; };
+
+inline cudaError_t current_device_index(int *dev) {
+  cudaError_t e = cudaGetDevice(dev);
+  if (e != cudaSuccess) return e;
+  return (*dev < 0 || *dev >= MAX_DEVICES) ? cudaErrorInvalidDevice : cudaSuccess;
+}
+
+// Raise a kernel's dynamic shared-memory limit once per device.
+template <typename Kernel>
+inline cudaError_t allow_dynamic_smem(Kernel kernel, int bytes, PerDeviceFlag &flag) {
+  int dev = 0;
+  cudaError_t e = current_device_index(&dev);
+  if (e != cudaSuccess) return e;
+  if (flag.done[dev]) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) flag.done[dev] = true;
+  return e;
+}
+
+// Number of SMs of the current device (148 if it cannot be read), looked up once per device.
+inline int sm_count_of_current_device() {
+  static int count[MAX_DEVICES] = {};
+  int dev = 0;
+  if (current_device_index(&dev) != cudaSuccess) { cudaGetLastError(); return 148; }
+  if (count[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+      cudaGetLastError();
+      n = 148;
+    }
+    count[dev] = n;
+  }
+  return count[dev];
+}
+
 // ---------------------------------------------------------------- launchers (host)
 // Every launcher enqueues on `st` and returns the cudaError_t of the launch.
 

@@ -679,17 +679,13 @@ cudaError_t launch_attention_decode(const bf16 *q_rot, const bf16 *k_rot, const 
   if ((int)grid.x * (int)grid.z > 32 * 16 || n_splits > 64) return cudaErrorInvalidValue;
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)d);
   const Int4Half qq = q4 ? *q4 : Int4Half{nullptr, nullptr, nullptr, nullptr};
-  auto launch = [&](auto kern, int smem, bool &attr_set) -> cudaError_t {
-    if (!attr_set) {
-      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-      if (e != cudaSuccess) return e;
-      attr_set = true;
-    }
+  auto launch = [&](auto kern, int smem, PerDeviceFlag &attr_set) -> cudaError_t {
+    if (cudaError_t e = allow_dynamic_smem(kern, smem, attr_set); e != cudaSuccess) return e;
     kern<<<grid, DA_THREADS, smem, st>>>(q_rot, k_rot, v, part_o, part_ml, h, h_kv, cap, n, n_splits,
                                          scale_log2, counters, out, qq, cs);
     return cudaGetLastError();
   };
-  static bool set_done[2][3] = {};
+  static PerDeviceFlag set_done[2][3];
   const int qi = q4 ? 1 : 0;
   switch (d) {
     case 64:

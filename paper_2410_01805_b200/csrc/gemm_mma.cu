@@ -179,13 +179,8 @@ int rh_num_tiles(int d_R) { return (d_R + BN - 1) / BN; }
 cudaError_t launch_gemm_bf16(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, int ldc,
                              int M, int N, int K, cudaStream_t st) {
   if (K % BK != 0 || (lda % 8) || (ldb % 8)) return cudaErrorInvalidValue;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_mma_kernel<0>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, PIPE_BYTES);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static PerDeviceFlag attr_set;
+  if (cudaError_t e = allow_dynamic_smem(gemm_mma_kernel<0>, PIPE_BYTES, attr_set); e != cudaSuccess) return e;
   dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM);
   gemm_mma_kernel<0><<<grid, THREADS, PIPE_BYTES, st>>>(A, lda, Bt, ldb, C, ldc, M, N, K, nullptr,
                                                          nullptr, 0, 0);
@@ -195,14 +190,9 @@ cudaError_t launch_gemm_bf16(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf
 cudaError_t launch_rh_gemm(const bf16 *A, int lda, const bf16 *W1t, const float *W2, float *partial,
                            int M, int d_R, int K, int h_kv, int act, int *n_tiles, cudaStream_t st) {
   if (K % BK != 0 || (lda % 8) || h_kv > MAX_HKV) return cudaErrorInvalidValue;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_mma_kernel<1>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         rh_smem_bytes(MAX_HKV));
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static PerDeviceFlag attr_set;
+  if (cudaError_t e = allow_dynamic_smem(gemm_mma_kernel<1>, rh_smem_bytes(MAX_HKV), attr_set); e != cudaSuccess)
+    return e;
   dim3 grid((d_R + BN - 1) / BN, (M + BM - 1) / BM);
   *n_tiles = grid.x;
   gemm_mma_kernel<1><<<grid, THREADS, rh_smem_bytes(MAX_HKV), st>>>(

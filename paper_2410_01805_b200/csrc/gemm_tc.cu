@@ -533,26 +533,14 @@ cudaError_t launch_t(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, i
                      int K, const float *W2, float *partial, int h_kv, int act, const RopeAppendArgs &ra,
                      int *status, cudaStream_t st, const bf16 *resid = nullptr, int ldr = 0) {
   using Cfg = GemmCfg<BN>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, MODE, HD>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         Cfg::smem_bytes(MODE));
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static PerDeviceFlag attr_set;
+  if (cudaError_t e = allow_dynamic_smem(gemm_tc_kernel<BN, MODE, HD>, Cfg::smem_bytes(MODE), attr_set);
+      e != cudaSuccess)
+    return e;
   const CUtensorMap *ma = cached_map(A, K, M, (uint64_t)lda * 2, BM);
   const CUtensorMap *mb = cached_map(Bt, K, N, (uint64_t)ldb * 2, BN);
   if (!ma || !mb) return cudaErrorInvalidValue;
-  static int num_sms = 0;
-  if (num_sms == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0) {
-      cudaGetLastError();
-      num_sms = 148;
-    }
-  }
+  const int num_sms = sm_count_of_current_device();
   const int total = ((N + BN - 1) / BN) * ((M + BM - 1) / BM);
   const int grid = total < num_sms ? total : num_sms;
   // B is the larger operand: keep a B tile resident and sweep the rows (each B tile is then read

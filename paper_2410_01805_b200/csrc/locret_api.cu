@@ -21,6 +21,7 @@ namespace {
 // flight on a stream at a time).
 struct ScratchPool {
   cudaStream_t st = nullptr;
+  int device = 0;
   int refs = 0;
   // Second stream for the work that is off the critical path of a decoder layer (retaining
   // head, selection, compaction): it overlaps the tail of the attention kernel and the next
@@ -47,7 +48,8 @@ struct ScratchPool {
 };
 
 std::mutex g_mu;
-std::map<cudaStream_t, ScratchPool *> g_pools;
+// keyed by (device, stream): the default stream has the same handle on every device
+std::map<std::pair<int, cudaStream_t>, ScratchPool *> g_pools;
 
 template <typename T>
 bool grow(T **p, size_t *have, size_t want, cudaStream_t st) {
@@ -80,6 +82,7 @@ struct locret_layer {
   float *s[2];
   int64_t *tid[2];
   int cur;
+  int device;  // the device that was current at create: every later call must find it current
   const float2 *cs;
   int *d_status;
   int len;
@@ -134,7 +137,7 @@ void release_pool(ScratchPool *p) {
   cudaFree(p->q_rot); cudaFree(p->partial); cudaFree(p->keep); cudaFree(p->dec_o); cudaFree(p->dec_ml); cudaFree(p->dec_cnt);
   cudaFree(p->k_exp); cudaFree(p->v_exp);
   for (auto &t : p->cs) cudaFree(t.ptr);
-  g_pools.erase(p->st);
+  g_pools.erase(std::make_pair(p->device, p->st));
   delete p;
   cudaGetLastError();
 }
@@ -187,6 +190,13 @@ struct Timed {
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// A layer's buffers, streams and events belong to the device that was current at create.
+bool on_layer_device(const locret_layer *L) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return false; }
+  return dev == L->device;
+}
+
 // Wait for everything this layer has in flight, on both streams.
 cudaError_t sync_all(locret_layer *L) {
   cudaError_t e = cudaStreamSynchronize(L->st);
@@ -229,8 +239,9 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   const long long cap_ll = (long long)budget + chunk + cfg->reserve;
   if (cap_ll > (1ll << 24)) return LOCRET_ERR_INVALID;
 
-  int ndev = 0;
+  int ndev = 0, dev = 0;
   if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) { cudaGetLastError(); return LOCRET_ERR_CUDA; }
+  if (current_device_index(&dev) != cudaSuccess) { cudaGetLastError(); return LOCRET_ERR_CUDA; }
 
   locret_layer *L = new (std::nothrow) locret_layer();
   if (!L) return LOCRET_ERR_ALLOC;
@@ -239,6 +250,7 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   L->h = h; L->h_kv = hk; L->d = d; L->D = D; L->d_R = dR;
   L->d_in = (h + 2 * hk) * d;
   L->st = (cudaStream_t)cfg->stream;
+  L->device = dev;
   L->n_prefix = 0;
   L->cur = 0; L->len = 0; L->seen = 0; L->launches = 0; L->timing = false; L->serialize = false; L->attn_only = false; L->events_used = 0;
   L->pool = nullptr;
@@ -283,8 +295,8 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   // shared scratch
   {
     std::lock_guard<std::mutex> lk(g_mu);
-    ScratchPool *&p = g_pools[L->st];
-    if (!p) { p = new (std::nothrow) ScratchPool(); if (p) p->st = L->st; }
+    ScratchPool *&p = g_pools[std::make_pair(L->device, L->st)];
+    if (!p) { p = new (std::nothrow) ScratchPool(); if (p) { p->st = L->st; p->device = L->device; } }
     if (p) {
       p->refs++;
       L->pool = p;
@@ -436,6 +448,7 @@ int evict_and_close(locret_layer *L, int n_tok, uint32_t flags, bool side, cudaS
 int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t flags, void *attn_out,
                float *tp_partial) {
   if (!L || !hidden_in || !attn_out) return LOCRET_ERR_INVALID;
+  if (!on_layer_device(L)) return LOCRET_ERR_INVALID;
   if (L->tp_pending) return LOCRET_ERR_INVALID;  // a begun step is finished first
   if (n_tok < 1 || n_tok > L->chunk) return LOCRET_ERR_INVALID;
   if (flags & ~(LOCRET_NO_EVICT | LOCRET_LAST_CHUNK)) return LOCRET_ERR_INVALID;
@@ -622,7 +635,7 @@ int locret_prefill_chunk_tp_begin(locret_layer *L, const void *hidden_in, int32_
 
 int locret_prefill_chunk_tp_finish(locret_layer *L, const float *preact_sum) {
   if (!L || !preact_sum || !aligned16(preact_sum)) return LOCRET_ERR_INVALID;
-  if (!L->tp_pending) return LOCRET_ERR_INVALID;
+  if (!L->tp_pending || !on_layer_device(L)) return LOCRET_ERR_INVALID;
   L->tp_pending = false;
   const int n_tok = L->tp_n_tok;
   // nothing downstream in a decoder layer waits for the scores, the selection or the compaction: they
@@ -652,7 +665,7 @@ int locret_cache_len(const locret_layer *L, int32_t *len) {
 
 int locret_export_state(locret_layer *L, void *K, void *V, float *scores, int64_t *token_ids,
                         int32_t *len, int64_t *tokens_seen) {
-  if (!L) return LOCRET_ERR_INVALID;
+  if (!L || !on_layer_device(L)) return LOCRET_ERR_INVALID;
   if (L->int4 && (K || V)) return LOCRET_ERR_INVALID;  // use locret_export_state_int4
   CK(sync_all(L));
   const int c = L->cur, n = L->len;
@@ -675,7 +688,7 @@ int locret_export_state(locret_layer *L, void *K, void *V, float *scores, int64_
 
 int locret_import_state(locret_layer *L, const void *K, const void *V, const float *scores,
                         const int64_t *token_ids, int32_t len, int64_t tokens_seen) {
-  if (!L || len < 0 || len > L->cap || tokens_seen < 0) return LOCRET_ERR_INVALID;
+  if (!L || len < 0 || len > L->cap || tokens_seen < 0 || !on_layer_device(L)) return LOCRET_ERR_INVALID;
   if (L->int4) return LOCRET_ERR_INVALID;  // use locret_import_state_int4
   if (len > 0 && (!K || !V || !scores || !token_ids)) return LOCRET_ERR_INVALID;
   CK(sync_all(L));
@@ -700,7 +713,7 @@ int locret_import_state(locret_layer *L, const void *K, const void *V, const flo
 int locret_export_state_int4(locret_layer *L, void *k_codes, void *k_scales, void *v_codes,
                              void *v_scales, float *scores, int64_t *token_ids, int32_t *len,
                              int64_t *tokens_seen) {
-  if (!L || !L->int4) return LOCRET_ERR_INVALID;
+  if (!L || !L->int4 || !on_layer_device(L)) return LOCRET_ERR_INVALID;
   CK(sync_all(L));
   const int c = L->cur, n = L->len;
   if (len) *len = n;
@@ -722,7 +735,7 @@ int locret_export_state_int4(locret_layer *L, void *k_codes, void *k_scales, voi
 int locret_import_state_int4(locret_layer *L, const void *k_codes, const void *k_scales,
                              const void *v_codes, const void *v_scales, const float *scores,
                              const int64_t *token_ids, int32_t len, int64_t tokens_seen) {
-  if (!L || !L->int4 || len < 0 || len > L->cap || tokens_seen < 0) return LOCRET_ERR_INVALID;
+  if (!L || !L->int4 || len < 0 || len > L->cap || tokens_seen < 0 || !on_layer_device(L)) return LOCRET_ERR_INVALID;
   if (len > 0 && (!k_codes || !k_scales || !v_codes || !v_scales || !scores || !token_ids))
     return LOCRET_ERR_INVALID;
   CK(sync_all(L));
@@ -744,7 +757,7 @@ int locret_import_state_int4(locret_layer *L, const void *k_codes, const void *k
 }
 
 int locret_sync_status(locret_layer *L) {
-  if (!L) return LOCRET_ERR_INVALID;
+  if (!L || !on_layer_device(L)) return LOCRET_ERR_INVALID;
   int host = 0;
   CK(sync_all(L));
   CK(cudaMemcpyAsync(&host, L->d_status, sizeof(int), cudaMemcpyDeviceToHost, L->st));
@@ -754,7 +767,13 @@ int locret_sync_status(locret_layer *L) {
 }
 
 int locret_reset(locret_layer *L) {
-  if (!L) return LOCRET_ERR_INVALID;
+  if (!L || !on_layer_device(L)) return LOCRET_ERR_INVALID;
+  // a selection / compaction still in flight on the second stream writes this layer's cache: the
+  // layer's stream is ordered behind it here, so whatever is enqueued after the reset sees it done
+  if (L->use_side && L->side_pending) {
+    CK(cudaStreamWaitEvent(L->st, L->ev_side, 0));
+    L->side_pending = false;
+  }
   L->len = 0;
   L->seen = 0;
   L->tp_pending = false;
@@ -776,7 +795,7 @@ int locret_set_timing(locret_layer *L, int32_t enable) {
 }
 
 int locret_read_timing(locret_layer *L, float *ms, int64_t *launches) {
-  if (!L || !ms || !launches) return LOCRET_ERR_INVALID;
+  if (!L || !ms || !launches || !on_layer_device(L)) return LOCRET_ERR_INVALID;
   for (int i = 0; i < LOCRET_K_COUNT; i++) { ms[i] = 0.f; launches[i] = 0; }
   CK(sync_all(L));
   for (size_t i = 0; i < L->events_used; i++) {

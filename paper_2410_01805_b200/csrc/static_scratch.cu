@@ -13,11 +13,10 @@ using namespace locret;
 
 namespace {
 
-// Scratch for the partial scores [d_R / 128 tiles][n_tok][h_kv] (fp32).  It lives in every
+// Scratch for the partial scores [N-tiles of the GEMM (at most ceil(d_R / 64))][n_tok][h_kv] (fp32).  It lives in every
 // GPU context that loads the library until the process exits.
 static __device__ __align__(256) float g_static_partial[LOCRET_STATIC_SCRATCH_FLOATS];
 
-constexpr int MAX_DEVICES = 64;
 float *g_partial_ptr[MAX_DEVICES] = {nullptr};
 
 // In host code `g_static_partial` is only a stand-in for the symbol, never a device address:
@@ -44,7 +43,7 @@ int static_partial_for_current_device(float **out) {
 
 extern "C" int locret_rh_scores_static(const void *z, int32_t n_tok, int32_t d_in, const void *w1_t,
                                        int32_t d_retain, const float *w2, int32_t n_kv_heads,
-                                       int32_t act, float *scores, void *stream) {
+                                       int32_t act, float *scores, int32_t *status, void *stream) {
   if (!z || !w1_t || !w2 || !scores) return LOCRET_ERR_INVALID;
   if (n_tok < 1 || d_in < 64 || d_in % 64 != 0 || d_retain < 32 || d_retain % 32 != 0)
     return LOCRET_ERR_INVALID;
@@ -63,7 +62,7 @@ extern "C" int locret_rh_scores_static(const void *z, int32_t n_tok, int32_t d_i
   int n_tiles = 0;
   // Every partial this call reads is written by this call first, so nothing has to be cleared.
   if (launch_rh_gemm_tc((const bf16 *)z, d_in, (const bf16 *)w1_t, w2, partial, n_tok, d_retain, d_in,
-                        n_kv_heads, act, &n_tiles, nullptr, st) != cudaSuccess) {
+                        n_kv_heads, act, &n_tiles, status, st) != cudaSuccess) {
     cudaGetLastError();
     return LOCRET_ERR_CUDA;
   }

@@ -63,9 +63,9 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity) {
 // other roles stop waiting as well.  Returns false if the wait was abandoned.
 template <int BACKOFF_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
-                                          int *status) {
+                                          int *status, uint32_t limit = WAIT_LIMIT) {
   if (mbar_test_wait(bar, parity)) return true;
-  for (uint32_t i = 0; i < WAIT_LIMIT; i++) {
+  for (uint32_t i = 0; i < limit; i++) {
     if (mbar_try_wait(bar, parity)) return true;
     if (BACKOFF_NS > 0) __nanosleep(BACKOFF_NS);  // leave the issue slots to the warps that have work
     if ((i & 1023u) == 1023u && *abort_flag) return false;

@@ -17,6 +17,8 @@ V_ULP = 2.0 ** -7     # a stored V element may round to either bf16 neighbour (f
 SCORE_TOL = 1e-2      # |delta| <= SCORE_TOL * max(|ref|, rms(ref over the chunk))
 BAND = 1e-2           # index sets must agree outside this band around the cut
 FLIP_FRACTION = 5e-3  # share of stored chunk K/V elements allowed to sit one bf16 ulp apart (measured 2.3e-3 at K = 4096)
+ORDINARY_ABS = 2.0    # a query row is "ordinary" when sum_i p_i |v_i| stays below this in every column:
+                      # it puts no noticeable weight on a 20x-norm outlier token (typical rows: 0.8)
 
 
 def bf16_dev(x: np.ndarray) -> torch.Tensor:
@@ -51,6 +53,37 @@ def check_attention(got: np.ndarray, ref: np.ndarray, what="", abs_ref=None, fli
     worst = float(np.max(err / bound)) if err.size else 0.0
     assert worst <= 1.0, f"{what} attention: worst err/bound {worst:.3f}, max abs {err.max():.4g}"
     return float(err.max()) if err.size else 0.0
+
+
+def attention_stats(got: np.ndarray, ref: np.ndarray, abs_ref=None, flip_sens=None, pure_ref=None):
+    """How much of the derived bound the comparison uses, and how the CUDA path fares against the
+    plain stated tolerance (max-abs 2e-2), per chunk:
+      plain_max_abs            largest |delta| over all compared elements
+      plain_exceed_share       share of elements beyond the plain mixed bound 2e-2 * max(1, |ref|)
+                               (these are the ones that need the derived terms)
+      ordinary_rows / ordinary_max_abs   rows with sum p|v| < ORDINARY_ABS in every column, and the
+                               largest |delta| on them (must stay within the plain 2e-2)
+      bound_used_max           worst err / full bound
+      pure_within_2e-2_share   share of elements within plain 2e-2 of the oracle WITHOUT bf16 mirroring
+    """
+    rows = ~np.isnan(ref).any(axis=1)
+    g, r = got[rows], ref[rows]
+    err = np.abs(g - r)
+    st = {"plain_max_abs": float(err.max()) if err.size else 0.0,
+          "plain_exceed_share": float(np.mean(err > ATTN_TOL * np.maximum(1.0, np.abs(r)))) if err.size else 0.0}
+    if abs_ref is not None:
+        bound = ATTN_TOL * np.maximum(1.0, np.abs(r)) + (P_ULP + V_ULP) * abs_ref[rows]
+        if flip_sens is not None:
+            bound = bound + flip_sens[rows]
+        st["bound_used_max"] = float(np.max(err / bound)) if err.size else 0.0
+        ordinary = abs_ref[rows].max(axis=1) < ORDINARY_ABS
+        st["ordinary_rows"] = int(ordinary.sum())
+        st["rows"] = int(rows.sum())
+        st["ordinary_max_abs"] = float(err[ordinary].max()) if ordinary.any() else 0.0
+    if pure_ref is not None:
+        st["pure_within_2e-2_share"] = float(np.mean(np.abs(g - pure_ref[rows]) <= ATTN_TOL))
+        st["pure_max_abs"] = float(np.max(np.abs(g - pure_ref[rows])))
+    return st
 
 
 def check_scores(got: np.ndarray, ref: np.ndarray, what=""):
@@ -97,8 +130,12 @@ def import_oracle_state(gpu, st, int4: bool):
         gpu.import_state(st["K"], st["V"], st["S"], st["T"], st["seen"])
 
 
-def lockstep_chunk(ora, gpu, x: np.ndarray, flags: int = 0, rows=None, what=""):
-    """Import the oracle's state, run one chunk on both, compare everything.  Advances the oracle."""
+def lockstep_chunk(ora, gpu, x: np.ndarray, flags: int = 0, rows=None, what="", pure=None, plain=False):
+    """Import the oracle's state, run one chunk on both, compare everything.  Advances the oracle.
+    pure: an OracleLayer with mirror=False that is given the same state and chunk; its output only
+    feeds the statistics (how the CUDA path fares against the un-mirrored fp64 result).
+    plain: also assert the plain stated tolerances (attention max-abs 2e-2; workloads without
+    outlier tokens)."""
     shape = ora.s
     h, hk, d = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
     n_tok = x.shape[0]
@@ -121,10 +158,20 @@ def lockstep_chunk(ora, gpu, x: np.ndarray, flags: int = 0, rows=None, what=""):
     assert gpu.sync_status() == 0
     assert torch.equal(out_a, out_b), f"{what}: attention output not reproducible"
 
+    pure_out = None
+    if pure is not None:
+        pure.import_state(st)
+        pure_out = pure.prefill_chunk(x, flags, rows=rows)
     ref_out = ora.prefill_chunk(x, flags, rows=rows)
     stats = {}
-    stats["attn_max_abs"] = check_attention(out_b.float().cpu().numpy().astype(np.float64), ref_out, what,
-                                            ora.last_abs_out, ora.last_flip_sens)
+    got_out = out_b.float().cpu().numpy().astype(np.float64)
+    stats["attn_max_abs"] = check_attention(got_out, ref_out, what, ora.last_abs_out, ora.last_flip_sens)
+    stats.update(attention_stats(got_out, ref_out, ora.last_abs_out, ora.last_flip_sens, pure_out))
+    # rows that put no weight on an outlier token meet the stated tolerance as it is written
+    assert stats["ordinary_max_abs"] <= ATTN_TOL, \
+        f"{what}: ordinary rows off by {stats['ordinary_max_abs']:.4g} (plain tolerance {ATTN_TOL})"
+    if plain:
+        assert stats["plain_max_abs"] <= ATTN_TOL, f"{what}: plain max-abs {stats['plain_max_abs']:.4g}"
 
     n = ln + n_tok
     assert pre["K"].shape[1] == n and pre["seen"] == st["seen"] + n_tok
@@ -156,7 +203,11 @@ def lockstep_chunk(ora, gpu, x: np.ndarray, flags: int = 0, rows=None, what=""):
             f"{what}: chunk {name} off by more than one bf16 ulp"
         flips = float(np.mean(diff != 0))
         assert flips < FLIP_FRACTION, f"{what}: too many rounding flips in chunk {name}: {flips:.4f}"
-    stats["score_worst"] = check_scores(pre["S"][:, ln:].T.astype(np.float64), ora.last_scores, what)
+        stats[f"flip_rate_{name}"] = flips
+    got_s = pre["S"][:, ln:].T.astype(np.float64)
+    stats["score_worst"] = check_scores(got_s, ora.last_scores, what)
+    stats["score_plain_rel_worst"] = float(np.max(np.abs(got_s - ora.last_scores) /
+                                                  np.maximum(np.abs(ora.last_scores), 1e-3)))
 
     evict = not (flags & O.NO_EVICT) and n > ora.budget
     if evict:
@@ -177,4 +228,66 @@ def lockstep_chunk(ora, gpu, x: np.ndarray, flags: int = 0, rows=None, what=""):
         for key in state_keys + ("T",):
             assert np.array_equal(post[key], pre[key])
     assert gpu.cache_len == ora.len
+    return stats
+
+
+def forced_state(shape, budget: int, chunk: int, seed: int = 0, unmoved: int = 64):
+    """A full cache whose next eviction is decided before any chunk score is known: budget - chunk
+    units score +100 and chunk units score -100 (interleaved at random behind a short all-high
+    prefix), so a full chunk with the last n_stab protected evicts exactly the -100 units whatever
+    the chunk's own scores (|score| << 100): both sides keep the same set, the kept high units
+    behind the prefix all move to new slots, and the prefix stays where it is."""
+    import workloads as W
+    hk, d = shape.n_kv_heads, shape.head_dim
+    g = np.random.default_rng(7000 + seed)
+    K = W.to_bf16_grid(g.standard_normal((hk, budget, d)).astype(np.float32)).astype(np.float64)
+    V = W.to_bf16_grid(g.standard_normal((hk, budget, d)).astype(np.float32)).astype(np.float64)
+    n_high = budget - chunk
+    unmoved = min(unmoved, n_high)
+    S = np.full((hk, budget), -100.0)
+    for m in range(hk):
+        S[m, :unmoved] = 100.0
+        pick = unmoved + g.choice(budget - unmoved, size=n_high - unmoved, replace=False)
+        S[m, pick] = 100.0
+    T = np.broadcast_to(np.arange(budget, dtype=np.int64), (hk, budget)).copy()
+    return dict(K=K, V=V, S=S, T=T, seen=budget)
+
+
+def run_pair_without_reimport(ora, gpu, st, x_a, x_b, rows_a=None, rows_b=None, what=""):
+    """Chunk A evicts and compacts from the forced state `st`; chunk B then runs on BOTH sides from
+    what each side's own step A left (no import in between), so the attention of B reads the rotated
+    keys that the CUDA compaction wrote.  Returns B's statistics."""
+    h, d = ora.s.n_q_heads, ora.s.head_dim
+    budget = ora.budget
+    ora.import_state(st)
+    gpu.import_state(st["K"], st["V"], st["S"], st["T"], st["seen"])
+    out_a = torch.zeros((x_a.shape[0], h * d), dtype=torch.bfloat16, device="cuda")
+    gpu.prefill_chunk(bf16_dev(x_a), out_a, 0)
+    ref_a = ora.prefill_chunk(x_a, 0, rows=rows_a)
+    check_attention(out_a.float().cpu().numpy().astype(np.float64), ref_a, f"{what} A", ora.last_abs_out,
+                    ora.last_flip_sens)
+    post = gpu.export_state()                       # reads the state; rotated keys are left as compaction wrote them
+    assert gpu.sync_status() == 0
+    assert np.array_equal(post["T"], ora.T), f"{what}: retained token ids differ after the forced eviction"
+    keep = ora.last_keep
+    moved = sum(int(np.sum(keep[m] != np.arange(budget))) for m in range(ora.hk))
+    stay = sum(int(np.sum(keep[m] == np.arange(budget))) for m in range(ora.hk))
+    assert moved > 0 and stay > 0, f"{what}: the forced eviction must both move and leave units"
+    # the cache contents agree up to the rare one-ulp flips of the chunk's stored K, V
+    for name in ("K", "V"):
+        diff = np.abs(post[name] - getattr(ora, name))
+        assert np.all(diff <= np.abs(getattr(ora, name)) * 2.0 ** -7 + 1e-5 * np.abs(getattr(ora, name)).max())
+        assert np.mean(diff != 0) < FLIP_FRACTION
+    out_b = torch.zeros((x_b.shape[0], h * d), dtype=torch.bfloat16, device="cuda")
+    ln = ora.len
+    gpu.prefill_chunk(bf16_dev(x_b), out_b, O.NO_EVICT)
+    ref_b = ora.prefill_chunk(x_b, O.NO_EVICT, rows=rows_b)
+    got_b = out_b.float().cpu().numpy().astype(np.float64)
+    stats = {"attn_max_abs": check_attention(got_b, ref_b, f"{what} B", ora.last_abs_out, ora.last_flip_sens)}
+    stats.update(attention_stats(got_b, ref_b, ora.last_abs_out, ora.last_flip_sens))
+    assert stats["ordinary_max_abs"] <= ATTN_TOL, f"{what} B: ordinary rows off by {stats['ordinary_max_abs']:.4g}"
+    after = gpu.export_state()
+    stats["score_worst"] = check_scores(after["S"][:, ln:].T.astype(np.float64), ora.last_scores, f"{what} B")
+    stats["moved"], stats["stayed"] = moved, stay
+    assert gpu.sync_status() == 0
     return stats

@@ -20,26 +20,43 @@ def sampled_rows(n_tok, seed):
     return sorted(rows)
 
 
-def run_workload_chunks(name, n_chunks, layer=0, extra_rows=()):
+def run_workload_chunks(name, n_chunks, layer=0, extra_rows=(), plain=False, with_pure=False, block_chunks=()):
+    """block_chunks: chunk indices whose sampled rows also hold one whole 128-row query block (the block
+    walks through the chunk from one listed chunk to the next, so causal-diagonal tiles of different
+    row blocks are covered)."""
     from parity_util import lockstep_chunk, make_pair
     w = W.get_workload(name)
-    ora, gpu = make_pair(w.shape, W.layer_weights(w.shape, layer), w.budget, w.chunk, w.n_stab)
+    wts = W.layer_weights(w.shape, layer)
+    ora, gpu = make_pair(w.shape, wts, w.budget, w.chunk, w.n_stab)
+    pure = O.OracleLayer(w.shape, *wts, w.budget, w.chunk, w.n_stab, mirror=False) if with_pure else None
     start, stats = 0, []
     for i, n_tok in enumerate(w.chunk_sizes()[:n_chunks]):
         x = W.hidden_states(w, start, n_tok)
         rows = sampled_rows(n_tok, i)
         # always include the outlier tokens of the chunk: they are the ill-conditioned rows
         norms = np.linalg.norm(x, axis=1)
-        rows = sorted(set(rows) | set(np.flatnonzero(norms > 5 * np.median(norms)).tolist()[:4]) | set(extra_rows))
-        stats.append(lockstep_chunk(ora, gpu, x, 0, rows=rows, what=f"{name} chunk {i}"))
+        rows = set(rows) | set(np.flatnonzero(norms > 5 * np.median(norms)).tolist()[:4]) | set(extra_rows)
+        if i in block_chunks:
+            n_rb = (n_tok + 127) // 128
+            rb = (5 + 7 * list(block_chunks).index(i)) % n_rb
+            rows |= set(range(rb * 128, min(n_tok, (rb + 1) * 128)))
+        stats.append(lockstep_chunk(ora, gpu, x, 0, rows=sorted(rows), what=f"{name} chunk {i}", pure=pure, plain=plain))
         start += n_tok
     assert gpu.sync_status() == 0
     gpu.destroy()
+    summary = {k: max(s[k] for s in stats if k in s) for k in
+               ("plain_max_abs", "plain_exceed_share", "ordinary_max_abs", "bound_used_max", "flip_rate_K", "flip_rate_V",
+                "score_worst", "score_plain_rel_worst", "pure_max_abs") if any(k in s for s in stats)}
+    if with_pure:
+        summary["pure_within_2e-2_share_min"] = min(s["pure_within_2e-2_share"] for s in stats)
+    summary["rows_compared"] = sum(s.get("rows", 0) for s in stats)
+    summary["ordinary_rows"] = sum(s.get("ordinary_rows", 0) for s in stats)
+    print(f"{name}: worst over {len(stats)} chunks: {summary}")
     return w, ora, stats
 
 
 def test_c3_llama_shape_first_chunks_through_steady_state():
-    w, ora, stats = run_workload_chunks("c3_llama_128k", 4)
+    w, ora, stats = run_workload_chunks("c3_llama_128k", 4, block_chunks=(1, 2, 3))
     assert ora.len == w.budget
     assert all("sets_identical" in s for s in stats[1:])
 
@@ -56,8 +73,11 @@ def test_c5_llama_shape_int4_cache():
 
 def test_c4_phi3_shape_until_the_cache_is_full():
     # 16 chunks fill the 16384-unit budget; chunks 17 and 18 evict
-    w, ora, stats = run_workload_chunks("c4_phi3_128k", 18)
+    # no outlier tokens in this workload: the plain stated tolerance (max-abs 2e-2) is asserted as written,
+    # and the un-mirrored fp64 oracle runs beside the mirrored one for the statistics
+    w, ora, stats = run_workload_chunks("c4_phi3_128k", 18, plain=True, with_pure=True, block_chunks=(3, 16, 17))
     assert ora.len == w.budget and "sets_identical" in stats[-1]
+    assert min(s["pure_within_2e-2_share"] for s in stats) > 0.999
 
 
 def test_llama_shape_short_chunks():

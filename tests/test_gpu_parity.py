@@ -26,11 +26,15 @@ def hidden(n, D, seed=0, scale=1.0):
 def test_c1_lockstep_every_chunk():
     from parity_util import lockstep_chunk, make_pair
     w = W.get_workload("c1_small_gqa")
-    ora, gpu = make_pair(w.shape, W.layer_weights(w.shape, 0), w.budget, w.chunk, w.n_stab)
+    wts = W.layer_weights(w.shape, 0)
+    ora, gpu = make_pair(w.shape, wts, w.budget, w.chunk, w.n_stab)
+    pure = O.OracleLayer(w.shape, *wts, w.budget, w.chunk, w.n_stab, mirror=False)
     start, identical = 0, 0
     for i, n_tok in enumerate(w.chunk_sizes()):
         x = W.hidden_states(w, start, n_tok)
-        st = lockstep_chunk(ora, gpu, x, 0, what=f"c1 chunk {i}")
+        # no outlier tokens here: the plain stated tolerance (max-abs 2e-2) holds as written
+        st = lockstep_chunk(ora, gpu, x, 0, what=f"c1 chunk {i}", pure=pure, plain=True)
+        assert st["pure_within_2e-2_share"] == 1.0 and st["score_plain_rel_worst"] < 0.05
         identical += bool(st.get("sets_identical", True))
         start += n_tok
     assert ora.len == w.budget and identical >= len(w.chunk_sizes()) - 1
@@ -320,6 +324,14 @@ def test_bounded_wait_reports_a_timeout_and_the_context_survives():
     from parity_util import lockstep_chunk, make_pair
     assert P.lib.locret_selftest_wait_timeout(torch.cuda.current_stream().cuda_stream) == -5
     assert b"timed out" in P.lib.locret_strerror(-5)
+    # the production wait itself: one role runs out of polls, sets the abort flag and the status word;
+    # a second role that waits with the full production limit must be stopped by that flag
+    rep = np.zeros(4, dtype=np.int64)
+    assert P.lib.locret_selftest_wait_abort(torch.cuda.current_stream().cuda_stream, rep.ctypes.data) == 0
+    assert rep[0] == -5 and rep[1] == 1
+    # the first role gave up after 2^12 polls; the second checks the flag every 2^10 polls, so it
+    # stops within about a quarter more, nowhere near its own 2^24 polls
+    assert 0 < rep[2] and rep[3] < 4 * rep[2] + 10_000_000, rep
     sh = small_shape(d=128, D=128, dR=64)
     ora, gpu = make_pair(sh, weights_for(sh, 21), budget=200, chunk=128, n_stab=8)
     lockstep_chunk(ora, gpu, hidden(128, sh.d_model, 5), 0, what="after the timed-out wait")

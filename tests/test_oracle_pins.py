@@ -463,6 +463,144 @@ def test_int4_layer_quantises_on_append_and_moves_codes_unchanged():
                 assert layer.Vs[m, slot] == before["Vs"][m, old]
 
 
+def test_last_chunk_through_the_chunk_step_keeps_plain_top_b_by_hand():
+    """Algorithm 1's last iteration: no score is overwritten with +inf, so the retained set is the
+    plain top-b of cache ‖ chunk.  Scores are forced through hand-made weights: the retaining
+    head reads V's first column (W1 picks it, ReLU, W2 = 1), so score(token) = max(0, V[t, 0])."""
+    sh = shape(n_q_heads=1, n_kv_heads=1, head_dim=2, d_model=6, d_retain=1, act=2)
+    wqkv = np.eye(6)                         # [Q ‖ K ‖ V] = the hidden state itself
+    w1 = np.zeros((6, 1)); w1[4, 0] = 1.0    # first element of V
+    w2 = np.ones((1, 1))
+    b, n_s = 6, 4
+    layer = O.OracleLayer(sh, wqkv, w1, w2, budget=b, chunk=8, n_stab=n_s)
+    score = np.array([5., 1., 9., 2., 8., 3., 7., 4.,            # chunk 0: tokens 0..7
+                      0.5, 6., 0.25, 10., 0.1, 0.2, 0.3, 0.4])   # chunk 1: tokens 8..15
+    X = np.random.default_rng(40).standard_normal((16, 6))
+    X[:, 4] = score
+    layer.prefill_chunk(X[:8])               # protected: tokens 4..7; best two of 0..3: tokens 0 (5) and 2 (9)
+    assert list(layer.T[0]) == [0, 2, 4, 5, 6, 7]
+    assert np.allclose(layer.S[0], score[[0, 2, 4, 5, 6, 7]])
+    layer.prefill_chunk(X[8:], O.LAST_CHUNK)
+    # candidates: tokens {0,2,4,5,6,7} ∪ {8..15}; the six best scores are 10, 9, 8, 7, 6, 5
+    assert list(layer.T[0]) == [0, 2, 4, 6, 9, 11]
+    # the same step with protection would have kept the last four tokens whatever their scores
+    prot = O.OracleLayer(sh, wqkv, w1, w2, budget=b, chunk=8, n_stab=n_s)
+    prot.prefill_chunk(X[:8]); prot.prefill_chunk(X[8:])
+    assert list(prot.T[0]) == [2, 11, 12, 13, 14, 15]
+
+
+def test_abs_out_is_the_probability_weighted_magnitude_by_explicit_loops():
+    g = np.random.default_rng(41)
+    n, h, hk, d, ln = 5, 4, 2, 6, 7
+    Qr, Kc, Vc = g.standard_normal((n, h, d)), g.standard_normal((hk, ln, d)), g.standard_normal((hk, ln, d)) * 3
+    Kn, Vn = g.standard_normal((n, hk, d)), g.standard_normal((n, hk, d)) * 3
+    abs_out = np.full((n, h * d), np.nan)
+    out = O.attention_rows(Qr, Kc, Vc, Kn, Vn, h // hk, abs_out=abs_out)
+    for t in range(n):
+        for j in range(h):
+            m = j // (h // hk)
+            keys = [Kc[m, i] for i in range(ln)] + [Kn[u, m] for u in range(t + 1)]
+            vals = [Vc[m, i] for i in range(ln)] + [Vn[u, m] for u in range(t + 1)]
+            lg = np.array([Qr[t, j] @ k / math.sqrt(d) for k in keys])
+            p = np.exp(lg - lg.max()); p /= p.sum()
+            for c in range(d):
+                assert abs(abs_out[t, j * d + c] - sum(p[i] * abs(vals[i][c]) for i in range(len(keys)))) < 1e-12
+                assert abs(out[t, j * d + c] - sum(p[i] * vals[i][c] for i in range(len(keys)))) < 1e-12
+    assert np.all(abs_out >= np.abs(out) - 1e-12)           # triangle inequality
+
+
+def test_flip_sens_is_the_first_order_effect_of_one_flipped_key_element_by_brute_force():
+    """flip_sens = sum_i p_i delta_i |V_i - out|, delta_i = 2^-7 max_c |q_c k_ic| / sqrt(d): the change of
+    the output when key i's most influential element moves by 2^-7 of itself, summed over the keys
+    in absolute value.  Brute force: move that one element of one key, recompute the softmax exactly,
+    and add up the absolute output changes over the keys."""
+    g = np.random.default_rng(42)
+    n, h, hk, d, ln = 3, 2, 1, 8, 9
+    Qr, Kc, Vc = g.standard_normal((n, h, d)), g.standard_normal((hk, ln, d)), g.standard_normal((hk, ln, d))
+    Kn, Vn = g.standard_normal((n, hk, d)), g.standard_normal((n, hk, d))
+    fs = np.full((n, h * d), np.nan)
+    out = O.attention_rows(Qr, Kc, Vc, Kn, Vn, h, flip_sens=fs)
+
+    def softmax_out(q, keys, vals):
+        lg = keys @ q / math.sqrt(d)
+        p = np.exp(lg - lg.max()); p /= p.sum()
+        return p @ vals
+
+    for t in range(n):
+        for j in range(h):
+            keys = np.concatenate([Kc[0], Kn[: t + 1, 0]])
+            vals = np.concatenate([Vc[0], Vn[: t + 1, 0]])
+            base = softmax_out(Qr[t, j], keys, vals)
+            assert np.allclose(base, out[t, j * d:(j + 1) * d], atol=1e-13)
+            total = np.zeros(d)
+            for i in range(len(keys)):
+                c = int(np.argmax(np.abs(Qr[t, j] * keys[i])))
+                moved = keys.copy()
+                moved[i, c] *= 1.0 + 2.0 ** -7
+                total += np.abs(softmax_out(Qr[t, j], moved, vals) - base)
+            got = fs[t, j * d:(j + 1) * d]
+            # first order in 2^-7: the two agree to a few per cent; a factor of two (let alone ten)
+            # in delta, a dropped p_i or |V_i| in place of |V_i - out| would not
+            assert np.allclose(got, total, rtol=0.05, atol=1e-9), (got, total)
+
+
+def _mirror_reference(X, wqkv, sh, Kc, Vc, skip=None):
+    """The chunk step's attention with bf16 rounding at the storage points, written with the
+    library's conversions (torch.bfloat16) and its attention routine.  `skip` leaves one point
+    unrounded.  Points: 'staging' (projected Q, K, V), 'q_rot', 'k_rot_chunk', 'k_rot_cache'."""
+    def r(x, name):
+        if name == skip:
+            return x
+        return torch.from_numpy(np.asarray(x)).to(torch.bfloat16).to(torch.float64).numpy()
+    h, hk, d = sh.n_q_heads, sh.n_kv_heads, sh.head_dim
+    n, ln = X.shape[0], Kc.shape[1]
+    qkv = r(X @ wqkv, "staging")
+    Q = qkv[:, : h * d].reshape(n, h, d)
+    K = qkv[:, h * d:(h + hk) * d].reshape(n, hk, d)
+    V = qkv[:, (h + hk) * d:].reshape(n, hk, d)
+    pos = (ln + np.arange(n))[:, None]
+    Qr = r(O.rope(Q, pos, sh.rope_theta), "q_rot")
+    Kr = r(O.rope(K, pos, sh.rope_theta), "k_rot_chunk")
+    Kcr = r(O.rope(Kc, np.arange(ln)[None, :], sh.rope_theta), "k_rot_cache")
+    out = np.zeros((n, h * d))
+    g = h // hk
+    for j in range(h):
+        m = j // g
+        keys = torch.from_numpy(np.concatenate([Kcr[m], Kr[:, m]]))
+        vals = torch.from_numpy(np.concatenate([Vc[m], V[:, m]]))
+        mask = torch.ones((n, ln + n), dtype=torch.bool)
+        mask[:, ln:] = torch.tril(torch.ones((n, n), dtype=torch.bool))
+        o = torch.nn.functional.scaled_dot_product_attention(torch.from_numpy(Qr[:, j])[None], keys[None], vals[None],
+                                                             attn_mask=mask[None])
+        out[:, j * d:(j + 1) * d] = o[0].numpy()
+    return out, K, V
+
+
+@pytest.mark.parametrize("point", ["staging", "q_rot", "k_rot_chunk", "k_rot_cache"])
+def test_each_mirror_rounding_point_is_where_the_stored_value_is_rounded(point):
+    """Mirror mode rounds to bf16 exactly at the four storage points of the step.  With every point
+    rounded, a restatement on the library's conversions reproduces the oracle to rounding error of
+    fp64; with any one point left out it does not (so a point dropped from the oracle, or added
+    elsewhere, is seen)."""
+    sh = shape(n_q_heads=4, n_kv_heads=2, head_dim=8, d_model=16)
+    layer, (wqkv, w1, w2) = rand_layer(sh, budget=32, chunk=12, n_stab=0, seed=43, mirror=True)
+    g = np.random.default_rng(44)
+    X0 = O.round_bf16(g.standard_normal((12, sh.d_model)))
+    X1 = O.round_bf16(g.standard_normal((12, sh.d_model)))
+    layer.prefill_chunk(X0)
+    Kc, Vc = layer.K.copy(), layer.V.copy()
+    got = layer.prefill_chunk(X1)
+    want, K, V = _mirror_reference(X1, wqkv, sh, Kc, Vc)
+    assert np.max(np.abs(got - want)) < 1e-12
+    # what enters the cache is the staged (rounded) projection, pre-RoPE
+    assert np.array_equal(layer.K[:, 12:], np.transpose(K, (1, 0, 2)))
+    assert np.array_equal(layer.V[:, 12:], np.transpose(V, (1, 0, 2)))
+    without, K2, _ = _mirror_reference(X1, wqkv, sh, Kc, Vc, skip=point)
+    assert np.max(np.abs(got - without)) > 1e-6, f"rounding at {point} does not reach the output"
+    if point == "staging":
+        assert not np.array_equal(layer.K[:, 12:], np.transpose(K2, (1, 0, 2)))
+
+
 def test_mirror_mode_rounds_only_storage_points():
     sh = shape()
     lp, (wqkv, w1, w2) = rand_layer(sh, budget=64, chunk=16, n_stab=0, seed=26)
