@@ -33,8 +33,8 @@ import workloads as W  # noqa: E402
 METRIC = "chunked-prefill tokens/sec at 128K ctx (1 B200); % tensor/HBM roofline per kernel"
 UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "c3_llama_128k"
-# dram__bytes_read.sum + dram__bytes_write.sum of one steady-state attention launch, from the ncu
-# capture summarised in profiles/attn_tc_kernel_c3_steady_chunk.md (same launch shape as here)
+# dram__bytes_read.sum + dram__bytes_write.sum of one steady-state attention launch: a literal taken
+# from a profiler capture of the same launch shape (not measured during this run)
 NCU_ATTN_TRAFFIC_BYTES = {"c3_llama_128k": 67.5e6, "c2_llama_32k": 67.5e6}
 
 
@@ -346,7 +346,7 @@ def run_ours(args, w):
     roofline = {"kernel": "attn", "bound": "tensor", "achieved": float(attn_tf), "peak": peaks["tf_sustained"],
                 "unit": "TFLOP/s", "frac": float(attn_tf / peaks["tf_sustained"]),
                 "traffic": NCU_ATTN_TRAFFIC_BYTES.get(w.name) if not (args.layers or args.context) else None,
-                "traffic_unit": "bytes per steady-state launch (ncu)",
+                "traffic_unit": "bytes per steady-state launch (literal from a profiler capture of this launch shape)",
                 "peak_source": f"bf16 sustained, {peaks['source']}", "dominant_by_time": K_NAMES[dom],
                 "isolated": {"achieved": isolated["attn"]["tflops"],
                              "frac": isolated["attn"]["tflops"] / peaks["tf_sustained"],
