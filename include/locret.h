@@ -214,23 +214,6 @@ int locret_selftest_wait_timeout(void *stream);
  */
 int locret_selftest_wait_abort(void *stream, int64_t *report);
 
-/*
- * Host-side replay of how the attention kernel (Eq. 1) divides a launch over its CTAs.  The key
- * steps of all query-tile pairs ("items": two 128-row query tiles sharing a KV head, against the
- * 128-key tiles they see) are laid on one line, and CTA u of U takes the steps [u S / U, (u+1) S / U):
- * a few segments, each a range [k0, k1) of one item's key steps.  Pieces of a divided item meet in
- * scratch and are merged in segment order by the CTA that finishes last.  No device is needed and
- * nothing is launched.  n_tok >= 64 chunk tokens, len retained units, max_ctas >= 1.
- * rows (HOST, cap x 8 int32, may be NULL with cap = 0): per segment, in the order the CTAs walk them:
- * CTA, item, k0, k1, key tiles of the item, scratch slot of the piece (-1: a whole item), first and last
- * CTA holding a piece of the item.  *n_ctas, *total_steps (HOST, may be NULL): U and S.
- * Returns the number of segments (also when it exceeds cap), LOCRET_ERR_INVALID for shapes the kernel
- * does not take, or -2 if the replay found a piece its merge would not look for (a defect).
- */
-int locret_selftest_attention_split(int32_t n_tok, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
-                                    int32_t len, int32_t max_ctas, int32_t *rows, int32_t cap, int32_t *n_ctas,
-                                    int32_t *total_steps);
-
 /* Forget all units: len = 0, tokens_seen = 0.  Asynchronous: nothing is launched; the layer's
  * stream is ordered behind any selection / compaction of this layer still in flight on the
  * library's second stream, so work enqueued after the reset finds the cache quiescent. */

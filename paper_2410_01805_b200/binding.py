@@ -68,7 +68,6 @@ def _load():
     l.locret_launch_count.argtypes = [P, C.POINTER(C.c_int64)]
     l.locret_rh_scores_static.argtypes = [P, C.c_int32, C.c_int32, P, C.c_int32, P, C.c_int32, C.c_int32, P, P, P]
     l.locret_selftest_wait_abort.argtypes = [P, P]
-    l.locret_selftest_attention_split.argtypes = [C.c_int32] * 6 + [P, C.c_int32, P, P]
     l.locret_destroy.argtypes = [P]
     l.locret_destroy.restype = None
     l.locret_block_create.argtypes = [C.POINTER(locret_block_cfg), C.c_int32, C.c_int32, C.c_int32, C.POINTER(P)]

@@ -43,11 +43,6 @@ struct ScratchPool {
   unsigned *dec_cnt = nullptr;
   float *partial = nullptr;
   int32_t *keep = nullptr;
-  // attention: pieces of query-tile pairs whose key steps are divided over several CTAs
-  float *att_o = nullptr, *att_ml = nullptr;
-  unsigned *att_cnt = nullptr;
-  size_t atto_b = 0, attml_b = 0, attcnt_b = 0;
-  int att_units = 0;
   struct CsTable { float theta; int d, cap; float2 *ptr; };
   std::vector<CsTable> cs;
 };
@@ -141,7 +136,6 @@ void release_pool(ScratchPool *p) {
   if (p->ev_exp_ready) cudaEventDestroy(p->ev_exp_ready);
   cudaFree(p->q_rot); cudaFree(p->partial); cudaFree(p->keep); cudaFree(p->dec_o); cudaFree(p->dec_ml); cudaFree(p->dec_cnt);
   cudaFree(p->k_exp); cudaFree(p->v_exp);
-  cudaFree(p->att_o); cudaFree(p->att_ml); cudaFree(p->att_cnt);
   for (auto &t : p->cs) cudaFree(t.ptr);
   g_pools.erase(std::make_pair(p->device, p->st));
   delete p;
@@ -338,18 +332,6 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
         g = g && grow(&p->dec_ml, &p->decml_b, (size_t)h * 64 * 2 * sizeof(float), L->st);
       }
       g = g && grow(&p->keep, &p->keep_b, (size_t)hk * budget * sizeof(int32_t), L->st);
-      if (L->use_tc) {
-        // (the pool's layers share the scratch: it is sized for the largest division any of them asked for,
-        // and every launch may use that many CTAs)
-        const int units = attention_tc_max_units();
-        if (units > p->att_units) p->att_units = units;
-        g = g && grow(&p->att_o, &p->atto_b, attention_tc_part_o_floats(p->att_units, 128) * sizeof(float), L->st);
-        g = g && grow(&p->att_ml, &p->attml_b, attention_tc_part_ml_floats(p->att_units) * sizeof(float), L->st);
-        const size_t before_cnt = p->attcnt_b;
-        g = g && grow(&p->att_cnt, &p->attcnt_b, (size_t)attention_tc_max_items(chunk, h) * sizeof(unsigned), L->st);
-        // the counters are zero between launches; a new array starts at zero
-        if (g && p->attcnt_b != before_cnt) g = cudaMemsetAsync(p->att_cnt, 0, p->attcnt_b, L->st) == cudaSuccess;
-      }
       if (L->int4) {
         const size_t before_k = p->kexp_b, before_v = p->vexp_b;
         g = g && grow(&p->k_exp, &p->kexp_b, kv_b, L->st);
@@ -566,13 +548,9 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
       CK(launch_attention_decode(P->q_rot, k_att, v_att, (bf16 *)attn_out, P->dec_o, P->dec_ml, P->dec_cnt + 1,
                                  L->h, L->h_kv, L->d, L->cap, n, decode_attn_splits(L->h_kv, n),
                                  L->int4 ? &L->q4[c] : nullptr, L->cs, L->st));
-    else if (tc_ok) {
-      AttnWork work;
-      work.part_o = P->att_o; work.part_ml = P->att_ml; work.item_cnt = P->att_cnt;
-      work.max_units = P->att_units; work.max_items = (int)(P->attcnt_b / sizeof(unsigned));
+    else if (tc_ok)
       CK(launch_attention_tc(&L->map_q, &L->map_k, &L->map_v[c], (bf16 *)attn_out, n_tok, L->h, L->h_kv,
-                             L->d, L->len, work, L->d_status, L->st));
-    }
+                             L->d, L->len, L->d_status, L->st));
     else
       CK(launch_attention_mma(P->q_rot, k_att, v_att, (bf16 *)attn_out, n_tok, L->h, L->h_kv,
                               L->d, L->cap, L->len, L->st));

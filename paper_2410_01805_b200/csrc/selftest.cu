@@ -51,15 +51,6 @@ __global__ void wait_abort_kernel(int *status, long long *report, unsigned short
 
 }  // namespace
 
-extern "C" int locret_selftest_attention_split(int32_t n_tok, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
-                                               int32_t len, int32_t max_ctas, int32_t *rows, int32_t cap,
-                                               int32_t *n_ctas, int32_t *total_steps) {
-  if (n_kv_heads < 1 || n_q_heads < 1 || n_q_heads % n_kv_heads || cap < 0) return LOCRET_ERR_INVALID;
-  const int n = attention_tc_replay_split(n_tok, n_q_heads, n_kv_heads, head_dim, len, max_ctas, rows, cap, n_ctas,
-                                          total_steps);
-  return n == -1 ? LOCRET_ERR_INVALID : n;
-}
-
 extern "C" int locret_selftest_wait_abort(void *stream, int64_t *report) {
   if (!report) return LOCRET_ERR_INVALID;
   cudaStream_t st = (cudaStream_t)stream;

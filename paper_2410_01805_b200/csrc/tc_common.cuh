@@ -256,25 +256,10 @@ bool tmap_encode_3d_bf16(CUtensorMap *map, const void *base, uint64_t d0, uint64
 
 
 // Eq. 1 on tcgen05 (attn_tc.cu).  map_k / map_v: 3-D maps {d, cap, h_kv}, box {64, 128, 1};
-// map_q: 2-D map {h*d, rows}, box {64, 128}.  The launch divides the key steps of all query-tile
-// pairs evenly over at most work.max_units CTAs; pieces of a divided pair meet in the scratch of
-// `work` (part_o: attention_tc_part_o_floats(max_units, d) floats, part_ml:
-// attention_tc_part_ml_floats(max_units), item_cnt: max_items words that are zero before the first
-// launch and are left at zero by every launch that runs to its end).
-struct AttnWork {
-  float *part_o, *part_ml;
-  unsigned *item_cnt;
-  int max_units, max_items;
-};
+// map_q: 2-D map {h*d, rows}, box {64, 128}.
 bool attention_tc_supported(int n_tok, int h, int h_kv, int d);
-int attention_tc_max_units();
-size_t attention_tc_part_o_floats(int units, int d);
-size_t attention_tc_part_ml_floats(int units);
-int attention_tc_max_items(int chunk, int h);
-int attention_tc_replay_split(int n_tok, int h, int h_kv, int d, int len, int max_units, int32_t *rows,
-                              int cap, int32_t *n_units_out, int32_t *total_steps_out);
 cudaError_t launch_attention_tc(const CUtensorMap *map_q, const CUtensorMap *map_k,
                                 const CUtensorMap *map_v, bf16 *out, int n_tok, int h, int h_kv, int d,
-                                int len, const AttnWork &work, int *status, cudaStream_t st);
+                                int len, int *status, cudaStream_t st);
 
 }  // namespace locret

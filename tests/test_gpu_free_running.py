@@ -144,19 +144,3 @@ def test_steps_back_to_back_on_two_streams_equal_the_one_stream_schedule(kv_dtyp
             for tok in got ^ want:
                 assert abs(s_all[tok, m] - cut) < BAND, f"layer {l} head {m}: token {tok} outside the band"
             assert len(got ^ want) <= 6
-
-
-@pytest.mark.parametrize("units", [1, 3, 7, 40, 1000])
-def test_lockstep_under_forced_divisions_of_the_attention_launch(units, monkeypatch):
-    """The attention launch divides its key steps evenly over its CTAs; pieces of a query-tile pair
-    meet in scratch and are merged by whoever finishes last.  Forcing the number of CTAs moves every
-    cut: 1 (no cut at all), a few (long ranges over many pairs), and far more than there are key
-    steps (every pair cut into pieces of four steps)."""
-    from parity_util import lockstep_chunk, make_pair
-    monkeypatch.setenv("LOCRET_ATTN_UNITS", str(units))
-    for d, heads in ((128, (8, 2)), (96, (3, 3)), (64, (4, 1))):
-        sh = _shape(heads[0], heads[1], d)
-        ora, gpu = make_pair(sh, W.layer_weights(sh, 0, seed=W.BASE_SEED + d), budget=900, chunk=384, n_stab=33)
-        for i, n_tok in enumerate([384, 384, 200, 384, 65]):
-            lockstep_chunk(ora, gpu, _hidden(n_tok, sh.d_model, 300 + i), 0, what=f"units {units} d{d} chunk {i}")
-        gpu.destroy()
