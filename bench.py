@@ -36,6 +36,12 @@ DEFAULT_WORKLOAD = "c3_llama_128k"
 # dram__bytes_read.sum + dram__bytes_write.sum of one steady-state attention launch: a literal taken
 # from a profiler capture of the same launch shape (not measured during this run)
 NCU_ATTN_TRAFFIC_BYTES = {"c3_llama_128k": 67.5e6, "c2_llama_32k": 67.5e6}
+# sm__pipe_tensor_cycles_active of the same capture (per cent of cycles; clock-independent)
+NCU_ATTN_TENSOR_PIPE_PCT = 54.7
+# the other benchmark configurations are sampled in the default run: this many layers, contexts cut to this
+OTHER_CONFIGS = ("c2_llama_32k", "c4_phi3_128k", "c5_llama_stream_int4")
+OTHER_LAYERS = 4
+OTHER_CONTEXT = 65536
 
 
 def measured_peaks():
@@ -196,6 +202,111 @@ def job_throughput(world: int, tokens_per_rank: int, ms: float) -> float:
     return world * tokens_per_rank / (ms * 1e-3)
 
 
+# ----------------------------------------------------------------------------- per-kernel rates
+
+def summarise(w, k_ms, k_cnt, steps, peaks):
+    """Per kernel family: launches, time, share, and the rate against the roofline that bounds it
+    (tensor kernels: TFLOP/s of the algorithmic flops against the sustained bf16 peak; compaction:
+    GB/s of the bytes a kept unit costs against the measured copy bandwidth)."""
+    from paper_2410_01805_b200 import K_NAMES
+    s = w.shape
+    fl = step_flops(w) * steps
+    out_k = {}
+    tot = float(k_ms.sum())
+    for i, name in enumerate(K_NAMES):
+        if k_cnt[i]:
+            out_k[name] = {"launches": int(k_cnt[i]), "ms_total": float(k_ms[i]), "share": float(k_ms[i] / tot),
+                           "us_per_launch": float(k_ms[i] / k_cnt[i] * 1e3)}
+    for name, f in (("qkv", fl[0]), ("attn", fl[1]), ("rh", fl[2])):
+        if name in out_k:
+            out_k[name]["tflops"] = float(f / (k_ms[K_NAMES.index(name)] * 1e-3) / 1e12)
+            out_k[name]["frac_of_sustained_bf16"] = out_k[name]["tflops"] / peaks["tf_sustained"]
+    ic = K_NAMES.index("compact")
+    if k_cnt[ic]:
+        if s.kv_dtype == 1:
+            unit_b = 2 * (s.head_dim // 2) * 2 + 2 * 2 * 2 + 2 * (4 + 8)   # codes, scales, score, id: read + write
+        else:
+            unit_b = 2 * s.head_dim * 2 * 2 + 2 * (4 + 8) + s.head_dim * 2   # K, V read + write; score, id; rotated K
+        out_k["compact"]["gbs"] = float(k_cnt[ic] * s.n_kv_heads * w.budget * unit_b / (k_ms[ic] * 1e-3) / 1e9)
+        out_k["compact"]["frac_of_hbm_copy"] = out_k["compact"]["gbs"] / peaks["hbm_gbs"]
+    return out_k
+
+
+def sample_config(name, dev, peaks, n_layers, context, x_shared=None, weights_shared=None):
+    """A short sample of another benchmark configuration, so that the line carries figures for it that
+    were measured in the same run: `n_layers` layers of the stack (the layers are identical in shape
+    and every layer receives the same chunk, so a pass over the whole stack costs full / n_layers times
+    the sample), context cut to `context` tokens; 1 warm-up pass, 2 timed passes, 1 pass with every
+    kernel on one stream for the per-kernel rates."""
+    import torch
+    from paper_2410_01805_b200 import K_NAMES, LocretLayer
+    full = W.get_workload(name)
+    w = full.with_(n_layers=n_layers, context=min(context, full.context))
+    s = w.shape
+    stream = torch.cuda.current_stream()
+    sizes = w.chunk_sizes()
+    if x_shared is not None and x_shared.shape[0] >= w.context and x_shared.shape[1] == s.d_model:
+        x_dev = x_shared[:w.context]
+    else:
+        x_host = torch.empty((w.context, s.d_model), dtype=torch.bfloat16)
+        pos = 0
+        while pos < w.context:
+            n_tok = min(8 * w.chunk, w.context - pos)
+            x_host[pos:pos + n_tok] = torch.from_numpy(W.hidden_states(full, pos, n_tok)).to(torch.bfloat16)
+            pos += n_tok
+        x_dev = x_host.to(dev)
+    layers = []
+    for l in range(n_layers):
+        if weights_shared is not None and l < len(weights_shared):
+            wq, w1, w2 = weights_shared[l]
+        else:
+            wq, w1, w2 = (torch.from_numpy(a).to(torch.bfloat16).to(dev) for a in W.layer_weights(s, l))
+        layers.append(LocretLayer(s, wq, w1, w2, w.budget, w.chunk, w.n_stab, stream=stream))
+    out = torch.empty((w.chunk, s.n_q_heads * s.head_dim), dtype=torch.bfloat16, device=dev)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+
+    def one_pass():
+        for L in layers:
+            L.reset()
+        p = 0
+        for n_tok in sizes:
+            for L in layers:
+                L.prefill_chunk(x_dev[p:p + n_tok], out, 0, n_tok)
+            p += n_tok
+
+    one_pass()
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(2):
+        flush.zero_()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream); one_pass(); b.record(stream)
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b))
+    for L in layers:
+        L.set_timing(2)
+    flush.zero_()
+    one_pass()
+    k_ms = np.zeros(len(K_NAMES)); k_cnt = np.zeros(len(K_NAMES), dtype=np.int64)
+    for L in layers:
+        a, c = L.read_timing(); k_ms += a; k_cnt += c
+        L.set_timing(0)
+    status = max(abs(L.sync_status()) for L in layers)
+    for L in layers:
+        L.destroy()
+    t_ms = float(np.mean(times))
+    scale = full.n_layers / n_layers
+    return {"workload": name,
+            "sample": f"{n_layers} of {full.n_layers} layers, first {w.context} of {full.context} tokens, "
+                      f"1 warm-up + 2 timed passes; tokens_per_s = tokens / (pass time x {scale:g})",
+            "tokens_per_s": w.context / (t_ms * 1e-3 * scale), "ms_per_sampled_pass": t_ms,
+            "us_per_chunk_layer": t_ms * 1e3 / (len(sizes) * n_layers),
+            "tflops_step": float(step_flops(w).sum() / (t_ms * 1e-3) / 1e12),
+            "frac_of_sustained_bf16": float(step_flops(w).sum() / (t_ms * 1e-3) / 1e12 / peaks["tf_sustained"]),
+            "device_status": status,
+            "kernels_isolated": summarise(w, k_ms, k_cnt, 1, peaks)}
+
+
 # ----------------------------------------------------------------------------- our arm
 
 def run_ours(args, w):
@@ -228,10 +339,13 @@ def run_ours(args, w):
     x_dev = x_host.to(dev, non_blocking=True)
     stream = torch.cuda.current_stream()
     layers = []
+    kept_weights = []   # the first layers' weights stay on the device for the samples of the other configurations
     for l in range(w.n_layers):
         wq, w1, w2 = (torch.from_numpy(a).to(torch.bfloat16).to(dev) for a in W.layer_weights(s, l))
         layers.append(LocretLayer(s, wq, w1, w2, w.budget, w.chunk, w.n_stab, reserve=args.decode_steps,
                                   stream=stream))
+        if l < OTHER_LAYERS and not args.no_other_configs:
+            kept_weights.append((wq, w1, w2))
         del wq, w1, w2
     gen_s = time.perf_counter() - t0
 
@@ -309,24 +423,6 @@ def run_ours(args, w):
     # on the library's second stream and overlap attention / the next projection, so their event
     # times (and attention's) include the time they share the SMs; one extra pass with every
     # kernel on one stream gives each kernel's rate when it runs alone.
-    def summarise(k_ms, k_cnt, steps):
-        fl = step_flops(w) * steps
-        out_k = {}
-        tot = float(k_ms.sum())
-        for i, name in enumerate(K_NAMES):
-            if k_cnt[i]:
-                out_k[name] = {"launches": int(k_cnt[i]), "ms_total": float(k_ms[i]), "share": float(k_ms[i] / tot)}
-        for name, f in (("qkv", fl[0]), ("attn", fl[1]), ("rh", fl[2])):
-            out_k[name]["tflops"] = float(f / (k_ms[K_NAMES.index(name)] * 1e-3) / 1e12)
-        ic = K_NAMES.index("compact")
-        if k_cnt[ic]:
-            if s.kv_dtype == 1:
-                unit_b = 2 * (s.head_dim // 2) * 2 + 2 * 2 * 2 + 2 * (4 + 8)   # codes, scales, score, id: read + write
-            else:
-                unit_b = 2 * s.head_dim * 2 * 2 + 2 * (4 + 8) + s.head_dim * 2   # K, V read + write; score, id; rotated K
-            out_k["compact"]["gbs"] = float(k_cnt[ic] * s.n_kv_heads * w.budget * unit_b / (k_ms[ic] * 1e-3) / 1e9)
-        return out_k
-
     # live in the timed region: only the dominant kernel (attention) is bracketed with events, to
     # keep the measurement's own cost out of `value`; the full split comes from the extra pass
     ia = K_NAMES.index("attn")
@@ -340,11 +436,14 @@ def run_ours(args, w):
     for L in layers:
         a, c = L.read_timing(); iso_ms += a; iso_cnt += c
         L.set_timing(0)
-    isolated = summarise(iso_ms, iso_cnt, 1)
+    isolated = summarise(w, iso_ms, iso_cnt, 1, peaks)
     attn_tf = per_kernel["attn"]["tflops"]
     dom = int(np.argmax(iso_ms))
     roofline = {"kernel": "attn", "bound": "tensor", "achieved": float(attn_tf), "peak": peaks["tf_sustained"],
                 "unit": "TFLOP/s", "frac": float(attn_tf / peaks["tf_sustained"]),
+                "frac_of_measured_sustained": float(attn_tf / peaks["tf_sustained"]),
+                "frac_of_datasheet_dense_bf16": float(attn_tf / 2250.0),
+                "ncu_tensor_pipe_active_pct": NCU_ATTN_TENSOR_PIPE_PCT,
                 "traffic": NCU_ATTN_TRAFFIC_BYTES.get(w.name) if not (args.layers or args.context) else None,
                 "traffic_unit": "bytes per steady-state launch (literal from a profiler capture of this launch shape)",
                 "peak_source": f"bf16 sustained, {peaks['source']}", "dominant_by_time": K_NAMES[dom],
@@ -378,6 +477,28 @@ def run_ours(args, w):
                   "frac_of_hbm_peak": step_bytes / (dms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                   "cache_units_per_head": ln, "note": "one request, all layers per token, after the prefill"}
 
+    # ---- the other benchmark configurations, sampled (rank 0 of a single-GPU run only)
+    other = None
+    for L in layers:
+        L.destroy()
+    layers = []
+    if rank == 0 and world == 1 and not args.no_other_configs and not (args.layers or args.context):
+        del out, x_stage
+        torch.cuda.empty_cache()
+        other = []
+        for name in OTHER_CONFIGS:
+            if name == w.name:
+                continue
+            share = W.get_workload(name).shape.d_model == s.d_model and W.get_workload(name).hidden == w.hidden
+            same_w = W.get_workload(name).shape.d_in == s.d_in and W.get_workload(name).shape.d_retain == s.d_retain
+            try:
+                other.append(sample_config(name, dev, peaks, OTHER_LAYERS, OTHER_CONTEXT,
+                                           x_shared=x_dev if share else None,
+                                           weights_shared=kept_weights if (share and same_w) else None))
+            except Exception as e:  # a sample must never take the headline down with it
+                other.append({"workload": name, "error": repr(e)})
+    kept_weights = []
+
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": t_ms, "higher_is_better": True, "scaling": "weak",
@@ -396,14 +517,13 @@ def run_ours(args, w):
         "decode": decode,
         "tflops_step": float(step_flops(w).sum() / (t_ms * 1e-3) / 1e12),
         "setup_s": gen_s,
+        "other_configs": other,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, cores, sample, _ = oracle_sample(w, 2)  # two steady-state chunk-layers: about 15 s of host work
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
     if rank == 0:
         print(json.dumps(line), flush=True)
-    for L in layers:
-        L.destroy()
     if world > 1:
         dist.destroy_process_group()
 
@@ -651,6 +771,8 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling only)")
     ap.add_argument("--context", type=int, default=0, help="override the context length (profiling only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the short samples of the other benchmark configurations")
     ap.add_argument("--no-kernel-timing", action="store_true",
                     help="do not bracket kernels with events in the timed region (to measure that overhead)")
     ap.add_argument("--decode-steps", type=int, default=64, help="decode steps timed after the prefill (0 = none)")
