@@ -204,10 +204,23 @@ def job_throughput(world: int, tokens_per_rank: int, ms: float) -> float:
 
 # ----------------------------------------------------------------------------- per-kernel rates
 
-def summarise(w, k_ms, k_cnt, steps, peaks):
+def compaction_bytes(w, evictions, moved, rotated):
+    """Algorithmic bytes of the in-place gather: per evicting launch the index and position arrays of
+    every slot; per unit moved to another slot K and V read and written, its score and token id; per
+    rotated key rewritten the pre-RoPE key read (a moved unit's is already counted) and the rotated key
+    written."""
+    s = w.shape
+    idx = evictions * s.n_kv_heads * w.budget * 12
+    if s.kv_dtype == 1:
+        return idx + moved * (2 * (s.head_dim // 2) * 2 + 2 * 2 * 2 + 2 * (4 + 8))
+    row = s.head_dim * 2
+    return idx + moved * (4 * row + 2 * (4 + 8)) + (rotated - moved) * row + rotated * row
+
+
+def summarise(w, k_ms, k_cnt, steps, peaks, compact_bytes=None):
     """Per kernel family: launches, time, share, and the rate against the roofline that bounds it
     (tensor kernels: TFLOP/s of the algorithmic flops against the sustained bf16 peak; compaction:
-    GB/s of the bytes a kept unit costs against the measured copy bandwidth)."""
+    GB/s of the bytes it had to move, counted by the library, against the measured copy bandwidth)."""
     from paper_2410_01805_b200 import K_NAMES
     s = w.shape
     fl = step_flops(w) * steps
@@ -222,12 +235,9 @@ def summarise(w, k_ms, k_cnt, steps, peaks):
             out_k[name]["tflops"] = float(f / (k_ms[K_NAMES.index(name)] * 1e-3) / 1e12)
             out_k[name]["frac_of_sustained_bf16"] = out_k[name]["tflops"] / peaks["tf_sustained"]
     ic = K_NAMES.index("compact")
-    if k_cnt[ic]:
-        if s.kv_dtype == 1:
-            unit_b = 2 * (s.head_dim // 2) * 2 + 2 * 2 * 2 + 2 * (4 + 8)   # codes, scales, score, id: read + write
-        else:
-            unit_b = 2 * s.head_dim * 2 * 2 + 2 * (4 + 8) + s.head_dim * 2   # K, V read + write; score, id; rotated K
-        out_k["compact"]["gbs"] = float(k_cnt[ic] * s.n_kv_heads * w.budget * unit_b / (k_ms[ic] * 1e-3) / 1e9)
+    if k_cnt[ic] and compact_bytes is not None:
+        out_k["compact"]["bytes_per_launch"] = float(compact_bytes / k_cnt[ic])
+        out_k["compact"]["gbs"] = float(compact_bytes / (k_ms[ic] * 1e-3) / 1e9)
         out_k["compact"]["frac_of_hbm_copy"] = out_k["compact"]["gbs"] / peaks["hbm_gbs"]
     return out_k
 
@@ -286,11 +296,14 @@ def sample_config(name, dev, peaks, n_layers, context, x_shared=None, weights_sh
     for L in layers:
         L.set_timing(2)
     flush.zero_()
+    c0 = np.sum([L.compaction_counters for L in layers], axis=0)
     one_pass()
+    c1 = np.sum([L.compaction_counters for L in layers], axis=0)
     k_ms = np.zeros(len(K_NAMES)); k_cnt = np.zeros(len(K_NAMES), dtype=np.int64)
     for L in layers:
         a, c = L.read_timing(); k_ms += a; k_cnt += c
         L.set_timing(0)
+    cbytes = compaction_bytes(w, int(k_cnt[K_NAMES.index("compact")]), int(c1[0] - c0[0]), int(c1[1] - c0[1]))
     status = max(abs(L.sync_status()) for L in layers)
     for L in layers:
         L.destroy()
@@ -304,7 +317,7 @@ def sample_config(name, dev, peaks, n_layers, context, x_shared=None, weights_sh
             "tflops_step": float(step_flops(w).sum() / (t_ms * 1e-3) / 1e12),
             "frac_of_sustained_bf16": float(step_flops(w).sum() / (t_ms * 1e-3) / 1e12 / peaks["tf_sustained"]),
             "device_status": status,
-            "kernels_isolated": summarise(w, k_ms, k_cnt, 1, peaks)}
+            "kernels_isolated": summarise(w, k_ms, k_cnt, 1, peaks, cbytes)}
 
 
 # ----------------------------------------------------------------------------- our arm
@@ -431,12 +444,16 @@ def run_ours(args, w):
     for L in layers:
         L.set_timing(2)
     flush.zero_()
+    cc0 = np.sum([L.compaction_counters for L in layers], axis=0)
     prefill_resident()
+    cc1 = np.sum([L.compaction_counters for L in layers], axis=0)
     iso_ms = np.zeros(len(K_NAMES)); iso_cnt = np.zeros(len(K_NAMES), dtype=np.int64)
     for L in layers:
         a, c = L.read_timing(); iso_ms += a; iso_cnt += c
         L.set_timing(0)
-    isolated = summarise(w, iso_ms, iso_cnt, 1, peaks)
+    isolated = summarise(w, iso_ms, iso_cnt, 1, peaks,
+                         compaction_bytes(w, int(iso_cnt[K_NAMES.index("compact")]), int(cc1[0] - cc0[0]),
+                                          int(cc1[1] - cc0[1])))
     attn_tf = per_kernel["attn"]["tflops"]
     dom = int(np.argmax(iso_ms))
     roofline = {"kernel": "attn", "bound": "tensor", "achieved": float(attn_tf), "peak": peaks["tf_sustained"],

@@ -69,7 +69,8 @@ enum {
   LOCRET_K_RH_REDUCE,   /* (c) sum of the retaining head's partial scores (a      */
                         /*     one-token step sums them inside LOCRET_K_RH)        */
   LOCRET_K_TOPK,        /* (d) per-head selection                                 */
-  LOCRET_K_COMPACT,     /* (d) gather / compaction + re-RoPE of kept keys         */
+  LOCRET_K_COMPACT,     /* (d) gather in place + re-RoPE of keys whose position   */
+                        /*     changed                                            */
   LOCRET_K_DEQUANT,     /* 4-bit cache: expansion of the retained units to bf16   */
   LOCRET_K_QUANT,       /* 4-bit cache: quantisation of the chunk's units         */
   LOCRET_K_COUNT
@@ -99,9 +100,9 @@ typedef struct {
 /*
  * Create one layer's state for chunked prefill with a fixed cache budget (Section 3.4;
  * hyper-parameters b, B, n_s of Table 4).  Requires 1 <= chunk, 1 <= budget,
- * 0 <= n_stab <= budget.  Allocates device memory (cache for budget + chunk + reserve
- * units per KV head, double-buffered; scratch), repacks the weights, and synchronises
- * the stream once.  On failure *out is NULL and nothing stays allocated.
+ * 0 <= n_stab <= budget, budget + chunk + reserve <= 262144.  Allocates device memory (cache
+ * for budget + chunk + reserve units per KV head; scratch), repacks the weights, and
+ * synchronises the stream once.  On failure *out is NULL and nothing stays allocated.
  */
 int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, int32_t n_stab,
                   locret_layer **out);
@@ -160,7 +161,8 @@ int locret_cache_len(const locret_layer *layer, int32_t *len);
 /*
  * Copy the retained state to HOST buffers (any may be NULL to skip it): K and V as bf16
  * [h_kv × len × d] (K pre-RoPE), scores fp32 [h_kv × len], token_ids int64 [h_kv × len]
- * (index of the token in the stream), *len, *tokens_seen.  Synchronises the stream.
+ * (index of the token in the stream), *len, *tokens_seen.  Units come in temporal order (the
+ * order of Algorithm 1's gather), whatever slots they occupy on the device.  Synchronises the stream.
  * A layer with a 4-bit cache returns LOCRET_ERR_INVALID if K or V is asked for (its state
  * is exchanged exactly through locret_export_state_int4).
  */
@@ -248,6 +250,15 @@ int locret_read_timing(locret_layer *layer, float *ms, int64_t *launches);
 
 /* Total number of this library's kernels launched for the layer since create. */
 int locret_launch_count(const locret_layer *layer, int64_t *count);
+
+/*
+ * How much the evictions of this layer have moved since create (Algorithm 1's gather, done in place:
+ * kept units stay in their slots, units kept from the chunk refill the freed slots, and a rotated key
+ * is rewritten only where the unit's position in temporal order changed, Section 3.4).  *units_moved:
+ * units (one token of one KV head) copied to another slot; *keys_rotated: rotated keys rewritten.
+ * Either pointer may be NULL.  Synchronises the layer's streams.
+ */
+int locret_compaction_counters(locret_layer *layer, int64_t *units_moved, int64_t *keys_rotated);
 
 /*
  * ---- The rest of the decoder layer (beyond the scope of the chunk step itself) ----

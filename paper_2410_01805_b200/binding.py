@@ -66,6 +66,7 @@ def _load():
     l.locret_set_timing.argtypes = [P, C.c_int32]
     l.locret_read_timing.argtypes = [P, P, P]
     l.locret_launch_count.argtypes = [P, C.POINTER(C.c_int64)]
+    l.locret_compaction_counters.argtypes = [P, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
     l.locret_rh_scores_static.argtypes = [P, C.c_int32, C.c_int32, P, C.c_int32, P, C.c_int32, C.c_int32, P, P, P]
     l.locret_selftest_wait_abort.argtypes = [P, P]
     l.locret_destroy.argtypes = [P]
@@ -231,6 +232,13 @@ class LocretLayer:
         n = C.c_int64()
         _check(lib.locret_launch_count(self._h, C.byref(n)), "locret_launch_count")
         return n.value
+
+    @property
+    def compaction_counters(self):
+        """(units moved to another slot, rotated keys rewritten) by this layer's evictions since create."""
+        a, b = C.c_int64(), C.c_int64()
+        _check(lib.locret_compaction_counters(self._h, C.byref(a), C.byref(b)), "locret_compaction_counters")
+        return a.value, b.value
 
     def destroy(self):
         if self._h:

@@ -179,21 +179,30 @@ cudaError_t launch_attention_mma(const bf16 *q_rot, const bf16 *k_rot, const bf1
                                  int n_tok, int h, int h_kv, int d, int cap, int len,
                                  cudaStream_t st);
 
-// keep[m][0..budget) = ascending slots kept among n candidates (the first n_pre and the last n_prot
-// protected).
-cudaError_t launch_topk(const float *scores, int score_stride, int h_kv, int n, int budget,
-                        int n_prot, int n_pre, int32_t *keep, cudaStream_t st);
+// Eviction in place.  Kept units stay in their slots and freed slots below `budget` are refilled, so
+// slot order is not temporal order: a unit's position in temporal order is its RANK, stored per slot
+// for slots below `ranked_len`; slots from there on (appended since the last eviction) are in order,
+// rank = slot.
+struct TopkArgs {
+  const float *scores;      // [h_kv][stride]
+  const int32_t *rank_old;  // [h_kv][stride]
+  int stride, ranked_len;
+  int n, budget, n_prot, n_pre;   // candidates: slots [0, n); ranks [0, n_pre) and [n - n_prot, n) protected
+  int32_t *src_of;          // [h_kv][budget]  out: the slot whose unit ends up in slot i
+  int32_t *rank_new;        // [h_kv][stride]  out: rank after the eviction, for slots < budget (the
+                            //                 entries from budget on are used as scratch)
+  unsigned long long *counters;  // [2] or null: units moved to another slot, rotated keys rewritten (added to)
+};
+cudaError_t launch_topk(const TopkArgs &a, int h_kv, cudaStream_t st);
 
 struct CompactArgs {
-  const bf16 *k_src, *v_src;
-  const float *s_src;
-  const int64_t *t_src;
-  bf16 *k_dst, *v_dst, *k_rot;
-  float *s_dst;
-  int64_t *t_dst;
-  const int32_t *keep;  // [h_kv][budget]
+  bf16 *k, *v, *k_rot;      // [h_kv][cap][d]
+  float *s;                 // [h_kv][cap]
+  int64_t *t;
+  const int32_t *src_of;    // [h_kv][budget]
+  const int32_t *rank_new, *rank_old;  // [h_kv][cap]
   const float2 *cs;
-  int h_kv, d, cap, budget;
+  int h_kv, d, cap, budget, ranked_len;
 };
 cudaError_t launch_compact(const CompactArgs &a, cudaStream_t st);
 
@@ -206,17 +215,18 @@ struct Int4Half {
   uint8_t *kq, *vq;  // [h_kv][cap][d/2] two codes per byte, even element in the low nibble
   __half *ks, *vs;   // [h_kv][cap] one scale per head vector
 };
-// Expand slots [0, len) into bf16: keys rotated at position = slot when `rotate`, values plain.
+// Expand slots [0, len) into bf16: keys rotated at the unit's position in temporal order when `rotate`
+// (rank[m * cap + slot] for slot < ranked_len, the slot itself above; rank may be null: position = slot),
+// values plain.
 cudaError_t launch_dequant(const Int4Half &q, bf16 *k_out, bf16 *v_out, const float2 *cs, int h_kv, int d,
-                           int cap, int len, bool rotate, cudaStream_t st);
+                           int cap, int len, bool rotate, const int32_t *rank, int ranked_len, cudaStream_t st);
 // Quantise n_tok vectors per KV head into slots [slot0, slot0 + n_tok).  Vector (t, m) of K is at
 // k_src + t * tok_stride + m * head_stride (elements), likewise V.
 cudaError_t launch_quantize(const bf16 *k_src, const bf16 *v_src, long long tok_stride,
                             long long head_stride, const Int4Half &q, int n_tok, int h_kv, int d, int cap,
                             int slot0, cudaStream_t st);
-cudaError_t launch_compact_int4(const Int4Half &src, const Int4Half &dst, const float *s_src,
-                                const int64_t *t_src, float *s_dst, int64_t *t_dst, const int32_t *keep,
-                                int h_kv, int d, int cap, int budget, cudaStream_t st);
+cudaError_t launch_compact_int4(const Int4Half &q, float *s, int64_t *t, const int32_t *src_of, int h_kv, int d,
+                                int cap, int budget, cudaStream_t st);
 
 // ---- decoding (decode.cu): one token
 cudaError_t launch_gemv(const bf16 *x, const bf16 *Wt, int N, int K, bf16 *y, cudaStream_t st);
@@ -239,12 +249,13 @@ int decode_attn_splits(int h_kv, int n);
 // part_o: fp32 [h][n_splits][d]; part_ml: fp32 [h][n_splits][2]; counters: one zeroed word per
 // (KV head, group of 16 query heads), left at zero (the last split merges the partial results).
 // q4 != nullptr: keys [0, n - 1) are read from the 4-bit cache (expanded and rotated with `cs` on the
-// way into shared memory) and only key n - 1, the token of this step, from k_rot / v.
+// way into shared memory, at position rank[m * cap + slot] for slot < ranked_len and slot above) and only
+// key n - 1, the token of this step, from k_rot / v.
 struct Int4Half;
 cudaError_t launch_attention_decode(const bf16 *q_rot, const bf16 *k_rot, const bf16 *v, bf16 *out,
                                     float *part_o, float *part_ml, unsigned *counters, int h, int h_kv, int d,
                                     int cap, int n, int n_splits, const Int4Half *q4, const float2 *cs,
-                                    cudaStream_t st);
+                                    const int32_t *rank, int ranked_len, cudaStream_t st);
 
 // dst[c][r] = src[r][c]  (weight repack at create)
 cudaError_t launch_transpose_bf16(const bf16 *src, bf16 *dst, int rows, int cols, cudaStream_t st);

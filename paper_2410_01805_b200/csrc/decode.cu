@@ -301,8 +301,8 @@ __device__ __forceinline__ uint4 to_bf16x8(const float (&x)[8]) {
 // order (a wrapping atomic counter, left at zero for the next step).
 constexpr int DA_THREADS = 128, DA_G = 16, DA_KT = 64;
 
-// INT4: keys [0, n - 1) come from the 4-bit cache (codes and scales expanded, keys rotated at
-// position = slot, with the arithmetic of the expansion pre-pass, as the tile is brought into shared
+// INT4: keys [0, n - 1) come from the 4-bit cache (codes and scales expanded, keys rotated at the
+// unit's position in temporal order, with the arithmetic of the expansion pre-pass, as the tile is brought into shared
 // memory); key n - 1, the token of this step, comes from the bf16 arrays k_rot / v like every key of
 // a bf16 cache.
 template <int D, bool INT4>
@@ -311,7 +311,7 @@ attn_decode_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_ro
                    const bf16 *__restrict__ v, float *__restrict__ part_o, float *__restrict__ part_ml,
                    int h, int h_kv, int cap, int n, int n_splits, float scale_log2,
                    unsigned *__restrict__ counters, bf16 *__restrict__ out, Int4Half q4,
-                   const float2 *__restrict__ cs) {
+                   const float2 *__restrict__ cs, const int32_t *__restrict__ rank, int ranked_len) {
   constexpr int LD = D + 8;
   constexpr int VPR = D / 8;  // 16-byte vectors per row
   extern __shared__ __align__(16) unsigned char da_smem[];
@@ -359,7 +359,8 @@ attn_decode_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_ro
         float a[8], b[8];
         dequant8(*reinterpret_cast<const uint32_t *>(kc + c / 2), ks, a);
         dequant8(*reinterpret_cast<const uint32_t *>(kc + (c + HALF) / 2), ks, b);
-        const float2 *t = cs + (size_t)key * HALF + c;
+        const int pos = key < ranked_len ? rank[u] : key;  // the unit's place in temporal order
+        const float2 *t = cs + (size_t)pos * HALF + c;
 #pragma unroll
         for (int e = 0; e < 8; e++) {
           const float x1 = a[e], x2 = b[e];
@@ -673,7 +674,7 @@ int decode_attn_splits(int h_kv, int n) {
 cudaError_t launch_attention_decode(const bf16 *q_rot, const bf16 *k_rot, const bf16 *v, bf16 *out,
                                     float *part_o, float *part_ml, unsigned *counters, int h, int h_kv, int d,
                                     int cap, int n, int n_splits, const Int4Half *q4, const float2 *cs,
-                                    cudaStream_t st) {
+                                    const int32_t *rank, int ranked_len, cudaStream_t st) {
   const int g = h / h_kv;
   dim3 grid(h_kv, n_splits, (g + DA_G - 1) / DA_G);
   if ((int)grid.x * (int)grid.z > 32 * 16 || n_splits > 64) return cudaErrorInvalidValue;
@@ -682,7 +683,7 @@ cudaError_t launch_attention_decode(const bf16 *q_rot, const bf16 *k_rot, const 
   auto launch = [&](auto kern, int smem, PerDeviceFlag &attr_set) -> cudaError_t {
     if (cudaError_t e = allow_dynamic_smem(kern, smem, attr_set); e != cudaSuccess) return e;
     kern<<<grid, DA_THREADS, smem, st>>>(q_rot, k_rot, v, part_o, part_ml, h, h_kv, cap, n, n_splits,
-                                         scale_log2, counters, out, qq, cs);
+                                         scale_log2, counters, out, qq, cs, rank, rank ? ranked_len : 0);
     return cudaGetLastError();
   };
   static PerDeviceFlag set_done[2][3];

@@ -3,8 +3,8 @@
 // scale per head vector: scale = fp16(absmax / 7) (1 if that is zero),
 // code = clamp(rint(x / scale), -8, 7), decided in fp32.  Units are quantised when they enter
 // the cache; the keys are stored pre-RoPE.  Before attention a pre-pass expands the retained
-// units into bf16 scratch (keys rotated at position = slot), so the attention kernels are the
-// same as for a bf16 cache; compaction moves codes and scales unchanged.
+// units into bf16 scratch (keys rotated at the unit's position in temporal order, its rank), so
+// the attention kernels are the same as for a bf16 cache; eviction moves codes and scales unchanged.
 #include "common.cuh"
 
 namespace locret {
@@ -33,7 +33,7 @@ __device__ __forceinline__ uint4 to_bf16x8(const float (&x)[8]) {
 // One thread: elements [c, c+8) and [c+half, c+half+8) of one (head, slot) vector of K and V.
 __global__ void dequant_rope_kernel(Int4Half q, bf16 *__restrict__ k_rot, bf16 *__restrict__ v_out,
                                     const float2 *__restrict__ cs, int h_kv, int d, int cap, int len,
-                                    int rotate) {
+                                    int rotate, const int32_t *__restrict__ rank, int ranked_len) {
   const int row = blockIdx.x * blockDim.y + threadIdx.y;
   if (row >= h_kv * len) return;
   const int m = row / len, i = row - m * len;
@@ -45,7 +45,8 @@ __global__ void dequant_rope_kernel(Int4Half q, bf16 *__restrict__ k_rot, bf16 *
   dequant8(*reinterpret_cast<const uint32_t *>(kc + c / 2), ks, a);
   dequant8(*reinterpret_cast<const uint32_t *>(kc + (c + half) / 2), ks, b);
   if (rotate) {
-    const float2 *t = cs + (size_t)i * half + c;
+    const int pos = i < ranked_len ? rank[u] : i;
+    const float2 *t = cs + (size_t)pos * half + c;
 #pragma unroll
     for (int e = 0; e < 8; e++) {
       const float x1 = a[e], x2 = b[e];
@@ -105,40 +106,41 @@ __global__ void quantize_kernel(const bf16 *__restrict__ k_src, const bf16 *__re
   if (lane == 0) (is_v ? q.vs : q.ks)[u] = sh;
 }
 
-// Gather codes, scales, scores and token ids of the kept units (temporal order kept).
-__global__ void compact_int4_kernel(Int4Half src, Int4Half dst, const float *__restrict__ s_src,
-                                    const int64_t *__restrict__ t_src, float *__restrict__ s_dst,
-                                    int64_t *__restrict__ t_dst, const int32_t *__restrict__ keep,
-                                    int h_kv, int d, int cap, int budget) {
+// Eviction in place: the units that come from another slot bring their codes, scales, score and
+// token id along (src_of[m][i] is the slot whose unit ends up in slot i; sources lie at or above
+// budget, destinations below).
+__global__ void compact_int4_kernel(Int4Half q, float *__restrict__ s, int64_t *__restrict__ t,
+                                    const int32_t *__restrict__ src_of, int h_kv, int d, int cap, int budget) {
   const int row = blockIdx.x * blockDim.y + threadIdx.y;
   if (row >= h_kv * budget) return;
   const int m = row / budget, i = row - m * budget;
-  const int from = keep[(size_t)m * budget + i];
+  const int from = src_of[(size_t)m * budget + i];
+  if (from == i) return;
   const size_t us = (size_t)m * cap + from, ud = (size_t)m * cap + i;
   const int vecs = d / 32;  // 16-byte vectors per code row (d/2 bytes)
   const int x = threadIdx.x;
   if (x < vecs)
-    reinterpret_cast<uint4 *>(dst.kq + ud * (d / 2))[x] = reinterpret_cast<const uint4 *>(src.kq + us * (d / 2))[x];
+    reinterpret_cast<uint4 *>(q.kq + ud * (d / 2))[x] = reinterpret_cast<const uint4 *>(q.kq + us * (d / 2))[x];
   else if (x < 2 * vecs)
-    reinterpret_cast<uint4 *>(dst.vq + ud * (d / 2))[x - vecs] =
-        reinterpret_cast<const uint4 *>(src.vq + us * (d / 2))[x - vecs];
+    reinterpret_cast<uint4 *>(q.vq + ud * (d / 2))[x - vecs] =
+        reinterpret_cast<const uint4 *>(q.vq + us * (d / 2))[x - vecs];
   if (x == 0) {
-    dst.ks[ud] = src.ks[us];
-    dst.vs[ud] = src.vs[us];
-    s_dst[ud] = s_src[us];
-    t_dst[ud] = t_src[us];
+    q.ks[ud] = q.ks[us];
+    q.vs[ud] = q.vs[us];
+    s[ud] = s[us];
+    t[ud] = t[us];
   }
 }
 
 }  // namespace
 
 cudaError_t launch_dequant(const Int4Half &q, bf16 *k_out, bf16 *v_out, const float2 *cs, int h_kv, int d,
-                           int cap, int len, bool rotate, cudaStream_t st) {
+                           int cap, int len, bool rotate, const int32_t *rank, int ranked_len, cudaStream_t st) {
   if (len == 0) return cudaSuccess;
   const int tx = d / 16, ty = 256 / tx;
   const int rows = h_kv * len;
   dequant_rope_kernel<<<(rows + ty - 1) / ty, dim3(tx, ty), 0, st>>>(q, k_out, v_out, cs, h_kv, d, cap, len,
-                                                                    rotate ? 1 : 0);
+                                                                    rotate ? 1 : 0, rank, rank ? ranked_len : 0);
   return cudaGetLastError();
 }
 
@@ -153,13 +155,11 @@ cudaError_t launch_quantize(const bf16 *k_src, const bf16 *v_src, long long tok_
   return cudaGetLastError();
 }
 
-cudaError_t launch_compact_int4(const Int4Half &src, const Int4Half &dst, const float *s_src,
-                                const int64_t *t_src, float *s_dst, int64_t *t_dst, const int32_t *keep,
-                                int h_kv, int d, int cap, int budget, cudaStream_t st) {
+cudaError_t launch_compact_int4(const Int4Half &q, float *s, int64_t *t, const int32_t *src_of, int h_kv, int d,
+                                int cap, int budget, cudaStream_t st) {
   const int tx = 2 * (d / 32), ty = 256 / tx;
   const int rows = h_kv * budget;
-  compact_int4_kernel<<<(rows + ty - 1) / ty, dim3(tx, ty), 0, st>>>(src, dst, s_src, t_src, s_dst, t_dst,
-                                                                    keep, h_kv, d, cap, budget);
+  compact_int4_kernel<<<(rows + ty - 1) / ty, dim3(tx, ty), 0, st>>>(q, s, t, src_of, h_kv, d, cap, budget);
   return cudaGetLastError();
 }
 

@@ -75,13 +75,18 @@ struct locret_layer {
   ScratchPool *pool;
   bf16 *wqkv_t, *w1_t;
   float *w2f;
-  bf16 *k_pre[2], *v[2], *k_rot;  // bf16 cache (null for a 4-bit cache)
+  bf16 *k_pre, *v, *k_rot;        // bf16 cache (null for a 4-bit cache)
   bool int4;
-  Int4Half q4[2];                 // 4-bit cache
+  Int4Half q4;                    // 4-bit cache
   const void *map_kv_base;
-  float *s[2];
-  int64_t *tid[2];
-  int cur;
+  float *s;
+  int64_t *tid;
+  // Eviction works in place, so slot order is not temporal order: rank[rcur][m][slot] is the unit's
+  // position in temporal order for slot < ranked_len; slots from there on are in order (rank = slot).
+  // The other array receives the ranks of the next eviction.
+  int32_t *rank[2];
+  int rcur, ranked_len;
+  unsigned long long *d_counters;  // [2]: units moved to another slot, rotated keys rewritten
   int device;  // the device that was current at create: every later call must find it current
   const float2 *cs;
   int *d_status;
@@ -100,7 +105,7 @@ struct locret_layer {
   uint32_t tp_flags;
   cudaEvent_t ev_ready, ev_attn, ev_side, ev_tp;  // ev_tp: the divided-heads exchange (both directions)
   bool tc_attn;  // tensor maps for the tcgen05 attention kernel are valid
-  CUtensorMap map_k, map_v[2], map_q;
+  CUtensorMap map_k, map_v, map_q;
   const void *map_q_base;
   std::vector<TimedEvent> events;
   size_t events_used;
@@ -110,10 +115,9 @@ namespace {
 
 void free_layer_memory(locret_layer *L) {
   cudaFree(L->wqkv_t); cudaFree(L->w1_t); cudaFree(L->w2f);
-  for (int i = 0; i < 2; i++) {
-    cudaFree(L->k_pre[i]); cudaFree(L->v[i]); cudaFree(L->s[i]); cudaFree(L->tid[i]);
-    cudaFree(L->q4[i].kq); cudaFree(L->q4[i].vq); cudaFree(L->q4[i].ks); cudaFree(L->q4[i].vs);
-  }
+  cudaFree(L->k_pre); cudaFree(L->v); cudaFree(L->s); cudaFree(L->tid);
+  cudaFree(L->q4.kq); cudaFree(L->q4.vq); cudaFree(L->q4.ks); cudaFree(L->q4.vs);
+  cudaFree(L->rank[0]); cudaFree(L->rank[1]); cudaFree(L->d_counters);
   cudaFree(L->k_rot); cudaFree(L->d_status);
   for (auto &e : L->events) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
   if (L->ev_ready) cudaEventDestroy(L->ev_ready);
@@ -204,6 +208,42 @@ cudaError_t sync_all(locret_layer *L) {
   return e;
 }
 
+// Export in temporal order.  The cache keeps units where eviction left them; slot `i` of head `m`
+// holds the unit of position rank[m][i] (for i below ranked_len; the slot itself above).  The arrays
+// are copied to the host as they lie and put in order there (an export is a diagnostic path).
+struct TemporalOrder {
+  std::vector<int32_t> rank;  // [h_kv][ranked] or empty when the cache is in order
+  int ranked = 0;
+  int load(locret_layer *L) {
+    ranked = L->ranked_len < L->len ? L->ranked_len : L->len;
+    if (ranked == 0) return LOCRET_OK;
+    rank.resize((size_t)L->h_kv * ranked);
+    CK(cudaMemcpy2D(rank.data(), (size_t)ranked * 4, L->rank[L->rcur], (size_t)L->cap * 4, (size_t)ranked * 4,
+                    L->h_kv, cudaMemcpyDeviceToHost));
+    return LOCRET_OK;
+  }
+  // rows of `row_bytes` bytes, device pitch cap * row_bytes per head -> out [h_kv][len][row_bytes]
+  int copy_out(locret_layer *L, const void *dev, size_t row_bytes, void *out) {
+    const int n = L->len;
+    const size_t dense = (size_t)n * row_bytes, pitch = (size_t)L->cap * row_bytes;
+    if (ranked == 0) {
+      CK(cudaMemcpy2D(out, dense, dev, pitch, dense, L->h_kv, cudaMemcpyDeviceToHost));
+      return LOCRET_OK;
+    }
+    std::vector<unsigned char> tmp;
+    try { tmp.resize((size_t)L->h_kv * dense); } catch (...) { return LOCRET_ERR_ALLOC; }
+    CK(cudaMemcpy2D(tmp.data(), dense, dev, pitch, dense, L->h_kv, cudaMemcpyDeviceToHost));
+    unsigned char *o = static_cast<unsigned char *>(out);
+    for (int m = 0; m < L->h_kv; m++)
+      for (int i = 0; i < n; i++) {
+        const int r = i < ranked ? rank[(size_t)m * ranked + i] : i;
+        if (r < 0 || r >= n) return LOCRET_ERR_CUDA;  // a rank outside the cache: the state is corrupt
+        memcpy(o + ((size_t)m * n + r) * row_bytes, tmp.data() + ((size_t)m * n + i) * row_bytes, row_bytes);
+      }
+    return LOCRET_OK;
+  }
+};
+
 }  // namespace
 
 extern "C" {
@@ -237,7 +277,7 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   if (!cfg->w_qkv || !cfg->w1 || !cfg->w2) return LOCRET_ERR_INVALID;
   if (!aligned16(cfg->w_qkv) || !aligned16(cfg->w1)) return LOCRET_ERR_INVALID;
   const long long cap_ll = (long long)budget + chunk + cfg->reserve;
-  if (cap_ll > (1ll << 24)) return LOCRET_ERR_INVALID;
+  if (cap_ll > (1ll << 18)) return LOCRET_ERR_INVALID;  // (the selection keeps bitmaps of all candidates in shared memory)
 
   int ndev = 0, dev = 0;
   if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) { cudaGetLastError(); return LOCRET_ERR_CUDA; }
@@ -252,7 +292,7 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   L->st = (cudaStream_t)cfg->stream;
   L->device = dev;
   L->n_prefix = 0;
-  L->cur = 0; L->len = 0; L->seen = 0; L->launches = 0; L->timing = false; L->serialize = false; L->attn_only = false; L->events_used = 0;
+  L->rcur = 0; L->ranked_len = 0; L->len = 0; L->seen = 0; L->launches = 0; L->timing = false; L->serialize = false; L->attn_only = false; L->events_used = 0;
   L->pool = nullptr;
   {
     const char *e = getenv("LOCRET_LEGACY_MMA");
@@ -271,24 +311,25 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   const size_t code_b = (size_t)hk * L->cap * (d / 2), scale_b = (size_t)hk * L->cap * sizeof(__half);
   const size_t sc_b = (size_t)hk * L->cap * sizeof(float);
   const size_t td_b = (size_t)hk * L->cap * sizeof(int64_t);
+  const size_t rk_b = (size_t)hk * L->cap * sizeof(int32_t);
   bool ok = true;
   ok = ok && cudaMalloc(&L->wqkv_t, (size_t)L->d_in * D * sizeof(bf16)) == cudaSuccess;
   ok = ok && cudaMalloc(&L->w1_t, (size_t)dR * L->d_in * sizeof(bf16)) == cudaSuccess;
   ok = ok && cudaMalloc(&L->w2f, (size_t)dR * hk * sizeof(float)) == cudaSuccess;
-  for (int i = 0; i < 2 && ok; i++) {
-    if (L->int4) {
-      ok = ok && cudaMalloc(&L->q4[i].kq, code_b) == cudaSuccess;
-      ok = ok && cudaMalloc(&L->q4[i].vq, code_b) == cudaSuccess;
-      ok = ok && cudaMalloc(&L->q4[i].ks, scale_b) == cudaSuccess;
-      ok = ok && cudaMalloc(&L->q4[i].vs, scale_b) == cudaSuccess;
-    } else {
-      ok = ok && cudaMalloc(&L->k_pre[i], kv_b) == cudaSuccess;
-      ok = ok && cudaMalloc(&L->v[i], kv_b) == cudaSuccess;
-    }
-    ok = ok && cudaMalloc(&L->s[i], sc_b) == cudaSuccess;
-    ok = ok && cudaMalloc(&L->tid[i], td_b) == cudaSuccess;
+  if (L->int4) {
+    ok = ok && cudaMalloc(&L->q4.kq, code_b) == cudaSuccess;
+    ok = ok && cudaMalloc(&L->q4.vq, code_b) == cudaSuccess;
+    ok = ok && cudaMalloc(&L->q4.ks, scale_b) == cudaSuccess;
+    ok = ok && cudaMalloc(&L->q4.vs, scale_b) == cudaSuccess;
+  } else {
+    ok = ok && cudaMalloc(&L->k_pre, kv_b) == cudaSuccess;
+    ok = ok && cudaMalloc(&L->v, kv_b) == cudaSuccess;
+    ok = ok && cudaMalloc(&L->k_rot, kv_b) == cudaSuccess;
   }
-  if (!L->int4) ok = ok && cudaMalloc(&L->k_rot, kv_b) == cudaSuccess;
+  ok = ok && cudaMalloc(&L->s, sc_b) == cudaSuccess;
+  ok = ok && cudaMalloc(&L->tid, td_b) == cudaSuccess;
+  for (int i = 0; i < 2; i++) ok = ok && cudaMalloc(&L->rank[i], rk_b) == cudaSuccess;
+  ok = ok && cudaMalloc(&L->d_counters, 2 * sizeof(unsigned long long)) == cudaSuccess;
   ok = ok && cudaMalloc(&L->d_status, sizeof(int)) == cudaSuccess;
   if (!ok) { cudaGetLastError(); free_layer_memory(L); delete L; return LOCRET_ERR_ALLOC; }
 
@@ -364,9 +405,7 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
     L->tc_attn = L->use_tc &&
                  tmap_encode_3d_bf16(&L->map_k, L->k_rot, d, L->cap, hk, (uint64_t)d * 2,
                                      (uint64_t)L->cap * d * 2, 64, 128, 1) &&
-                 tmap_encode_3d_bf16(&L->map_v[0], L->v[0], d, L->cap, hk, (uint64_t)d * 2,
-                                     (uint64_t)L->cap * d * 2, 64, 128, 1) &&
-                 tmap_encode_3d_bf16(&L->map_v[1], L->v[1], d, L->cap, hk, (uint64_t)d * 2,
+                 tmap_encode_3d_bf16(&L->map_v, L->v, d, L->cap, hk, (uint64_t)d * 2,
                                      (uint64_t)L->cap * d * 2, 64, 128, 1);
 
   // repack the weights: K-major copies for both GEMMs, W2 in fp32
@@ -374,20 +413,22 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   if (e == cudaSuccess) e = launch_transpose_bf16((const bf16 *)cfg->w_qkv, L->wqkv_t, D, L->d_in, L->st);
   if (e == cudaSuccess) e = launch_transpose_bf16((const bf16 *)cfg->w1, L->w1_t, L->d_in, dR, L->st);
   if (e == cudaSuccess) e = launch_bf16_to_f32((const bf16 *)cfg->w2, L->w2f, dR * hk, L->st);
-  for (int i = 0; i < 2 && e == cudaSuccess; i++) {
+  if (e == cudaSuccess) {
     if (L->int4) {
-      e = cudaMemsetAsync(L->q4[i].kq, 0, code_b, L->st);
-      if (e == cudaSuccess) e = cudaMemsetAsync(L->q4[i].vq, 0, code_b, L->st);
-      if (e == cudaSuccess) e = cudaMemsetAsync(L->q4[i].ks, 0, scale_b, L->st);
-      if (e == cudaSuccess) e = cudaMemsetAsync(L->q4[i].vs, 0, scale_b, L->st);
+      e = cudaMemsetAsync(L->q4.kq, 0, code_b, L->st);
+      if (e == cudaSuccess) e = cudaMemsetAsync(L->q4.vq, 0, code_b, L->st);
+      if (e == cudaSuccess) e = cudaMemsetAsync(L->q4.ks, 0, scale_b, L->st);
+      if (e == cudaSuccess) e = cudaMemsetAsync(L->q4.vs, 0, scale_b, L->st);
     } else {
-      e = cudaMemsetAsync(L->k_pre[i], 0, kv_b, L->st);
-      if (e == cudaSuccess) e = cudaMemsetAsync(L->v[i], 0, kv_b, L->st);
+      e = cudaMemsetAsync(L->k_pre, 0, kv_b, L->st);
+      if (e == cudaSuccess) e = cudaMemsetAsync(L->v, 0, kv_b, L->st);
+      if (e == cudaSuccess) e = cudaMemsetAsync(L->k_rot, 0, kv_b, L->st);
     }
-    if (e == cudaSuccess) e = cudaMemsetAsync(L->s[i], 0, sc_b, L->st);
-    if (e == cudaSuccess) e = cudaMemsetAsync(L->tid[i], 0, td_b, L->st);
   }
-  if (e == cudaSuccess && !L->int4) e = cudaMemsetAsync(L->k_rot, 0, kv_b, L->st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(L->s, 0, sc_b, L->st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(L->tid, 0, td_b, L->st);
+  for (int i = 0; i < 2 && e == cudaSuccess; i++) e = cudaMemsetAsync(L->rank[i], 0, rk_b, L->st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(L->d_counters, 0, 2 * sizeof(unsigned long long), L->st);
   if (e == cudaSuccess) e = cudaMemsetAsync(L->d_status, 0, sizeof(int), L->st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(L->st);
   if (e != cudaSuccess) {
@@ -406,30 +447,34 @@ namespace {
 // (d) of the step: protect, top-b, gather; then the bookkeeping that closes the step
 int evict_and_close(locret_layer *L, int n_tok, uint32_t flags, bool side, cudaStream_t S) {
   ScratchPool *P = L->pool;
-  const int c = L->cur, n = L->len + n_tok;
+  const int n = L->len + n_tok;
   if (!(flags & LOCRET_NO_EVICT) && n > L->budget) {
     const int n_prot = (flags & LOCRET_LAST_CHUNK) ? 0 : (L->n_stab < n ? L->n_stab : n);
+    int32_t *const rank_old = L->rank[L->rcur], *const rank_new = L->rank[L->rcur ^ 1];
     {
       Timed t(L, LOCRET_K_TOPK, S);
       // (n_prefix + n_stab <= budget < n, so the prefix never reaches into the protected tail)
-      CK(launch_topk(L->s[c], L->cap, L->h_kv, n, L->budget, n_prot, L->n_prefix, P->keep, S));
+      TopkArgs a;
+      a.scores = L->s; a.rank_old = rank_old; a.stride = L->cap; a.ranked_len = L->ranked_len;
+      a.n = n; a.budget = L->budget; a.n_prot = n_prot; a.n_pre = L->n_prefix;
+      a.src_of = P->keep; a.rank_new = rank_new; a.counters = L->d_counters;
+      CK(launch_topk(a, L->h_kv, S));
     }
-    // compaction rewrites the rotated keys the attention kernel reads
+    // the gather rewrites keys and values that the attention kernel reads
     if (side) CK(cudaStreamWaitEvent(S, L->ev_attn, 0));
     if (L->int4) {
       Timed t(L, LOCRET_K_COMPACT, S);
-      CK(launch_compact_int4(L->q4[c], L->q4[c ^ 1], L->s[c], L->tid[c], L->s[c ^ 1], L->tid[c ^ 1],
-                             P->keep, L->h_kv, L->d, L->cap, L->budget, S));
+      CK(launch_compact_int4(L->q4, L->s, L->tid, P->keep, L->h_kv, L->d, L->cap, L->budget, S));
     } else {
       Timed t(L, LOCRET_K_COMPACT, S);
       CompactArgs a;
-      a.k_src = L->k_pre[c]; a.v_src = L->v[c]; a.s_src = L->s[c]; a.t_src = L->tid[c];
-      a.k_dst = L->k_pre[c ^ 1]; a.v_dst = L->v[c ^ 1]; a.s_dst = L->s[c ^ 1]; a.t_dst = L->tid[c ^ 1];
-      a.k_rot = L->k_rot; a.keep = P->keep; a.cs = L->cs;
-      a.h_kv = L->h_kv; a.d = L->d; a.cap = L->cap; a.budget = L->budget;
+      a.k = L->k_pre; a.v = L->v; a.k_rot = L->k_rot; a.s = L->s; a.t = L->tid;
+      a.src_of = P->keep; a.rank_new = rank_new; a.rank_old = rank_old; a.cs = L->cs;
+      a.h_kv = L->h_kv; a.d = L->d; a.cap = L->cap; a.budget = L->budget; a.ranked_len = L->ranked_len;
       CK(launch_compact(a, S));
     }
-    L->cur = c ^ 1;
+    L->rcur ^= 1;
+    L->ranked_len = L->budget;
     L->len = L->budget;
   } else {
     L->len = n;
@@ -456,7 +501,6 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
   const int n = L->len + n_tok;
   if (n > L->cap) return LOCRET_ERR_CAPACITY;
   ScratchPool *P = L->pool;
-  const int c = L->cur;
   const bool tp = tp_partial != nullptr;
   const bool decode = n_tok == 1 && L->use_tc && !tp;  // one token: bandwidth-bound kernels of decode.cu
   const bool side = L->use_side && !L->serialize;
@@ -476,11 +520,11 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
 
   // a 4-bit cache is expanded into bf16 scratch first: keys rotated at position = slot
   bf16 *const k_att = L->int4 ? P->k_exp : L->k_rot;
-  bf16 *const v_att = L->int4 ? P->v_exp : L->v[c];
+  bf16 *const v_att = L->int4 ? P->v_exp : L->v;
   RopeAppendArgs ra;  // positions, RoPE, append of the chunk's units at slots [len, len + n_tok)
   ra.staging = staging; ra.q_rot = P->q_rot;
   ra.z_post = L->cfg.rh_input == 1 ? z_post : nullptr;
-  ra.k_pre = L->int4 ? nullptr : L->k_pre[c]; ra.k_rot = k_att; ra.v = v_att; ra.tid = L->tid[c]; ra.cs = L->cs;
+  ra.k_pre = L->int4 ? nullptr : L->k_pre; ra.k_rot = k_att; ra.v = v_att; ra.tid = L->tid; ra.cs = L->cs;
   ra.n_tok = n_tok; ra.h = L->h; ra.h_kv = L->h_kv; ra.d = L->d; ra.cap = L->cap; ra.len = L->len;
   ra.seen = L->seen;
   // with a tensor-core projection whose width is a whole number of tiles the epilogue of the GEMM does the RoPE pass
@@ -495,7 +539,8 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
     if (side && P->exp_busy) { CK(cudaStreamWaitEvent(S, P->ev_exp_free, 0)); P->exp_busy = false; }
     {
       Timed t(L, LOCRET_K_DEQUANT, S);
-      CK(launch_dequant(L->q4[c], P->k_exp, P->v_exp, L->cs, L->h_kv, L->d, L->cap, L->len, true, S));
+      CK(launch_dequant(L->q4, P->k_exp, P->v_exp, L->cs, L->h_kv, L->d, L->cap, L->len, true, L->rank[L->rcur],
+                        L->ranked_len, S));
     }
     if (side) CK(cudaEventRecord(P->ev_exp_ready, S));
   }
@@ -520,7 +565,7 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
   auto quantize_chunk = [&](cudaStream_t R) -> int {  // the chunk's units enter the cache quantised (keys pre-RoPE)
     Timed t(L, LOCRET_K_QUANT, R);
     const bf16 *ks = staging + (size_t)L->h * L->d, *vs = ks + (size_t)L->h_kv * L->d;
-    CK(launch_quantize(ks, vs, L->d_in, L->d, L->q4[c], n_tok, L->h_kv, L->d, L->cap, L->len, R));
+    CK(launch_quantize(ks, vs, L->d_in, L->d, L->q4, n_tok, L->h_kv, L->d, L->cap, L->len, R));
     return LOCRET_OK;
   };
   // the codes are read by the compaction of this step and by later steps, never by this step's
@@ -534,9 +579,8 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
     if (tc_ok && L->int4 && L->map_kv_base != P->k_exp) {
       tc_ok = tmap_encode_3d_bf16(&L->map_k, P->k_exp, L->d, L->cap, L->h_kv, (uint64_t)L->d * 2,
                                   (uint64_t)L->cap * L->d * 2, 64, 128, 1) &&
-              tmap_encode_3d_bf16(&L->map_v[0], P->v_exp, L->d, L->cap, L->h_kv, (uint64_t)L->d * 2,
+              tmap_encode_3d_bf16(&L->map_v, P->v_exp, L->d, L->cap, L->h_kv, (uint64_t)L->d * 2,
                                   (uint64_t)L->cap * L->d * 2, 64, 128, 1);
-      L->map_v[1] = L->map_v[0];
       L->map_kv_base = tc_ok ? P->k_exp : nullptr;
     }
     if (tc_ok && L->map_q_base != P->q_rot) {
@@ -547,9 +591,9 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
     if (decode)
       CK(launch_attention_decode(P->q_rot, k_att, v_att, (bf16 *)attn_out, P->dec_o, P->dec_ml, P->dec_cnt + 1,
                                  L->h, L->h_kv, L->d, L->cap, n, decode_attn_splits(L->h_kv, n),
-                                 L->int4 ? &L->q4[c] : nullptr, L->cs, L->st));
+                                 L->int4 ? &L->q4 : nullptr, L->cs, L->rank[L->rcur], L->ranked_len, L->st));
     else if (tc_ok)
-      CK(launch_attention_tc(&L->map_q, &L->map_k, &L->map_v[c], (bf16 *)attn_out, n_tok, L->h, L->h_kv,
+      CK(launch_attention_tc(&L->map_q, &L->map_k, &L->map_v, (bf16 *)attn_out, n_tok, L->h, L->h_kv,
                              L->d, L->len, L->d_status, L->st));
     else
       CK(launch_attention_mma(P->q_rot, k_att, v_att, (bf16 *)attn_out, n_tok, L->h, L->h_kv,
@@ -599,7 +643,7 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
     const bf16 *z = L->cfg.rh_input == 1 ? z_post : staging;
     if (decode)
       CK(launch_rh_gemv(z, L->w1_t, L->w2f, P->partial, L->d_R, L->d_in, L->h_kv, L->cfg.act, P->dec_cnt,
-                        L->s[c] + L->len, L->cap, S));
+                        L->s + L->len, L->cap, S));
     else if (L->use_tc && n_tok >= 32 && gemm_tc_supported(n_tok, L->d_R, L->d_in, L->d_in, L->d_in))
       CK(launch_rh_gemm_tc(z, L->d_in, L->w1_t, L->w2f, P->partial, n_tok, L->d_R, L->d_in, L->h_kv,
                            L->cfg.act, &n_tiles, L->d_status, S));
@@ -609,7 +653,7 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
   }
   if (!decode) {  // (the one-token kernel sums its own partial scores)
     Timed t(L, LOCRET_K_RH_REDUCE, S);
-    CK(launch_rh_reduce(P->partial, n_tiles, n_tok, L->h_kv, L->s[c], L->cap, L->len, S));
+    CK(launch_rh_reduce(P->partial, n_tiles, n_tok, L->h_kv, L->s, L->cap, L->len, S));
   }
   if (side) {
     CK(cudaEventRecord(P->ev_stage_free[sb], S));
@@ -648,7 +692,7 @@ int locret_prefill_chunk_tp_finish(locret_layer *L, const float *preact_sum) {
   }
   {  // (c) finished: activation and this GPU's columns of W2, into the score cache
     Timed t(L, LOCRET_K_RH_REDUCE, S);
-    CK(launch_rh_finish(preact_sum, L->w2f, L->s[L->cur], L->cap, L->len, n_tok, L->d_R, L->h_kv, L->cfg.act, S));
+    CK(launch_rh_finish(preact_sum, L->w2f, L->s, L->cap, L->len, n_tok, L->d_R, L->h_kv, L->cfg.act, S));
   }
   return evict_and_close(L, n_tok, L->tp_flags, side, S);
 }
@@ -668,21 +712,19 @@ int locret_export_state(locret_layer *L, void *K, void *V, float *scores, int64_
   if (!L || !on_layer_device(L)) return LOCRET_ERR_INVALID;
   if (L->int4 && (K || V)) return LOCRET_ERR_INVALID;  // use locret_export_state_int4
   CK(sync_all(L));
-  const int c = L->cur, n = L->len;
+  const int n = L->len;
   if (len) *len = n;
   if (tokens_seen) *tokens_seen = L->seen;
   if (n > 0) {
-    const size_t row = (size_t)n * L->d * sizeof(bf16), pitch = (size_t)L->cap * L->d * sizeof(bf16);
-    if (K) CK(cudaMemcpy2DAsync(K, row, L->k_pre[c], pitch, row, L->h_kv, cudaMemcpyDeviceToHost, L->st));
-    if (V) CK(cudaMemcpy2DAsync(V, row, L->v[c], pitch, row, L->h_kv, cudaMemcpyDeviceToHost, L->st));
-    if (scores)
-      CK(cudaMemcpy2DAsync(scores, (size_t)n * 4, L->s[c], (size_t)L->cap * 4, (size_t)n * 4, L->h_kv,
-                           cudaMemcpyDeviceToHost, L->st));
-    if (token_ids)
-      CK(cudaMemcpy2DAsync(token_ids, (size_t)n * 8, L->tid[c], (size_t)L->cap * 8, (size_t)n * 8,
-                           L->h_kv, cudaMemcpyDeviceToHost, L->st));
+    TemporalOrder ord;
+    int rc = ord.load(L);
+    if (rc != LOCRET_OK) return rc;
+    const size_t row = (size_t)L->d * sizeof(bf16);
+    if (K && (rc = ord.copy_out(L, L->k_pre, row, K)) != LOCRET_OK) return rc;
+    if (V && (rc = ord.copy_out(L, L->v, row, V)) != LOCRET_OK) return rc;
+    if (scores && (rc = ord.copy_out(L, L->s, 4, scores)) != LOCRET_OK) return rc;
+    if (token_ids && (rc = ord.copy_out(L, L->tid, 8, token_ids)) != LOCRET_OK) return rc;
   }
-  CK(cudaStreamSynchronize(L->st));
   return LOCRET_OK;
 }
 
@@ -692,20 +734,20 @@ int locret_import_state(locret_layer *L, const void *K, const void *V, const flo
   if (L->int4) return LOCRET_ERR_INVALID;  // use locret_import_state_int4
   if (len > 0 && (!K || !V || !scores || !token_ids)) return LOCRET_ERR_INVALID;
   CK(sync_all(L));
-  const int c = L->cur;
   if (len > 0) {
     const size_t row = (size_t)len * L->d * sizeof(bf16), pitch = (size_t)L->cap * L->d * sizeof(bf16);
-    CK(cudaMemcpy2DAsync(L->k_pre[c], pitch, K, row, row, L->h_kv, cudaMemcpyHostToDevice, L->st));
-    CK(cudaMemcpy2DAsync(L->v[c], pitch, V, row, row, L->h_kv, cudaMemcpyHostToDevice, L->st));
-    CK(cudaMemcpy2DAsync(L->s[c], (size_t)L->cap * 4, scores, (size_t)len * 4, (size_t)len * 4, L->h_kv,
+    CK(cudaMemcpy2DAsync(L->k_pre, pitch, K, row, row, L->h_kv, cudaMemcpyHostToDevice, L->st));
+    CK(cudaMemcpy2DAsync(L->v, pitch, V, row, row, L->h_kv, cudaMemcpyHostToDevice, L->st));
+    CK(cudaMemcpy2DAsync(L->s, (size_t)L->cap * 4, scores, (size_t)len * 4, (size_t)len * 4, L->h_kv,
                          cudaMemcpyHostToDevice, L->st));
-    CK(cudaMemcpy2DAsync(L->tid[c], (size_t)L->cap * 8, token_ids, (size_t)len * 8, (size_t)len * 8,
+    CK(cudaMemcpy2DAsync(L->tid, (size_t)L->cap * 8, token_ids, (size_t)len * 8, (size_t)len * 8,
                          L->h_kv, cudaMemcpyHostToDevice, L->st));
     L->launches++;
-    CK(launch_rerope(L->k_pre[c], L->k_rot, L->cs, L->h_kv, L->d, L->cap, len, L->st));
+    CK(launch_rerope(L->k_pre, L->k_rot, L->cs, L->h_kv, L->d, L->cap, len, L->st));
   }
   CK(cudaStreamSynchronize(L->st));
   L->len = len;
+  L->ranked_len = 0;  // imported units are in temporal order: position = slot
   L->seen = tokens_seen;
   return LOCRET_OK;
 }
@@ -715,20 +757,22 @@ int locret_export_state_int4(locret_layer *L, void *k_codes, void *k_scales, voi
                              int64_t *tokens_seen) {
   if (!L || !L->int4 || !on_layer_device(L)) return LOCRET_ERR_INVALID;
   CK(sync_all(L));
-  const int c = L->cur, n = L->len;
+  const int n = L->len;
   if (len) *len = n;
   if (tokens_seen) *tokens_seen = L->seen;
   if (n > 0) {
-    const size_t crow = (size_t)n * (L->d / 2), cpitch = (size_t)L->cap * (L->d / 2);
-    const Int4Half &q = L->q4[c];
-    if (k_codes) CK(cudaMemcpy2DAsync(k_codes, crow, q.kq, cpitch, crow, L->h_kv, cudaMemcpyDeviceToHost, L->st));
-    if (v_codes) CK(cudaMemcpy2DAsync(v_codes, crow, q.vq, cpitch, crow, L->h_kv, cudaMemcpyDeviceToHost, L->st));
-    if (k_scales) CK(cudaMemcpy2DAsync(k_scales, (size_t)n * 2, q.ks, (size_t)L->cap * 2, (size_t)n * 2, L->h_kv, cudaMemcpyDeviceToHost, L->st));
-    if (v_scales) CK(cudaMemcpy2DAsync(v_scales, (size_t)n * 2, q.vs, (size_t)L->cap * 2, (size_t)n * 2, L->h_kv, cudaMemcpyDeviceToHost, L->st));
-    if (scores) CK(cudaMemcpy2DAsync(scores, (size_t)n * 4, L->s[c], (size_t)L->cap * 4, (size_t)n * 4, L->h_kv, cudaMemcpyDeviceToHost, L->st));
-    if (token_ids) CK(cudaMemcpy2DAsync(token_ids, (size_t)n * 8, L->tid[c], (size_t)L->cap * 8, (size_t)n * 8, L->h_kv, cudaMemcpyDeviceToHost, L->st));
+    TemporalOrder ord;
+    int rc = ord.load(L);
+    if (rc != LOCRET_OK) return rc;
+    const size_t crow = (size_t)(L->d / 2);
+    const Int4Half &q = L->q4;
+    if (k_codes && (rc = ord.copy_out(L, q.kq, crow, k_codes)) != LOCRET_OK) return rc;
+    if (v_codes && (rc = ord.copy_out(L, q.vq, crow, v_codes)) != LOCRET_OK) return rc;
+    if (k_scales && (rc = ord.copy_out(L, q.ks, 2, k_scales)) != LOCRET_OK) return rc;
+    if (v_scales && (rc = ord.copy_out(L, q.vs, 2, v_scales)) != LOCRET_OK) return rc;
+    if (scores && (rc = ord.copy_out(L, L->s, 4, scores)) != LOCRET_OK) return rc;
+    if (token_ids && (rc = ord.copy_out(L, L->tid, 8, token_ids)) != LOCRET_OK) return rc;
   }
-  CK(cudaStreamSynchronize(L->st));
   return LOCRET_OK;
 }
 
@@ -739,20 +783,30 @@ int locret_import_state_int4(locret_layer *L, const void *k_codes, const void *k
   if (len > 0 && (!k_codes || !k_scales || !v_codes || !v_scales || !scores || !token_ids))
     return LOCRET_ERR_INVALID;
   CK(sync_all(L));
-  const int c = L->cur;
   if (len > 0) {
     const size_t crow = (size_t)len * (L->d / 2), cpitch = (size_t)L->cap * (L->d / 2);
-    const Int4Half &q = L->q4[c];
+    const Int4Half &q = L->q4;
     CK(cudaMemcpy2DAsync(q.kq, cpitch, k_codes, crow, crow, L->h_kv, cudaMemcpyHostToDevice, L->st));
     CK(cudaMemcpy2DAsync(q.vq, cpitch, v_codes, crow, crow, L->h_kv, cudaMemcpyHostToDevice, L->st));
     CK(cudaMemcpy2DAsync(q.ks, (size_t)L->cap * 2, k_scales, (size_t)len * 2, (size_t)len * 2, L->h_kv, cudaMemcpyHostToDevice, L->st));
     CK(cudaMemcpy2DAsync(q.vs, (size_t)L->cap * 2, v_scales, (size_t)len * 2, (size_t)len * 2, L->h_kv, cudaMemcpyHostToDevice, L->st));
-    CK(cudaMemcpy2DAsync(L->s[c], (size_t)L->cap * 4, scores, (size_t)len * 4, (size_t)len * 4, L->h_kv, cudaMemcpyHostToDevice, L->st));
-    CK(cudaMemcpy2DAsync(L->tid[c], (size_t)L->cap * 8, token_ids, (size_t)len * 8, (size_t)len * 8, L->h_kv, cudaMemcpyHostToDevice, L->st));
+    CK(cudaMemcpy2DAsync(L->s, (size_t)L->cap * 4, scores, (size_t)len * 4, (size_t)len * 4, L->h_kv, cudaMemcpyHostToDevice, L->st));
+    CK(cudaMemcpy2DAsync(L->tid, (size_t)L->cap * 8, token_ids, (size_t)len * 8, (size_t)len * 8, L->h_kv, cudaMemcpyHostToDevice, L->st));
   }
   CK(cudaStreamSynchronize(L->st));
   L->len = len;
+  L->ranked_len = 0;
   L->seen = tokens_seen;
+  return LOCRET_OK;
+}
+
+int locret_compaction_counters(locret_layer *L, int64_t *units_moved, int64_t *keys_rotated) {
+  if (!L || !on_layer_device(L)) return LOCRET_ERR_INVALID;
+  unsigned long long host[2] = {0, 0};
+  CK(sync_all(L));
+  CK(cudaMemcpy(host, L->d_counters, sizeof(host), cudaMemcpyDeviceToHost));
+  if (units_moved) *units_moved = (int64_t)host[0];
+  if (keys_rotated) *keys_rotated = (int64_t)host[1];
   return LOCRET_OK;
 }
 
@@ -775,6 +829,7 @@ int locret_reset(locret_layer *L) {
     L->side_pending = false;
   }
   L->len = 0;
+  L->ranked_len = 0;
   L->seen = 0;
   L->tp_pending = false;
   return LOCRET_OK;

@@ -17,8 +17,10 @@ V_ULP = 2.0 ** -7     # a stored V element may round to either bf16 neighbour (f
 SCORE_TOL = 1e-2      # |delta| <= SCORE_TOL * max(|ref|, rms(ref over the chunk))
 BAND = 1e-2           # index sets must agree outside this band around the cut
 FLIP_FRACTION = 5e-3  # share of stored chunk K/V elements allowed to sit one bf16 ulp apart (measured 2.3e-3 at K = 4096)
-ORDINARY_ABS = 2.0    # a (query row, head) is "ordinary" when sum_i p_i |v_i| stays below this in every column:
-                      # it puts no noticeable weight on a 20x-norm outlier token (typical rows: 0.8)
+WELL_CONDITIONED = 5e-3  # an output element is well conditioned when the oracle's own first-order estimate of what
+                         # the legitimate storage differences can do to it, (P_ULP + V_ULP) sum p|v| + flip_sens,
+                         # stays below this: the row puts no weight worth mentioning on a 20x-norm outlier
+                         # token.  There the stated tolerance (max-abs 2e-2) is asserted as it is written.
 
 
 def bf16_dev(x: np.ndarray) -> torch.Tensor:
@@ -61,8 +63,8 @@ def attention_stats(got: np.ndarray, ref: np.ndarray, abs_ref=None, flip_sens=No
       plain_max_abs            largest |delta| over all compared elements
       plain_exceed_share       share of elements beyond the plain mixed bound 2e-2 * max(1, |ref|)
                                (these are the ones that need the derived terms)
-      ordinary_rows / ordinary_max_abs   (query row, head) pairs with sum p|v| < ORDINARY_ABS in every column
-                               of the head, out of `rows` pairs, and the largest |delta| on them (must stay
+      wellcond_share / wellcond_max_abs   share of elements whose derived terms stay below WELL_CONDITIONED
+                               (no weight on an outlier token), and the largest |delta| on them (must stay
                                within the plain 2e-2)
       bound_used_max           worst err / full bound
       pure_within_2e-2_share   share of elements within plain 2e-2 of the oracle WITHOUT bf16 mirroring
@@ -77,15 +79,11 @@ def attention_stats(got: np.ndarray, ref: np.ndarray, abs_ref=None, flip_sens=No
         if flip_sens is not None:
             bound = bound + flip_sens[rows]
         st["bound_used_max"] = float(np.max(err / bound)) if err.size else 0.0
-        # per (query row, head): heads attend independently, and in the outlier workloads nearly
-        # every row has SOME head that puts weight on an outlier token
-        d = head_dim or err.shape[1]
-        a3 = abs_ref[rows].reshape(err.shape[0], -1, d)
-        ordinary = a3.max(axis=2) < ORDINARY_ABS                              # [rows, heads]
-        st["ordinary_rows"] = int(ordinary.sum())
-        st["rows"] = int(ordinary.size)
-        e3 = err.reshape(a3.shape)
-        st["ordinary_max_abs"] = float(e3[ordinary].max()) if ordinary.any() else 0.0
+        extra = bound - ATTN_TOL * np.maximum(1.0, np.abs(r))
+        well = extra <= WELL_CONDITIONED
+        st["rows"] = int(rows.sum())
+        st["wellcond_share"] = float(np.mean(well)) if well.size else 0.0
+        st["wellcond_max_abs"] = float(err[well].max()) if well.any() else 0.0
     if pure_ref is not None:
         st["pure_within_2e-2_share"] = float(np.mean(np.abs(g - pure_ref[rows]) <= ATTN_TOL))
         st["pure_max_abs"] = float(np.max(np.abs(g - pure_ref[rows])))
@@ -173,9 +171,9 @@ def lockstep_chunk(ora, gpu, x: np.ndarray, flags: int = 0, rows=None, what="", 
     got_out = out_b.float().cpu().numpy().astype(np.float64)
     stats["attn_max_abs"] = check_attention(got_out, ref_out, what, ora.last_abs_out, ora.last_flip_sens)
     stats.update(attention_stats(got_out, ref_out, ora.last_abs_out, ora.last_flip_sens, pure_out, head_dim=d))
-    # rows that put no weight on an outlier token meet the stated tolerance as it is written
-    assert stats["ordinary_max_abs"] <= ATTN_TOL, \
-        f"{what}: ordinary rows off by {stats['ordinary_max_abs']:.4g} (plain tolerance {ATTN_TOL})"
+    # elements that put no weight on an outlier token meet the stated tolerance as it is written
+    assert stats["wellcond_max_abs"] <= ATTN_TOL, \
+        f"{what}: well-conditioned elements off by {stats['wellcond_max_abs']:.4g} (plain tolerance {ATTN_TOL})"
     if plain:
         assert stats["plain_max_abs"] <= ATTN_TOL, f"{what}: plain max-abs {stats['plain_max_abs']:.4g}"
 
@@ -291,7 +289,7 @@ def run_pair_without_reimport(ora, gpu, st, x_a, x_b, rows_a=None, rows_b=None, 
     got_b = out_b.float().cpu().numpy().astype(np.float64)
     stats = {"attn_max_abs": check_attention(got_b, ref_b, f"{what} B", ora.last_abs_out, ora.last_flip_sens)}
     stats.update(attention_stats(got_b, ref_b, ora.last_abs_out, ora.last_flip_sens, head_dim=d))
-    assert stats["ordinary_max_abs"] <= ATTN_TOL, f"{what} B: ordinary rows off by {stats['ordinary_max_abs']:.4g}"
+    assert stats["wellcond_max_abs"] <= ATTN_TOL, f"{what} B: well-conditioned elements off by {stats['wellcond_max_abs']:.4g}"
     after = gpu.export_state()
     stats["score_worst"] = check_scores(after["S"][:, ln:].T.astype(np.float64), ora.last_scores, f"{what} B")
     stats["moved"], stats["stayed"] = moved, stay

@@ -144,3 +144,101 @@ def test_steps_back_to_back_on_two_streams_equal_the_one_stream_schedule(kv_dtyp
             for tok in got ^ want:
                 assert abs(s_all[tok, m] - cut) < BAND, f"layer {l} head {m}: token {tok} outside the band"
             assert len(got ^ want) <= 6
+
+
+def _hand_scored_layer(h, hk, d, D, seed):
+    """Weights under which the retaining head's score of token t for KV head m is exactly
+    relu(x[t, m]): W_qkv routes hidden element m unchanged into the first element of value head m,
+    W1 picks that element, the activation is ReLU and W2 passes it on.  With small integers in
+    x[:, :h_kv] the scores are exact on both sides and full of ties."""
+    sh = W.LayerShape(d_model=D, n_q_heads=h, n_kv_heads=hk, head_dim=d, d_retain=8, rope_theta=500000.0, act=2)
+    g = np.random.default_rng(seed)
+    d_in = sh.d_in
+    wqkv = W.to_bf16_grid((g.standard_normal((D, d_in)) / np.sqrt(D)).astype(np.float32))
+    w1 = np.zeros((d_in, 8), dtype=np.float32)
+    w2 = np.zeros((8, hk), dtype=np.float32)
+    for m in range(hk):
+        col = (h + hk + m) * d
+        wqkv[:, col] = 0.0
+        wqkv[m, col] = 1.0
+        w1[col, m] = 1.0
+        w2[m, m] = 1.0
+    return sh, (wqkv, w1, w2)
+
+
+@pytest.mark.parametrize("d,heads,n_prefix,last", [(64, (4, 2), 0, False), (128, (8, 2), 5, True), (96, (3, 3), 0, True)])
+def test_many_evictions_in_place_stay_identical_to_the_oracle(d, heads, n_prefix, last):
+    """Eviction leaves kept units in their slots and refills freed ones, so after a few steps slot order
+    and temporal order have nothing in common.  Hand-made scores (exact small integers, many ties) keep
+    both sides on the same retained set without any import: after every step the exported state must be
+    the oracle's (token ids and scores exactly, K and V up to the rare one-ulp flips of a projection),
+    and attention - which reads keys rotated at the units' positions in temporal order - must agree."""
+    from parity_util import FLIP_FRACTION, bf16_dev, check_attention, make_pair
+    h, hk = heads
+    sh, wts = _hand_scored_layer(h, hk, d, 64, seed=d)
+    budget, chunk, n_stab = 150, 96, 20
+    ora, gpu = make_pair(sh, wts, budget, chunk, n_stab, reserve=8)
+    if n_prefix:
+        ora.set_protected_prefix(n_prefix)
+        gpu.set_protected_prefix(n_prefix)
+    g = np.random.default_rng(500 + d)
+    sizes = [96, 96, 41, 96, 1, 96, 77, 96, 96, 13]
+    for i, n_tok in enumerate(sizes):
+        x = W.to_bf16_grid(g.standard_normal((n_tok, 64)).astype(np.float32))
+        x[:, :hk] = g.integers(-3, 40, size=(n_tok, hk)).astype(np.float32)
+        flags = O.LAST_CHUNK if (last and i == len(sizes) - 1) else 0
+        out = torch.zeros((n_tok, h * d), dtype=torch.bfloat16, device="cuda")
+        gpu.prefill_chunk(bf16_dev(x), out, flags)
+        ref = ora.prefill_chunk(x, flags)
+        check_attention(out.float().cpu().numpy().astype(np.float64), ref, f"step {i}", ora.last_abs_out,
+                        ora.last_flip_sens)
+        st = gpu.export_state()
+        assert np.array_equal(st["T"], ora.T), f"step {i}: retained token ids differ"
+        assert np.array_equal(st["S"].astype(np.float64), ora.S), f"step {i}: scores differ"
+        for name in ("K", "V"):
+            diff = np.abs(st[name] - getattr(ora, name))
+            assert np.all(diff <= np.abs(getattr(ora, name)) * 2.0 ** -7 + 1e-6), f"step {i}: {name} differs"
+            assert np.mean(diff != 0) < FLIP_FRACTION
+        assert gpu.sync_status() == 0
+    moved, rotated = gpu.compaction_counters
+    assert 0 < moved <= rotated
+    # a few one-token steps on top (appended in order behind the shuffled slots)
+    for t in range(4):
+        x = W.to_bf16_grid(g.standard_normal((1, 64)).astype(np.float32))
+        out = torch.zeros((1, h * d), dtype=torch.bfloat16, device="cuda")
+        gpu.decode_step(bf16_dev(x), out)
+        ref = ora.decode_step(x[0])
+        check_attention(out.float().cpu().numpy().astype(np.float64), ref, f"decode {t}", ora.last_abs_out,
+                        ora.last_flip_sens)
+    assert np.array_equal(gpu.export_state()["T"], ora.T)
+    gpu.destroy()
+
+
+def test_many_evictions_in_place_with_the_4_bit_cache():
+    """The same with codes and scales moving in place: they must arrive unchanged, in temporal order."""
+    from parity_util import bf16_dev, check_attention, make_pair
+    import dataclasses
+    sh, wts = _hand_scored_layer(8, 2, 128, 64, seed=9)
+    sh = dataclasses.replace(sh, kv_dtype=1)
+    ora, gpu = make_pair(sh, wts, 150, 96, 20, reserve=8)
+    g = np.random.default_rng(77)
+    for i, n_tok in enumerate([96, 96, 41, 96, 1, 96, 77]):
+        x = W.to_bf16_grid(g.standard_normal((n_tok, 64)).astype(np.float32))
+        x[:, :2] = g.integers(-3, 40, size=(n_tok, 2)).astype(np.float32)
+        out = torch.zeros((n_tok, 8 * 128), dtype=torch.bfloat16, device="cuda")
+        gpu.prefill_chunk(bf16_dev(x), out, 0)
+        ref = ora.prefill_chunk(x, 0)
+        check_attention(out.float().cpu().numpy().astype(np.float64), ref, f"int4 step {i}", ora.last_abs_out,
+                        ora.last_flip_sens)
+        st = gpu.export_state()
+        assert np.array_equal(st["T"], ora.T), f"step {i}"
+        for name in ("Kc", "Vc"):
+            assert np.mean(st[name] != getattr(ora, name)) < 0.01, f"step {i}: {name}"
+    for t in range(3):
+        x = W.to_bf16_grid(g.standard_normal((1, 64)).astype(np.float32))
+        out = torch.zeros((1, 8 * 128), dtype=torch.bfloat16, device="cuda")
+        gpu.decode_step(bf16_dev(x), out)
+        ref = ora.decode_step(x[0])
+        check_attention(out.float().cpu().numpy().astype(np.float64), ref, f"int4 decode {t}", ora.last_abs_out,
+                        ora.last_flip_sens)
+    gpu.destroy()

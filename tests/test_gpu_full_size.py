@@ -45,12 +45,12 @@ def run_workload_chunks(name, n_chunks, layer=0, extra_rows=(), plain=False, wit
     assert gpu.sync_status() == 0
     gpu.destroy()
     summary = {k: max(s[k] for s in stats if k in s) for k in
-               ("plain_max_abs", "plain_exceed_share", "ordinary_max_abs", "bound_used_max", "flip_rate_K", "flip_rate_V",
+               ("plain_max_abs", "plain_exceed_share", "wellcond_max_abs", "bound_used_max", "flip_rate_K", "flip_rate_V",
                 "score_worst", "score_plain_rel_worst", "pure_max_abs") if any(k in s for s in stats)}
     if with_pure:
         summary["pure_within_2e-2_share_min"] = min(s["pure_within_2e-2_share"] for s in stats)
     summary["rows_compared"] = sum(s.get("rows", 0) for s in stats)
-    summary["ordinary_rows"] = sum(s.get("ordinary_rows", 0) for s in stats)
+    summary["wellcond_share_min"] = min(s.get("wellcond_share", 0.0) for s in stats)
     print(f"{name}: worst over {len(stats)} chunks: {summary}")
     return w, ora, stats
 
