@@ -67,6 +67,27 @@ __device__ __forceinline__ float apply_act(float x, int act) {
   return fmaxf(x, 0.0f);                         // ReLU
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// Consecutive kernels of one stream launched with `pdl` may overlap: the later one starts once every
+// CTA of the earlier one has called pdl_launch_dependents() (or exited) and runs up to its
+// pdl_wait(), which returns when the earlier grid has completed and its writes are visible.  In a
+// kernel launched the ordinary way both calls do nothing.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                 bool pdl, Args &&...args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---------------------------------------------------------------- per-device launch state (host)
 // cudaFuncSetAttribute acts on the current device only, so "already done" is remembered per
 // device: one process may drive several GPUs.
@@ -238,24 +259,29 @@ cudaError_t launch_gemv_resid(const bf16 *x, const bf16 *Wt, int N, int K, const
 cudaError_t launch_gemv_gated(const bf16 *x, const bf16 *Wt, int F, int K, bf16 *act, cudaStream_t st);
 // projection + positions + RoPE + cache append of one token (a.staging is not used: `staging` is written)
 cudaError_t launch_gemv_rope(const bf16 *x, const bf16 *Wt, int K, bf16 *staging, const RopeAppendArgs &a,
-                             cudaStream_t st);
+                             cudaStream_t st, bool pdl = false);
 // retaining head of one token; the last block sums the per-block partials into
 // score_out[m * score_stride]; counter: one zeroed word, left at zero
+// pdl: the kernel is the third of a one-token step's chain (projection, attention, retaining head)
+// launched with programmatic dependent launch; it needs only the projection's output, so it runs beside
+// the attention kernel and waits for that kernel just before it ends (which keeps the chain ordered)
 cudaError_t launch_rh_gemv(const bf16 *z, const bf16 *W1t, const float *W2, float *partial, int d_R, int K,
                            int h_kv, int act, unsigned *counter, float *score_out, int score_stride,
-                           cudaStream_t st);
+                           cudaStream_t st, bool pdl = false);
 int rh_gemv_blocks(int d_R);
 int decode_attn_splits(int h_kv, int n);
 // part_o: fp32 [h][n_splits][d]; part_ml: fp32 [h][n_splits][2]; counters: one zeroed word per
 // (KV head, group of 16 query heads), left at zero (the last split merges the partial results).
 // q4 != nullptr: keys [0, n - 1) are read from the 4-bit cache (expanded and rotated with `cs` on the
 // way into shared memory, at position rank[m * cap + slot] for slot < ranked_len and slot above) and only
-// key n - 1, the token of this step, from k_rot / v.
+// key n - 1, the token of this step, from k_rot / v.  tok_k / tok_v (4-bit cache only, may be null): the
+// token's pre-RoPE keys and values [h_kv][d], which the kernel quantises into slot n - 1 of the cache.
 struct Int4Half;
 cudaError_t launch_attention_decode(const bf16 *q_rot, const bf16 *k_rot, const bf16 *v, bf16 *out,
                                     float *part_o, float *part_ml, unsigned *counters, int h, int h_kv, int d,
                                     int cap, int n, int n_splits, const Int4Half *q4, const float2 *cs,
-                                    const int32_t *rank, int ranked_len, cudaStream_t st);
+                                    const int32_t *rank, int ranked_len, const bf16 *tok_k, const bf16 *tok_v,
+                                    cudaStream_t st, bool pdl = false);
 
 // dst[c][r] = src[r][c]  (weight repack at create)
 cudaError_t launch_transpose_bf16(const bf16 *src, bf16 *dst, int rows, int cols, cudaStream_t st);

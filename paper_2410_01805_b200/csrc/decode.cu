@@ -46,6 +46,10 @@ gemv_kernel(const bf16 *__restrict__ x, const bf16 *__restrict__ Wt, int N, int 
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint4 *sx = reinterpret_cast<uint4 *>(smem_raw);  // K / 8 vectors
   float *swarp = reinterpret_cast<float *>(sx + K / 8);  // [8 warps][32]
+  // MODE 1 in a one-token step's chain: the input is the projection's output, complete since the
+  // attention kernel before this one passed its own wait, so nothing is waited for here; the next
+  // layer's projection may start (and request its weights) at once
+  if (MODE == 1) pdl_launch_dependents();
   for (int i = threadIdx.x; i < K / 8; i += GV_THREADS) sx[i] = reinterpret_cast<const uint4 *>(x)[i];
   __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -110,6 +114,9 @@ gemv_kernel(const bf16 *__restrict__ x, const bf16 *__restrict__ Wt, int N, int 
         }
       }
     }
+    // the attention kernel of this step must have finished before the next layer's projection (which
+    // waits for THIS kernel) overwrites the buffers attention reads
+    pdl_wait();
   }
 }
 
@@ -121,6 +128,8 @@ gemv_rope_kernel(const bf16 *__restrict__ x, const bf16 *__restrict__ Wt, int K,
                  RopeAppendArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint4 *sx = reinterpret_cast<uint4 *>(smem_raw);  // K / 8 vectors
+  pdl_wait();
+  pdl_launch_dependents();
   for (int i = threadIdx.x; i < K / 8; i += GV_THREADS) sx[i] = reinterpret_cast<const uint4 *>(x)[i];
   __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -206,6 +215,12 @@ gemv_rope_wide_kernel(const bf16 *__restrict__ x, const bf16 *__restrict__ Wt, i
     }
   };
   load_batch(p_lo);
+  // the weights do not depend on anything before this kernel: the first batch is in flight while the
+  // kernel waits for the step before it (whose buffers it is about to overwrite).  The attention
+  // kernel may start only after that wait: it requests retained keys before its own, and an
+  // eviction of the previous step may still be rewriting them until then.
+  pdl_wait();
+  pdl_launch_dependents();
   const uint4 xv = act ? __ldg(reinterpret_cast<const uint4 *>(x) + tid) : make_uint4(0, 0, 0, 0);
   int par = 0;
   for (int p0 = p_lo; p0 < p_hi; p0 += GW_PB, par ^= 1) {
@@ -311,7 +326,8 @@ attn_decode_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_ro
                    const bf16 *__restrict__ v, float *__restrict__ part_o, float *__restrict__ part_ml,
                    int h, int h_kv, int cap, int n, int n_splits, float scale_log2,
                    unsigned *__restrict__ counters, bf16 *__restrict__ out, Int4Half q4,
-                   const float2 *__restrict__ cs, const int32_t *__restrict__ rank, int ranked_len) {
+                   const float2 *__restrict__ cs, const int32_t *__restrict__ rank, int ranked_len,
+                   const bf16 *__restrict__ tok_k, const bf16 *__restrict__ tok_v) {
   constexpr int LD = D + 8;
   constexpr int VPR = D / 8;  // 16-byte vectors per row
   extern __shared__ __align__(16) unsigned char da_smem[];
@@ -380,11 +396,50 @@ attn_decode_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_ro
       *reinterpret_cast<uint4 *>(vd + c) = va; *reinterpret_cast<uint4 *>(vd + c + HALF) = vb;
     }
   };
+  // The retained keys and values were written by earlier steps: a first tile that does not reach
+  // the token of this step is requested before the wait for this step's projection.
+  const bool early = !INT4 && NKT > 0 && k0 + DA_KT <= n - 1;
+  if (early) load_kv(0, 0);
+  pdl_wait();
+  pdl_launch_dependents();  // the retaining head reads only what the projection wrote: it may run beside this kernel
+  if (INT4 && tok_k && split == 0 && hg == 0 && warp < 2) {
+    // The token of this step enters the 4-bit cache (this step still reads it in bf16): one warp
+    // quantises its pre-RoPE key, one its value, with the arithmetic of the chunk kernel.
+    const bf16 *src = (warp == 0 ? tok_k : tok_v) + (size_t)m * D;
+    float x0[2], x1[2], amax = 0.f;
+#pragma unroll
+    for (int k = 0; k < 2; k++) {
+      const int p = lane + 32 * k;
+      x0[k] = x1[k] = 0.f;
+      if (2 * p < D) {
+        const __nv_bfloat162 v2 = *reinterpret_cast<const __nv_bfloat162 *>(src + 2 * p);
+        x0[k] = __bfloat162float(v2.x);
+        x1[k] = __bfloat162float(v2.y);
+        amax = fmaxf(amax, fmaxf(fabsf(x0[k]), fabsf(x1[k])));
+      }
+    }
+    amax = warp_max(amax);
+    __half sh = __float2half_rn(__fdiv_rn(amax, 7.0f));
+    if (__half2float(sh) == 0.f) sh = __float2half_rn(1.0f);
+    const float sf = __half2float(sh);
+    const size_t u = (size_t)m * cap + (n - 1);
+    uint8_t *dst = (warp == 0 ? q4.kq : q4.vq) + u * (D / 2);
+#pragma unroll
+    for (int k = 0; k < 2; k++) {
+      const int p = lane + 32 * k;
+      if (2 * p < D) {
+        const int c0 = (int)fminf(fmaxf(rintf(__fdiv_rn(x0[k], sf)), -8.f), 7.f);
+        const int c1 = (int)fminf(fmaxf(rintf(__fdiv_rn(x1[k], sf)), -8.f), 7.f);
+        dst[p] = (uint8_t)((c0 & 0xF) | ((c1 & 0xF) << 4));
+      }
+    }
+    if (lane == 0) (warp == 0 ? q4.ks : q4.vs)[u] = sh;
+  }
   for (int x = tid; x < DA_G * VPR; x += DA_THREADS) {
     const int r = x / VPR, c = (x - r * VPR) * 8;
     cp_async16(sQ + r * LD + c, q_rot + (size_t)(h0 + min(r, gh - 1)) * D + c, r < gh);
   }
-  if (!INT4 && NKT > 0) load_kv(0, 0);
+  if (!INT4 && NKT > 0 && !early) load_kv(0, 0);
   cp_async_commit();
 
   uint32_t qf[D / 16][4];
@@ -637,30 +692,28 @@ cudaError_t launch_gemv_gated(const bf16 *x, const bf16 *Wt, int F, int K, bf16 
 int rh_gemv_blocks(int d_R) { return min((d_R + 3) / 4, 148 * 4); }
 
 cudaError_t launch_gemv_rope(const bf16 *x, const bf16 *Wt, int K, bf16 *staging, const RopeAppendArgs &a,
-                             cudaStream_t st) {
+                             cudaStream_t st, bool pdl) {
   if (K % 8 || a.d % 2) return cudaErrorInvalidValue;
   const int items = (a.h + 2 * a.h_kv) * (a.d / 2);
   if (K / 8 <= GW_THREADS) {
     const int blocks = min((items + GW_PB - 1) / GW_PB, 148 * 2);
-    gemv_rope_wide_kernel<<<blocks, GW_THREADS, 0, st>>>(x, Wt, K, staging, a);
-    return cudaGetLastError();
+    return launch_kernel(gemv_rope_wide_kernel, dim3(blocks), dim3(GW_THREADS), 0, st, pdl, x, Wt, K, staging, a);
   }
   const int blocks = min((items + 7) / 8, 148 * 4);
-  gemv_rope_kernel<<<blocks, GV_THREADS, K * 2, st>>>(x, Wt, K, staging, a);
-  return cudaGetLastError();
+  return launch_kernel(gemv_rope_kernel, dim3(blocks), dim3(GV_THREADS), (size_t)K * 2, st, pdl, x, Wt, K, staging, a);
 }
 
 // score_out: where the token's scores go (element m * score_stride for KV head m); counter: one
 // zero-initialised word that the kernel leaves at zero
 cudaError_t launch_rh_gemv(const bf16 *z, const bf16 *W1t, const float *W2, float *partial, int d_R, int K,
                            int h_kv, int act, unsigned *counter, float *score_out, int score_stride,
-                           cudaStream_t st) {
+                           cudaStream_t st, bool pdl) {
   if (K % 16 || h_kv > 32) return cudaErrorInvalidValue;
   const int smem = K * 2 + 8 * 32 * 4;
   const int blocks = rh_gemv_blocks(d_R);
-  gemv_kernel<1><<<blocks, GV_THREADS, smem, st>>>(z, W1t, d_R, K, nullptr, W2, partial, h_kv, act, counter,
-                                                  score_out, score_stride, nullptr);
-  return cudaGetLastError();
+  return launch_kernel(gemv_kernel<1>, dim3(blocks), dim3(GV_THREADS), (size_t)smem, st, pdl, z, W1t, d_R, K,
+                       (bf16 *)nullptr, W2, partial, h_kv, act, counter, score_out, score_stride,
+                       (const bf16 *)nullptr);
 }
 
 int decode_attn_splits(int h_kv, int n) {
@@ -674,7 +727,8 @@ int decode_attn_splits(int h_kv, int n) {
 cudaError_t launch_attention_decode(const bf16 *q_rot, const bf16 *k_rot, const bf16 *v, bf16 *out,
                                     float *part_o, float *part_ml, unsigned *counters, int h, int h_kv, int d,
                                     int cap, int n, int n_splits, const Int4Half *q4, const float2 *cs,
-                                    const int32_t *rank, int ranked_len, cudaStream_t st) {
+                                    const int32_t *rank, int ranked_len, const bf16 *tok_k, const bf16 *tok_v,
+                                    cudaStream_t st, bool pdl) {
   const int g = h / h_kv;
   dim3 grid(h_kv, n_splits, (g + DA_G - 1) / DA_G);
   if ((int)grid.x * (int)grid.z > 32 * 16 || n_splits > 64) return cudaErrorInvalidValue;
@@ -682,9 +736,8 @@ cudaError_t launch_attention_decode(const bf16 *q_rot, const bf16 *k_rot, const 
   const Int4Half qq = q4 ? *q4 : Int4Half{nullptr, nullptr, nullptr, nullptr};
   auto launch = [&](auto kern, int smem, PerDeviceFlag &attr_set) -> cudaError_t {
     if (cudaError_t e = allow_dynamic_smem(kern, smem, attr_set); e != cudaSuccess) return e;
-    kern<<<grid, DA_THREADS, smem, st>>>(q_rot, k_rot, v, part_o, part_ml, h, h_kv, cap, n, n_splits,
-                                         scale_log2, counters, out, qq, cs, rank, rank ? ranked_len : 0);
-    return cudaGetLastError();
+    return launch_kernel(kern, grid, dim3(DA_THREADS), (size_t)smem, st, pdl, q_rot, k_rot, v, part_o, part_ml, h, h_kv,
+                         cap, n, n_splits, scale_log2, counters, out, qq, cs, rank, rank ? ranked_len : 0, tok_k, tok_v);
   };
   static PerDeviceFlag set_done[2][3];
   const int qi = q4 ? 1 : 0;

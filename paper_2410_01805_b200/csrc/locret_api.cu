@@ -99,6 +99,7 @@ struct locret_layer {
   bool use_tc;  // tcgen05 kernels (default); LOCRET_LEGACY_MMA=1 keeps the mma.sync kernels for A/B runs
   bool fuse_rope;  // RoPE + append in the projection's epilogue (LOCRET_UNFUSED_ROPE=1 disables)
   bool use_side;  // off-critical-path kernels go to the pool's second stream (LOCRET_SERIAL=1 disables)
+  bool use_pdl;   // one-token steps overlap their kernels by programmatic dependent launch (LOCRET_NO_PDL=1 disables)
   bool side_pending;
   bool tp_pending;  // a divided-heads step was begun and waits for the summed product
   int tp_n_tok;
@@ -301,6 +302,8 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
     L->use_side = !(ser && ser[0] == '1');
     const char *unf = getenv("LOCRET_UNFUSED_ROPE");
     L->fuse_rope = !(unf && unf[0] == '1');
+    const char *np = getenv("LOCRET_NO_PDL");
+    L->use_pdl = !(np && np[0] == '1');
     L->side_pending = false;
     L->ev_ready = L->ev_attn = L->ev_side = L->ev_tp = nullptr;
   }
@@ -503,7 +506,10 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
   ScratchPool *P = L->pool;
   const bool tp = tp_partial != nullptr;
   const bool decode = n_tok == 1 && L->use_tc && !tp;  // one token: bandwidth-bound kernels of decode.cu
-  const bool side = L->use_side && !L->serialize;
+  // (a one-token step is a chain of three short kernels on the layer's own stream, overlapped by
+  // programmatic dependent launch: an event between them would serialise them again)
+  const bool side = L->use_side && !L->serialize && !decode;
+  const bool pdl = decode && L->use_pdl && !L->timing;
   cudaStream_t S = side ? P->side : L->st;  // stream of the off-critical-path kernels
   const int sb = P->flip;                    // staging buffer of this call
   P->flip ^= 1;
@@ -547,7 +553,7 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
   {  // (a) projections
     Timed t(L, LOCRET_K_QKV);
     if (decode)  // projection, positions, RoPE and append of the one token in one kernel
-      CK(launch_gemv_rope((const bf16 *)hidden_in, L->wqkv_t, L->D, staging, ra, L->st));
+      CK(launch_gemv_rope((const bf16 *)hidden_in, L->wqkv_t, L->D, staging, ra, L->st, pdl));
     else if (fused_rope)
       CK(launch_qkv_rope_tc((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, staging, n_tok, L->d_in, L->D,
                             ra, L->d_status, L->st));
@@ -570,7 +576,8 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
   };
   // the codes are read by the compaction of this step and by later steps, never by this step's
   // attention (the chunk attends to its own keys and values in bf16): second stream
-  if (L->int4 && !side) { const int rc = quantize_chunk(L->st); if (rc != LOCRET_OK) return rc; }
+  // (a one-token step quantises its token inside the attention kernel)
+  if (L->int4 && !side && !decode) { const int rc = quantize_chunk(L->st); if (rc != LOCRET_OK) return rc; }
   if (side) CK(cudaEventRecord(L->ev_ready, L->st));
   if (side && deq) CK(cudaStreamWaitEvent(L->st, P->ev_exp_ready, 0));
   {  // (b) Eq. 1
@@ -591,7 +598,9 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
     if (decode)
       CK(launch_attention_decode(P->q_rot, k_att, v_att, (bf16 *)attn_out, P->dec_o, P->dec_ml, P->dec_cnt + 1,
                                  L->h, L->h_kv, L->d, L->cap, n, decode_attn_splits(L->h_kv, n),
-                                 L->int4 ? &L->q4 : nullptr, L->cs, L->rank[L->rcur], L->ranked_len, L->st));
+                                 L->int4 ? &L->q4 : nullptr, L->cs, L->rank[L->rcur], L->ranked_len,
+                                 L->int4 ? staging + (size_t)L->h * L->d : nullptr,
+                                 L->int4 ? staging + (size_t)(L->h + L->h_kv) * L->d : nullptr, L->st, pdl));
     else if (tc_ok)
       CK(launch_attention_tc(&L->map_q, &L->map_k, &L->map_v, (bf16 *)attn_out, n_tok, L->h, L->h_kv,
                              L->d, L->len, L->d_status, L->st));
@@ -643,7 +652,7 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
     const bf16 *z = L->cfg.rh_input == 1 ? z_post : staging;
     if (decode)
       CK(launch_rh_gemv(z, L->w1_t, L->w2f, P->partial, L->d_R, L->d_in, L->h_kv, L->cfg.act, P->dec_cnt,
-                        L->s + L->len, L->cap, S));
+                        L->s + L->len, L->cap, S, pdl));
     else if (L->use_tc && n_tok >= 32 && gemm_tc_supported(n_tok, L->d_R, L->d_in, L->d_in, L->d_in))
       CK(launch_rh_gemm_tc(z, L->d_in, L->w1_t, L->w2f, P->partial, n_tok, L->d_R, L->d_in, L->h_kv,
                            L->cfg.act, &n_tiles, L->d_status, S));
