@@ -127,6 +127,17 @@ int locret_prefill_chunk(locret_layer *layer, const void *hidden_in, int32_t n_t
 int locret_decode_step(locret_layer *layer, const void *hidden_in, void *attn_out);
 
 /*
+ * locret_decode_step for several layers in one call, in order: every layer receives the same
+ * hidden_in and layer i writes attn_out + i * out_stride elements (out_stride a multiple of 8; 0:
+ * all layers write the same buffer).  For harnesses that drive the attention blocks of a stack
+ * alone, where the cost of crossing into the library once per layer is comparable to a layer-step
+ * on the device; in a model the caller computes the next layer's input in between and calls
+ * locret_decode_step per layer.  Stops at the first layer that returns an error and returns it.
+ */
+int locret_decode_step_stack(locret_layer *const *layers, int32_t n_layers, const void *hidden_in,
+                             void *attn_out, int64_t out_stride);
+
+/*
  * The same step with the KV heads (and the query heads of their groups) divided over several
  * GPUs, one layer object per GPU.  Heads attend and evict independently (Algorithm 1 runs per
  * head) and only the retaining head reads every head's [Q, K, V] (Section 3.3), so the GPUs

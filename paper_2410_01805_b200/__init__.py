@@ -9,6 +9,7 @@ built library raises.
 from .binding import (  # noqa: F401
     K_NAMES,
     LAST_CHUNK,
+    LayerStack,
     NO_EVICT,
     LocretBlock,
     LocretError,

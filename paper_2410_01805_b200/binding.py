@@ -52,6 +52,7 @@ def _load():
     l.locret_create.argtypes = [C.POINTER(locret_layer_cfg), C.c_int32, C.c_int32, C.c_int32, C.POINTER(P)]
     l.locret_prefill_chunk.argtypes = [P, P, C.c_int32, C.c_uint32, P]
     l.locret_decode_step.argtypes = [P, P, P]
+    l.locret_decode_step_stack.argtypes = [P, C.c_int32, P, P, C.c_int64]
     l.locret_prefill_chunk_tp_begin.argtypes = [P, P, C.c_int32, C.c_uint32, P, P]
     l.locret_prefill_chunk_tp_finish.argtypes = [P, P]
     l.locret_cache_len.argtypes = [P, C.POINTER(C.c_int32)]
@@ -250,6 +251,18 @@ class LocretLayer:
             self.destroy()
         except Exception:
             pass
+
+
+class LayerStack:
+    """Handles of several layers as one C array, for locret_decode_step_stack."""
+
+    def __init__(self, layers):
+        self.layers = list(layers)
+        self._arr = (C.c_void_p * len(self.layers))(*[L._h.value for L in self.layers])
+
+    def decode_step(self, hidden_in: torch.Tensor, attn_out: torch.Tensor, out_stride: int = 0):
+        _check(lib.locret_decode_step_stack(self._arr, len(self.layers), hidden_in.data_ptr(), attn_out.data_ptr(),
+                                            int(out_stride)), "locret_decode_step_stack")
 
 
 def shard_by_kv_head(w_qkv: torch.Tensor, w1: torch.Tensor, w2: torch.Tensor, n_q_heads: int,

@@ -710,6 +710,18 @@ int locret_decode_step(locret_layer *L, const void *hidden_in, void *attn_out) {
   return locret_prefill_chunk(L, hidden_in, 1, LOCRET_NO_EVICT, attn_out);
 }
 
+int locret_decode_step_stack(locret_layer *const *layers, int32_t n_layers, const void *hidden_in, void *attn_out,
+                             int64_t out_stride) {
+  if (!layers || n_layers < 1 || !attn_out || out_stride < 0 || (out_stride % 8) != 0) return LOCRET_ERR_INVALID;
+  for (int i = 0; i < n_layers; i++) {
+    if (!layers[i]) return LOCRET_ERR_INVALID;
+    bf16 *out = static_cast<bf16 *>(attn_out) + (size_t)i * out_stride;
+    const int rc = locret_prefill_chunk(layers[i], hidden_in, 1, LOCRET_NO_EVICT, out);
+    if (rc != LOCRET_OK) return rc;
+  }
+  return LOCRET_OK;
+}
+
 int locret_cache_len(const locret_layer *L, int32_t *len) {
   if (!L || !len) return LOCRET_ERR_INVALID;
   *len = L->len;

@@ -242,3 +242,35 @@ def test_many_evictions_in_place_with_the_4_bit_cache():
         check_attention(out.float().cpu().numpy().astype(np.float64), ref, f"int4 decode {t}", ora.last_abs_out,
                         ora.last_flip_sens)
     gpu.destroy()
+
+
+def test_one_call_for_a_stack_of_layers_equals_one_call_per_layer():
+    from paper_2410_01805_b200 import LayerStack, LocretLayer
+    from parity_util import bf16_dev
+    sh = _shape(8, 2, 128, D=256, dR=128)
+    weights = [W.layer_weights(sh, l, seed=W.BASE_SEED + 5) for l in range(3)]
+    runs = []
+    for use_stack in (False, True):
+        layers = [LocretLayer(sh, *(bf16_dev(a) for a in wts), 300, 128, 40, reserve=8) for wts in weights]
+        x0 = bf16_dev(_hidden(128, sh.d_model, 1))
+        out = torch.zeros((128, 8 * 128), dtype=torch.bfloat16, device="cuda")
+        for L in layers:
+            L.prefill_chunk(x0, out, 0)
+        outs = torch.zeros((4, 3, 8 * 128), dtype=torch.bfloat16, device="cuda")
+        stack = LayerStack(layers)
+        for t in range(4):
+            x = bf16_dev(_hidden(1, sh.d_model, 50 + t))
+            if use_stack:
+                stack.decode_step(x, outs[t], out_stride=8 * 128)
+            else:
+                for l, L in enumerate(layers):
+                    L.decode_step(x, outs[t, l])
+        states = [L.export_state() for L in layers]
+        assert all(L.sync_status() == 0 for L in layers)
+        runs.append((outs.clone(), states))
+        for L in layers:
+            L.destroy()
+    assert torch.equal(runs[0][0], runs[1][0])
+    for a, b in zip(runs[0][1], runs[1][1]):
+        for k in ("K", "V", "S", "T"):
+            assert np.array_equal(a[k], b[k])

@@ -135,3 +135,25 @@ def test_decode_steps_after_prefill_at_the_llama_shape(name):
         assert np.all(np.abs(got - want) <= 1e-2 * np.maximum(np.abs(want), np.sqrt(np.mean(ora.S ** 2)))), f"decode {t} score"
     assert gpu.cache_len == w.budget + 6 and gpu.sync_status() == 0
     gpu.destroy()
+
+
+def test_deep_in_the_headline_stream_chunk_40_of_the_last_layer():
+    """A spot check far into the 128K run: the oracle walks layer 31 through the first 40 chunks (one query
+    row per chunk, so the walk costs projections and scores only), its state - 122880 tokens seen, the
+    cache long since at its budget - is imported, and chunk 40 is compared in lock-step like the first ones."""
+    from parity_util import lockstep_chunk, make_pair
+    w = W.get_workload("c3_llama_128k")
+    ora, gpu = make_pair(w.shape, W.layer_weights(w.shape, 31), w.budget, w.chunk, w.n_stab)
+    start = 0
+    for i in range(40):
+        ora.prefill_chunk(W.hidden_states(w, start, w.chunk), 0, rows=[0])
+        start += w.chunk
+    assert ora.seen == 40 * w.chunk and ora.len == w.budget
+    # the cache holds the last 2500 tokens and 3500 older ones from all over the stream
+    assert ora.T[0][0] < w.chunk * 20 and ora.T[0][-1] == start - 1
+    x = W.hidden_states(w, start, w.chunk)
+    norms = np.linalg.norm(x, axis=1)
+    rows = sorted(set(sampled_rows(w.chunk, 40)) | set(np.flatnonzero(norms > 5 * np.median(norms)).tolist()[:4]))
+    st = lockstep_chunk(ora, gpu, x, 0, rows=rows, what="c3 chunk 40, layer 31")
+    assert "sets_identical" in st and gpu.sync_status() == 0
+    gpu.destroy()
