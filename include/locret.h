@@ -166,6 +166,27 @@ int locret_prefill_chunk_tp_begin(locret_layer *layer, const void *hidden_in, in
                                   uint32_t flags, void *attn_out, float *preact_partial);
 int locret_prefill_chunk_tp_finish(locret_layer *layer, const float *preact_sum);
 
+/*
+ * The exchange of the divided step done by the GEMM itself (Section 3.3: the retaining head reads
+ * every head).  locret_tp_set_peers registers, once, the sum buffers of all n_peers GPUs, this GPU's
+ * among them: peer_sums is a HOST array of n_peers device pointers, each fp32 [chunk x d_R], 16-byte
+ * aligned; a buffer of another GPU must be mapped into this process (peer access or an IPC handle).
+ * Synchronises the layer's streams; allocates a few hundred bytes (and a [chunk x d_R] scratch).
+ * locret_prefill_chunk_tp_begin_peers is locret_prefill_chunk_tp_begin whose first product is not
+ * written to a buffer of the caller but ADDED, tile by tile in the GEMM's epilogue, into rows
+ * [0, n_tok) of EVERY registered buffer, with plain reductions to global memory at system scope (no
+ * TMA and no multicast ever touches a peer's memory).  The caller provides the two orderings an
+ * all-reduce would: every buffer is zero before any GPU starts adding, and every GPU has finished
+ * adding (its begin call's work on the layer's stream is complete) before any GPU's
+ * locret_prefill_chunk_tp_finish reads its own buffer.  Each GPU sends its product n_peers - 1 times
+ * over the links; sums may differ from an all-reduce's in the last bits (the order of the additions is
+ * not fixed).  Not run on more than one GPU by the tests of this library: there all the buffers live on
+ * one device.
+ */
+int locret_tp_set_peers(locret_layer *layer, float *const *peer_sums, int32_t n_peers);
+int locret_prefill_chunk_tp_begin_peers(locret_layer *layer, const void *hidden_in, int32_t n_tok, uint32_t flags,
+                                        void *attn_out);
+
 /* Number of retained units per KV head (the same for every head).  No device work. */
 int locret_cache_len(const locret_layer *layer, int32_t *len);
 
@@ -326,7 +347,7 @@ void locret_block_destroy(locret_block *block);
  * q_ans: device bf16 [n_a × h × d] (queries of the answer tokens as they enter the scores, i.e.
  * after RoPE); k_prompt: device bf16 [n_q × h_kv × d]; labels: device fp32 [h_kv × n_q]
  * (overwritten).  The passage prints the product without the 1/sqrt(d) of Eq. 1: scale = 1
- * reproduces it as printed; scale must be > 0.  head_dim 64 or 128; pointers 16-byte aligned.
+ * reproduces it as printed; scale must be > 0.  head_dim 64, 96 or 128; pointers 16-byte aligned.
  * One tensor-core contraction per query head whose epilogue keeps only row maxima (the
  * n_q × n_a score matrix is never written).  Synchronises the stream before it returns.
  */

@@ -55,6 +55,8 @@ def _load():
     l.locret_decode_step_stack.argtypes = [P, C.c_int32, P, P, C.c_int64]
     l.locret_prefill_chunk_tp_begin.argtypes = [P, P, C.c_int32, C.c_uint32, P, P]
     l.locret_prefill_chunk_tp_finish.argtypes = [P, P]
+    l.locret_tp_set_peers.argtypes = [P, P, C.c_int32]
+    l.locret_prefill_chunk_tp_begin_peers.argtypes = [P, P, C.c_int32, C.c_uint32, P]
     l.locret_cache_len.argtypes = [P, C.POINTER(C.c_int32)]
     l.locret_export_state.argtypes = [P, P, P, P, P, C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
     l.locret_import_state.argtypes = [P, P, P, P, P, C.c_int32, C.c_int64]
@@ -135,6 +137,17 @@ class LocretLayer:
             raise ValueError("preact_partial must be a contiguous CUDA float32 tensor of n_tok x d_retain")
         _check(lib.locret_prefill_chunk_tp_begin(self._h, hidden_in.data_ptr(), n_tok, flags, attn_out.data_ptr(),
                                                  preact_partial.data_ptr()), "locret_prefill_chunk_tp_begin")
+
+    def tp_set_peers(self, peer_sums):
+        """peer_sums: float32 CUDA tensors [chunk, d_retain], one per GPU (this GPU's among them)."""
+        arr = (C.c_void_p * len(peer_sums))(*[t.data_ptr() for t in peer_sums])
+        _check(lib.locret_tp_set_peers(self._h, arr, len(peer_sums)), "locret_tp_set_peers")
+
+    def prefill_chunk_tp_begin_peers(self, hidden_in: torch.Tensor, attn_out: torch.Tensor, flags: int = 0,
+                                     n_tok: int | None = None):
+        n_tok = hidden_in.shape[0] if n_tok is None else n_tok
+        _check(lib.locret_prefill_chunk_tp_begin_peers(self._h, hidden_in.data_ptr(), n_tok, flags,
+                                                       attn_out.data_ptr()), "locret_prefill_chunk_tp_begin_peers")
 
     def prefill_chunk_tp_finish(self, preact_sum: torch.Tensor):
         if not (preact_sum.is_cuda and preact_sum.dtype == torch.float32 and preact_sum.is_contiguous()):

@@ -292,7 +292,7 @@ __device__ int g_cis_status;
 extern "C" int locret_cis_labels(const void *q_ans, const void *k_prompt, int32_t n_a, int32_t n_q, int32_t h,
                                  int32_t h_kv, int32_t d, float scale, float *labels, void *stream) {
   if (!q_ans || !k_prompt || !labels) return LOCRET_ERR_INVALID;
-  if (n_a < 1 || n_q < 1 || h < 1 || h_kv < 1 || h % h_kv || (d != 64 && d != 128) || !(scale > 0.f))
+  if (n_a < 1 || n_q < 1 || h < 1 || h_kv < 1 || h % h_kv || (d != 64 && d != 96 && d != 128) || !(scale > 0.f))
     return LOCRET_ERR_INVALID;
   if ((reinterpret_cast<uintptr_t>(q_ans) | reinterpret_cast<uintptr_t>(k_prompt)) & 15u) return LOCRET_ERR_INVALID;
   cudaStream_t st = (cudaStream_t)stream;

@@ -163,6 +163,12 @@ cudaError_t launch_rh_finish(const float *pre, const float *w2, float *s, int sc
                              int n_tok, int d_R, int h_kv, int act, cudaStream_t st);
 cudaError_t launch_gemm_tc_f32(const bf16 *A, int lda, const bf16 *Bt, int ldb, float *C, int ldc, int M, int N,
                                int K, int *status, cudaStream_t st);
+// the same product ADDED into n_peers fp32 buffers (device array of device pointers; the buffers may be
+// other GPUs' memory): reductions to global memory at system scope, no TMA on peer memory
+cudaError_t launch_gemm_tc_f32_add_peers(const bf16 *A, int lda, const bf16 *Bt, int ldb, float *const *peers,
+                                         int n_peers, int ldc, int M, int N, int K, int *status, cudaStream_t st);
+// peers[p][i] += src[i] for i < count (the fallback beside the GEMM above)
+cudaError_t launch_add_to_peers(const float *src, float *const *peers, int n_peers, size_t count, cudaStream_t st);
 bool gemm_tc_gated_supported(int M, int N, int K, int lda, int ldb);
 cudaError_t launch_gemm_tc_gated(const bf16 *A, int lda, const bf16 *Bt, int ldb, bf16 *C, int ldc, int M,
                                  int N, int K, int *status, cudaStream_t st);

@@ -116,7 +116,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int KB = K / BK;
+  // K-blocks of 64; a last partial block reads past the operands' inner extent, where TMA fills zeros
+  const int KB = (K + BK - 1) / BK;
   const int tiles_n = (N + BN - 1) / BN;
   const int tiles_m = (M + BM - 1) / BM;
   const int total = tiles_m * tiles_n;
@@ -271,6 +272,31 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               for (int v = 0; v < 8; v++)
                 dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
                                      __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+            }
+          }
+        }
+      } else if (MODE == 6) {
+        // Heads divided over GPUs: this GPU's partial product is ADDED into the sum buffer of every
+        // GPU (`partial` holds h_kv = n_peers device pointers to fp32 [M x ldc] buffers, which may be
+        // other GPUs' memory mapped into this process).  Plain reductions to global memory at system
+        // scope, 16 bytes each: no TMA and no multicast touches a peer's memory.
+        if (ok) {
+          float *const *peers = reinterpret_cast<float *const *>(partial);
+#pragma unroll 1
+          for (int c0 = 0; c0 < BN; c0 += 32) {
+            uint32_t r[32];
+            tmem_ld32(taddr + c0, r);
+            tmem_wait_ld();
+            if (row < M && n0 + c0 < N) {
+              for (int pe = 0; pe < h_kv; pe++) {
+                float *dst = peers[pe] + (size_t)row * ldc + n0 + c0;
+#pragma unroll
+                for (int v = 0; v < 8; v++)
+                  asm volatile("red.relaxed.sys.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + 4 * v),
+                               "f"(__uint_as_float(r[4 * v])), "f"(__uint_as_float(r[4 * v + 1])),
+                               "f"(__uint_as_float(r[4 * v + 2])), "f"(__uint_as_float(r[4 * v + 3]))
+                               : "memory");
+              }
             }
           }
         }
@@ -595,8 +621,19 @@ cudaError_t launch_gemm_tc_f32(const bf16 *A, int lda, const bf16 *Bt, int ldb, 
   return launch_t<128, 5>(A, lda, Bt, ldb, Cb, ldc, M, N, K, nullptr, nullptr, 0, 0, RopeAppendArgs{}, status, st);
 }
 
+// peers[p][m][n] += (A Bt^T)[m][n] for every p < n_peers (fp32 buffers with leading dimension ldc floats;
+// `peers` is a DEVICE array of n_peers pointers)
+cudaError_t launch_gemm_tc_f32_add_peers(const bf16 *A, int lda, const bf16 *Bt, int ldb, float *const *peers,
+                                         int n_peers, int ldc, int M, int N, int K, int *status, cudaStream_t st) {
+  float *pl = reinterpret_cast<float *>(const_cast<float **>(peers));
+  if (N >= 256)
+    return launch_t<256, 6>(A, lda, Bt, ldb, nullptr, ldc, M, N, K, nullptr, pl, n_peers, 0, RopeAppendArgs{}, status, st);
+  return launch_t<128, 6>(A, lda, Bt, ldb, nullptr, ldc, M, N, K, nullptr, pl, n_peers, 0, RopeAppendArgs{}, status, st);
+}
+
 // out[m] = max(out[m], scale * max_n (A Bt^T)[m][n]) for m < M (out fp32, initialised by the
-// caller, e.g. to -inf); scale > 0.  K % 64 == 0; any N.
+// caller, e.g. to -inf); scale > 0.  K % 8 == 0 (a last K-block that is not full is zero-filled by
+// TMA); any N.
 cudaError_t launch_gemm_tc_rowmax(const bf16 *A, int lda, const bf16 *Bt, int ldb, float *out, int M, int N,
                                   int K, float scale, int *status, cudaStream_t st) {
   int bits;

@@ -101,6 +101,9 @@ struct locret_layer {
   bool use_side;  // off-critical-path kernels go to the pool's second stream (LOCRET_SERIAL=1 disables)
   bool use_pdl;   // one-token steps overlap their kernels by programmatic dependent launch (LOCRET_NO_PDL=1 disables)
   bool side_pending;
+  float **d_peers;  // divided heads, fused exchange: device array of the GPUs' sum buffers
+  int n_peers;
+  float *tp_scratch;  // this GPU's product for shapes the tensor-core GEMM does not take
   bool tp_pending;  // a divided-heads step was begun and waits for the summed product
   int tp_n_tok;
   uint32_t tp_flags;
@@ -119,7 +122,7 @@ void free_layer_memory(locret_layer *L) {
   cudaFree(L->k_pre); cudaFree(L->v); cudaFree(L->s); cudaFree(L->tid);
   cudaFree(L->q4.kq); cudaFree(L->q4.vq); cudaFree(L->q4.ks); cudaFree(L->q4.vs);
   cudaFree(L->rank[0]); cudaFree(L->rank[1]); cudaFree(L->d_counters);
-  cudaFree(L->k_rot); cudaFree(L->d_status);
+  cudaFree(L->k_rot); cudaFree(L->d_status); cudaFree(L->d_peers); cudaFree(L->tp_scratch);
   for (auto &e : L->events) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
   if (L->ev_ready) cudaEventDestroy(L->ev_ready);
   if (L->ev_tp) cudaEventDestroy(L->ev_tp);
@@ -295,6 +298,7 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   L->n_prefix = 0;
   L->rcur = 0; L->ranked_len = 0; L->len = 0; L->seen = 0; L->launches = 0; L->timing = false; L->serialize = false; L->attn_only = false; L->events_used = 0;
   L->pool = nullptr;
+  L->d_peers = nullptr; L->n_peers = 0; L->tp_scratch = nullptr;
   {
     const char *e = getenv("LOCRET_LEGACY_MMA");
     L->use_tc = !(e && e[0] == '1');
@@ -494,7 +498,7 @@ int evict_and_close(locret_layer *L, int n_tok, uint32_t flags, bool side, cudaS
 // one GPU's share: the step stops after attention and this GPU's partial first product of the
 // retaining head (fp32 [n_tok x d_R], written to tp_partial), everything on the layer's stream.
 int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t flags, void *attn_out,
-               float *tp_partial) {
+               float *tp_partial, bool tp_peers = false) {
   if (!L || !hidden_in || !attn_out) return LOCRET_ERR_INVALID;
   if (!on_layer_device(L)) return LOCRET_ERR_INVALID;
   if (L->tp_pending) return LOCRET_ERR_INVALID;  // a begun step is finished first
@@ -504,7 +508,7 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
   const int n = L->len + n_tok;
   if (n > L->cap) return LOCRET_ERR_CAPACITY;
   ScratchPool *P = L->pool;
-  const bool tp = tp_partial != nullptr;
+  const bool tp = tp_partial != nullptr || tp_peers;
   const bool decode = n_tok == 1 && L->use_tc && !tp;  // one token: bandwidth-bound kernels of decode.cu
   // (a one-token step is a chain of three short kernels on the layer's own stream, overlapped by
   // programmatic dependent launch: an event between them would serialise them again)
@@ -624,11 +628,21 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
     {
       Timed t(L, LOCRET_K_RH, S);
       const bf16 *z = L->cfg.rh_input == 1 ? z_post : staging;
-      if (L->use_tc && gemm_tc_supported(n_tok, L->d_R, L->d_in, L->d_in, L->d_in))
+      const bool tc = L->use_tc && gemm_tc_supported(n_tok, L->d_R, L->d_in, L->d_in, L->d_in);
+      if (tp_peers && tc) {
+        // the exchange inside the GEMM: the epilogue adds each tile into every GPU's sum buffer
+        CK(launch_gemm_tc_f32_add_peers(z, L->d_in, L->w1_t, L->d_in, L->d_peers, L->n_peers, L->d_R, n_tok, L->d_R,
+                                        L->d_in, L->d_status, S));
+      } else if (tp_peers) {
+        CK(launch_preact_naive(z, L->w1_t, L->tp_scratch, n_tok, L->d_R, L->d_in, S));
+        L->launches++;
+        CK(launch_add_to_peers(L->tp_scratch, L->d_peers, L->n_peers, (size_t)n_tok * L->d_R, S));
+      } else if (tc) {
         CK(launch_gemm_tc_f32(z, L->d_in, L->w1_t, L->d_in, tp_partial, L->d_R, n_tok, L->d_R, L->d_in,
                               L->d_status, S));
-      else
+      } else {
         CK(launch_preact_naive(z, L->w1_t, tp_partial, n_tok, L->d_R, L->d_in, S));
+      }
     }
     if (side) {
       CK(cudaEventRecord(P->ev_stage_free[sb], S));
@@ -684,6 +698,27 @@ int locret_prefill_chunk_tp_begin(locret_layer *L, const void *hidden_in, int32_
                                   void *attn_out, float *preact_partial) {
   if (!preact_partial || !aligned16(preact_partial)) return LOCRET_ERR_INVALID;
   return chunk_step(L, hidden_in, n_tok, flags, attn_out, preact_partial);
+}
+
+int locret_tp_set_peers(locret_layer *L, float *const *peer_sums, int32_t n_peers) {
+  if (!L || !peer_sums || n_peers < 1 || n_peers > 64 || !on_layer_device(L) || L->tp_pending) return LOCRET_ERR_INVALID;
+  for (int i = 0; i < n_peers; i++)
+    if (!peer_sums[i] || !aligned16(peer_sums[i])) return LOCRET_ERR_INVALID;
+  CK(sync_all(L));
+  if (!L->d_peers && cudaMalloc(&L->d_peers, 64 * sizeof(float *)) != cudaSuccess) { cudaGetLastError(); return LOCRET_ERR_ALLOC; }
+  if (!L->tp_scratch && cudaMalloc(&L->tp_scratch, (size_t)L->chunk * L->d_R * sizeof(float)) != cudaSuccess) {
+    cudaGetLastError();
+    return LOCRET_ERR_ALLOC;
+  }
+  CK(cudaMemcpy(L->d_peers, peer_sums, (size_t)n_peers * sizeof(float *), cudaMemcpyHostToDevice));
+  L->n_peers = n_peers;
+  return LOCRET_OK;
+}
+
+int locret_prefill_chunk_tp_begin_peers(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t flags,
+                                        void *attn_out) {
+  if (!L || L->n_peers < 1) return LOCRET_ERR_INVALID;
+  return chunk_step(L, hidden_in, n_tok, flags, attn_out, nullptr, true);
 }
 
 int locret_prefill_chunk_tp_finish(locret_layer *L, const float *preact_sum) {

@@ -46,7 +46,21 @@ __global__ void rh_finish_kernel(const float *__restrict__ pre, const float *__r
   }
 }
 
+__global__ void add_to_peers_kernel(const float *__restrict__ src, float *const *__restrict__ peers, int n_peers,
+                                    size_t count) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  const float v = src[i];
+  for (int p = 0; p < n_peers; p++)
+    asm volatile("red.relaxed.sys.global.add.f32 [%0], %1;" ::"l"(peers[p] + i), "f"(v) : "memory");
+}
+
 }  // namespace
+
+cudaError_t launch_add_to_peers(const float *src, float *const *peers, int n_peers, size_t count, cudaStream_t st) {
+  add_to_peers_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(src, peers, n_peers, count);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_preact_naive(const bf16 *z, const bf16 *W1t, float *pre, int n_tok, int d_R, int d_in,
                                 cudaStream_t st) {

@@ -16,7 +16,7 @@ def draw(shape, seed, scale=1.0):
 
 
 @pytest.mark.parametrize("n_a,n_q,h,hk,d", [(40, 300, 4, 2, 64), (257, 1000, 8, 2, 128), (1, 129, 3, 3, 64),
-                                            (300, 70, 4, 1, 128)])
+                                            (300, 70, 4, 1, 128), (257, 1000, 6, 3, 96), (33, 129, 32, 32, 96)])
 def test_cis_labels_match_the_definition(n_a, n_q, h, hk, d):
     from parity_util import bf16_dev
     from paper_2410_01805_b200 import cis_labels
@@ -34,10 +34,10 @@ def test_cis_labels_match_the_definition(n_a, n_q, h, hk, d):
 
 def test_cis_labels_argument_checks():
     from paper_2410_01805_b200 import LocretError, cis_labels
-    q = torch.zeros((4, 2, 96), dtype=torch.bfloat16, device="cuda")
-    k = torch.zeros((8, 2, 96), dtype=torch.bfloat16, device="cuda")
+    q = torch.zeros((4, 2, 80), dtype=torch.bfloat16, device="cuda")
+    k = torch.zeros((8, 2, 80), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(LocretError):
-        cis_labels(q, k)                          # head_dim 96 is not supported here
+        cis_labels(q, k)                          # head_dim 64, 96 or 128
     q = torch.zeros((4, 2, 64), dtype=torch.bfloat16, device="cuda")
     k = torch.zeros((8, 2, 64), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(LocretError):

@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
 class ShardsOnOneGpu:
     """Presents `world` per-rank layer objects as one layer to the lock-step comparison."""
 
-    def __init__(self, shape, weights, budget, chunk, n_stab, world, reserve=0):
+    def __init__(self, shape, weights, budget, chunk, n_stab, world, reserve=0, fused=False):
         from dataclasses import replace
         from paper_2410_01805_b200 import LocretLayer, shard_by_kv_head
         from parity_util import bf16_dev
@@ -30,9 +30,25 @@ class ShardsOnOneGpu:
         self.layers = [LocretLayer(local, *c, budget, chunk, n_stab, reserve=reserve) for c in self.cuts]
         self.pre = [torch.empty(chunk, shape.d_retain, dtype=torch.float32, device="cuda") for _ in range(world)]
         self.outs = [torch.zeros(chunk, self.hl * self.d, dtype=torch.bfloat16, device="cuda") for _ in range(world)]
+        # fused: every rank's GEMM adds its product into every rank's sum buffer (here all on this device)
+        self.fused = fused
+        if fused:
+            for L in self.layers:
+                L.tp_set_peers(self.pre)
 
     def prefill_chunk(self, x, out, flags=0):
         n_tok = x.shape[0]
+        if self.fused:
+            for p in self.pre:
+                p.zero_()                      # first ordering of the exchange: all buffers zero before anyone adds
+            for r, L in enumerate(self.layers):
+                L.prefill_chunk_tp_begin_peers(x, self.outs[r], flags, n_tok)
+            torch.cuda.synchronize()           # second ordering: everybody has added before anybody reads
+            for r, L in enumerate(self.layers):
+                L.prefill_chunk_tp_finish(self.pre[r])
+                out[:n_tok, r * self.hl * self.d:(r + 1) * self.hl * self.d] = self.outs[r][:n_tok]
+            torch.cuda.synchronize()           # (the buffers are zeroed again at the next step)
+            return
         for r, L in enumerate(self.layers):
             L.prefill_chunk_tp_begin(x, self.outs[r], self.pre[r], flags, n_tok)
         total = torch.stack([p[:n_tok] for p in self.pre]).sum(dim=0).contiguous()   # the exchange step
@@ -174,3 +190,35 @@ def test_wrapper_with_one_rank_and_call_order_errors():
     L.prefill_chunk(xd, out)
     assert L.cache_len == 80 and L.sync_status() == 0
     tp.destroy()
+
+
+@pytest.mark.parametrize("world,h,hk,d,D,dR", [(2, 8, 4, 64, 128, 96), (4, 8, 4, 128, 128, 256), (3, 6, 3, 64, 96, 72)])
+def test_exchange_inside_the_gemm_epilogue_all_buffers_on_one_device(world, h, hk, d, D, dR):
+    """The divided step whose first product is added, tile by tile, into every rank's sum buffer by the
+    GEMM's epilogue (reductions to global memory; on several GPUs the buffers are peers' memory, here they
+    all live on this device).  D = 96 / d_R = 72 takes the fallback kernels."""
+    from parity_util import lockstep_chunk
+    sh = W.LayerShape(d_model=D, n_q_heads=h, n_kv_heads=hk, head_dim=d, d_retain=dR, rope_theta=500000.0)
+    weights = W.layer_weights(sh, 0, seed=W.BASE_SEED + 990 + world)
+    ora = oracle_for(sh, weights, 300, 200, 17)
+    gpu = ShardsOnOneGpu(sh, weights, 300, 200, 17, world, fused=True)
+    g = np.random.default_rng(777)
+    for i, n_tok in enumerate([200, 127, 200, 33, 200]):
+        x = W.to_bf16_grid(g.standard_normal((n_tok, sh.d_model)).astype(np.float32))
+        lockstep_chunk(ora, gpu, x, 0, what=f"fused tp{world} chunk {i}")
+    assert ora.len == 300 and gpu.sync_status() == 0
+    gpu.destroy()
+
+
+def test_exchange_inside_the_gemm_epilogue_at_the_llama_shape():
+    from parity_util import lockstep_chunk
+    w = W.get_workload("c3_llama_128k")
+    weights = W.layer_weights(w.shape, 0)
+    ora = oracle_for(w.shape, weights, 1024, 512, 100)
+    gpu = ShardsOnOneGpu(w.shape, weights, 1024, 512, 100, 4, fused=True)
+    start = 0
+    for i in range(3):
+        x = W.hidden_states(w, start, 512)
+        lockstep_chunk(ora, gpu, x, 0, rows=np.array([0, 130, 511]), what=f"llama fused tp4 chunk {i}")
+        start += 512
+    gpu.destroy()
