@@ -25,6 +25,8 @@ What each function follows:
                              per head), the retaining head reads every head's [Q, K, V]
                              (Section 3.3), so the workers exchange one thing, the sum of
                              their partial products z_local · W1_local, before the activation.
+* ``OracleLayerHeadBudgets`` – the same step with one budget per KV head (Appendix H: heads evict
+                             independently, so budgets may differ between them).
 * ``quantize_int4`` / ``dequantize_int4`` – the 4-bit cache variant (Appendix H combines
                              a 4-bit KV cache with the method; the number format is the
                              workload's: symmetric, one fp16 scale per head vector).
@@ -371,6 +373,126 @@ class OracleLayer:
     def decode_step(self, x):
         """The B = 1 case of Eq. 1: append without eviction."""
         return self.prefill_chunk(np.asarray(x, np.float64).reshape(1, -1), NO_EVICT)
+
+
+# --------------------------------------------------------------------------- a budget per head
+#
+# Appendix H (the combination with head-wise budget allocation): "Locret evicts cache units across the
+# attention heads independently", so the budget may differ from head to head.  Every KV head m then has
+# its own cache length len_m = min(b_m, tokens seen), its own re-assigned positions (cache slot i of head
+# m sits at position i, the chunk's token t at len_m + t, Section 3.4) and its own eviction; the
+# retaining head still reads the token's [Q, K, V] of all heads (Section 3.3).  Reading: stabilizers and
+# the protected prefix are the same for every head; the query heads of a group use their KV head's
+# positions.
+
+class OracleLayerHeadBudgets(OracleLayer):
+    """OracleLayer with one budget per KV head.  State per head: Kh[m] [len_m, d], Vh[m], Sh[m] [len_m],
+    Th[m] [len_m]."""
+
+    def __init__(self, shape, w_qkv, w1, w2, head_budgets, chunk: int, n_stab: int, reserve: int = 0,
+                 mirror: bool = False):
+        budgets = [int(b) for b in head_budgets]
+        if len(budgets) != shape.n_kv_heads or min(budgets) < 1 or n_stab > min(budgets):
+            raise ValueError("need one budget >= max(1, n_stab) per KV head")
+        super().__init__(shape, w_qkv, w1, w2, max(budgets), chunk, n_stab, reserve=reserve, mirror=mirror)
+        if self.int4:
+            raise ValueError("per-head budgets are defined for the bf16 cache only")
+        self.budgets = budgets
+        self.reset()
+
+    def set_protected_prefix(self, n_prefix: int):
+        if n_prefix < 0 or n_prefix + self.n_stab > min(self.budgets):
+            raise ValueError("need 0 <= n_prefix and n_prefix + n_stab <= every head's budget")
+        self.n_prefix = int(n_prefix)
+
+    def reset(self):
+        super().reset()
+        hk, d = self.hk, self.d
+        self.Kh = [np.zeros((0, d)) for _ in range(hk)]
+        self.Vh = [np.zeros((0, d)) for _ in range(hk)]
+        self.Sh = [np.zeros(0) for _ in range(hk)]
+        self.Th = [np.zeros(0, dtype=np.int64) for _ in range(hk)]
+
+    @property
+    def lens(self):
+        return [k.shape[0] for k in self.Kh]
+
+    @property
+    def len(self) -> int:
+        return max(self.lens) if hasattr(self, "Kh") else 0
+
+    def export_state(self):
+        return dict(K=[a.copy() for a in self.Kh], V=[a.copy() for a in self.Vh], S=[a.copy() for a in self.Sh],
+                    T=[a.copy() for a in self.Th], seen=self.seen)
+
+    def import_state(self, st):
+        self.Kh = [np.array(a, np.float64) for a in st["K"]]
+        self.Vh = [np.array(a, np.float64) for a in st["V"]]
+        self.Sh = [np.array(a, np.float64) for a in st["S"]]
+        self.Th = [np.array(a, np.int64) for a in st["T"]]
+        self.seen = int(st["seen"])
+
+    def prefill_chunk(self, X, flags: int = 0, rows=None, preact=None):
+        X = np.asarray(X, np.float64)
+        n_tok = X.shape[0]
+        h, hk, d, g = self.h, self.hk, self.d, self.g
+        lens = self.lens
+        if n_tok < 1 or n_tok > self.chunk:
+            raise ValueError("n_tok must be in [1, chunk]")
+        for m in range(hk):
+            if lens[m] + n_tok > self.budgets[m] + self.chunk + (self.cap - self.budget - self.chunk):
+                raise CapacityError("cache capacity exceeded")
+
+        # (a) projections; the staging buffer is a storage point
+        qkv = self._r(project_qkv(X, self.w_qkv, h, hk, d))
+        Q, K, V = split_qkv(qkv, h, hk, d)
+
+        # (b) Eq. 1, head by head: head m's cache slot i sits at position i, the chunk's token t at len_m + t
+        out = np.full((n_tok, h * d), np.nan)
+        self.last_abs_out = np.full((n_tok, h * d), np.nan)
+        self.last_flip_sens = np.full((n_tok, h * d), np.nan) if self.want_flip_sens else None
+        Qr_all = np.zeros_like(Q)
+        Kr_all = np.zeros_like(K)
+        for m in range(hk):
+            pos = (lens[m] + np.arange(n_tok))[:, None]
+            js = slice(m * g, (m + 1) * g)
+            Qr = self._r(rope(Q[:, js, :], pos, self.s.rope_theta))
+            Kr_chunk = self._r(rope(K[:, m:m + 1, :], pos, self.s.rope_theta))
+            Kr_cache = self._r(rope(self.Kh[m][None], np.arange(lens[m])[None, :], self.s.rope_theta))
+            Qr_all[:, js, :], Kr_all[:, m:m + 1, :] = Qr, Kr_chunk
+            cols = slice(m * g * d, (m + 1) * g * d)
+            ab = np.full((n_tok, g * d), np.nan)
+            fs = np.full((n_tok, g * d), np.nan) if self.want_flip_sens else None
+            out[:, cols] = attention_rows(Qr, Kr_cache, self.Vh[m][None], Kr_chunk, V[:, m:m + 1, :], g, rows, ab, fs)
+            self.last_abs_out[:, cols] = ab
+            if fs is not None:
+                self.last_flip_sens[:, cols] = fs
+
+        # (c) retaining head on the token's concatenated [Q ‖ K ‖ V] of all heads
+        if self.s.rh_input == 0:
+            z = qkv
+        else:
+            z = np.concatenate([Qr_all.reshape(n_tok, -1), Kr_all.reshape(n_tok, -1), V.reshape(n_tok, -1)], axis=1)
+        s_chunk = retaining_scores(z, self.w1, self.w2, self.s.act)     # [n_tok, h_kv]
+        self.last_scores = s_chunk
+
+        # (d) per head: concat, protect, top-b_m, gather
+        tid = self.seen + np.arange(n_tok, dtype=np.int64)
+        self.last_keep = [None] * hk
+        for m in range(hk):
+            Km = np.concatenate([self.Kh[m], K[:, m, :]], axis=0)
+            Vm = np.concatenate([self.Vh[m], V[:, m, :]], axis=0)
+            Sm = np.concatenate([self.Sh[m], s_chunk[:, m]])
+            Tm = np.concatenate([self.Th[m], tid])
+            n = Km.shape[0]
+            if not (flags & NO_EVICT) and n > self.budgets[m]:
+                n_prot = 0 if (flags & LAST_CHUNK) else min(self.n_stab, n)
+                keep = select_keep(Sm, self.budgets[m], n_prot, self.n_prefix)
+                self.last_keep[m] = keep
+                Km, Vm, Sm, Tm = Km[keep], Vm[keep], Sm[keep], Tm[keep]
+            self.Kh[m], self.Vh[m], self.Sh[m], self.Th[m] = Km, Vm, Sm, Tm
+        self.seen += n_tok
+        return out
 
 
 # --------------------------------------------------------------------------- heads divided over workers

@@ -601,6 +601,95 @@ def test_each_mirror_rounding_point_is_where_the_stored_value_is_rounded(point):
         assert not np.array_equal(layer.K[:, 12:], np.transpose(K2, (1, 0, 2)))
 
 
+# ------------------------------------------------------------------ a budget per head (Appendix H)
+
+def rand_head_layer(sh, budgets, chunk, n_stab, seed=0, **kw):
+    g = np.random.default_rng(seed)
+    d_in = (sh.n_q_heads + 2 * sh.n_kv_heads) * sh.head_dim
+    wqkv = g.standard_normal((sh.d_model, d_in)) / math.sqrt(sh.d_model)
+    w1 = g.standard_normal((d_in, sh.d_retain)) / math.sqrt(d_in)
+    w2 = g.standard_normal((sh.d_retain, sh.n_kv_heads)) / math.sqrt(sh.d_retain)
+    return O.OracleLayerHeadBudgets(sh, wqkv, w1, w2, budgets, chunk, n_stab, **kw), (wqkv, w1, w2)
+
+
+@pytest.mark.parametrize("mirror", [False, True])
+def test_equal_head_budgets_reproduce_the_single_budget_layer(mirror):
+    sh = shape(n_q_heads=6, n_kv_heads=3)
+    lh, (wqkv, w1, w2) = rand_head_layer(sh, [9, 9, 9], 5, 2, seed=50, mirror=mirror)
+    lu = O.OracleLayer(sh, wqkv, w1, w2, 9, 5, 2, mirror=mirror)
+    X = np.random.default_rng(51).standard_normal((23, sh.d_model))
+    for s0 in range(0, 23, 5):
+        a, b = lh.prefill_chunk(X[s0:s0 + 5]), lu.prefill_chunk(X[s0:s0 + 5])
+        assert np.array_equal(a, b)
+        for m in range(3):
+            assert np.array_equal(lh.Th[m], lu.T[m]) and np.array_equal(lh.Kh[m], lu.K[m])
+            assert np.array_equal(lh.Sh[m], lu.S[m]) and np.array_equal(lh.Vh[m], lu.V[m])
+
+
+@pytest.mark.parametrize("B", [3, 8, 16])
+def test_head_budgets_closed_form_per_head_and_sizes(B):
+    """Scores depend on the token alone, so head m ends with Last_{n_s} ∪ Top_{b_m - n_s} of the earlier
+    tokens whatever the chunking and whatever the other heads keep; its size is min(b_m, seen) throughout."""
+    sh = shape(n_q_heads=4, n_kv_heads=4, head_dim=4, d_model=12)
+    budgets, n_stab, ctx = [5, 11, 40, 7], 3, 37
+    layer, (wqkv, w1, w2) = rand_head_layer(sh, budgets, 16, n_stab, seed=52)
+    X = np.random.default_rng(53).standard_normal((ctx, sh.d_model))
+    seen = 0
+    for s0 in range(0, ctx, B):
+        layer.prefill_chunk(X[s0:s0 + B])
+        seen = min(ctx, s0 + B)
+        assert layer.lens == [min(b, seen) for b in budgets]
+        for m in range(4):
+            assert np.all(np.diff(layer.Th[m]) > 0)
+    s_all = O.retaining_scores(X @ wqkv, w1, w2)
+    for m, b in enumerate(budgets):
+        if b >= ctx:
+            assert list(layer.Th[m]) == list(range(ctx))
+            continue
+        rest = ctx - n_stab
+        order = sorted(range(rest), key=lambda i: (-s_all[i, m], -i))
+        assert list(layer.Th[m]) == sorted(order[: b - n_stab] + list(range(rest, ctx)))
+        assert np.allclose(layer.Sh[m], s_all[layer.Th[m], m], atol=1e-12)
+
+
+def test_a_head_whose_budget_covers_the_context_attends_to_everything_while_others_evict():
+    sh = shape(n_q_heads=4, n_kv_heads=2, head_dim=8, d_model=16)
+    ctx = 29
+    layer, (wqkv, _, _) = rand_head_layer(sh, [ctx, 6], 7, 2, seed=54)
+    X = np.random.default_rng(55).standard_normal((ctx, sh.d_model))
+    got = run_chunks(layer, X, 7)
+    want = brute_force_causal_attention(X, wqkv, sh)
+    # query heads 0, 1 belong to KV head 0 (nothing evicted): full causal attention at true positions
+    assert np.allclose(got[:, :16], want[:, :16], rtol=0, atol=1e-11)
+    # query heads 2, 3 see a cache of 6 units: different from full attention, and equal to the hand gather
+    assert not np.allclose(got[8:, 16:], want[8:, 16:], atol=1e-3)
+    assert layer.lens == [ctx, 6]
+
+
+def test_head_budget_attention_over_an_evicted_head_uses_that_heads_positions():
+    """After eviction head m's kept units sit at positions 0..len_m-1 and the chunk follows at len_m + t:
+    checked by an explicit gather for a head with a small budget beside one with a large budget."""
+    sh = shape(n_q_heads=2, n_kv_heads=2, head_dim=8, d_model=16)
+    layer, (wqkv, w1, w2) = rand_head_layer(sh, [4, 12], 5, 1, seed=56)
+    X = np.random.default_rng(57).standard_normal((15, sh.d_model))
+    layer.prefill_chunk(X[:5]); layer.prefill_chunk(X[5:10])
+    kept = [t.copy() for t in layer.Th]
+    assert [len(k) for k in kept] == [4, 10]
+    out = layer.prefill_chunk(X[10:15])
+    proj = X @ wqkv
+    h, hk, d = 2, 2, 8
+    for m in range(2):
+        toks = list(kept[m]) + list(range(10, 15))
+        ln = len(kept[m])
+        Kr = O.rope(proj[toks, (h + m) * d:(h + m + 1) * d], np.arange(len(toks)), sh.rope_theta)
+        Vv = proj[toks, (h + hk + m) * d:(h + hk + m + 1) * d]
+        for t in range(5):
+            q = O.rope(proj[10 + t, m * d:(m + 1) * d], ln + t, sh.rope_theta)
+            lg = Kr[: ln + t + 1] @ q / math.sqrt(d)
+            p = np.exp(lg - lg.max()); p /= p.sum()
+            assert np.allclose(out[t, m * d:(m + 1) * d], p @ Vv[: ln + t + 1], atol=1e-12)
+
+
 def test_mirror_mode_rounds_only_storage_points():
     sh = shape()
     lp, (wqkv, w1, w2) = rand_layer(sh, budget=64, chunk=16, n_stab=0, seed=26)
