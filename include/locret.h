@@ -268,6 +268,29 @@ int locret_reset(locret_layer *layer);
 int locret_set_protected_prefix(locret_layer *layer, int32_t n_prefix);
 
 /*
+ * A budget per KV head (Appendix H, the combination with head-wise budget allocation: "Locret evicts
+ * cache units across the attention heads independently", so budgets may differ between heads; a budget
+ * per layer is simply the `budget` each layer is created with).  budgets: HOST int32 [n_kv_heads], each
+ * 1 <= b_m <= the budget given at create (which sizes the cache) and >= n_stab + protected prefix.
+ * Allowed only while the layer is empty (right after create or locret_reset); LOCRET_ERR_INVALID for a
+ * 4-bit cache.  From then on head m keeps min(b_m, tokens seen) units: its cache slot i sits at position i
+ * and the chunk's token t at len_m + t (Section 3.4), its query heads use those positions, and it is cut
+ * to b_m by every evicting step in which it holds more; the retaining head still reads all heads'
+ * [Q, K, V].  Steps with head budgets use the general kernels (projection, then positions / RoPE / append
+ * in a pass of their own; one-token steps take the chunk kernels); the divided-heads calls are refused.
+ * locret_cache_len then returns the largest length; locret_cache_lens all of them (HOST int32
+ * [n_kv_heads]; also valid without head budgets).  State is exchanged with the _heads calls below:
+ * arrays as in locret_export_state but with `pitch` rows per head (pitch >= the largest length), head
+ * m's first lens[m] rows valid, in temporal order; the plain export / import calls are refused.
+ */
+int locret_set_head_budgets(locret_layer *layer, const int32_t *budgets);
+int locret_cache_lens(const locret_layer *layer, int32_t *lens);
+int locret_export_state_heads(locret_layer *layer, void *K, void *V, float *scores, int64_t *token_ids,
+                              int32_t pitch, int32_t *lens, int64_t *tokens_seen);
+int locret_import_state_heads(locret_layer *layer, const void *K, const void *V, const float *scores,
+                              const int64_t *token_ids, int32_t pitch, const int32_t *lens, int64_t tokens_seen);
+
+/*
  * Per-kernel timing.  With enable != 0 every kernel launched for this layer is
  * bracketed by CUDA events on the stream it runs on (kernels on the two streams overlap, so
  * the per-kernel times of a step add up to more than its duration); enable = 2 also keeps

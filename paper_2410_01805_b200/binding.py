@@ -70,6 +70,10 @@ def _load():
     l.locret_read_timing.argtypes = [P, P, P]
     l.locret_launch_count.argtypes = [P, C.POINTER(C.c_int64)]
     l.locret_compaction_counters.argtypes = [P, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+    l.locret_set_head_budgets.argtypes = [P, P]
+    l.locret_cache_lens.argtypes = [P, P]
+    l.locret_export_state_heads.argtypes = [P, P, P, P, P, C.c_int32, P, C.POINTER(C.c_int64)]
+    l.locret_import_state_heads.argtypes = [P, P, P, P, P, C.c_int32, P, C.c_int64]
     l.locret_rh_scores_static.argtypes = [P, C.c_int32, C.c_int32, P, C.c_int32, P, C.c_int32, C.c_int32, P, P, P]
     l.locret_selftest_wait_abort.argtypes = [P, P]
     l.locret_destroy.argtypes = [P]
@@ -220,6 +224,52 @@ class LocretLayer:
         n = Kb.shape[1]
         _check(lib.locret_import_state(self._h, Kb.data_ptr(), Vb.data_ptr(), Sb.ctypes.data,
                                        Tb.ctypes.data, n, int(seen)), "locret_import_state")
+
+    # -- a budget per KV head
+    def set_head_budgets(self, budgets):
+        b = np.ascontiguousarray(budgets, dtype=np.int32)
+        if b.shape != (self.h_kv,):
+            raise ValueError("one budget per KV head")
+        _check(lib.locret_set_head_budgets(self._h, b.ctypes.data), "locret_set_head_budgets")
+
+    @property
+    def cache_lens(self):
+        lens = np.zeros(self.h_kv, dtype=np.int32)
+        _check(lib.locret_cache_lens(self._h, lens.ctypes.data), "locret_cache_lens")
+        return lens.tolist()
+
+    def export_state_heads(self):
+        """dict(K, V: lists of [len_m, d] float32 arrays; S, T: lists of [len_m]; seen)."""
+        lens = self.cache_lens
+        pitch = max(max(lens), 1)
+        K = torch.zeros((self.h_kv, pitch, self.d), dtype=torch.bfloat16)
+        V = torch.zeros_like(K)
+        S = np.zeros((self.h_kv, pitch), dtype=np.float32)
+        T = np.zeros((self.h_kv, pitch), dtype=np.int64)
+        out_lens = np.zeros(self.h_kv, dtype=np.int32)
+        seen = C.c_int64()
+        _check(lib.locret_export_state_heads(self._h, K.data_ptr(), V.data_ptr(), S.ctypes.data, T.ctypes.data, pitch,
+                                             out_lens.ctypes.data, C.byref(seen)), "locret_export_state_heads")
+        Kf, Vf = K.float().numpy(), V.float().numpy()
+        return dict(K=[Kf[m, :n] for m, n in enumerate(out_lens)], V=[Vf[m, :n] for m, n in enumerate(out_lens)],
+                    S=[S[m, :n] for m, n in enumerate(out_lens)], T=[T[m, :n] for m, n in enumerate(out_lens)],
+                    seen=seen.value)
+
+    def import_state_heads(self, K, V, S, T, seen: int):
+        lens = np.array([len(t) for t in T], dtype=np.int32)
+        pitch = max(int(lens.max()), 1)
+        Kb = torch.zeros((self.h_kv, pitch, self.d), dtype=torch.bfloat16)
+        Vb = torch.zeros_like(Kb)
+        Sb = np.zeros((self.h_kv, pitch), dtype=np.float32)
+        Tb = np.zeros((self.h_kv, pitch), dtype=np.int64)
+        for m, n in enumerate(lens):
+            if n:
+                Kb[m, :n] = torch.from_numpy(np.ascontiguousarray(K[m], dtype=np.float32)).to(torch.bfloat16)
+                Vb[m, :n] = torch.from_numpy(np.ascontiguousarray(V[m], dtype=np.float32)).to(torch.bfloat16)
+                Sb[m, :n] = S[m]
+                Tb[m, :n] = T[m]
+        _check(lib.locret_import_state_heads(self._h, Kb.data_ptr(), Vb.data_ptr(), Sb.ctypes.data, Tb.ctypes.data, pitch,
+                                             lens.ctypes.data, int(seen)), "locret_import_state_heads")
 
     def sync_status(self) -> int:
         return lib.locret_sync_status(self._h)

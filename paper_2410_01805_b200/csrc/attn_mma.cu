@@ -15,7 +15,7 @@ template <int D>
 __global__ void __launch_bounds__(ATHREADS)
 attn_mma_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_rot,
                 const bf16 *__restrict__ v, bf16 *__restrict__ out, int n_tok, int h, int h_kv,
-                int cap, int len, float scale_log2) {
+                int cap, int len_all, float scale_log2, int per_head, PerHead len_m) {
   constexpr int LD = D + 8;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   bf16 *sQ = reinterpret_cast<bf16 *>(smem_raw);
@@ -28,6 +28,7 @@ attn_mma_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_rot,
   const int q0 = qtile * QT;
   const int j = blockIdx.y;
   const int m = j / (h / h_kv);
+  const int len = per_head ? len_m.v[m] : len_all;  // (a budget per head: this KV head's cache length)
   const int n = len + n_tok;
   const int n_keys = min(n, len + q0 + QT);
   const int NKT = (n_keys + KT_ - 1) / KT_;
@@ -182,14 +183,14 @@ attn_mma_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_rot,
 
 template <int D>
 cudaError_t launch_d(const bf16 *q_rot, const bf16 *k_rot, const bf16 *v, bf16 *out, int n_tok, int h,
-                     int h_kv, int cap, int len, cudaStream_t st) {
+                     int h_kv, int cap, int len, cudaStream_t st, const PerHead *len_m) {
   constexpr int smem = (QT + 4 * KT_) * (D + 8) * 2;
   static PerDeviceFlag attr_set;
   if (cudaError_t e = allow_dynamic_smem(attn_mma_kernel<D>, smem, attr_set); e != cudaSuccess) return e;
   dim3 grid((n_tok + QT - 1) / QT, h);
   float scale_log2 = 1.4426950408889634f / sqrtf((float)D);
   attn_mma_kernel<D><<<grid, ATHREADS, smem, st>>>(q_rot, k_rot, v, out, n_tok, h, h_kv, cap, len,
-                                                   scale_log2);
+                                                   scale_log2, len_m ? 1 : 0, len_m ? *len_m : PerHead{});
   return cudaGetLastError();
 }
 
@@ -197,11 +198,11 @@ cudaError_t launch_d(const bf16 *q_rot, const bf16 *k_rot, const bf16 *v, bf16 *
 
 cudaError_t launch_attention_mma(const bf16 *q_rot, const bf16 *k_rot, const bf16 *v, bf16 *out,
                                  int n_tok, int h, int h_kv, int d, int cap, int len,
-                                 cudaStream_t st) {
+                                 cudaStream_t st, const PerHead *len_m) {
   switch (d) {
-    case 64: return launch_d<64>(q_rot, k_rot, v, out, n_tok, h, h_kv, cap, len, st);
-    case 96: return launch_d<96>(q_rot, k_rot, v, out, n_tok, h, h_kv, cap, len, st);
-    case 128: return launch_d<128>(q_rot, k_rot, v, out, n_tok, h, h_kv, cap, len, st);
+    case 64: return launch_d<64>(q_rot, k_rot, v, out, n_tok, h, h_kv, cap, len, st, len_m);
+    case 96: return launch_d<96>(q_rot, k_rot, v, out, n_tok, h, h_kv, cap, len, st, len_m);
+    case 128: return launch_d<128>(q_rot, k_rot, v, out, n_tok, h, h_kv, cap, len, st, len_m);
   }
   return cudaErrorInvalidValue;
 }

@@ -83,6 +83,8 @@ struct AttnParams {
   int n_tok, h, h_kv, d, len, pair_heads;
   float scale_log2;
   int *status;
+  int per_head;   // a budget per head: KV head m holds len_m.v[m] retained units
+  PerHead len_m;
 };
 
 template <int D>
@@ -110,7 +112,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = p.h / p.h_kv;
-  const int n = p.len + p.n_tok;
   const int n_rb = (p.n_tok + TILE - 1) / TILE;
 
   // which two query tiles; longest key ranges first
@@ -128,12 +129,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     head[0] = head[1] = (int)blockIdx.x % p.h;
   }
   const int kvh = head[0] / g;
-  int NK = (p.len + row0[1] + TILE + TILE - 1) / TILE;
+  const int len = p.per_head ? p.len_m.v[kvh] : p.len;   // retained units of this KV head
+  const int n = len + p.n_tok;
+  int NK = (len + row0[1] + TILE + TILE - 1) / TILE;
   NK = min(NK, (n + TILE - 1) / TILE);
   // The softmax is order independent, so every CTA walks the key tiles that need no mask in its
   // own rotated order: CTAs of one KV head start together, and in a common order they would all
   // ask the L2 for the same K and V lines at the same moment (measured: 1.4x slower).
-  const int NF = min(NK, (p.len + row0[0] + 1) / TILE);  // tiles fully visible to every row
+  const int NF = min(NK, (len + row0[0] + 1) / TILE);  // tiles fully visible to every row
   const int rot = NF > 0 ? (int)((blockIdx.x * 29u + 7u) % (unsigned)NF) : 0;
   auto tile_of = [&](int j) { int x = j + rot; return j < NF ? (x >= NF ? x - NF : x) : j; };
 
@@ -286,7 +289,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 #pragma unroll
       for (int t = 0; t < 2; t++) {
         const int row = row0[t] + r;
-        const int limit = p.len + row;  // last visible key
+        const int limit = len + row;  // last visible key
         const uint32_t s_addr = tmem_base + lane_off + t * TILE;
         const uint32_t o_addr = tmem_base + lane_off + 2 * TILE + t * HD;
         if (ok) ok = mbar_wait(&s_full[t], j & 1, abort_flag, p.status);
@@ -298,7 +301,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
         const int key0 = tile_of(j) * TILE;
         float tmax;
-        if (key0 + TILE - 1 > p.len + row0[t]) {  // a tile that crosses the causal boundary
+        if (key0 + TILE - 1 > len + row0[t]) {  // a tile that crosses the causal boundary
           tmax = -INFINITY;
 #pragma unroll
           for (int i = 0; i < 64; i++) {
@@ -436,9 +439,11 @@ static cudaError_t launch_attn_d(const CUtensorMap *map_q, const CUtensorMap *ma
 
 cudaError_t launch_attention_tc(const CUtensorMap *map_q, const CUtensorMap *map_k,
                                 const CUtensorMap *map_v, bf16 *out, int n_tok, int h, int h_kv, int d,
-                                int len, int *status, cudaStream_t st) {
+                                int len, int *status, cudaStream_t st, const PerHead *len_m) {
   AttnParams p;
   p.out = out; p.n_tok = n_tok; p.h = h; p.h_kv = h_kv; p.d = d; p.len = len;
+  p.per_head = len_m ? 1 : 0;
+  p.len_m = len_m ? *len_m : PerHead{};
   p.pair_heads = ((h / h_kv) % 2 == 0) ? 1 : 0;
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)d);
   p.status = status;

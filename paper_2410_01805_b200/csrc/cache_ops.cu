@@ -50,7 +50,9 @@ __global__ void rope_append_kernel(RopeAppendArgs a) {
   const bf16 *src = a.staging + (size_t)t * d_in + (size_t)hd * a.d;
   Vec8 self, partner;
   self.raw = *reinterpret_cast<const uint4 *>(src + c);
-  const int slot = a.len + t;
+  // the head's own cache length when the heads have budgets of their own (a query head uses its KV head's)
+  const int kvh = hd < a.h ? hd / (a.h / a.h_kv) : (hd < a.h + a.h_kv ? hd - a.h : hd - a.h - a.h_kv);
+  const int slot = (a.per_head ? a.len_m.v[kvh] : a.len) + t;
   const float2 *cs_row = a.cs + (size_t)slot * half;
   if (hd < a.h + a.h_kv) {
     partner.raw = *reinterpret_cast<const uint4 *>(src + (c < half ? c + half : c - half));
@@ -106,12 +108,15 @@ __device__ __forceinline__ void rope_pairs8(const uint4 &lo, const uint4 &hi, co
 // blockDim.x = d / 16 threads per row, blockDim.y rows per block.
 __global__ void compact_kernel(CompactArgs a) {
   const int row = blockIdx.x * blockDim.y + threadIdx.y;
-  if (row >= a.h_kv * a.budget) return;
-  const int m = row / a.budget, i = row - m * a.budget;
+  if (row >= a.h_kv * a.src_stride) return;
+  const int m = row / a.src_stride, i = row - m * a.src_stride;
+  if (a.per_head ? (!a.evict_m.v[m] || i >= a.budget_m.v[m]) : i >= a.budget) return;
+  const int ranked_len = a.per_head ? a.ranked_m.v[m] : a.ranked_len;
+  const int rcur = a.per_head ? a.rcur_m.v[m] : a.rcur;
   const size_t u = (size_t)m * a.cap + i;
-  const int src = a.src_of[(size_t)m * a.budget + i];
-  const int pos = a.rank_new[u];
-  const int pos_old = i < a.ranked_len ? a.rank_old[u] : i;
+  const int src = a.src_of[(size_t)m * a.src_stride + i];
+  const int pos = a.rank[rcur ^ 1][u];
+  const int pos_old = i < ranked_len ? a.rank[rcur][u] : i;
   if (src == i && pos == pos_old) return;  // stays, and stays where it was in the order
   const int c = threadIdx.x * 8;
   const int half = a.d / 2;
@@ -310,7 +315,8 @@ topk_kernel(TopkArgs a, int cache_in_smem) {
   __shared__ int s_total_eq;
 
   const int m = blockIdx.x, tid = threadIdx.x;
-  const int n = a.n, budget = a.budget;
+  const int n = a.per_head ? a.n_m.v[m] : a.n, budget = a.per_head ? a.budget_m.v[m] : a.budget;
+  if (n <= budget) return;  // (a budget per head: this head keeps everything in this step)
   const int W = (n + 31) / 32;
   uint32_t *keptbits = tk_smem;          // bit s: slot s is kept
   uint32_t *evbits = tk_smem + W;        // bit r: the unit of rank r is evicted
@@ -320,12 +326,14 @@ topk_kernel(TopkArgs a, int cache_in_smem) {
   int32_t *sranks = reinterpret_cast<int32_t *>(tk_smem + 5 * W + n);
 
   const float *sc = a.scores + (size_t)m * a.stride;
-  const int32_t *rk = a.rank_old + (size_t)m * a.stride;
-  int32_t *src_of = a.src_of + (size_t)m * budget;
-  int32_t *rank_new = a.rank_new + (size_t)m * a.stride;
-  const int ranked_len = a.ranked_len;
-  const int lo_rank = a.n_pre, hi_rank = n - a.n_prot;   // ranks [lo_rank, hi_rank) compete
-  const int k = budget - a.n_prot - a.n_pre;              // 0 <= k < hi_rank - lo_rank (n > budget)
+  const int rcur = a.per_head ? a.rcur_m.v[m] : a.rcur;
+  const int32_t *rk = a.rank[rcur] + (size_t)m * a.stride;
+  int32_t *src_of = a.src_of + (size_t)m * a.src_stride;
+  int32_t *rank_new = a.rank[rcur ^ 1] + (size_t)m * a.stride;
+  const int ranked_len = a.per_head ? a.ranked_m.v[m] : a.ranked_len;
+  const int n_prot = a.per_head ? a.nprot_m.v[m] : a.n_prot;
+  const int lo_rank = a.n_pre, hi_rank = n - n_prot;   // ranks [lo_rank, hi_rank) compete
+  const int k = budget - n_prot - a.n_pre;              // 0 <= k < hi_rank - lo_rank (n > budget)
 
   auto key_at = [&](int i) -> uint32_t { return cache_in_smem ? skeys[i] : score_key(sc[i]); };
   auto rank_at = [&](int i) -> int { return cache_in_smem ? sranks[i] : (i < ranked_len ? rk[i] : i); };
@@ -489,7 +497,7 @@ cudaError_t launch_rope_append(const RopeAppendArgs &a, cudaStream_t st) {
 
 cudaError_t launch_compact(const CompactArgs &a, cudaStream_t st) {
   const int tpr = a.d / 16, rpb = 256 / tpr;  // threads per row, rows per block
-  const int rows = a.h_kv * a.budget;
+  const int rows = a.h_kv * a.src_stride;
   compact_kernel<<<(rows + rpb - 1) / rpb, dim3(tpr, rpb), 0, st>>>(a);
   return cudaGetLastError();
 }
@@ -513,9 +521,14 @@ cudaError_t launch_topk(const TopkArgs &a, int h_kv, cudaStream_t st) {
   const size_t max_dyn = 200 * 1024;
   static PerDeviceFlag attr_set;
   if (cudaError_t e = allow_dynamic_smem(topk_kernel, (int)max_dyn, attr_set); e != cudaSuccess) return e;
-  const int cached = topk_smem_bytes(a.n, true) <= max_dyn;
-  const size_t bytes = topk_smem_bytes(a.n, cached);
-  if (bytes > max_dyn || a.n > a.stride) return cudaErrorInvalidValue;
+  int n_max = a.n;
+  if (a.per_head) {
+    n_max = 0;
+    for (int m = 0; m < h_kv; m++) n_max = a.n_m.v[m] > n_max ? a.n_m.v[m] : n_max;
+  }
+  const int cached = topk_smem_bytes(n_max, true) <= max_dyn;
+  const size_t bytes = topk_smem_bytes(n_max, cached);
+  if (bytes > max_dyn || n_max > a.stride) return cudaErrorInvalidValue;
   topk_kernel<<<h_kv, TK_THREADS, bytes, st>>>(a, cached);
   return cudaGetLastError();
 }

@@ -128,6 +128,11 @@ inline int sm_count_of_current_device() {
   return count[dev];
 }
 
+// One value per KV head, handed to kernels by value (a layer has at most 32 KV heads).  Used when the
+// heads have budgets of their own (Appendix H: heads evict independently): cache lengths, and with
+// them append slots and positions, then differ from head to head.
+struct PerHead { int v[32]; };
+
 // ---------------------------------------------------------------- launchers (host)
 // Every launcher enqueues on `st` and returns the cudaError_t of the launch.
 
@@ -181,7 +186,7 @@ int rh_tc_num_tiles(int d_R);
 
 // scores[m][slot0 + t] = sum_nt partial[nt][t][m]
 cudaError_t launch_rh_reduce(const float *partial, int n_tiles, int M, int h_kv, float *scores,
-                             int score_stride, int slot0, cudaStream_t st);
+                             int score_stride, int slot0, cudaStream_t st, const PerHead *slot0_m = nullptr);
 
 struct RopeAppendArgs {
   const bf16 *staging;  // [n_tok x d_in]  pre-RoPE Q | K | V
@@ -194,6 +199,8 @@ struct RopeAppendArgs {
   const float2 *cs;     // [cap][d/2] (cos, sin)
   int n_tok, h, h_kv, d, cap, len;
   int64_t seen;
+  int per_head;    // the chunk is appended at slot len_m.v[m] + t of KV head m (query heads use their KV head's)
+  PerHead len_m;   // (read by rope_append_kernel only: the fused epilogue and the one-token kernel take `len`)
 };
 cudaError_t launch_rope_append(const RopeAppendArgs &a, cudaStream_t st);
 // The projection GEMM with rope_append's work done in its epilogue (a.staging is written, not read).
@@ -204,7 +211,7 @@ cudaError_t launch_qkv_rope_tc(const bf16 *X, int ldx, const bf16 *Wt, int ldw, 
 // Attention (Eq. 1): query row t of head j sees keys [0, len + t] of KV head j / g.
 cudaError_t launch_attention_mma(const bf16 *q_rot, const bf16 *k_rot, const bf16 *v, bf16 *out,
                                  int n_tok, int h, int h_kv, int d, int cap, int len,
-                                 cudaStream_t st);
+                                 cudaStream_t st, const PerHead *len_m = nullptr);
 
 // Eviction in place.  Kept units stay in their slots and freed slots below `budget` are refilled, so
 // slot order is not temporal order: a unit's position in temporal order is its RANK, stored per slot
@@ -212,13 +219,17 @@ cudaError_t launch_attention_mma(const bf16 *q_rot, const bf16 *k_rot, const bf1
 // rank = slot.
 struct TopkArgs {
   const float *scores;      // [h_kv][stride]
-  const int32_t *rank_old;  // [h_kv][stride]
+  int32_t *rank[2];         // [h_kv][stride] each: rank[rcur] holds the ranks, the other receives the new ones
+  int rcur;                 //   (for slots < budget; its entries from budget on are used as scratch)
   int stride, ranked_len;
   int n, budget, n_prot, n_pre;   // candidates: slots [0, n); ranks [0, n_pre) and [n - n_prot, n) protected
-  int32_t *src_of;          // [h_kv][budget]  out: the slot whose unit ends up in slot i
-  int32_t *rank_new;        // [h_kv][stride]  out: rank after the eviction, for slots < budget (the
-                            //                 entries from budget on are used as scratch)
+  int32_t *src_of;          // [h_kv][src_stride]  out: the slot whose unit ends up in slot i
+  int src_stride;
   unsigned long long *counters;  // [2] or null: units moved to another slot, rotated keys rewritten (added to)
+  // a budget per head: head m has n_m candidates, budget_m, nprot_m protected at the end, ranks valid
+  // below ranked_m, its ranks in rank[rcur_m]; a head with n_m <= budget_m keeps everything and is skipped
+  int per_head;
+  PerHead n_m, budget_m, nprot_m, ranked_m, rcur_m;
 };
 cudaError_t launch_topk(const TopkArgs &a, int h_kv, cudaStream_t st);
 
@@ -226,10 +237,13 @@ struct CompactArgs {
   bf16 *k, *v, *k_rot;      // [h_kv][cap][d]
   float *s;                 // [h_kv][cap]
   int64_t *t;
-  const int32_t *src_of;    // [h_kv][budget]
-  const int32_t *rank_new, *rank_old;  // [h_kv][cap]
+  const int32_t *src_of;    // [h_kv][src_stride]
+  const int32_t *rank[2];   // [h_kv][cap]: rank[rcur] before the eviction, the other after
+  int rcur;
   const float2 *cs;
-  int h_kv, d, cap, budget, ranked_len;
+  int h_kv, d, cap, budget, ranked_len, src_stride;
+  int per_head;             // (see TopkArgs) evict_m: 1 where head m evicts in this step
+  PerHead budget_m, ranked_m, rcur_m, evict_m;
 };
 cudaError_t launch_compact(const CompactArgs &a, cudaStream_t st);
 

@@ -159,13 +159,14 @@ gemm_mma_kernel(const bf16 *__restrict__ A, int lda, const bf16 *__restrict__ Bt
 }
 
 __global__ void rh_reduce_kernel(const float *__restrict__ partial, int n_tiles, int M, int h_kv,
-                                 float *__restrict__ scores, int score_stride, int slot0) {
+                                 float *__restrict__ scores, int score_stride, int slot0, int per_head,
+                                 PerHead slot0_m) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= M * h_kv) return;
   int t = i / h_kv, m = i - t * h_kv;
   float s = 0.f;
   for (int nt = 0; nt < n_tiles; nt++) s += partial[((size_t)nt * M + t) * h_kv + m];
-  scores[(size_t)m * score_stride + slot0 + t] = s;
+  scores[(size_t)m * score_stride + (per_head ? slot0_m.v[m] : slot0) + t] = s;
 }
 
 constexpr int rh_smem_bytes(int h_kv) {
@@ -201,10 +202,10 @@ cudaError_t launch_rh_gemm(const bf16 *A, int lda, const bf16 *W1t, const float 
 }
 
 cudaError_t launch_rh_reduce(const float *partial, int n_tiles, int M, int h_kv, float *scores,
-                             int score_stride, int slot0, cudaStream_t st) {
+                             int score_stride, int slot0, cudaStream_t st, const PerHead *slot0_m) {
   int total = M * h_kv;
-  rh_reduce_kernel<<<(total + 255) / 256, 256, 0, st>>>(partial, n_tiles, M, h_kv, scores,
-                                                        score_stride, slot0);
+  rh_reduce_kernel<<<(total + 255) / 256, 256, 0, st>>>(partial, n_tiles, M, h_kv, scores, score_stride, slot0,
+                                                        slot0_m ? 1 : 0, slot0_m ? *slot0_m : PerHead{});
   return cudaGetLastError();
 }
 

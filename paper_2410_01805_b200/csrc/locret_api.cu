@@ -86,6 +86,10 @@ struct locret_layer {
   // The other array receives the ranks of the next eviction.
   int32_t *rank[2];
   int rcur, ranked_len;
+  // a budget per KV head (Appendix H): lengths, valid-rank counts and the array that holds the ranks
+  // then differ from head to head; `len` is the largest length
+  bool per_head;
+  PerHead budget_m, len_m, ranked_m, rcur_m;
   unsigned long long *d_counters;  // [2]: units moved to another slot, rotated keys rewritten
   int device;  // the device that was current at create: every later call must find it current
   const float2 *cs;
@@ -296,7 +300,9 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   L->st = (cudaStream_t)cfg->stream;
   L->device = dev;
   L->n_prefix = 0;
-  L->rcur = 0; L->ranked_len = 0; L->len = 0; L->seen = 0; L->launches = 0; L->timing = false; L->serialize = false; L->attn_only = false; L->events_used = 0;
+  L->rcur = 0; L->ranked_len = 0; L->len = 0;
+  L->per_head = false;
+  for (int m = 0; m < 32; m++) { L->budget_m.v[m] = budget; L->len_m.v[m] = 0; L->ranked_m.v[m] = 0; L->rcur_m.v[m] = 0; } L->seen = 0; L->launches = 0; L->timing = false; L->serialize = false; L->attn_only = false; L->events_used = 0;
   L->pool = nullptr;
   L->d_peers = nullptr; L->n_peers = 0; L->tp_scratch = nullptr;
   {
@@ -455,16 +461,30 @@ namespace {
 int evict_and_close(locret_layer *L, int n_tok, uint32_t flags, bool side, cudaStream_t S) {
   ScratchPool *P = L->pool;
   const int n = L->len + n_tok;
-  if (!(flags & LOCRET_NO_EVICT) && n > L->budget) {
+  const bool may_evict = !(flags & LOCRET_NO_EVICT);
+  bool evicts = may_evict && n > L->budget;
+  PerHead n_m{}, nprot_m{}, evict_m{};
+  if (L->per_head) {
+    evicts = false;
+    for (int m = 0; m < L->h_kv; m++) {
+      n_m.v[m] = L->len_m.v[m] + n_tok;
+      nprot_m.v[m] = (flags & LOCRET_LAST_CHUNK) ? 0 : (L->n_stab < n_m.v[m] ? L->n_stab : n_m.v[m]);
+      evict_m.v[m] = may_evict && n_m.v[m] > L->budget_m.v[m];
+      evicts = evicts || evict_m.v[m];
+    }
+  }
+  if (evicts) {
     const int n_prot = (flags & LOCRET_LAST_CHUNK) ? 0 : (L->n_stab < n ? L->n_stab : n);
-    int32_t *const rank_old = L->rank[L->rcur], *const rank_new = L->rank[L->rcur ^ 1];
     {
       Timed t(L, LOCRET_K_TOPK, S);
       // (n_prefix + n_stab <= budget < n, so the prefix never reaches into the protected tail)
       TopkArgs a;
-      a.scores = L->s; a.rank_old = rank_old; a.stride = L->cap; a.ranked_len = L->ranked_len;
+      a.scores = L->s; a.rank[0] = L->rank[0]; a.rank[1] = L->rank[1]; a.rcur = L->rcur;
+      a.stride = L->cap; a.ranked_len = L->ranked_len;
       a.n = n; a.budget = L->budget; a.n_prot = n_prot; a.n_pre = L->n_prefix;
-      a.src_of = P->keep; a.rank_new = rank_new; a.counters = L->d_counters;
+      a.src_of = P->keep; a.src_stride = L->budget; a.counters = L->d_counters;
+      a.per_head = L->per_head ? 1 : 0;
+      a.n_m = n_m; a.budget_m = L->budget_m; a.nprot_m = nprot_m; a.ranked_m = L->ranked_m; a.rcur_m = L->rcur_m;
       CK(launch_topk(a, L->h_kv, S));
     }
     // the gather rewrites keys and values that the attention kernel reads
@@ -476,10 +496,28 @@ int evict_and_close(locret_layer *L, int n_tok, uint32_t flags, bool side, cudaS
       Timed t(L, LOCRET_K_COMPACT, S);
       CompactArgs a;
       a.k = L->k_pre; a.v = L->v; a.k_rot = L->k_rot; a.s = L->s; a.t = L->tid;
-      a.src_of = P->keep; a.rank_new = rank_new; a.rank_old = rank_old; a.cs = L->cs;
+      a.src_of = P->keep; a.src_stride = L->budget; a.rank[0] = L->rank[0]; a.rank[1] = L->rank[1]; a.rcur = L->rcur;
+      a.cs = L->cs;
       a.h_kv = L->h_kv; a.d = L->d; a.cap = L->cap; a.budget = L->budget; a.ranked_len = L->ranked_len;
+      a.per_head = L->per_head ? 1 : 0;
+      a.budget_m = L->budget_m; a.ranked_m = L->ranked_m; a.rcur_m = L->rcur_m; a.evict_m = evict_m;
       CK(launch_compact(a, S));
     }
+  }
+  if (L->per_head) {
+    int mx = 0;
+    for (int m = 0; m < L->h_kv; m++) {
+      if (evict_m.v[m]) {
+        L->len_m.v[m] = L->budget_m.v[m];
+        L->ranked_m.v[m] = L->budget_m.v[m];
+        L->rcur_m.v[m] ^= 1;
+      } else {
+        L->len_m.v[m] = n_m.v[m];
+      }
+      mx = L->len_m.v[m] > mx ? L->len_m.v[m] : mx;
+    }
+    L->len = mx;
+  } else if (evicts) {
     L->rcur ^= 1;
     L->ranked_len = L->budget;
     L->len = L->budget;
@@ -507,9 +545,13 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
   if (!aligned16(hidden_in) || !aligned16(attn_out)) return LOCRET_ERR_INVALID;
   const int n = L->len + n_tok;
   if (n > L->cap) return LOCRET_ERR_CAPACITY;
+  const PerHead *const len_m = L->per_head ? &L->len_m : nullptr;
   ScratchPool *P = L->pool;
   const bool tp = tp_partial != nullptr || tp_peers;
-  const bool decode = n_tok == 1 && L->use_tc && !tp;  // one token: bandwidth-bound kernels of decode.cu
+  if (L->per_head && tp) return LOCRET_ERR_INVALID;  // (a budget per head and divided heads are not combined)
+  // one token: bandwidth-bound kernels of decode.cu (with a budget per head a one-token step takes the
+  // chunk's general kernels, which know the heads' own lengths)
+  const bool decode = n_tok == 1 && L->use_tc && !tp && !L->per_head;
   // (a one-token step is a chain of three short kernels on the layer's own stream, overlapped by
   // programmatic dependent launch: an event between them would serialise them again)
   const bool side = L->use_side && !L->serialize && !decode;
@@ -537,8 +579,10 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
   ra.k_pre = L->int4 ? nullptr : L->k_pre; ra.k_rot = k_att; ra.v = v_att; ra.tid = L->tid; ra.cs = L->cs;
   ra.n_tok = n_tok; ra.h = L->h; ra.h_kv = L->h_kv; ra.d = L->d; ra.cap = L->cap; ra.len = L->len;
   ra.seen = L->seen;
+  ra.per_head = L->per_head ? 1 : 0;
+  ra.len_m = L->len_m;
   // with a tensor-core projection whose width is a whole number of tiles the epilogue of the GEMM does the RoPE pass
-  const bool fused_rope = !decode && L->fuse_rope && L->use_tc && n_tok >= 32 &&
+  const bool fused_rope = !decode && !L->per_head && L->fuse_rope && L->use_tc && n_tok >= 32 &&
                           qkv_rope_tc_supported(n_tok, L->d_in, L->D, L->D, L->D, L->d);
   const bool deq = L->int4 && L->len > 0 && !decode;
   if (deq) {
@@ -607,10 +651,10 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
                                  L->int4 ? staging + (size_t)(L->h + L->h_kv) * L->d : nullptr, L->st, pdl));
     else if (tc_ok)
       CK(launch_attention_tc(&L->map_q, &L->map_k, &L->map_v, (bf16 *)attn_out, n_tok, L->h, L->h_kv,
-                             L->d, L->len, L->d_status, L->st));
+                             L->d, L->len, L->d_status, L->st, len_m));
     else
       CK(launch_attention_mma(P->q_rot, k_att, v_att, (bf16 *)attn_out, n_tok, L->h, L->h_kv,
-                              L->d, L->cap, L->len, L->st));
+                              L->d, L->cap, L->len, L->st, len_m));
   }
   if (side && L->int4) {  // the attention kernel just launched is the scratch's last reader (a one-token step reads its own token there)
     CK(cudaEventRecord(P->ev_exp_free, L->st));
@@ -676,7 +720,7 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
   }
   if (!decode) {  // (the one-token kernel sums its own partial scores)
     Timed t(L, LOCRET_K_RH_REDUCE, S);
-    CK(launch_rh_reduce(P->partial, n_tiles, n_tok, L->h_kv, L->s, L->cap, L->len, S));
+    CK(launch_rh_reduce(P->partial, n_tiles, n_tok, L->h_kv, L->s, L->cap, L->len, S, len_m));
   }
   if (side) {
     CK(cudaEventRecord(P->ev_stage_free[sb], S));
@@ -766,6 +810,7 @@ int locret_cache_len(const locret_layer *L, int32_t *len) {
 int locret_export_state(locret_layer *L, void *K, void *V, float *scores, int64_t *token_ids,
                         int32_t *len, int64_t *tokens_seen) {
   if (!L || !on_layer_device(L)) return LOCRET_ERR_INVALID;
+  if (L->per_head) return LOCRET_ERR_INVALID;           // use locret_export_state_heads
   if (L->int4 && (K || V)) return LOCRET_ERR_INVALID;  // use locret_export_state_int4
   CK(sync_all(L));
   const int n = L->len;
@@ -788,6 +833,7 @@ int locret_import_state(locret_layer *L, const void *K, const void *V, const flo
                         const int64_t *token_ids, int32_t len, int64_t tokens_seen) {
   if (!L || len < 0 || len > L->cap || tokens_seen < 0 || !on_layer_device(L)) return LOCRET_ERR_INVALID;
   if (L->int4) return LOCRET_ERR_INVALID;  // use locret_import_state_int4
+  if (L->per_head) return LOCRET_ERR_INVALID;  // use locret_import_state_heads
   if (len > 0 && (!K || !V || !scores || !token_ids)) return LOCRET_ERR_INVALID;
   CK(sync_all(L));
   if (len > 0) {
@@ -856,6 +902,96 @@ int locret_import_state_int4(locret_layer *L, const void *k_codes, const void *k
   return LOCRET_OK;
 }
 
+int locret_set_head_budgets(locret_layer *L, const int32_t *budgets) {
+  if (!L || !budgets || !on_layer_device(L)) return LOCRET_ERR_INVALID;
+  if (L->int4 || L->len != 0 || L->seen != 0 || L->tp_pending) return LOCRET_ERR_INVALID;
+  for (int m = 0; m < L->h_kv; m++)
+    if (budgets[m] < 1 || budgets[m] > L->budget || L->n_stab + L->n_prefix > budgets[m]) return LOCRET_ERR_INVALID;
+  L->per_head = true;
+  for (int m = 0; m < L->h_kv; m++) {
+    L->budget_m.v[m] = budgets[m]; L->len_m.v[m] = 0; L->ranked_m.v[m] = 0; L->rcur_m.v[m] = 0;
+  }
+  return LOCRET_OK;
+}
+
+int locret_cache_lens(const locret_layer *L, int32_t *lens) {
+  if (!L || !lens) return LOCRET_ERR_INVALID;
+  for (int m = 0; m < L->h_kv; m++) lens[m] = L->per_head ? L->len_m.v[m] : L->len;
+  return LOCRET_OK;
+}
+
+int locret_export_state_heads(locret_layer *L, void *K, void *V, float *scores, int64_t *token_ids, int32_t pitch,
+                              int32_t *lens, int64_t *tokens_seen) {
+  if (!L || !on_layer_device(L) || L->int4 || pitch < L->len) return LOCRET_ERR_INVALID;
+  CK(sync_all(L));
+  if (tokens_seen) *tokens_seen = L->seen;
+  std::vector<int32_t> rank;
+  std::vector<unsigned char> tmp;
+  for (int m = 0; m < L->h_kv; m++) {
+    const int n = L->per_head ? L->len_m.v[m] : L->len;
+    const int ranked = L->per_head ? L->ranked_m.v[m] : L->ranked_len;
+    const int rc = L->per_head ? L->rcur_m.v[m] : L->rcur;
+    if (lens) lens[m] = n;
+    if (n == 0) continue;
+    const int nr = ranked < n ? ranked : n;
+    rank.resize(nr);
+    if (nr) CK(cudaMemcpy(rank.data(), L->rank[rc] + (size_t)m * L->cap, (size_t)nr * 4, cudaMemcpyDeviceToHost));
+    auto copy = [&](const void *dev, size_t row_bytes, void *out) -> int {
+      if (!out) return LOCRET_OK;
+      tmp.resize((size_t)n * row_bytes);
+      CK(cudaMemcpy(tmp.data(), (const unsigned char *)dev + (size_t)m * L->cap * row_bytes, (size_t)n * row_bytes,
+                    cudaMemcpyDeviceToHost));
+      unsigned char *o = (unsigned char *)out + (size_t)m * pitch * row_bytes;
+      for (int i = 0; i < n; i++) {
+        const int r = i < nr ? rank[i] : i;
+        if (r < 0 || r >= n) return LOCRET_ERR_CUDA;
+        memcpy(o + (size_t)r * row_bytes, tmp.data() + (size_t)i * row_bytes, row_bytes);
+      }
+      return LOCRET_OK;
+    };
+    int e;
+    if ((e = copy(L->k_pre, (size_t)L->d * 2, K)) != LOCRET_OK) return e;
+    if ((e = copy(L->v, (size_t)L->d * 2, V)) != LOCRET_OK) return e;
+    if ((e = copy(L->s, 4, scores)) != LOCRET_OK) return e;
+    if ((e = copy(L->tid, 8, token_ids)) != LOCRET_OK) return e;
+  }
+  return LOCRET_OK;
+}
+
+int locret_import_state_heads(locret_layer *L, const void *K, const void *V, const float *scores,
+                              const int64_t *token_ids, int32_t pitch, const int32_t *lens, int64_t tokens_seen) {
+  if (!L || !on_layer_device(L) || L->int4 || !L->per_head || !lens || pitch < 0 || tokens_seen < 0)
+    return LOCRET_ERR_INVALID;
+  int mx = 0;
+  for (int m = 0; m < L->h_kv; m++) {
+    if (lens[m] < 0 || lens[m] > pitch || lens[m] > L->cap) return LOCRET_ERR_INVALID;
+    mx = lens[m] > mx ? lens[m] : mx;
+  }
+  if (mx > 0 && (!K || !V || !scores || !token_ids)) return LOCRET_ERR_INVALID;
+  CK(sync_all(L));
+  for (int m = 0; m < L->h_kv; m++) {
+    const int n = lens[m];
+    L->len_m.v[m] = n;
+    L->ranked_m.v[m] = 0;  // imported units are in temporal order
+    if (n == 0) continue;
+    const size_t row = (size_t)L->d * 2;
+    CK(cudaMemcpyAsync(L->k_pre + (size_t)m * L->cap * L->d, (const unsigned char *)K + (size_t)m * pitch * row,
+                       (size_t)n * row, cudaMemcpyHostToDevice, L->st));
+    CK(cudaMemcpyAsync(L->v + (size_t)m * L->cap * L->d, (const unsigned char *)V + (size_t)m * pitch * row,
+                       (size_t)n * row, cudaMemcpyHostToDevice, L->st));
+    CK(cudaMemcpyAsync(L->s + (size_t)m * L->cap, scores + (size_t)m * pitch, (size_t)n * 4, cudaMemcpyHostToDevice, L->st));
+    CK(cudaMemcpyAsync(L->tid + (size_t)m * L->cap, token_ids + (size_t)m * pitch, (size_t)n * 8,
+                       cudaMemcpyHostToDevice, L->st));
+    L->launches++;
+    CK(launch_rerope(L->k_pre + (size_t)m * L->cap * L->d, L->k_rot + (size_t)m * L->cap * L->d, L->cs, 1, L->d, L->cap,
+                     n, L->st));
+  }
+  CK(cudaStreamSynchronize(L->st));
+  L->len = mx;
+  L->seen = tokens_seen;
+  return LOCRET_OK;
+}
+
 int locret_compaction_counters(locret_layer *L, int64_t *units_moved, int64_t *keys_rotated) {
   if (!L || !on_layer_device(L)) return LOCRET_ERR_INVALID;
   unsigned long long host[2] = {0, 0};
@@ -886,6 +1022,7 @@ int locret_reset(locret_layer *L) {
   }
   L->len = 0;
   L->ranked_len = 0;
+  for (int m = 0; m < 32; m++) { L->len_m.v[m] = 0; L->ranked_m.v[m] = 0; }
   L->seen = 0;
   L->tp_pending = false;
   return LOCRET_OK;
@@ -893,6 +1030,9 @@ int locret_reset(locret_layer *L) {
 
 int locret_set_protected_prefix(locret_layer *L, int32_t n_prefix) {
   if (!L || n_prefix < 0 || n_prefix + L->n_stab > L->budget) return LOCRET_ERR_INVALID;
+  if (L->per_head)
+    for (int m = 0; m < L->h_kv; m++)
+      if (n_prefix + L->n_stab > L->budget_m.v[m]) return LOCRET_ERR_INVALID;
   L->n_prefix = n_prefix;
   return LOCRET_OK;
 }

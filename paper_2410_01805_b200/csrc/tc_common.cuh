@@ -260,6 +260,6 @@ bool tmap_encode_3d_bf16(CUtensorMap *map, const void *base, uint64_t d0, uint64
 bool attention_tc_supported(int n_tok, int h, int h_kv, int d);
 cudaError_t launch_attention_tc(const CUtensorMap *map_q, const CUtensorMap *map_k,
                                 const CUtensorMap *map_v, bf16 *out, int n_tok, int h, int h_kv, int d,
-                                int len, int *status, cudaStream_t st);
+                                int len, int *status, cudaStream_t st, const PerHead *len_m = nullptr);
 
 }  // namespace locret
