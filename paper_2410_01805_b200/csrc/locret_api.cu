@@ -30,6 +30,10 @@ struct ScratchPool {
   cudaEvent_t ev_stage_free[2] = {nullptr, nullptr};
   // 4-bit caches: the bf16 expansion is written on the second stream while the projection runs
   cudaEvent_t ev_exp_free = nullptr, ev_exp_ready = nullptr;
+  // work of ANY layer may be pending on the second stream: a step that uses the shared scratch of the
+  // off-critical-path kernels (partial scores, index lists) on the layer's own stream waits for it first
+  cudaEvent_t ev_side_idle = nullptr;
+  bool side_dirty = false;
   bool exp_busy = false;  // ev_exp_free recorded and not yet waited for
   bool stage_busy[2] = {false, false};  // recorded and not yet waited for
   int flip = 0;
@@ -146,6 +150,7 @@ void release_pool(ScratchPool *p) {
   }
   if (p->ev_exp_free) cudaEventDestroy(p->ev_exp_free);
   if (p->ev_exp_ready) cudaEventDestroy(p->ev_exp_ready);
+  if (p->ev_side_idle) cudaEventDestroy(p->ev_side_idle);
   cudaFree(p->q_rot); cudaFree(p->partial); cudaFree(p->keep); cudaFree(p->dec_o); cudaFree(p->dec_ml); cudaFree(p->dec_cnt);
   cudaFree(p->k_exp); cudaFree(p->v_exp);
   for (auto &t : p->cs) cudaFree(t.ptr);
@@ -362,7 +367,8 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
         for (int i = 0; i < 2 && g; i++)
           g = cudaEventCreateWithFlags(&p->ev_stage_free[i], cudaEventDisableTiming) == cudaSuccess;
         g = g && cudaEventCreateWithFlags(&p->ev_exp_free, cudaEventDisableTiming) == cudaSuccess &&
-            cudaEventCreateWithFlags(&p->ev_exp_ready, cudaEventDisableTiming) == cudaSuccess;
+            cudaEventCreateWithFlags(&p->ev_exp_ready, cudaEventDisableTiming) == cudaSuccess &&
+            cudaEventCreateWithFlags(&p->ev_side_idle, cudaEventDisableTiming) == cudaSuccess;
       }
       if (g && !p->dec_cnt) {
         g = cudaMalloc(&p->dec_cnt, DEC_CNT_WORDS * sizeof(unsigned)) == cudaSuccess &&
@@ -561,6 +567,14 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
   P->flip ^= 1;
   bf16 *const staging = P->staging[sb];
   bf16 *const z_post = P->z_post[sb];
+  if (L->use_side && !side && P->side_dirty) {
+    // this step runs the retaining head (and an eviction) on the layer's own stream, with the scratch
+    // other layers' steps may still be using on the second stream
+    CK(cudaEventRecord(P->ev_side_idle, P->side));
+    CK(cudaStreamWaitEvent(L->st, P->ev_side_idle, 0));
+    P->side_dirty = false;
+  }
+  if (side) P->side_dirty = true;
   if (L->use_side) {
     // the staging buffer is free once the retaining head that last read it has run, and this
     // layer's cache once its previous selection / compaction has finished
@@ -775,6 +789,7 @@ int locret_prefill_chunk_tp_finish(locret_layer *L, const float *preact_sum) {
   const bool side = L->use_side && !L->serialize;
   cudaStream_t S = side ? L->pool->side : L->st;
   if (side) {
+    L->pool->side_dirty = true;
     CK(cudaEventRecord(L->ev_tp, L->st));
     CK(cudaStreamWaitEvent(S, L->ev_tp, 0));
   }
