@@ -289,7 +289,7 @@ cudaError_t launch_rh_gemv(const bf16 *z, const bf16 *W1t, const float *W2, floa
                            int h_kv, int act, unsigned *counter, float *score_out, int score_stride,
                            cudaStream_t st, bool pdl = false);
 int rh_gemv_blocks(int d_R);
-int decode_attn_splits(int h_kv, int n);
+int decode_attn_splits(int h_kv, int n, bool int4);
 // part_o: fp32 [h][n_splits][d]; part_ml: fp32 [h][n_splits][2]; counters: one zeroed word per
 // (KV head, group of 16 query heads), left at zero (the last split merges the partial results).
 // q4 != nullptr: keys [0, n - 1) are read from the 4-bit cache (expanded and rotated with `cs` on the

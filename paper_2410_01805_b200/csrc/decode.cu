@@ -1,6 +1,8 @@
 // Decoding (the B = 1 case of Eq. 1): one token per step, so every kernel is bound by the bytes
 // it must read once: the weights for the two projections, the retained keys and values for
 // attention.  Plain CUDA cores, 16-byte loads, no tensor cores (there is no contraction to tile).
+#include <stdlib.h>
+
 #include "common.cuh"
 
 namespace locret {
@@ -716,8 +718,18 @@ cudaError_t launch_rh_gemv(const bf16 *z, const bf16 *W1t, const float *W2, floa
                        (const bf16 *)nullptr);
 }
 
-int decode_attn_splits(int h_kv, int n) {
-  int s = (148 * 2 + h_kv - 1) / h_kv;          // about two CTAs per SM in total
+// Splits of the key range per KV head.  Measured at the Llama shape (8 KV heads, 6000 keys, 256 steps through
+// 32 layers): with a bf16 cache 64 / 96 / 120 / 148 / 200 / 296 / 444 CTAs in total give 914 / 1058 / 1130 /
+// 1152 / 1224 / 1133 / 1052 tokens/s (more splits shorten each CTA's chain of tiles, but the last split of a
+// head merges them all); a 4-bit cache, whose CTAs also expand and rotate the codes (and load a tile's codes
+// without overlapping the previous tile's arithmetic), wants more: 96 / 148 / 296 / 444 CTAs give 501 / 639 /
+// 825 / 700 tokens/s.
+int decode_attn_splits(int h_kv, int n, bool int4) {
+  static int forced = -1;
+  if (forced < 0) { const char *e = getenv("LOCRET_DEC_CTAS"); forced = e ? atoi(e) : 0; if (forced < 0 || forced > 2048) forced = 0; }
+  const int sms = sm_count_of_current_device();
+  const int total = forced ? forced : (int4 ? 2 * sms : (sms * 27) / 20);
+  int s = (total + h_kv - 1) / h_kv;
   const int max_s = (n + 127) / 128;            // at least one 128-key tile per split
   if (s > max_s) s = max_s;
   if (s > 64) s = 64;

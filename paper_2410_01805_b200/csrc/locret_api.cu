@@ -659,7 +659,7 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
     }
     if (decode)
       CK(launch_attention_decode(P->q_rot, k_att, v_att, (bf16 *)attn_out, P->dec_o, P->dec_ml, P->dec_cnt + 1,
-                                 L->h, L->h_kv, L->d, L->cap, n, decode_attn_splits(L->h_kv, n),
+                                 L->h, L->h_kv, L->d, L->cap, n, decode_attn_splits(L->h_kv, n, L->int4),
                                  L->int4 ? &L->q4 : nullptr, L->cs, L->rank[L->rcur], L->ranked_len,
                                  L->int4 ? staging + (size_t)L->h * L->d : nullptr,
                                  L->int4 ? staging + (size_t)(L->h + L->h_kv) * L->d : nullptr, L->st, pdl));
