@@ -58,9 +58,34 @@ def test_training_argument_checks():
         rh_loss_grad(z, lab, w1, w2)
 
 
+def test_adamw_step_matches_the_oracle_on_seeded_inputs():
+    """The optimiser kernel alone: parameters, gradients and moments come from the seeded generator
+    (nothing the CUDA path computed goes into the oracle)."""
+    from paper_2410_01805_b200 import adamw_step
+    g = np.random.default_rng(8000)
+    n = 100_003
+    p = g.standard_normal(n).astype(np.float32)
+    gr = (g.standard_normal(n) * 0.1).astype(np.float32)
+    m = (g.standard_normal(n) * 0.01).astype(np.float32)
+    v = (g.random(n) * 1e-3).astype(np.float32)
+    for step, lr in ((1, 5e-4), (7, 2e-2)):
+        rp, rm, rv = O.adamw_step(p, gr, m, v, step, lr)
+        P, G, M, V = (torch.from_numpy(a.copy()).cuda() for a in (p, gr, m, v))
+        B = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+        adamw_step(P, G, M, V, step, lr, param_bf16=B)
+        torch.cuda.synchronize()
+        assert np.abs(P.cpu().numpy() - rp).max() <= 1e-6 * max(1.0, np.abs(rp).max())
+        assert np.abs(M.cpu().numpy() - rm).max() <= 1e-7 and np.abs(V.cpu().numpy() - rv).max() <= 1e-8
+        assert torch.equal(B, P.to(torch.bfloat16))
+
+
 def test_a_few_training_steps_follow_the_oracle_and_reduce_the_loss():
-    """Labels from the definition, loss and gradients, AdamW: three updates in lock-step with the
-    oracle's fp64 trajectory (the GPU's bf16 weights are fed to both sides at every step)."""
+    """Labels from the definition, loss and gradients, AdamW: three updates, each side on its OWN
+    trajectory (the oracle's fp64 master weights and moments are updated with the oracle's own
+    gradients; nothing the CUDA path computed is fed to it).  Both compute the forward pass from the
+    bf16 rounding of their master weights.  The first Adam updates have magnitude lr whatever the
+    gradient's size, so an element whose gradient is smaller than the gradient error may move the other
+    way on the two sides: parameters are compared where the oracle's gradient is well above that error."""
     from parity_util import bf16_dev
     from paper_2410_01805_b200 import adamw_step, cis_labels, rh_loss_grad
     g = np.random.default_rng(8100)
@@ -81,22 +106,28 @@ def test_a_few_training_steps_follow_the_oracle_and_reduce_the_loss():
     o1, o2 = w1.astype(np.float64), w2.astype(np.float64)
     om1, ov1, om2, ov2 = (np.zeros_like(a) for a in (o1, o1, o2, o2))
     zd = bf16_dev(z)
-    losses = []
+    losses, ref_losses = [], []
     lr = 2e-2
+    sure1 = np.ones_like(o1, dtype=bool)
+    sure2 = np.ones_like(o2, dtype=bool)
     for step in range(1, 4):
         loss, g1, g2 = rh_loss_grad(zd, labels, B1, B2, 2.5e-3)
-        # the oracle starts every step from the bf16 weights the GPU used
-        b1, b2 = B1.float().cpu().numpy().astype(np.float64), B2.float().cpu().numpy().astype(np.float64)
-        rl, r1, r2 = O.rh_loss_and_grads(z, ref_labels, b1, b2, 2.5e-3)
-        assert abs(float(loss.item()) - rl) <= 1e-3 * abs(rl)
-        assert np.abs(g2.cpu().numpy() - r2).max() <= 1e-3 * np.abs(r2).max()
-        assert np.abs(g1.cpu().numpy() - r1).max() <= 2e-2 * np.sqrt(np.mean(r1 ** 2))
-        losses.append(float(loss.item()))
-        o1, om1, ov1 = O.adamw_step(P1.cpu().numpy(), g1.cpu().numpy(), M1.cpu().numpy(), V1.cpu().numpy(), step, lr)
-        o2, om2, ov2 = O.adamw_step(P2.cpu().numpy(), g2.cpu().numpy(), M2.cpu().numpy(), V2.cpu().numpy(), step, lr)
+        rl, r1, r2 = O.rh_loss_and_grads(z, ref_labels, O.round_bf16(o1), O.round_bf16(o2), 2.5e-3)
+        losses.append(float(loss.item())); ref_losses.append(rl)
+        tol = 1e-3 if step == 1 else 5e-2          # later steps: the trajectories have parted on the unsure elements
+        assert abs(losses[-1] - rl) <= tol * abs(rl), (step, losses[-1], rl)
+        if step == 1:
+            assert np.abs(g2.cpu().numpy() - r2).max() <= 1e-3 * np.abs(r2).max()
+            assert np.abs(g1.cpu().numpy() - r1).max() <= 2e-2 * np.sqrt(np.mean(r1 ** 2))
+        sure1 &= np.abs(r1) > 0.2 * np.sqrt(np.mean(r1 ** 2))
+        sure2 &= np.abs(r2) > 0.2 * np.sqrt(np.mean(r2 ** 2))
+        o1, om1, ov1 = O.adamw_step(o1, r1, om1, ov1, step, lr)
+        o2, om2, ov2 = O.adamw_step(o2, r2, om2, ov2, step, lr)
         adamw_step(P1, g1, M1, V1, step, lr, param_bf16=B1)
         adamw_step(P2, g2, M2, V2, step, lr, param_bf16=B2)
         torch.cuda.synchronize()
-        assert np.abs(P1.cpu().numpy() - o1).max() <= 1e-5 and np.abs(P2.cpu().numpy() - o2).max() <= 1e-5
         assert torch.equal(B1, P1.to(torch.bfloat16))
-    assert losses[2] < losses[0]
+    assert sure1.mean() > 0.2 and sure2.mean() > 0.2      # (a third of the elements stay clear of zero gradient in all three steps)
+    assert np.abs(P1.cpu().numpy() - o1)[sure1].max() <= 0.25 * lr
+    assert np.abs(P2.cpu().numpy() - o2)[sure2].max() <= 0.25 * lr
+    assert losses[2] < losses[0] and ref_losses[2] < ref_losses[0]
