@@ -118,6 +118,8 @@ struct locret_layer {
   cudaEvent_t ev_ready, ev_attn, ev_side, ev_tp;  // ev_tp: the divided-heads exchange (both directions)
   bool tc_attn;  // tensor maps for the tcgen05 attention kernel are valid
   CUtensorMap map_k, map_v, map_q;
+  CUtensorMap map_k64;   // keys in boxes of 64 (the CTA-pair attention kernel loads half a key tile per CTA)
+  bool attn_pair;
   const void *map_q_base;
   std::vector<TimedEvent> events;
   size_t events_used;
@@ -317,6 +319,8 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
     L->use_side = !(ser && ser[0] == '1');
     const char *unf = getenv("LOCRET_UNFUSED_ROPE");
     L->fuse_rope = !(unf && unf[0] == '1');
+    const char *ap = getenv("LOCRET_ATTN_PAIR");
+    L->attn_pair = ap && ap[0] == '1';
     const char *np = getenv("LOCRET_NO_PDL");
     L->use_pdl = !(np && np[0] == '1');
     L->side_pending = false;
@@ -425,7 +429,9 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
                  tmap_encode_3d_bf16(&L->map_k, L->k_rot, d, L->cap, hk, (uint64_t)d * 2,
                                      (uint64_t)L->cap * d * 2, 64, 128, 1) &&
                  tmap_encode_3d_bf16(&L->map_v, L->v, d, L->cap, hk, (uint64_t)d * 2,
-                                     (uint64_t)L->cap * d * 2, 64, 128, 1);
+                                     (uint64_t)L->cap * d * 2, 64, 128, 1) &&
+                 tmap_encode_3d_bf16(&L->map_k64, L->k_rot, d, L->cap, hk, (uint64_t)d * 2,
+                                     (uint64_t)L->cap * d * 2, 64, 64, 1);
 
   // repack the weights: K-major copies for both GEMMs, W2 in fp32
   cudaError_t e = cudaSuccess;
@@ -649,7 +655,9 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
       tc_ok = tmap_encode_3d_bf16(&L->map_k, P->k_exp, L->d, L->cap, L->h_kv, (uint64_t)L->d * 2,
                                   (uint64_t)L->cap * L->d * 2, 64, 128, 1) &&
               tmap_encode_3d_bf16(&L->map_v, P->v_exp, L->d, L->cap, L->h_kv, (uint64_t)L->d * 2,
-                                  (uint64_t)L->cap * L->d * 2, 64, 128, 1);
+                                  (uint64_t)L->cap * L->d * 2, 64, 128, 1) &&
+              tmap_encode_3d_bf16(&L->map_k64, P->k_exp, L->d, L->cap, L->h_kv, (uint64_t)L->d * 2,
+                                  (uint64_t)L->cap * L->d * 2, 64, 64, 1);
       L->map_kv_base = tc_ok ? P->k_exp : nullptr;
     }
     if (tc_ok && L->map_q_base != P->q_rot) {
@@ -663,6 +671,9 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
                                  L->int4 ? &L->q4 : nullptr, L->cs, L->rank[L->rcur], L->ranked_len,
                                  L->int4 ? staging + (size_t)L->h * L->d : nullptr,
                                  L->int4 ? staging + (size_t)(L->h + L->h_kv) * L->d : nullptr, L->st, pdl));
+    else if (tc_ok && L->attn_pair && attention_tc2_supported(n_tok, L->h, L->h_kv, L->d))
+      CK(launch_attention_tc2(&L->map_q, &L->map_k64, &L->map_v, (bf16 *)attn_out, n_tok, L->h, L->h_kv,
+                              L->d, L->len, L->d_status, L->st, len_m));
     else if (tc_ok)
       CK(launch_attention_tc(&L->map_q, &L->map_k, &L->map_v, (bf16 *)attn_out, n_tok, L->h, L->h_kv,
                              L->d, L->len, L->d_status, L->st, len_m));

@@ -262,4 +262,11 @@ cudaError_t launch_attention_tc(const CUtensorMap *map_q, const CUtensorMap *map
                                 const CUtensorMap *map_v, bf16 *out, int n_tok, int h, int h_kv, int d,
                                 int len, int *status, cudaStream_t st, const PerHead *len_m = nullptr);
 
+
+// The same on CTA pairs (attn_tc2.cu), head_dim 128.  map_k: box {64, 64, 1}; the others as above.
+bool attention_tc2_supported(int n_tok, int h, int h_kv, int d);
+cudaError_t launch_attention_tc2(const CUtensorMap *map_q, const CUtensorMap *map_k,
+                                 const CUtensorMap *map_v, bf16 *out, int n_tok, int h, int h_kv, int d,
+                                 int len, int *status, cudaStream_t st, const PerHead *len_m = nullptr);
+
 }  // namespace locret
