@@ -319,8 +319,8 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
     L->use_side = !(ser && ser[0] == '1');
     const char *unf = getenv("LOCRET_UNFUSED_ROPE");
     L->fuse_rope = !(unf && unf[0] == '1');
-    const char *ap = getenv("LOCRET_ATTN_PAIR");
-    L->attn_pair = ap && ap[0] == '1';
+    const char *ap = getenv("LOCRET_ATTN_PAIR");   // "0": the one-CTA kernel also for head_dim 128
+    L->attn_pair = !(ap && ap[0] == '0');
     const char *np = getenv("LOCRET_NO_PDL");
     L->use_pdl = !(np && np[0] == '1');
     L->side_pending = false;
