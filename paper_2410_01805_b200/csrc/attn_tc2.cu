@@ -295,11 +295,16 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
         // Drain: the completions of the last uses of every stage are multicast to both CTAs and nobody
         // else waits for them; the CTA must not end (and its shared memory pass to another kernel's
-        // CTA) while such an arrival is still on its way.
+        // CTA) while such an arrival is still on its way.  This thread has nothing else left to do.
+#ifndef A2_NO_DRAIN
         for (int j = max(NK - NSTK, 0); j < NK && ok; j++)
           ok = mbar_wait(&k_empty[j % NSTK], (j / NSTK) & 1, abort_flag, p.status);
         for (int j = max(NK - NSTV, 0); j < NK && ok; j++)
           ok = mbar_wait(&v_empty[j % NSTV], (j / NSTV) & 1, abort_flag, p.status);
+        for (int j = max(NK - NBUF, 0); j < NK && ok; j++)
+          ok = mbar_wait(&pv_done[j % NBUF], (j / NBUF) & 1, abort_flag, p.status);
+        if (ok && NK > 0) ok = mbar_wait(o_final, 0, abort_flag, p.status);
+#endif
       }
     } else if (warp == 9 && cta == 0) {
       // ------------------------------------------------------------ issuer of O += P_j V_j (pair)
@@ -501,9 +506,6 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         if (m_fin != m_mine) { l = (l == 0.f) ? 0.f : l * exp2f(m_mine - m_fin); m_mine = m_fin; }
       }
       if (ok) ok = mbar_wait(o_final, 0, abort_flag, p.status);
-      // (same drain for the per-buffer completions: every phase of pv_done has landed in this CTA)
-      for (int j = max(NK - NBUF, 0); j < NK && ok; j++)
-        ok = mbar_wait(&pv_done[j % NBUF], (j / NBUF) & 1, abort_flag, p.status);
     }
     tc_fence_after();
     xch[G * TILE + r] = l;
