@@ -35,9 +35,9 @@ UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "c3_llama_128k"
 # dram__bytes_read.sum + dram__bytes_write.sum of one steady-state attention launch: a literal taken
 # from a profiler capture of the same launch shape (not measured during this run)
-NCU_ATTN_TRAFFIC_BYTES = {"c3_llama_128k": 67.5e6, "c2_llama_32k": 67.5e6}
+NCU_ATTN_TRAFFIC_BYTES = {"c3_llama_128k": 70.9e6, "c2_llama_32k": 70.9e6}
 # sm__pipe_tensor_cycles_active of the same capture (per cent of cycles; clock-independent)
-NCU_ATTN_TENSOR_PIPE_PCT = 54.7
+NCU_ATTN_TENSOR_PIPE_PCT = 60.9
 # the other benchmark configurations are sampled in the default run: this many layers, contexts cut to this
 OTHER_CONFIGS = ("c2_llama_32k", "c4_phi3_128k", "c5_llama_stream_int4")
 OTHER_LAYERS = 4

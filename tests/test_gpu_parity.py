@@ -381,3 +381,17 @@ def test_attention_rescales_the_accumulator_when_a_later_key_tile_dominates(d):
         top2 = np.sort(tile_max, axis=1)[:, -2:]
         forced += int(np.sum(top2[:, 1] - top2[:, 0] > 101.0))
     assert forced >= 50, forced
+
+
+def test_one_cta_attention_kernel_is_still_selectable_for_head_dim_128(monkeypatch):
+    """head_dim 128 runs the CTA-pair kernel by default; LOCRET_ATTN_PAIR=0 (read when a layer is
+    created) selects the one-CTA kernel, which must pass the same lock-step comparison."""
+    from parity_util import lockstep_chunk, make_pair
+    sh = small_shape(h=8, hk=2, d=128, D=256, dR=64)
+    for env in ("0", "1"):
+        monkeypatch.setenv("LOCRET_ATTN_PAIR", env)
+        ora, gpu = make_pair(sh, weights_for(sh, 44), budget=700, chunk=384, n_stab=16)
+        for i, n_tok in enumerate([384, 200, 384, 129]):
+            lockstep_chunk(ora, gpu, hidden(n_tok, sh.d_model, 90 + i), 0, what=f"LOCRET_ATTN_PAIR={env} chunk {i}")
+        assert gpu.sync_status() == 0
+        gpu.destroy()
