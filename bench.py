@@ -493,6 +493,8 @@ def run_ours(args, w):
         dms = a.elapsed_time(b) / args.decode_steps
         ln = min(w.budget, w.context)
         kv_bytes = 2 * s.n_kv_heads * ln * s.head_dim * 2          # rotated K + V read by attention
+        if s.kv_dtype == 1:   # 4-bit cache: codes of K and V, two fp16 scales and the rank per unit
+            kv_bytes = s.n_kv_heads * ln * (s.head_dim + 4 + 4)
         w_bytes = 2 * (s.d_model * s.d_in + s.d_in * s.d_retain)
         step_bytes = w.n_layers * (kv_bytes + w_bytes)
         decode = {"tokens_per_s": 1e3 / dms, "ms_per_token": dms, "steps": args.decode_steps,

@@ -362,23 +362,60 @@ attn_decode_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_ro
       cp_async16(sV + (buf * DA_KT + r) * LD + c, vbase + off, ok);
     }
   };
-  // 4-bit cache: one thread expands elements [c, c+8) and [c+half, c+half+8) of K and V of one key
-  auto load_kv_q4 = [&](int buf, int kt) {
+  // 4-bit cache: one thread expands elements [c, c+8) and [c+half, c+half+8) of K and V of one key.
+  // In two steps, so that a tile's codes, scales and ranks are already on their way while the
+  // previous tile is multiplied: fetch_q4 requests them into registers (one tile ahead), expand_q4
+  // reads the (cos, sin) rows of the units' positions, expands, rotates and fills the shared tile.
+  constexpr int Q4_ITER = DA_KT * (D / 16) / DA_THREADS;
+  static_assert(Q4_ITER * DA_THREADS == DA_KT * (D / 16), "whole iterations");
+  struct Q4Pre { uint32_t kw0, kw1, vw0, vw1; float ks, vs; int pos; };  // pos < 0: not a unit of the 4-bit cache
+  Q4Pre pre[INT4 ? Q4_ITER : 1];
+  auto fetch_q4 = [&](int kt) {
     constexpr int HALF = D / 2, HV = D / 16;
-    for (int x = tid; x < DA_KT * HV; x += DA_THREADS) {
+#pragma unroll
+    for (int i = 0; i < Q4_ITER; i++) {
+      const int x = tid + i * DA_THREADS;
+      const int r = x / HV, c = (x - r * HV) * 8;
+      const int key = k0 + kt * DA_KT + r;
+      pre[i].pos = -1;
+      if (key < n - 1) {
+        const size_t u = (size_t)m * cap + key;
+        const uint8_t *kc = q4.kq + u * HALF, *vc = q4.vq + u * HALF;
+        pre[i].kw0 = *reinterpret_cast<const uint32_t *>(kc + c / 2);
+        pre[i].kw1 = *reinterpret_cast<const uint32_t *>(kc + (c + HALF) / 2);
+        pre[i].vw0 = *reinterpret_cast<const uint32_t *>(vc + c / 2);
+        pre[i].vw1 = *reinterpret_cast<const uint32_t *>(vc + (c + HALF) / 2);
+        pre[i].ks = __half2float(q4.ks[u]);
+        pre[i].vs = __half2float(q4.vs[u]);
+        pre[i].pos = key < ranked_len ? rank[u] : key;  // the unit's place in temporal order
+      }
+    }
+  };
+  auto expand_q4 = [&](int buf, int kt) {
+    constexpr int HALF = D / 2, HV = D / 16;
+    float4 t4[Q4_ITER][4];   // 8 (cos, sin) pairs per item, all requested before any is used
+#pragma unroll
+    for (int i = 0; i < Q4_ITER; i++) {
+      const int x = tid + i * DA_THREADS;
+      const int c = (x - (x / HV) * HV) * 8;
+      if (pre[i].pos >= 0) {
+        const float4 *t = reinterpret_cast<const float4 *>(cs + (size_t)pre[i].pos * HALF + c);
+#pragma unroll
+        for (int e = 0; e < 4; e++) t4[i][e] = __ldg(t + e);
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < Q4_ITER; i++) {
+      const int x = tid + i * DA_THREADS;
       const int r = x / HV, c = (x - r * HV) * 8;
       const int key = k0 + kt * DA_KT + r;
       bf16 *kd = sK + (buf * DA_KT + r) * LD, *vd = sV + (buf * DA_KT + r) * LD;
       uint4 ka = make_uint4(0, 0, 0, 0), kb = ka, va = ka, vb = ka;
-      if (key < n - 1) {
-        const size_t u = (size_t)m * cap + key;
-        const uint8_t *kc = q4.kq + u * HALF, *vc = q4.vq + u * HALF;
-        const float ks = __half2float(q4.ks[u]), vs = __half2float(q4.vs[u]);
+      if (pre[i].pos >= 0) {
         float a[8], b[8];
-        dequant8(*reinterpret_cast<const uint32_t *>(kc + c / 2), ks, a);
-        dequant8(*reinterpret_cast<const uint32_t *>(kc + (c + HALF) / 2), ks, b);
-        const int pos = key < ranked_len ? rank[u] : key;  // the unit's place in temporal order
-        const float2 *t = cs + (size_t)pos * HALF + c;
+        dequant8(pre[i].kw0, pre[i].ks, a);
+        dequant8(pre[i].kw1, pre[i].ks, b);
+        const float2 *t = reinterpret_cast<const float2 *>(&t4[i][0]);
 #pragma unroll
         for (int e = 0; e < 8; e++) {
           const float x1 = a[e], x2 = b[e];
@@ -386,10 +423,10 @@ attn_decode_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_ro
           b[e] = x2 * t[e].x + x1 * t[e].y;
         }
         ka = to_bf16x8(a); kb = to_bf16x8(b);
-        dequant8(*reinterpret_cast<const uint32_t *>(vc + c / 2), vs, a);
-        dequant8(*reinterpret_cast<const uint32_t *>(vc + (c + HALF) / 2), vs, b);
+        dequant8(pre[i].vw0, pre[i].vs, a);
+        dequant8(pre[i].vw1, pre[i].vs, b);
         va = to_bf16x8(a); vb = to_bf16x8(b);
-      } else if (key < k1) {  // the token of this step
+      } else if (key >= n - 1 && key < k1) {  // the token of this step
         const size_t off = ((size_t)m * cap + key) * D + c;
         ka = *reinterpret_cast<const uint4 *>(k_rot + off); kb = *reinterpret_cast<const uint4 *>(k_rot + off + HALF);
         va = *reinterpret_cast<const uint4 *>(v + off); vb = *reinterpret_cast<const uint4 *>(v + off + HALF);
@@ -402,6 +439,7 @@ attn_decode_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_ro
   // the token of this step is requested before the wait for this step's projection.
   const bool early = !INT4 && NKT > 0 && k0 + DA_KT <= n - 1;
   if (early) load_kv(0, 0);
+  if (INT4 && NKT > 0) fetch_q4(0);   // (the token of this step is not among them: it is read in bf16, after the wait)
   pdl_wait();
   pdl_launch_dependents();  // the retaining head reads only what the projection wrote: it may run beside this kernel
   if (INT4 && tok_k && split == 0 && hg == 0 && warp < 2) {
@@ -454,7 +492,8 @@ attn_decode_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_ro
 
   for (int kt = 0; kt < NKT; kt++) {
     if (INT4) {
-      load_kv_q4(kt & 1, kt);  // (the other buffer may still be read by a slower warp)
+      expand_q4(kt & 1, kt);   // (the other buffer may still be read by a slower warp)
+      if (kt + 1 < NKT) fetch_q4(kt + 1);
       cp_async_wait<0>();
     } else {
       if (kt + 1 < NKT) load_kv((kt + 1) & 1, kt + 1);
