@@ -578,7 +578,9 @@ attn_decode_kernel(const bf16 *__restrict__ q_rot, const bf16 *__restrict__ k_ro
       mma_bf16_16816(o[2 * dn], pf, b0, b1);
       mma_bf16_16816(o[2 * dn + 1], pf, b2, b3);
     }
-    __syncthreads();
+    // bf16 cache: the next iteration's cp.async refills the buffer read here.  4-bit cache: the next
+    // expansion fills the other buffer, and the one after it comes behind the next iteration's barrier.
+    if (!INT4) __syncthreads();
   }
   cp_async_wait<0>();
 
