@@ -36,6 +36,12 @@
  *     (locret_destroy, locret_cache_len and the other host-only calls work from any device).
  *   - There is no CPU fallback: without a CUDA device every call that needs one
  *     returns LOCRET_ERR_CUDA.
+ *   - Kernel selection, read from the environment when a layer is created (for A/B measurements;
+ *     results agree within the stated tolerances): LOCRET_ATTN_PAIR=0 runs Eq. 1 for head_dim 128
+ *     on one CTA per pair of query tiles instead of a cluster of two (tcgen05 cta_group::2);
+ *     LOCRET_LEGACY_MMA=1 keeps every product on mma.sync kernels; LOCRET_UNFUSED_ROPE=1 runs
+ *     positions, RoPE and the cache append as a pass of their own; LOCRET_NO_PDL=1 launches the
+ *     one-token kernels without programmatic dependent launch.
  */
 #ifndef LOCRET_H_
 #define LOCRET_H_
