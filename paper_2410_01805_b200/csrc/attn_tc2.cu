@@ -47,7 +47,7 @@ constexpr int V_STAGE = TILE * 128;     // 128 keys x this CTA's 64 columns
 constexpr int A2_BAR_BYTES = 512;
 constexpr int A2_SMEM = 1024 + Q_BYTES + NSTK * K_STAGE + NSTV * V_STAGE + A2_BAR_BYTES + 2 * TILE * 4 + 2 * TILE * 4;
 constexpr float RESCALE_LOG2 = 100.0f;  // see attn_tc.cu: P and O stay finite, precision is scale free
-constexpr int PF = 6;
+constexpr int PF = 3;       // key tiles prefetched into L2 ahead of the shared-memory stages (0 / 3 / 6 / 10 measured: 3 is best by about 1 % of the step)
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
