@@ -37,11 +37,13 @@
  *   - There is no CPU fallback: without a CUDA device every call that needs one
  *     returns LOCRET_ERR_CUDA.
  *   - Kernel selection, read from the environment when a layer is created (for A/B measurements;
- *     results agree within the stated tolerances): LOCRET_ATTN_PAIR=0 runs Eq. 1 for head_dim 128
- *     on one CTA per pair of query tiles instead of a cluster of two (tcgen05 cta_group::2);
+ *     results agree within the stated tolerances): LOCRET_ATTN_PAIR=1 runs Eq. 1 for head_dim 128
+ *     on a cluster of two CTAs per pair of query tiles (tcgen05 cta_group::2) instead of one CTA;
+ *     it is faster and opt-in (bench.py sets it), and a divided-heads step never uses it.
  *     LOCRET_LEGACY_MMA=1 keeps every product on mma.sync kernels; LOCRET_UNFUSED_ROPE=1 runs
  *     positions, RoPE and the cache append as a pass of their own; LOCRET_NO_PDL=1 launches the
- *     one-token kernels without programmatic dependent launch.
+ *     one-token kernels without programmatic dependent launch; LOCRET_DIAG_STATUS=1 makes
+ *     locret_sync_status print which kernel family recorded a device-side time-out.
  */
 #ifndef LOCRET_H_
 #define LOCRET_H_

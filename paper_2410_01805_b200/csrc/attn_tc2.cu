@@ -542,6 +542,10 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     __syncwarp();
     tmem2_dealloc(tmem_base, 512);
   }
+  // Neither CTA leaves before BOTH have released the pair's tensor memory: if one SM were handed to
+  // another kernel's CTA while the partner's release (a cta_group::2 operation) is still to come,
+  // that release could reach the newcomer's allocation.
+  cluster_sync_all();
 #ifdef A2_TRACE
   if (blockIdx.x == 0 && threadIdx.x == 0 && NK > 60) {
     const long long t0 = a2_trace[0][32][0];

@@ -319,8 +319,9 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
     L->use_side = !(ser && ser[0] == '1');
     const char *unf = getenv("LOCRET_UNFUSED_ROPE");
     L->fuse_rope = !(unf && unf[0] == '1');
-    const char *ap = getenv("LOCRET_ATTN_PAIR");   // "0": the one-CTA kernel also for head_dim 128
-    L->attn_pair = !(ap && ap[0] == '0');
+    // "1": Eq. 1 for head_dim 128 on clusters of two CTAs (faster; opt-in, see the comment at its launch)
+    const char *ap = getenv("LOCRET_ATTN_PAIR");
+    L->attn_pair = ap && ap[0] == '1';
     const char *np = getenv("LOCRET_NO_PDL");
     L->use_pdl = !(np && np[0] == '1');
     L->side_pending = false;
@@ -352,7 +353,7 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   ok = ok && cudaMalloc(&L->tid, td_b) == cudaSuccess;
   for (int i = 0; i < 2; i++) ok = ok && cudaMalloc(&L->rank[i], rk_b) == cudaSuccess;
   ok = ok && cudaMalloc(&L->d_counters, 2 * sizeof(unsigned long long)) == cudaSuccess;
-  ok = ok && cudaMalloc(&L->d_status, sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMalloc(&L->d_status, 4 * sizeof(int)) == cudaSuccess;
   if (!ok) { cudaGetLastError(); free_layer_memory(L); delete L; return LOCRET_ERR_ALLOC; }
 
   // shared scratch
@@ -454,7 +455,7 @@ int locret_create(const locret_layer_cfg *cfg, int32_t budget, int32_t chunk, in
   if (e == cudaSuccess) e = cudaMemsetAsync(L->tid, 0, td_b, L->st);
   for (int i = 0; i < 2 && e == cudaSuccess; i++) e = cudaMemsetAsync(L->rank[i], 0, rk_b, L->st);
   if (e == cudaSuccess) e = cudaMemsetAsync(L->d_counters, 0, 2 * sizeof(unsigned long long), L->st);
-  if (e == cudaSuccess) e = cudaMemsetAsync(L->d_status, 0, sizeof(int), L->st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(L->d_status, 0, 4 * sizeof(int), L->st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(L->st);
   if (e != cudaSuccess) {
     cudaGetLastError();
@@ -624,10 +625,10 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
       CK(launch_gemv_rope((const bf16 *)hidden_in, L->wqkv_t, L->D, staging, ra, L->st, pdl));
     else if (fused_rope)
       CK(launch_qkv_rope_tc((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, staging, n_tok, L->d_in, L->D,
-                            ra, L->d_status, L->st));
+                            ra, L->d_status + 1, L->st));
     else if (L->use_tc && n_tok >= 32 && gemm_tc_supported(n_tok, L->d_in, L->D, L->D, L->D))
       CK(launch_gemm_tc((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, staging, L->d_in, n_tok,
-                        L->d_in, L->D, L->d_status, L->st));
+                        L->d_in, L->D, L->d_status + 1, L->st));
     else
       CK(launch_gemm_bf16((const bf16 *)hidden_in, L->D, L->wqkv_t, L->D, staging, L->d_in, n_tok,
                           L->d_in, L->D, L->st));
@@ -671,7 +672,12 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
                                  L->int4 ? &L->q4 : nullptr, L->cs, L->rank[L->rcur], L->ranked_len,
                                  L->int4 ? staging + (size_t)L->h * L->d : nullptr,
                                  L->int4 ? staging + (size_t)(L->h + L->h_kv) * L->d : nullptr, L->st, pdl));
-    else if (tc_ok && L->attn_pair && attention_tc2_supported(n_tok, L->h, L->h_kv, L->d))
+    // The CTA-pair kernel is opt-in (LOCRET_ATTN_PAIR=1) and never used in a divided-heads step.  In a test
+    // process in which it had run, the projection GEMM of a later divided-heads step (eight shards of the
+    // Llama shape on one GPU) reported a device-side time-out in about one full test run in three, also when
+    // that step itself used the one-CTA kernel; no run without the pair kernel ever did.  The cause has not
+    // been found, so the default is the kernel every earlier run validated.
+    else if (tc_ok && L->attn_pair && !tp && attention_tc2_supported(n_tok, L->h, L->h_kv, L->d))
       CK(launch_attention_tc2(&L->map_q, &L->map_k64, &L->map_v, (bf16 *)attn_out, n_tok, L->h, L->h_kv,
                               L->d, L->len, L->d_status, L->st, len_m));
     else if (tc_ok)
@@ -701,14 +707,14 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
       if (tp_peers && tc) {
         // the exchange inside the GEMM: the epilogue adds each tile into every GPU's sum buffer
         CK(launch_gemm_tc_f32_add_peers(z, L->d_in, L->w1_t, L->d_in, L->d_peers, L->n_peers, L->d_R, n_tok, L->d_R,
-                                        L->d_in, L->d_status, S));
+                                        L->d_in, L->d_status + 2, S));
       } else if (tp_peers) {
         CK(launch_preact_naive(z, L->w1_t, L->tp_scratch, n_tok, L->d_R, L->d_in, S));
         L->launches++;
         CK(launch_add_to_peers(L->tp_scratch, L->d_peers, L->n_peers, (size_t)n_tok * L->d_R, S));
       } else if (tc) {
         CK(launch_gemm_tc_f32(z, L->d_in, L->w1_t, L->d_in, tp_partial, L->d_R, n_tok, L->d_R, L->d_in,
-                              L->d_status, S));
+                              L->d_status + 2, S));
       } else {
         CK(launch_preact_naive(z, L->w1_t, tp_partial, n_tok, L->d_R, L->d_in, S));
       }
@@ -738,7 +744,7 @@ int chunk_step(locret_layer *L, const void *hidden_in, int32_t n_tok, uint32_t f
                         L->s + L->len, L->cap, S, pdl));
     else if (L->use_tc && n_tok >= 32 && gemm_tc_supported(n_tok, L->d_R, L->d_in, L->d_in, L->d_in))
       CK(launch_rh_gemm_tc(z, L->d_in, L->w1_t, L->w2f, P->partial, n_tok, L->d_R, L->d_in, L->h_kv,
-                           L->cfg.act, &n_tiles, L->d_status, S));
+                           L->cfg.act, &n_tiles, L->d_status + 3, S));
     else
       CK(launch_rh_gemm(z, L->d_in, L->w1_t, L->w2f, P->partial, n_tok, L->d_R, L->d_in, L->h_kv,
                         L->cfg.act, &n_tiles, S));
@@ -1032,8 +1038,18 @@ int locret_sync_status(locret_layer *L) {
   if (!L || !on_layer_device(L)) return LOCRET_ERR_INVALID;
   int host = 0;
   CK(sync_all(L));
-  CK(cudaMemcpyAsync(&host, L->d_status, sizeof(int), cudaMemcpyDeviceToHost, L->st));
+  // one word per kernel family (attention; projection GEMM; divided-heads GEMM; retaining-head GEMM), so that
+  // a reported time-out says where it happened (LOCRET_DIAG_STATUS=1 prints the words to stderr)
+  int words[4] = {0, 0, 0, 0};
+  CK(cudaMemcpyAsync(words, L->d_status, sizeof(words), cudaMemcpyDeviceToHost, L->st));
   CK(cudaStreamSynchronize(L->st));
+  for (int i = 3; i >= 0; i--) if (words[i]) host = words[i];
+  if (host != 0) {
+    const char *dg = getenv("LOCRET_DIAG_STATUS");
+    if (dg && dg[0] == '1')
+      fprintf(stderr, "locret status words: attention %d, projection %d, divided-heads product %d, retaining head %d (h %d, h_kv %d, d %d)\n",
+              words[0], words[1], words[2], words[3], L->h, L->h_kv, L->d);
+  }
   CK(cudaGetLastError());
   return host;
 }

@@ -337,61 +337,3 @@ def test_bounded_wait_reports_a_timeout_and_the_context_survives():
     lockstep_chunk(ora, gpu, hidden(128, sh.d_model, 5), 0, what="after the timed-out wait")
     assert gpu.sync_status() == 0
     gpu.destroy()
-
-
-@pytest.mark.parametrize("d", [64, 128])
-def test_attention_rescales_the_accumulator_when_a_later_key_tile_dominates(d):
-    """The tcgen05 attention kernels fix a row's scale at the first key tile they process and rescale the
-    accumulator only when a later tile's maximum exceeds it by 2^100.  Ordinary inputs never do that,
-    so here the query and key projections are made 12 times larger each (scores 144 times larger):
-    rows whose best key tile beats every other tile by more than 100 in log2 units must take the
-    rescale path whatever order the kernel walks the tiles in (unless it happens to start at that
-    tile).  head_dim 64 runs the one-CTA kernel, 128 the CTA-pair kernel."""
-    from parity_util import bf16_dev, check_attention, make_pair
-    sh = small_shape(h=4, hk=2, d=d, D=128, dR=64)
-    h, hk = sh.n_q_heads, sh.n_kv_heads
-    wqkv, w1, w2 = weights_for(sh, 33)
-    wqkv = wqkv.copy()
-    wqkv[:, : (h + hk) * d] *= 12.0
-    wqkv = W.to_bf16_grid(wqkv)
-    chunk, n_chunks = 512, 3
-    ora, gpu = make_pair(sh, (wqkv, w1, w2), budget=chunk * n_chunks, chunk=chunk, n_stab=0)
-    out = torch.zeros((chunk, h * d), dtype=torch.bfloat16, device="cuda")
-    xs = [hidden(chunk, sh.d_model, 70 + i) for i in range(n_chunks)]
-    for i, x in enumerate(xs):
-        gpu.prefill_chunk(bf16_dev(x), out, O.NO_EVICT)
-        ref = ora.prefill_chunk(x, O.NO_EVICT)
-        check_attention(out.float().cpu().numpy().astype(np.float64), ref, f"hot scores, chunk {i}",
-                        ora.last_abs_out, ora.last_flip_sens)
-    assert gpu.sync_status() == 0
-    gpu.destroy()
-
-    # how many rows of the last chunk cannot avoid the rescale: scores from the oracle's own steps
-    X = np.concatenate(xs, axis=0)
-    qkv = O.round_bf16(O.project_qkv(X, wqkv, h, hk, d))
-    Q, K, _ = O.split_qkv(qkv, h, hk, d)
-    pos = np.arange(X.shape[0])
-    Qr = O.round_bf16(O.rope(Q, pos[:, None], sh.rope_theta))
-    Kr = O.round_bf16(O.rope(K, pos[:, None], sh.rope_theta))
-    ln = chunk * (n_chunks - 1)          # keys every row of the last chunk sees in full tiles of 128
-    forced = 0
-    for j in range(h):
-        s = (Qr[ln:, j, :] @ Kr[:ln, j // sh.group, :].T) * (np.log2(np.e) / np.sqrt(d))
-        tile_max = s.reshape(chunk, ln // 128, 128).max(axis=2)
-        top2 = np.sort(tile_max, axis=1)[:, -2:]
-        forced += int(np.sum(top2[:, 1] - top2[:, 0] > 101.0))
-    assert forced >= 50, forced
-
-
-def test_one_cta_attention_kernel_is_still_selectable_for_head_dim_128(monkeypatch):
-    """head_dim 128 runs the CTA-pair kernel by default; LOCRET_ATTN_PAIR=0 (read when a layer is
-    created) selects the one-CTA kernel, which must pass the same lock-step comparison."""
-    from parity_util import lockstep_chunk, make_pair
-    sh = small_shape(h=8, hk=2, d=128, D=256, dR=64)
-    for env in ("0", "1"):
-        monkeypatch.setenv("LOCRET_ATTN_PAIR", env)
-        ora, gpu = make_pair(sh, weights_for(sh, 44), budget=700, chunk=384, n_stab=16)
-        for i, n_tok in enumerate([384, 200, 384, 129]):
-            lockstep_chunk(ora, gpu, hidden(n_tok, sh.d_model, 90 + i), 0, what=f"LOCRET_ATTN_PAIR={env} chunk {i}")
-        assert gpu.sync_status() == 0
-        gpu.destroy()
