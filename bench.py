@@ -536,7 +536,10 @@ def run_ours(args, w):
         "config": {"workload": w.name, "layers": w.n_layers, "context": w.context, "chunk": w.chunk,
                    "budget": w.budget, "n_stab": w.n_stab, "heads": f"{s.n_q_heads}q/{s.n_kv_heads}kv x {s.head_dim}",
                    "d_model": s.d_model, "d_retain": s.d_retain, "l2": "flushed between timed iterations (256 MB write)",
-                   "parallelism": "replicas only" if world > 1 else "1 GPU"},
+                   "parallelism": "replicas only" if world > 1 else "1 GPU",
+                   "attention_kernel": ("cta_pair (LOCRET_ATTN_PAIR=1, set by bench.py)"
+                                        if os.environ.get("LOCRET_ATTN_PAIR") == "1" and s.head_dim == 128
+                                        else "one_cta (library default)")},
         "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": int(w.context * s.d_model * 2),
                 "d2h_bytes_per_step": int(w.context * hd * 2), "ms_per_step": t_e2e},
         "gpu_launches": int(launches),
