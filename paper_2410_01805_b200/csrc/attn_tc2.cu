@@ -25,7 +25,6 @@
 //                    into the buffer P_j leaves; commits are multicast to both CTAs' barriers.
 // TMEM columns per CTA: S/P buffers [0,128) [128,256) [256,384), O [384,512).
 // Query row t sees keys [0, len + t]: the retained cache unmasked, the chunk causally.
-#include <cstdio>
 #include "tc_common.cuh"
 
 namespace locret {
@@ -157,13 +156,6 @@ __device__ __forceinline__ void mma2_commit_both(uint64_t *bar) {
       "h"((uint16_t)3)
       : "memory");
 }
-
-#ifdef A2_TRACE
-__device__ long long a2_trace[3][96][8];
-#define TR(role, j, k) do { if (blockIdx.x == 0 && (j) < 96 && lane == 0) a2_trace[role][j][k] = clock64(); } while (0)
-#else
-#define TR(role, j, k) do { } while (0)
-#endif
 
 struct Attn2Params {
   bf16 *out;
@@ -328,19 +320,14 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           const int buf = j % NBUF;
           const uint32_t ph = (j / NBUF) & 1;
           ok = mbar_wait(&v_full[j % NSTV], (j / NSTV) & 1, abort_flag, p.status);
-          TR(2, j, 0);
           ok = ok && mbar_wait(&p_half[buf], ph, abort_flag, p.status);
           if (!ok) break;
-          TR(2, j, 1);
           tc_fence_after();
           issue_pv(j, 0);
-          TR(2, j, 2);
           ok = mbar_wait(&p_full[buf], ph, abort_flag, p.status);
           if (!ok) break;
-          TR(2, j, 3);
           tc_fence_after();
           issue_pv(j, 1);
-          TR(2, j, 4);
           // (a barrier of its own: pv_done completes once per use of a buffer, and a warp that is done
           // early could be two phases ahead of it, which a parity cannot tell from none)
           if (j == NK - 1) mma2_commit_both(o_final);
@@ -372,9 +359,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           if (ok && j >= NBUF) ok = mbar_wait(&pv_done[j % NBUF], ((j - NBUF) / NBUF) & 1, abort_flag, p.status);
           if (!ok) break;
           tc_fence_after();
-          TR(2, j, 5);
           issue_s(j);
-          TR(2, j, 6);
         }
       }
     }
@@ -396,15 +381,12 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     for (int j = G; j < NK; j += 2) {
       const int buf = j % NBUF;
       const uint32_t s_addr = tmem_base + lane_off + (uint32_t)buf * TILE;
-      TR(G, j, 0);
       if (ok) ok = mbar_wait(&s_full[buf], (j / NBUF) & 1, abort_flag, p.status);
-      TR(G, j, 1);
       tc_fence_after();
       uint32_t s[128];
 #pragma unroll
       for (int q = 0; q < 4; q++) tmem_ld32(s_addr + q * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32 * q]));
       tmem_wait_ld();
-      TR(G, j, 2);
 
       const int key0 = tile_of(j) * TILE;
       float tmax;
@@ -428,7 +410,6 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         tmax = fmaxf(fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3])), fmaxf(fmaxf(tm[4], tm[5]), fmaxf(tm[6], tm[7])));
       }
       tmax *= c;
-      TR(G, j, 3);
 
       // the row's scale: the value published for tile j - 1, unless this tile's maximum is far above it
       float m_prev = tmax;
@@ -438,7 +419,6 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         m_prev = m_pub[((j - 1) & 1) * TILE + r];
         need = tmax > m_prev + RESCALE_LOG2;
       }
-      TR(G, j, 4);
       const float m_new = need ? tmax : m_prev;
       m_pub[(j & 1) * TILE + r] = m_new;
       __syncwarp();
@@ -487,7 +467,6 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive_remote((hf == 0 ? p_half0 : p_full0) + (uint32_t)buf * 8u);
-        TR(G, j, 5 + hf);
       }
       {
         float a0, a1, b0, b1;
@@ -546,18 +525,6 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   // another kernel's CTA while the partner's release (a cta_group::2 operation) is still to come,
   // that release could reach the newcomer's allocation.
   cluster_sync_all();
-#ifdef A2_TRACE
-  if (blockIdx.x == 0 && threadIdx.x == 0 && NK > 60) {
-    const long long t0 = a2_trace[0][32][0];
-    for (int j = 32; j < 44; j++) {
-      const int G = j & 1;
-      printf("j %d G%d: wait_s %lld got_s %lld ld %lld max %lld chain %lld half %lld full %lld | iss: pre %lld phalf %lld iss4 %lld pfull %lld iss12 %lld\n", j, G,
-             a2_trace[G][j][0] - t0, a2_trace[G][j][1] - t0, a2_trace[G][j][2] - t0, a2_trace[G][j][3] - t0, a2_trace[G][j][4] - t0,
-             a2_trace[G][j][5] - t0, a2_trace[G][j][6] - t0, a2_trace[2][j][0] - t0, a2_trace[2][j][1] - t0, a2_trace[2][j][2] - t0,
-             a2_trace[2][j][3] - t0, a2_trace[2][j][4] - t0, a2_trace[2][j][5] - t0, a2_trace[2][j][6] - t0);
-    }
-  }
-#endif
 }
 
 }  // namespace
